@@ -1,0 +1,216 @@
+"""CPU oracle (test infrastructure only).
+
+Thin numpy/ctypes front end of ``fpq_oracle.c``: the plain definition of the
+paper's floating-point quantizer (Sec. IV-B), its learned-rounding variant with
+hardened decisions (Sec. V-B) and the quantized linear / conv layer (Sec. V-B,
+Sec. VI-A), summed in double.  Nothing in the product path may import this
+package: it exists so that tests, the smoke check and the benchmark's
+CPU-baseline leg have something independent to compare the CUDA library with.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fpq_oracle.c")
+_SO = os.path.join(_HERE, "libfpq_oracle.so")
+
+SAT_PAPER = 0
+SAT_NATIVE = 1
+
+
+@dataclass(frozen=True)
+class Format:
+    """(exponent bits, mantissa bits, integer exponent bias, saturation mode)."""
+
+    e: int
+    m: int
+    B: int
+    sat: int = SAT_PAPER
+
+    @property
+    def bits(self) -> int:
+        return 4 if 1 + self.e + self.m <= 4 else 8
+
+
+E4M3 = Format(4, 3, 7, SAT_NATIVE)
+E5M2 = Format(5, 2, 15, SAT_NATIVE)
+E2M1 = Format(2, 1, 1, SAT_PAPER)
+E1M2 = Format(1, 2, 1, SAT_PAPER)
+E3M4 = Format(3, 4, 4, SAT_PAPER)
+E2M5 = Format(2, 5, 2, SAT_PAPER)
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain C, OpenMP over output rows)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fno-fast-math", "-fPIC",
+               "-shared", _SRC, "-o", _SO, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _SO
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        i32, i64, f32, f64 = ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_double
+        vp = ctypes.c_void_p
+        L.fpq_o_decode.restype = f64
+        L.fpq_o_decode.argtypes = [i32, i32, i32, i32]
+        L.fpq_o_cmax.restype = f64
+        L.fpq_o_cmax.argtypes = [i32, i32, i32, i32]
+        L.fpq_o_quantize_one.restype = i32
+        L.fpq_o_quantize_one.argtypes = [f32, f32, i32, i32, i32, i32, i32, vp]
+        L.fpq_o_quantize_weight.restype = i64
+        L.fpq_o_quantize_weight.argtypes = [vp, i64, i64, vp, i32, i32, i32, i32, vp, vp]
+        L.fpq_o_quantize_act.restype = i64
+        L.fpq_o_quantize_act.argtypes = [vp, i64, f32, i32, i32, i32, i32, vp]
+        L.fpq_o_linear.restype = i32
+        L.fpq_o_linear.argtypes = [vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, vp, i64, i64, i64,
+                                   vp, i64, vp, vp]
+        L.fpq_o_conv2d.restype = i32
+        L.fpq_o_conv2d.argtypes = [vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, vp,
+                                   i64, i64, i64, i64, i64, i64, i64, i64, i64, vp, i64, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f32(a):
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def decode(code: int, f: Format) -> float:
+    return lib().fpq_o_decode(int(code), f.e, f.m, f.B)
+
+
+def decode_table(f: Format) -> np.ndarray:
+    """Values of all 2^(1+e+m) codes, indexed by code."""
+    return np.array([decode(c, f) for c in range(1 << (1 + f.e + f.m))], dtype=np.float64)
+
+
+def cmax(f: Format) -> float:
+    return lib().fpq_o_cmax(f.e, f.m, f.B, f.sat)
+
+
+def scale_from_max(maxabs: float, f: Format) -> np.float32:
+    """Scale that maps maxabs onto the clipping value: FP32 division."""
+    return np.float32(np.float32(maxabs) / np.float32(cmax(f)))
+
+
+def quantize_one(x: float, scale: float, f: Format, h: int = -1) -> int:
+    return lib().fpq_o_quantize_one(float(np.float32(x)), float(np.float32(scale)), f.e, f.m, f.B,
+                                    f.sat, int(h), None)
+
+
+def pack_bits(bits01: np.ndarray) -> np.ndarray:
+    """[N][K] array of 0/1 -> [N][ceil(K/8)] bytes, LSB first along K."""
+    return np.packbits(np.ascontiguousarray(bits01, dtype=np.uint8), axis=1, bitorder="little")
+
+
+def quantize_weight(w, scale, f: Format, rounding_bits=None) -> np.ndarray:
+    """w: [N][K] (conv weights flattened to [Co][C*R*S]); scale: [N];
+    rounding_bits: packed bytes from pack_bits or None for round to nearest."""
+    w = _f32(w)
+    N, K = w.shape
+    scale = _f32(scale)
+    assert scale.shape == (N,)
+    row = K if f.bits == 8 else (K + 1) // 2
+    codes = np.zeros((N, row), dtype=np.uint8)
+    rb = None
+    if rounding_bits is not None:
+        rb = np.ascontiguousarray(rounding_bits, dtype=np.uint8)
+        assert rb.shape == (N, (K + 7) // 8)
+    lib().fpq_o_quantize_weight(_p(w), N, K, _p(scale), f.e, f.m, f.B, f.sat, _p(rb), _p(codes))
+    return codes
+
+
+def quantize_act(x, scale, f: Format) -> np.ndarray:
+    x = _f32(x)
+    n = x.size
+    codes = np.zeros(n if f.bits == 8 else (n + 1) // 2, dtype=np.uint8)
+    lib().fpq_o_quantize_act(_p(x), n, float(np.float32(scale)), f.e, f.m, f.B, f.sat, _p(codes))
+    return codes.reshape(x.shape) if f.bits == 8 else codes
+
+
+def linear_codes(xc, wc, w_scale, x_scale, fx: Format, fw: Format, bias, M, N, K, idx=None):
+    """Returns (y, absum) in double; with idx only those flat positions i*N+n."""
+    xc = np.ascontiguousarray(xc, dtype=np.uint8)
+    wc = np.ascontiguousarray(wc, dtype=np.uint8)
+    w_scale = _f32(w_scale)
+    bias = None if bias is None else _f32(bias)
+    if idx is not None:
+        idx = np.ascontiguousarray(idx, dtype=np.int64)
+        n_out = idx.size
+    else:
+        n_out = M * N
+    y = np.zeros(n_out, dtype=np.float64)
+    ab = np.zeros(n_out, dtype=np.float64)
+    rc = lib().fpq_o_linear(_p(xc), _p(wc), _p(w_scale), float(np.float32(x_scale)), fx.e, fx.m,
+                            fx.B, fw.e, fw.m, fw.B, _p(bias), M, N, K, _p(idx),
+                            0 if idx is None else idx.size, _p(y), _p(ab))
+    assert rc == 0
+    if idx is None:
+        return y.reshape(M, N), ab.reshape(M, N)
+    return y, ab
+
+
+def conv2d_codes(xc, wc, w_scale, x_scale, fx: Format, fw: Format, bias, B, C, H, W, Co, R, S, pad,
+                 stride, idx=None):
+    xc = np.ascontiguousarray(xc, dtype=np.uint8)
+    wc = np.ascontiguousarray(wc, dtype=np.uint8)
+    w_scale = _f32(w_scale)
+    bias = None if bias is None else _f32(bias)
+    Ho = (H + 2 * pad - R) // stride + 1
+    Wo = (W + 2 * pad - S) // stride + 1
+    if idx is not None:
+        idx = np.ascontiguousarray(idx, dtype=np.int64)
+        n_out = idx.size
+    else:
+        n_out = B * Co * Ho * Wo
+    y = np.zeros(n_out, dtype=np.float64)
+    ab = np.zeros(n_out, dtype=np.float64)
+    rc = lib().fpq_o_conv2d(_p(xc), _p(wc), _p(w_scale), float(np.float32(x_scale)), fx.e, fx.m,
+                            fx.B, fw.e, fw.m, fw.B, _p(bias), B, C, H, W, Co, R, S, pad, stride,
+                            _p(idx), 0 if idx is None else idx.size, _p(y), _p(ab))
+    assert rc == 0
+    if idx is None:
+        return y.reshape(B, Co, Ho, Wo), ab.reshape(B, Co, Ho, Wo)
+    return y, ab
+
+
+def linear(x, w, w_scale, x_scale, fx: Format, fw: Format, bias=None, rounding_bits=None, idx=None):
+    """The whole quantized linear layer from FP32 inputs: quantize weights
+    (first) and activations (Sec. VI-A), contract, rescale, add bias."""
+    x = _f32(x)
+    w = _f32(w)
+    M, K = x.shape
+    N = w.shape[0]
+    wc = quantize_weight(w, w_scale, fw, rounding_bits)
+    xc = quantize_act(x, x_scale, fx)
+    return linear_codes(xc, wc, w_scale, x_scale, fx, fw, bias, M, N, K, idx)
+
+
+def conv2d(x, w, w_scale, x_scale, fx: Format, fw: Format, bias=None, rounding_bits=None, pad=0,
+           stride=1, idx=None):
+    """The whole quantized conv layer from FP32 NCHW input and [Co][C][R][S] weights."""
+    x = _f32(x)
+    w = _f32(w)
+    B, C, H, W = x.shape
+    Co, C2, R, S = w.shape
+    assert C2 == C
+    wc = quantize_weight(w.reshape(Co, C * R * S), w_scale, fw, rounding_bits)
+    xc = quantize_act(x, x_scale, fx)
+    return conv2d_codes(xc, wc, w_scale, x_scale, fx, fw, bias, B, C, H, W, Co, R, S, pad, stride, idx)
