@@ -1,0 +1,178 @@
+/*
+ * fpq - low-bit floating-point quantized conv / linear layers for sm_100a.
+ *
+ * C ABI of the inference hot path of "Low-Bitwidth Floating Point Quantization
+ * for Efficient High-Quality Diffusion Models": the layer that every U-Net
+ * convolution and linear becomes once its weights are mapped to FP8 or FP4 and
+ * its input activations to FP8 (Sec. VI-A: weights and activations of conv and
+ * linear layers are quantized, everything else stays FP32).
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its name ends in _host.
+ *   - The caller owns every buffer.  The library allocates nothing in these
+ *     calls and keeps no state except one sticky device status word
+ *     (fpq_read_status).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Calls only enqueue work; they do not synchronise unless stated.
+ *   - Errors are return codes (negative).  Whatever the host can check (null or
+ *     misaligned pointers, impossible formats, shapes, workspace size) is
+ *     rejected before anything is launched.
+ *
+ * Number format (Sec. IV-B, format equation): a code has 1 sign bit, exp_bits
+ * exponent bits p and man_bits mantissa bits d, value
+ *     (-1)^s 2^(p - exp_bias) (1 + d / 2^man_bits)            for p > 0
+ *     (-1)^s d 2^(1 - exp_bias - man_bits)                    for p = 0
+ * bit (e+m) = sign, bits [m, e+m) = p, bits [0, m) = d.  1 + e + m <= 8; formats
+ * of up to 4 bits are stored two per byte (even index in the low nibble).
+ * `scale` is the real value of one unit of the code domain: real = scale *
+ * value(code).  It plays the role of the paper's real-valued exponent bias:
+ * b_paper = exp_bias - log2(scale).
+ */
+#ifndef FPQ_H
+#define FPQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t fpq_status;
+
+enum {
+    FPQ_OK = 0,
+    FPQ_ERR_NULL = -1,        /* a required pointer is NULL */
+    FPQ_ERR_FORMAT = -2,      /* impossible (exp_bits, man_bits, exp_bias, sat_mode) */
+    FPQ_ERR_SHAPE = -3,       /* negative / overflowing / inconsistent sizes */
+    FPQ_ERR_ALIGN = -4,       /* pointer not aligned as documented */
+    FPQ_ERR_UNSUPPORTED = -5, /* operand formats the contraction has no path for */
+    FPQ_ERR_WORKSPACE = -6,   /* workspace missing or too small */
+    FPQ_ERR_CUDA = -7,        /* a CUDA runtime / driver call failed */
+    FPQ_ERR_TIMEOUT = -8,     /* a bounded device-side wait expired (device status) */
+    FPQ_ERR_NAN_INPUT = -9    /* a NaN was quantized (to code 0) (device status) */
+};
+
+enum { FPQ_SAT_PAPER = 0, FPQ_SAT_NATIVE = 1 };
+
+/*
+ * sat_mode selects the clipping value c (Sec. IV-B, c = (2 - 2^-m) 2^(2^e - b - 1)):
+ *   FPQ_SAT_PAPER   every exponent field is finite, c as printed;
+ *   FPQ_SAT_NATIVE  c is lowered to the largest finite value of the OCP FP8 type
+ *                   with the same (e, m): E4M3 -> 1.75 * 2^(15-b) (448 at b = 7),
+ *                   E5M2 -> 1.75 * 2^(30-b); the reserved codes are never
+ *                   produced.  Other (e, m) are unaffected.
+ */
+typedef struct {
+    int32_t exp_bits, man_bits, exp_bias, sat_mode;
+} fpq_format;
+
+enum { FPQ_LINEAR = 0, FPQ_CONV2D = 1 };
+
+/* What a weight tensor belongs to.  Linear: [N][K] (C = K, R = S = 1).
+ * Conv: [N][C][R][S], K = C*R*S. */
+typedef struct {
+    int32_t kind;
+    int32_t N, C, R, S;
+} fpq_layer_desc;
+
+/* scale = maxabs / c(fmt), one FP32 division.  Host function. */
+float fpq_scale_from_max(float maxabs, fpq_format fmt);
+
+/* Clipping value c of a format (host function; 0 if the format is invalid). */
+float fpq_format_max(fpq_format fmt);
+
+/*
+ * Weight encode (offline, once per layer).  For each weight: t = w * (1.0f /
+ * scale[n]) in FP32, clip to +-c, then
+ *   rounding_bits == NULL : round to nearest on the element's own step, ties to
+ *                           even (Sec. IV-B, rounding equation and step equation);
+ *   rounding_bits != NULL : floor(t / s) + h on the signed value, h the weight's
+ *                           bit, then clamp (Sec. V-B, learned rounding with the
+ *                           decision hardened to 0 / 1 as at inference).
+ * w            [N][K] row-major FP32 (conv weights pass K = C*R*S in [C][R][S] order)
+ * scale        [N] FP32, one per output channel (per-tensor = N equal entries)
+ * rounding_bits 1 bit per weight, LSB first along K, each row padded to a byte:
+ *              [N][ceil(K/8)]
+ * codes (out)  [N][K] bytes, or [N][ceil(K/2)] for formats of <= 4 bits
+ * Zero results are always code 0.  NaN -> code 0 and FPQ_ERR_NAN_INPUT in the
+ * device status word.  +-Inf -> +-c.
+ */
+fpq_status fpq_quantize_weight(const float* w, int64_t N, int64_t K, const float* scale,
+                               fpq_format fmt, const uint8_t* rounding_bits, uint8_t* codes,
+                               void* stream);
+
+/*
+ * Activation quantize, standalone form (Sec. IV-B; one static per-tensor scale,
+ * Sec. VI-A).  x: n FP32 values; codes (out): n bytes (ceil(n/2) for <= 4 bits).
+ * Round to nearest, ties to even.
+ */
+fpq_status fpq_quantize_act(const float* x, int64_t n, float scale, fpq_format fmt, uint8_t* codes,
+                            void* stream);
+
+/*
+ * Contraction-ready copy of encoded weights.  `codes` is the output of
+ * fpq_quantize_weight for the layer `d`; `prepared` must hold
+ * fpq_prepared_size(fmt, d) bytes and be 128-byte aligned.  The layout is
+ * internal: rows of C padded with zero codes to a multiple of 128, taps
+ * outermost within a row ([N][R*S][C_pad]).  May be saved and reloaded as bytes.
+ */
+size_t fpq_prepared_size(fpq_format fmt, const fpq_layer_desc* d);
+fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_layer_desc* d,
+                              void* prepared, void* stream);
+
+/*
+ * Quantized linear layer (Sec. V-B, Y = W A, and Sec. VI-A):
+ *   y[i][n] = (x_scale * w_scale[n]) * sum_k value(q(x[i][k])) * value(wq[n][k]) + bias[n]
+ * x FP32 [M][K] row-major, y FP32 [M][N] row-major, both 16-byte aligned; bias
+ * [N] or NULL.  The activations are quantized with (fx, x_scale) exactly as
+ * fpq_quantize_act does; products are exact and accumulated in FP32 on the
+ * tensor cores.  Supported operand pairs: fx = E4M3 bias 7 FPQ_SAT_NATIVE with
+ * fw = the same, or fw = E2M1 bias 1.  Anything else: FPQ_ERR_UNSUPPORTED.
+ * workspace: fpq_linear_workspace_size bytes, 128-byte aligned; contents are
+ * scratch.
+ */
+size_t fpq_linear_workspace_size(int64_t M, int64_t N, int64_t K, fpq_format fx, fpq_format fw);
+fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_scale, float x_scale,
+                      fpq_format fx, fpq_format fw, const float* bias, float* y, int64_t M,
+                      int64_t N, int64_t K, void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * Quantized 2-D convolution (cross-correlation, zero padding, square stride):
+ * x FP32 NCHW [B][C][H][W], y FP32 NCHW [B][C_out][H_out][W_out],
+ * H_out = (H + 2 pad - R) / stride + 1.  Same arithmetic as fpq_linear with
+ * k running over (c, r, s); padding contributes code 0.
+ */
+size_t fpq_conv2d_workspace_size(int B, int C, int H, int W, int C_out, int R, int S, int pad,
+                                 int stride, fpq_format fx, fpq_format fw);
+fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_scale, float x_scale,
+                      fpq_format fx, fpq_format fw, const float* bias, float* y, int B, int C, int H,
+                      int W, int C_out, int R, int S, int pad, int stride, void* workspace,
+                      size_t ws_bytes, void* stream);
+
+/*
+ * Host-buffer forms of the two layers: x_host / y_host are host pointers
+ * (pinned memory for asynchronous copies), x_dev / y_dev are device staging
+ * buffers of the same sizes owned by the caller.  The call copies x in, runs the
+ * layer, copies y out and waits for the stream.
+ */
+fpq_status fpq_linear_host(const float* x_host, float* x_dev, const void* w_prepared,
+                           const float* w_scale, float x_scale, fpq_format fx, fpq_format fw,
+                           const float* bias, float* y_dev, float* y_host, int64_t M, int64_t N,
+                           int64_t K, void* workspace, size_t ws_bytes, void* stream);
+fpq_status fpq_conv2d_host(const float* x_host, float* x_dev, const void* w_prepared,
+                           const float* w_scale, float x_scale, fpq_format fx, fpq_format fw,
+                           const float* bias, float* y_dev, float* y_host, int B, int C, int H,
+                           int W, int C_out, int R, int S, int pad, int stride, void* workspace,
+                           size_t ws_bytes, void* stream);
+
+/* Waits for `stream`, then returns and clears the sticky device status word:
+ * FPQ_OK, FPQ_ERR_TIMEOUT, FPQ_ERR_NAN_INPUT, or FPQ_ERR_CUDA. */
+fpq_status fpq_read_status(void* stream);
+
+const char* fpq_status_string(fpq_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FPQ_H */

@@ -1,0 +1,255 @@
+// Shared device/host helpers of the fpq CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fpq.h"
+
+namespace fpq {
+
+// ---- format constants resolved on the host, passed to kernels by value --------
+struct QFormat {
+    int32_t e, m, B;
+    int32_t code_max;     // largest magnitude code that may be produced
+    uint32_t cmax_bits;   // FP32 bit pattern of the clipping value c
+    int32_t sign_shift;   // e + m
+    int32_t four_bit;     // 1 if codes are packed two per byte
+    int32_t native_e4m3;  // 1 if (4, 3, bias 7, native saturation): hardware convert applies
+};
+
+bool resolve_format(fpq_format f, QFormat* q);   // false if the format is impossible
+float format_cmax(fpq_format f);
+
+// sticky device status word (defined in fpq_api.cu)
+int* status_word();
+
+__host__ __device__ inline int64_t round_up(int64_t a, int64_t b) { return (a + b - 1) / b * b; }
+
+// ---- the quantizer on one element ---------------------------------------------
+// Clip, pick the step of the element's binade, round (nearest-even, or signed
+// floor plus the learned decision h), clamp and encode, all on the FP32 bit
+// pattern of t = x * (1/scale).  h < 0 selects round to nearest.
+__device__ __forceinline__ uint32_t quantize_bits(float t, const QFormat& f, int h, bool& nan)
+{
+    uint32_t u = __float_as_uint(t);
+    uint32_t neg = u >> 31;
+    uint32_t au = u & 0x7fffffffu;
+    if (au > 0x7f800000u) {
+        nan = true;
+        return 0;
+    }
+    au = min(au, f.cmax_bits);                       // clip (Inf included)
+    int Eb = (int)(au >> 23);
+    uint32_t mant = (au & 0x7fffffu) | (Eb ? 0x800000u : 0u);
+    int Ebn = max(Eb, 1);                            // |a| = mant * 2^(Ebn - 150)
+    int E = Ebn - 127;
+    int e_eff = max(E, 1 - f.B);                     // binade whose step applies
+    int shift = min(23 - f.m + (e_eff - E), 31);     // |a| / step = mant / 2^shift
+    uint32_t fl = mant >> shift;
+    uint32_t rem = mant & ((1u << shift) - 1u);
+    uint32_t kmag;
+    if (h < 0) {
+        uint32_t half = 1u << (shift - 1);
+        kmag = fl + ((rem > half) || (rem == half && (fl & 1u)) ? 1u : 0u);
+    } else if (!neg) {
+        kmag = fl + (uint32_t)h;
+    } else {
+        uint32_t c = fl + (rem ? 1u : 0u);           // floor of the signed value is -c
+        if (c == 0) {                                // minus zero
+            kmag = (uint32_t)h;
+            neg = 0;
+        } else {
+            kmag = c - (uint32_t)h;
+        }
+    }
+    int p1 = e_eff + f.B - 1;                        // exponent field - 1 of that binade
+    uint32_t code;
+    if (p1 >= 1 && kmag < (1u << f.m))               // fell into the finer binade below
+        code = ((uint32_t)(p1 - 1) << f.m) + 2u * kmag;
+    else
+        code = ((uint32_t)p1 << f.m) + kmag;
+    code = min(code, (uint32_t)f.code_max);
+    if (code == 0)
+        neg = 0;
+    return code | (neg << f.sign_shift);
+}
+
+// Four E4M3 (bias 7, saturating at 448) codes from four scaled floats with the
+// hardware convert; -0 and NaN are mapped to code 0 afterwards.
+__device__ __forceinline__ uint32_t e4m3x4_from_scaled(float t0, float t1, float t2, float t3, bool& nan)
+{
+    uint16_t lo, hi;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(t1), "f"(t0));
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(t3), "f"(t2));
+    uint32_t v = (uint32_t)lo | ((uint32_t)hi << 16);
+    uint32_t mag = v & 0x7f7f7f7fu;
+    uint32_t is_nan = __vcmpeq4(mag, 0x7f7f7f7fu);
+    uint32_t is_zero = __vcmpeq4(mag, 0u);
+    if (is_nan)
+        nan = true;
+    return v & ~is_nan & ~(is_zero & 0x80808080u);
+}
+
+// ---- PTX wrappers ----------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait: gives up after about two seconds and reports false.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    for (int i = 0; i < 64; ++i)
+        if (mbar_try_wait(bar, parity))
+            return true;
+    uint64_t t0;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity))
+                return true;
+        uint64_t t1;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+        if (t1 - t0 > 2000000000ull)
+            return false;
+    }
+}
+
+__device__ __forceinline__ void fence_barrier_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void tma_prefetch_desc(const void* tmap)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+// tensor memory
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+
+__device__ __forceinline__ void tmem_relinquish()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before()
+{
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+
+__device__ __forceinline__ void tc_fence_after()
+{
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem], 8-bit / 4-bit floating operands, FP32 accumulate
+__device__ __forceinline__ void mma_f8f6f4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// the barrier gets one arrival once all MMAs issued so far by this thread are done
+__device__ __forceinline__ void mma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 consecutive FP32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r)
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_wait()
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor: K-major rows of 128 bytes, 128-byte swizzle,
+// groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr)
+{
+    return (uint64_t)((addr >> 4) & 0x3fffu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor: FP32 accumulator, operand formats (0 = E4M3, 5 = E2M1),
+// both operands K-major, M = 128, N = n.
+__host__ __device__ inline uint32_t idesc_f8f6f4(uint32_t a_fmt, uint32_t b_fmt, uint32_t n)
+{
+    return (1u << 4) | (a_fmt << 7) | (b_fmt << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+}  // namespace fpq

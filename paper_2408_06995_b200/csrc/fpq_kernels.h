@@ -1,0 +1,43 @@
+// Internal launch interface between the translation units of the fpq library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fpq_common.cuh"
+
+namespace fpq {
+
+cudaError_t launch_quantize_act(const float* x, int64_t n, float scale, const QFormat& f, uint8_t* codes,
+                                cudaStream_t st);
+cudaError_t launch_quantize_weight(const float* w, int64_t N, int64_t K, const float* scale, const QFormat& f,
+                                   const uint8_t* rbits, uint8_t* codes, cudaStream_t st);
+cudaError_t launch_quantize_rows_e4m3(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, uint8_t* codes,
+                                      cudaStream_t st);
+cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int HW, int Cp, float scale,
+                                              uint8_t* codes, cudaStream_t st);
+cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, uint8_t* prepared,
+                                  cudaStream_t st);
+
+// Geometry of one contraction launch (linear: taps = 1, rows of Ca codes).
+struct GemmProblem {
+    int conv;            // 0 linear, 1 conv
+    int w4;              // weights are E2M1
+    int64_t M;           // linear rows
+    int N;               // outputs / out channels
+    int Cp;              // padded reduction length per tap in the weight copy (multiple of 128)
+    int Ca;              // padded channels (row length) of the activation codes (multiple of 16)
+    int B, H, W, Ho, Wo; // conv geometry
+    int R, S, pad, stride;
+    const uint8_t* a_codes;   // [M][Ca] or [B][H][W][Ca]
+    const void* w_prepared;   // [N][R*S][Cp]
+    const float* w_scale;
+    float x_scale;
+    const float* bias;
+    float* y;
+};
+
+// Returns FPQ_OK or an error; enqueues one kernel.
+fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st);
+
+}  // namespace fpq

@@ -1,0 +1,311 @@
+// Element-wise quantizer kernels: weight encode, activation quantize, and the
+// two layout-changing activation quantizers that feed the contraction.
+#include "fpq_common.cuh"
+#include "fpq_kernels.h"
+
+namespace fpq {
+
+// ---------------------------------------------------------------------------------
+// Activation quantize, flat: 16 elements per thread, 4 x 128-bit loads, one
+// 128-bit store.  HBM-bound: 5 bytes per element.
+// ---------------------------------------------------------------------------------
+template <bool FAST_E4M3>
+__global__ void __launch_bounds__(256) quantize_act_kernel(const float* __restrict__ x, int64_t n, float rinv,
+                                                           QFormat f, uint8_t* __restrict__ codes, int* status)
+{
+    bool nan = false;
+    int64_t nvec = n / 16;
+    int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += stride) {
+        const float4* px = reinterpret_cast<const float4*>(x) + v * 4;
+        float4 a[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            a[j] = __ldg(px + j);
+        uint32_t out[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float t0 = __fmul_rn(a[j].x, rinv), t1 = __fmul_rn(a[j].y, rinv);
+            float t2 = __fmul_rn(a[j].z, rinv), t3 = __fmul_rn(a[j].w, rinv);
+            if (FAST_E4M3) {
+                out[j] = e4m3x4_from_scaled(t0, t1, t2, t3, nan);
+            } else {
+                out[j] = quantize_bits(t0, f, -1, nan) | (quantize_bits(t1, f, -1, nan) << 8) |
+                         (quantize_bits(t2, f, -1, nan) << 16) | (quantize_bits(t3, f, -1, nan) << 24);
+            }
+        }
+        if (!f.four_bit) {
+            reinterpret_cast<uint4*>(codes)[v] = make_uint4(out[0], out[1], out[2], out[3]);
+        } else {
+            uint32_t p[2];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                uint32_t a0 = out[2 * j], a1 = out[2 * j + 1];
+                p[j] = (a0 & 0xf) | ((a0 >> 4) & 0xf0) | ((a0 >> 8) & 0xf00) | ((a0 >> 12) & 0xf000) |
+                       ((a1 & 0xf) << 16) | (((a1 >> 4) & 0xf0) << 16) | (((a1 >> 8) & 0xf00) << 16) |
+                       (((a1 >> 12) & 0xf000) << 16);
+            }
+            reinterpret_cast<uint2*>(codes)[v] = make_uint2(p[0], p[1]);
+        }
+    }
+    // tail (fewer than 16 elements): one thread, in order, so nibbles never race
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int64_t i = nvec * 16; i < n; ++i) {
+            uint32_t c = quantize_bits(__fmul_rn(x[i], rinv), f, -1, nan);
+            if (!f.four_bit) {
+                codes[i] = (uint8_t)c;
+            } else if (i & 1) {
+                codes[i >> 1] = (uint8_t)(codes[i >> 1] | (c << 4));
+            } else {
+                codes[i >> 1] = (uint8_t)c;
+            }
+        }
+    }
+    if (nan)
+        atomicMin(status, FPQ_ERR_NAN_INPUT);
+}
+
+// Unaligned input: one output byte per thread (two elements for 4-bit codes).
+__global__ void __launch_bounds__(256) quantize_act_scalar_kernel(const float* __restrict__ x, int64_t n, float rinv,
+                                                                  QFormat f, uint8_t* __restrict__ codes, int* status)
+{
+    bool nan = false;
+    int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    int64_t per = f.four_bit ? 2 : 1;
+    int64_t nout = (n + per - 1) / per;
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < nout; o += stride) {
+        uint32_t c = quantize_bits(__fmul_rn(x[o * per], rinv), f, -1, nan);
+        if (f.four_bit && o * 2 + 1 < n)
+            c |= quantize_bits(__fmul_rn(x[o * 2 + 1], rinv), f, -1, nan) << 4;
+        codes[o] = (uint8_t)c;
+    }
+    if (nan)
+        atomicMin(status, FPQ_ERR_NAN_INPUT);
+}
+
+// ---------------------------------------------------------------------------------
+// Weight encode: one thread per group of 8 weights of a row (one rounding byte).
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) quantize_weight_kernel(const float* __restrict__ w, int64_t N, int64_t K,
+                                                              const float* __restrict__ scale, QFormat f,
+                                                              const uint8_t* __restrict__ rbits,
+                                                              uint8_t* __restrict__ codes, int* status)
+{
+    bool nan = false;
+    int64_t groups = (K + 7) / 8;
+    int64_t total = N * groups;
+    int64_t row_bytes = f.four_bit ? (K + 1) / 2 : K;
+    int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += stride) {
+        int64_t n = t / groups, g = t % groups;
+        float rinv = __fdiv_rn(1.0f, __ldg(scale + n));
+        int hb = rbits ? (int)__ldg(rbits + n * groups + g) : 0;
+        const float* pw = w + n * K + g * 8;
+        int cnt = (int)min((int64_t)8, K - g * 8);
+        uint32_t c[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            c[j] = 0;
+            if (j < cnt) {
+                int h = rbits ? ((hb >> j) & 1) : -1;
+                c[j] = quantize_bits(__fmul_rn(__ldg(pw + j), rinv), f, h, nan);
+            }
+        }
+        if (!f.four_bit) {
+            uint8_t* po = codes + n * row_bytes + g * 8;
+            for (int j = 0; j < cnt; ++j)
+                po[j] = (uint8_t)c[j];
+        } else {
+            uint8_t* po = codes + n * row_bytes + g * 4;
+            for (int j = 0; j < (cnt + 1) / 2; ++j)
+                po[j] = (uint8_t)(c[2 * j] | (c[2 * j + 1] << 4));
+        }
+    }
+    if (nan)
+        atomicMin(status, FPQ_ERR_NAN_INPUT);
+}
+
+// ---------------------------------------------------------------------------------
+// Row-major activations [M][K] FP32 -> codes [M][Kp] (Kp = K rounded up to 16, pad = 0),
+// the A operand of the linear contraction.  16 elements per thread.
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const float* __restrict__ x, int64_t M, int64_t K,
+                                                                 int64_t Kp, float rinv, uint8_t* __restrict__ codes,
+                                                                 int* status)
+{
+    bool nan = false;
+    int64_t vec_per_row = Kp / 16;
+    int64_t total = M * vec_per_row;
+    int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const bool aligned = (K % 4) == 0;
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < total; v += stride) {
+        int64_t row = v / vec_per_row, k0 = (v % vec_per_row) * 16;
+        const float* px = x + row * K + k0;
+        uint32_t out[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+            int64_t k = k0 + 4 * j;
+            if (aligned && k + 4 <= K) {
+                float4 q = __ldg(reinterpret_cast<const float4*>(px + 4 * j));
+                a0 = q.x; a1 = q.y; a2 = q.z; a3 = q.w;
+            } else {
+                if (k + 0 < K) a0 = __ldg(px + 4 * j + 0);
+                if (k + 1 < K) a1 = __ldg(px + 4 * j + 1);
+                if (k + 2 < K) a2 = __ldg(px + 4 * j + 2);
+                if (k + 3 < K) a3 = __ldg(px + 4 * j + 3);
+            }
+            out[j] = e4m3x4_from_scaled(__fmul_rn(a0, rinv), __fmul_rn(a1, rinv), __fmul_rn(a2, rinv),
+                                        __fmul_rn(a3, rinv), nan);
+        }
+        reinterpret_cast<uint4*>(codes)[v] = make_uint4(out[0], out[1], out[2], out[3]);
+    }
+    if (nan)
+        atomicMin(status, FPQ_ERR_NAN_INPUT);
+}
+
+// ---------------------------------------------------------------------------------
+// NCHW FP32 -> NHWC codes [B][H*W][Cp] (Cp = C rounded up to 16, pad = 0), the A
+// operand of the implicit-GEMM convolution.  A block transposes a tile of
+// 64 channels x 32 pixels through shared memory: loads are coalesced along
+// pixels, stores along channels.
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const float* __restrict__ x, int C, int HW,
+                                                                         int Cp, float rinv,
+                                                                         uint8_t* __restrict__ codes, int* status)
+{
+    __shared__ __align__(16) uint8_t tile[32][64 + 16];
+    bool nan = false;
+    const int b = blockIdx.z;
+    const int c0 = blockIdx.y * 64;
+    const int p0 = blockIdx.x * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
+    const float* xb = x + (int64_t)b * C * HW;
+    const int p = p0 + tx;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        // this thread converts 4 consecutive channels of one pixel
+        int cl = (ty + 8 * j) * 4;
+        float a[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            int c = c0 + cl + q;
+            a[q] = (c < C && p < HW) ? __ldg(xb + (int64_t)c * HW + p) : 0.f;
+        }
+        uint32_t v = e4m3x4_from_scaled(__fmul_rn(a[0], rinv), __fmul_rn(a[1], rinv), __fmul_rn(a[2], rinv),
+                                        __fmul_rn(a[3], rinv), nan);
+        *reinterpret_cast<uint32_t*>(&tile[tx][cl]) = v;
+    }
+    __syncthreads();
+    // 32 pixels x 4 chunks of 16 channels
+    if (threadIdx.x < 128) {
+        int pl = threadIdx.x >> 2, ch = (threadIdx.x & 3) * 16;
+        int pp = p0 + pl, c = c0 + ch;
+        if (pp < HW && c < Cp) {
+            uint4 v = *reinterpret_cast<const uint4*>(&tile[pl][ch]);
+            *reinterpret_cast<uint4*>(codes + ((int64_t)b * HW + pp) * Cp + c) = v;
+        }
+    }
+    if (nan)
+        atomicMin(status, FPQ_ERR_NAN_INPUT);
+}
+
+// ---------------------------------------------------------------------------------
+// Contraction-ready weight copy: [N][C][R][S] codes -> [N][R*S][Cp] codes, zero padded.
+// One thread per output byte.
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) prepare_weight_kernel(const uint8_t* __restrict__ codes, int N, int C, int RS,
+                                                             int Cp, int four_bit, uint8_t* __restrict__ prepared)
+{
+    int64_t row_out = four_bit ? (int64_t)RS * Cp / 2 : (int64_t)RS * Cp;
+    int64_t total = (int64_t)N * row_out;
+    int64_t K = (int64_t)C * RS;
+    int64_t row_in = four_bit ? (K + 1) / 2 : K;
+    int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += stride) {
+        int64_t n = o / row_out, within = o % row_out;
+        uint32_t outb = 0;
+        int per = four_bit ? 2 : 1;
+        for (int q = 0; q < per; ++q) {
+            int64_t e = within * per + q;       // element index in [RS][Cp]
+            int tap = (int)(e / Cp), c = (int)(e % Cp);
+            uint32_t code = 0;
+            if (c < C) {
+                int64_t k = (int64_t)c * RS + tap;   // source order [C][R][S]
+                if (four_bit) {
+                    uint8_t bsrc = __ldg(codes + n * row_in + (k >> 1));
+                    code = (k & 1) ? (bsrc >> 4) : (bsrc & 0xf);
+                } else {
+                    code = __ldg(codes + n * row_in + k);
+                }
+            }
+            outb |= code << (4 * q * four_bit);
+        }
+        prepared[o] = (uint8_t)outb;
+    }
+}
+
+// ---- launchers ----------------------------------------------------------------------
+static int grid_for(int64_t work_items, int threads)
+{
+    int64_t blocks = (work_items + threads - 1) / threads;
+    const int64_t cap = 148 * 16;
+    if (blocks > cap)
+        blocks = cap;
+    if (blocks < 1)
+        blocks = 1;
+    return (int)blocks;
+}
+
+cudaError_t launch_quantize_act(const float* x, int64_t n, float scale, const QFormat& f, uint8_t* codes,
+                                cudaStream_t st)
+{
+    if (n == 0)
+        return cudaSuccess;
+    float rinv = 1.0f / scale;
+    bool aligned = ((uintptr_t)x % 16 == 0) && ((uintptr_t)codes % 16 == 0);
+    if (!aligned) {
+        quantize_act_scalar_kernel<<<grid_for(n, 256), 256, 0, st>>>(x, n, rinv, f, codes, status_word());
+    } else if (f.native_e4m3) {
+        quantize_act_kernel<true><<<grid_for(n / 16 + 1, 256), 256, 0, st>>>(x, n, rinv, f, codes, status_word());
+    } else {
+        quantize_act_kernel<false><<<grid_for(n / 16 + 1, 256), 256, 0, st>>>(x, n, rinv, f, codes, status_word());
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_weight(const float* w, int64_t N, int64_t K, const float* scale, const QFormat& f,
+                                   const uint8_t* rbits, uint8_t* codes, cudaStream_t st)
+{
+    if (N == 0 || K == 0)
+        return cudaSuccess;
+    int64_t total = N * ((K + 7) / 8);
+    quantize_weight_kernel<<<grid_for(total, 256), 256, 0, st>>>(w, N, K, scale, f, rbits, codes, status_word());
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_rows_e4m3(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, uint8_t* codes,
+                                      cudaStream_t st)
+{
+    int64_t total = M * (Kp / 16);
+    quantize_rows_e4m3_kernel<<<grid_for(total, 256), 256, 0, st>>>(x, M, K, Kp, 1.0f / scale, codes, status_word());
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int HW, int Cp, float scale,
+                                              uint8_t* codes, cudaStream_t st)
+{
+    dim3 grid((HW + 31) / 32, (Cp + 63) / 64, B);
+    quantize_nchw_to_nhwc_e4m3_kernel<<<grid, 256, 0, st>>>(x, C, HW, Cp, 1.0f / scale, codes, status_word());
+    return cudaGetLastError();
+}
+
+cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, uint8_t* prepared,
+                                  cudaStream_t st)
+{
+    int64_t total = (int64_t)N * RS * Cp / (four_bit ? 2 : 1);
+    prepare_weight_kernel<<<grid_for(total, 256), 256, 0, st>>>(codes, N, C, RS, Cp, four_bit, prepared);
+    return cudaGetLastError();
+}
+
+}  // namespace fpq
