@@ -1,0 +1,246 @@
+"""Python binding of libfpq.so: argument marshalling only.
+
+Every function here has the name of the C entry point it calls
+(include/fpq.h) and passes torch tensors' device pointers and the current CUDA
+stream.  All arithmetic runs in the library's kernels.  There is no fallback:
+if the shared library is missing the import of a symbol fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "libfpq.so")
+
+OK = 0
+ERR_NULL, ERR_FORMAT, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED = -1, -2, -3, -4, -5
+ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NAN_INPUT = -6, -7, -8, -9
+SAT_PAPER, SAT_NATIVE = 0, 1
+LINEAR, CONV2D = 0, 1
+
+
+class FpqError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+class _CFormat(ctypes.Structure):
+    _fields_ = [("exp_bits", ctypes.c_int32), ("man_bits", ctypes.c_int32),
+                ("exp_bias", ctypes.c_int32), ("sat_mode", ctypes.c_int32)]
+
+
+class _CLayerDesc(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int32), ("N", ctypes.c_int32), ("C", ctypes.c_int32),
+                ("R", ctypes.c_int32), ("S", ctypes.c_int32)]
+
+
+@dataclass(frozen=True)
+class Format:
+    exp_bits: int
+    man_bits: int
+    exp_bias: int
+    sat_mode: int = SAT_PAPER
+
+    def c(self) -> _CFormat:
+        return _CFormat(self.exp_bits, self.man_bits, self.exp_bias, self.sat_mode)
+
+    @property
+    def four_bit(self) -> bool:
+        return 1 + self.exp_bits + self.man_bits <= 4
+
+
+E4M3 = Format(4, 3, 7, SAT_NATIVE)
+E5M2 = Format(5, 2, 15, SAT_NATIVE)
+E2M1 = Format(2, 1, 1, SAT_PAPER)
+E1M2 = Format(1, 2, 1, SAT_PAPER)
+E3M4 = Format(3, 4, 4, SAT_PAPER)
+E2M5 = Format(2, 5, 2, SAT_PAPER)
+
+EXPORTS = [
+    "fpq_scale_from_max", "fpq_format_max", "fpq_quantize_weight", "fpq_quantize_act",
+    "fpq_prepared_size", "fpq_prepare_weight", "fpq_linear_workspace_size", "fpq_linear",
+    "fpq_conv2d_workspace_size", "fpq_conv2d", "fpq_linear_host", "fpq_conv2d_host",
+    "fpq_read_status", "fpq_status_string",
+]
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_SO):
+            raise FileNotFoundError(
+                f"{_SO} is missing: build it with `python -m paper_2408_06995_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(_SO)
+        i32, i64, f32 = ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+        vp, sz = ctypes.c_void_p, ctypes.c_size_t
+        F, D = _CFormat, ctypes.POINTER(_CLayerDesc)
+        L.fpq_scale_from_max.restype = f32
+        L.fpq_scale_from_max.argtypes = [f32, F]
+        L.fpq_format_max.restype = f32
+        L.fpq_format_max.argtypes = [F]
+        L.fpq_quantize_weight.restype = i32
+        L.fpq_quantize_weight.argtypes = [vp, i64, i64, vp, F, vp, vp, vp]
+        L.fpq_quantize_act.restype = i32
+        L.fpq_quantize_act.argtypes = [vp, i64, f32, F, vp, vp]
+        L.fpq_prepared_size.restype = sz
+        L.fpq_prepared_size.argtypes = [F, D]
+        L.fpq_prepare_weight.restype = i32
+        L.fpq_prepare_weight.argtypes = [vp, F, D, vp, vp]
+        L.fpq_linear_workspace_size.restype = sz
+        L.fpq_linear_workspace_size.argtypes = [i64, i64, i64, F, F]
+        L.fpq_linear.restype = i32
+        L.fpq_linear.argtypes = [vp, vp, vp, f32, F, F, vp, vp, i64, i64, i64, vp, sz, vp]
+        L.fpq_conv2d_workspace_size.restype = sz
+        L.fpq_conv2d_workspace_size.argtypes = [i32] * 9 + [F, F]
+        L.fpq_conv2d.restype = i32
+        L.fpq_conv2d.argtypes = [vp, vp, vp, f32, F, F, vp, vp] + [i32] * 9 + [vp, sz, vp]
+        L.fpq_linear_host.restype = i32
+        L.fpq_linear_host.argtypes = [vp, vp, vp, vp, f32, F, F, vp, vp, vp, i64, i64, i64, vp, sz, vp]
+        L.fpq_conv2d_host.restype = i32
+        L.fpq_conv2d_host.argtypes = [vp, vp, vp, vp, f32, F, F, vp, vp, vp] + [i32] * 9 + [vp, sz, vp]
+        L.fpq_read_status.restype = i32
+        L.fpq_read_status.argtypes = [vp]
+        L.fpq_status_string.restype = ctypes.c_char_p
+        L.fpq_status_string.argtypes = [i32]
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise FpqError(code, where)
+
+
+def status_string(code: int) -> str:
+    return lib().fpq_status_string(int(code)).decode()
+
+
+def fpq_format_max(fmt: Format) -> float:
+    return lib().fpq_format_max(fmt.c())
+
+
+def fpq_scale_from_max(maxabs: float, fmt: Format) -> float:
+    return lib().fpq_scale_from_max(float(maxabs), fmt.c())
+
+
+def fpq_quantize_weight(w: torch.Tensor, scale: torch.Tensor, fmt: Format, rounding_bits=None,
+                        codes: torch.Tensor = None) -> torch.Tensor:
+    """w [N][K] float32 (cuda, contiguous), scale [N], rounding_bits packed uint8
+    [N][ceil(K/8)] or None.  Returns codes [N][K] or [N][ceil(K/2)] uint8."""
+    assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous() and w.dim() == 2
+    N, K = w.shape
+    if codes is None:
+        codes = torch.empty((N, (K + 1) // 2 if fmt.four_bit else K), dtype=torch.uint8, device=w.device)
+    _check(lib().fpq_quantize_weight(_ptr(w), N, K, _ptr(scale), fmt.c(), _ptr(rounding_bits), _ptr(codes),
+                                     _stream()), "fpq_quantize_weight")
+    return codes
+
+
+def fpq_quantize_act(x: torch.Tensor, scale: float, fmt: Format, codes: torch.Tensor = None) -> torch.Tensor:
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    n = x.numel()
+    if codes is None:
+        shape = ((n + 1) // 2,) if fmt.four_bit else tuple(x.shape)
+        codes = torch.empty(shape, dtype=torch.uint8, device=x.device)
+    _check(lib().fpq_quantize_act(_ptr(x), n, float(scale), fmt.c(), _ptr(codes), _stream()), "fpq_quantize_act")
+    return codes
+
+
+def _desc(kind, N, C, R=1, S=1):
+    return _CLayerDesc(kind, N, C, R, S)
+
+
+def fpq_prepared_size(fmt: Format, kind: int, N: int, C: int, R: int = 1, S: int = 1) -> int:
+    d = _desc(kind, N, C, R, S)
+    return lib().fpq_prepared_size(fmt.c(), ctypes.byref(d))
+
+
+def fpq_prepare_weight(codes: torch.Tensor, fmt: Format, kind: int, N: int, C: int, R: int = 1, S: int = 1,
+                       prepared: torch.Tensor = None) -> torch.Tensor:
+    d = _desc(kind, N, C, R, S)
+    size = lib().fpq_prepared_size(fmt.c(), ctypes.byref(d))
+    if size == 0:
+        raise FpqError(ERR_SHAPE, "fpq_prepared_size")
+    if prepared is None:
+        prepared = torch.empty(size, dtype=torch.uint8, device=codes.device)
+    _check(lib().fpq_prepare_weight(_ptr(codes), fmt.c(), ctypes.byref(d), _ptr(prepared), _stream()),
+           "fpq_prepare_weight")
+    return prepared
+
+
+def fpq_linear_workspace_size(M, N, K, fx: Format, fw: Format) -> int:
+    return lib().fpq_linear_workspace_size(M, N, K, fx.c(), fw.c())
+
+
+def fpq_linear(x, w_prepared, w_scale, x_scale, fx: Format, fw: Format, bias, N: int, y=None, workspace=None):
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous() and x.dim() == 2
+    M, K = x.shape
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float32, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(max(1, fpq_linear_workspace_size(M, N, K, fx, fw)), dtype=torch.uint8, device=x.device)
+    _check(lib().fpq_linear(_ptr(x), _ptr(w_prepared), _ptr(w_scale), float(x_scale), fx.c(), fw.c(), _ptr(bias),
+                            _ptr(y), M, N, K, _ptr(workspace), workspace.numel(), _stream()), "fpq_linear")
+    return y
+
+
+def fpq_conv2d_workspace_size(B, C, H, W, C_out, R, S, pad, stride, fx: Format, fw: Format) -> int:
+    return lib().fpq_conv2d_workspace_size(B, C, H, W, C_out, R, S, pad, stride, fx.c(), fw.c())
+
+
+def fpq_conv2d(x, w_prepared, w_scale, x_scale, fx: Format, fw: Format, bias, C_out, R, S, pad, stride, y=None,
+               workspace=None):
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous() and x.dim() == 4
+    B, C, H, W = x.shape
+    Ho = (H + 2 * pad - R) // stride + 1
+    Wo = (W + 2 * pad - S) // stride + 1
+    if y is None:
+        y = torch.empty((B, C_out, Ho, Wo), dtype=torch.float32, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(max(1, fpq_conv2d_workspace_size(B, C, H, W, C_out, R, S, pad, stride, fx, fw)),
+                                dtype=torch.uint8, device=x.device)
+    _check(lib().fpq_conv2d(_ptr(x), _ptr(w_prepared), _ptr(w_scale), float(x_scale), fx.c(), fw.c(), _ptr(bias),
+                            _ptr(y), B, C, H, W, C_out, R, S, pad, stride, _ptr(workspace), workspace.numel(),
+                            _stream()), "fpq_conv2d")
+    return y
+
+
+def fpq_linear_host(x_host, x_dev, w_prepared, w_scale, x_scale, fx, fw, bias, y_dev, y_host, workspace):
+    """x_host / y_host: pinned CPU tensors; x_dev / y_dev: device staging tensors."""
+    M, K = x_host.shape
+    N = y_host.shape[1]
+    _check(lib().fpq_linear_host(_ptr(x_host), _ptr(x_dev), _ptr(w_prepared), _ptr(w_scale), float(x_scale),
+                                 fx.c(), fw.c(), _ptr(bias), _ptr(y_dev), _ptr(y_host), M, N, K, _ptr(workspace),
+                                 workspace.numel(), _stream()), "fpq_linear_host")
+    return y_host
+
+
+def fpq_conv2d_host(x_host, x_dev, w_prepared, w_scale, x_scale, fx, fw, bias, y_dev, y_host, R, S, pad, stride,
+                    workspace):
+    B, C, H, W = x_host.shape
+    C_out = y_host.shape[1]
+    _check(lib().fpq_conv2d_host(_ptr(x_host), _ptr(x_dev), _ptr(w_prepared), _ptr(w_scale), float(x_scale),
+                                 fx.c(), fw.c(), _ptr(bias), _ptr(y_dev), _ptr(y_host), B, C, H, W, C_out, R, S,
+                                 pad, stride, _ptr(workspace), workspace.numel(), _stream()), "fpq_conv2d_host")
+    return y_host
+
+
+def fpq_read_status() -> int:
+    return lib().fpq_read_status(_stream())

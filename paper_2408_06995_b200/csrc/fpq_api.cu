@@ -1,0 +1,406 @@
+// extern "C" entry points: argument checks, format resolution, dispatch.
+#include <math.h>
+#include <string.h>
+
+#include "fpq_common.cuh"
+#include "fpq_kernels.h"
+
+namespace fpq {
+
+__device__ int g_status = 0;
+
+int* status_word()
+{
+    // one lookup per device: the symbol has a separate instance on each GPU
+    static int* ptr[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
+        return nullptr;
+    if (!ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status) != cudaSuccess)
+            return nullptr;
+        ptr[dev] = (int*)p;
+    }
+    return ptr[dev];
+}
+
+float format_cmax(fpq_format f)
+{
+    int top = (1 << f.exp_bits) - 1;
+    if (f.sat_mode == FPQ_SAT_NATIVE && f.exp_bits == 4 && f.man_bits == 3)
+        return ldexpf(1.75f, top - f.exp_bias);
+    if (f.sat_mode == FPQ_SAT_NATIVE && f.exp_bits == 5 && f.man_bits == 2)
+        return ldexpf(1.75f, top - 1 - f.exp_bias);
+    return ldexpf(2.0f - ldexpf(1.0f, -f.man_bits), top - f.exp_bias);
+}
+
+bool resolve_format(fpq_format f, QFormat* q)
+{
+    if (f.exp_bits < 1 || f.man_bits < 1 || 1 + f.exp_bits + f.man_bits > 8)
+        return false;
+    if (f.sat_mode != FPQ_SAT_PAPER && f.sat_mode != FPQ_SAT_NATIVE)
+        return false;
+    int top = (1 << f.exp_bits) - 1;
+    // every grid value must be a normal FP32 number
+    if (top - f.exp_bias > 126 || 1 - f.exp_bias - f.man_bits < -125)
+        return false;
+    q->e = f.exp_bits;
+    q->m = f.man_bits;
+    q->B = f.exp_bias;
+    q->sign_shift = f.exp_bits + f.man_bits;
+    q->four_bit = (1 + f.exp_bits + f.man_bits <= 4) ? 1 : 0;
+    q->code_max = (1 << (f.exp_bits + f.man_bits)) - 1;
+    if (f.sat_mode == FPQ_SAT_NATIVE && f.exp_bits == 4 && f.man_bits == 3)
+        q->code_max = 0x7E;
+    if (f.sat_mode == FPQ_SAT_NATIVE && f.exp_bits == 5 && f.man_bits == 2)
+        q->code_max = 0x7B;
+    float c = format_cmax(f);
+    memcpy(&q->cmax_bits, &c, 4);
+    q->native_e4m3 = (f.exp_bits == 4 && f.man_bits == 3 && f.exp_bias == 7 && f.sat_mode == FPQ_SAT_NATIVE) ? 1 : 0;
+    return true;
+}
+
+static bool is_e4m3_native(fpq_format f)
+{
+    return f.exp_bits == 4 && f.man_bits == 3 && f.exp_bias == 7 && f.sat_mode == FPQ_SAT_NATIVE;
+}
+
+static bool is_e2m1(fpq_format f)
+{
+    return f.exp_bits == 2 && f.man_bits == 1 && f.exp_bias == 1;
+}
+
+static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+static int64_t padded_c(int64_t C) { return round_up(C, 128); }
+
+static fpq_status check_pair(fpq_format fx, fpq_format fw)
+{
+    QFormat q;
+    if (!resolve_format(fx, &q) || !resolve_format(fw, &q))
+        return FPQ_ERR_FORMAT;
+    if (!is_e4m3_native(fx))
+        return FPQ_ERR_UNSUPPORTED;
+    if (!is_e4m3_native(fw) && !is_e2m1(fw))
+        return FPQ_ERR_UNSUPPORTED;
+    return FPQ_OK;
+}
+
+}  // namespace fpq
+
+using namespace fpq;
+
+extern "C" {
+
+float fpq_format_max(fpq_format fmt)
+{
+    QFormat q;
+    if (!resolve_format(fmt, &q))
+        return 0.f;
+    return format_cmax(fmt);
+}
+
+float fpq_scale_from_max(float maxabs, fpq_format fmt)
+{
+    float c = fpq_format_max(fmt);
+    if (c == 0.f)
+        return 0.f;
+    return maxabs / c;
+}
+
+fpq_status fpq_quantize_weight(const float* w, int64_t N, int64_t K, const float* scale, fpq_format fmt,
+                               const uint8_t* rounding_bits, uint8_t* codes, void* stream)
+{
+    QFormat q;
+    if (!resolve_format(fmt, &q))
+        return FPQ_ERR_FORMAT;
+    if (N < 0 || K < 0 || (N > 0 && K > INT64_MAX / 8 / N))
+        return FPQ_ERR_SHAPE;
+    if (N == 0 || K == 0)
+        return FPQ_OK;
+    if (!w || !scale || !codes)
+        return FPQ_ERR_NULL;
+    if (!aligned(w, 4) || !aligned(scale, 4))
+        return FPQ_ERR_ALIGN;
+    if (!status_word())
+        return FPQ_ERR_CUDA;
+    return launch_quantize_weight(w, N, K, scale, q, rounding_bits, codes, (cudaStream_t)stream) == cudaSuccess
+               ? FPQ_OK
+               : FPQ_ERR_CUDA;
+}
+
+fpq_status fpq_quantize_act(const float* x, int64_t n, float scale, fpq_format fmt, uint8_t* codes, void* stream)
+{
+    QFormat q;
+    if (!resolve_format(fmt, &q))
+        return FPQ_ERR_FORMAT;
+    if (n < 0)
+        return FPQ_ERR_SHAPE;
+    if (n == 0)
+        return FPQ_OK;
+    if (!x || !codes)
+        return FPQ_ERR_NULL;
+    if (!aligned(x, 4))
+        return FPQ_ERR_ALIGN;
+    if (!status_word())
+        return FPQ_ERR_CUDA;
+    return launch_quantize_act(x, n, scale, q, codes, (cudaStream_t)stream) == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
+}
+
+static fpq_status check_desc(const fpq_layer_desc* d)
+{
+    if (!d)
+        return FPQ_ERR_NULL;
+    if (d->kind != FPQ_LINEAR && d->kind != FPQ_CONV2D)
+        return FPQ_ERR_SHAPE;
+    if (d->N < 1 || d->C < 1 || d->R < 1 || d->S < 1)
+        return FPQ_ERR_SHAPE;
+    if (d->kind == FPQ_LINEAR && (d->R != 1 || d->S != 1))
+        return FPQ_ERR_SHAPE;
+    if ((int64_t)d->R * d->S > 1024 || (int64_t)d->N * d->R * d->S * padded_c(d->C) > ((int64_t)1 << 40))
+        return FPQ_ERR_SHAPE;
+    return FPQ_OK;
+}
+
+size_t fpq_prepared_size(fpq_format fmt, const fpq_layer_desc* d)
+{
+    QFormat q;
+    if (!resolve_format(fmt, &q) || check_desc(d) != FPQ_OK)
+        return 0;
+    size_t elems = (size_t)d->N * d->R * d->S * (size_t)padded_c(d->C);
+    return q.four_bit ? elems / 2 : elems;
+}
+
+fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_layer_desc* d, void* prepared,
+                              void* stream)
+{
+    QFormat q;
+    if (!resolve_format(fmt, &q))
+        return FPQ_ERR_FORMAT;
+    fpq_status s = check_desc(d);
+    if (s != FPQ_OK)
+        return s;
+    if (!codes || !prepared)
+        return FPQ_ERR_NULL;
+    if (!aligned(prepared, 128))
+        return FPQ_ERR_ALIGN;
+    return launch_prepare_weight(codes, d->N, d->C, d->R * d->S, (int)padded_c(d->C), q.four_bit, (uint8_t*)prepared,
+                                 (cudaStream_t)stream) == cudaSuccess
+               ? FPQ_OK
+               : FPQ_ERR_CUDA;
+}
+
+size_t fpq_linear_workspace_size(int64_t M, int64_t N, int64_t K, fpq_format fx, fpq_format fw)
+{
+    (void)N;
+    if (check_pair(fx, fw) != FPQ_OK || M < 0 || K < 0)
+        return 0;
+    return (size_t)(M * round_up(K, 16));
+}
+
+fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_scale, float x_scale, fpq_format fx,
+                      fpq_format fw, const float* bias, float* y, int64_t M, int64_t N, int64_t K, void* workspace,
+                      size_t ws_bytes, void* stream)
+{
+    fpq_status s = check_pair(fx, fw);
+    if (s != FPQ_OK)
+        return s;
+    if (M < 0 || N < 0 || K < 0 || M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff)
+        return FPQ_ERR_SHAPE;
+    if (M == 0 || N == 0)
+        return FPQ_OK;
+    if (K == 0)
+        return FPQ_ERR_SHAPE;
+    if (!x || !w_prepared || !w_scale || !y)
+        return FPQ_ERR_NULL;
+    if (!aligned(x, 16) || !aligned(y, 16) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
+        (bias && !aligned(bias, 4)))
+        return FPQ_ERR_ALIGN;
+    const int64_t Kp = round_up(K, 16);
+    if (!workspace || ws_bytes < (size_t)(M * Kp))
+        return FPQ_ERR_WORKSPACE;
+    if (!aligned(workspace, 128))
+        return FPQ_ERR_ALIGN;
+    if (!status_word())
+        return FPQ_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (launch_quantize_rows_e4m3(x, M, K, Kp, x_scale, (uint8_t*)workspace, st) != cudaSuccess)
+        return FPQ_ERR_CUDA;
+    GemmProblem p{};
+    p.conv = 0;
+    p.w4 = is_e2m1(fw) ? 1 : 0;
+    p.M = M;
+    p.N = (int)N;
+    p.Cp = (int)padded_c(K);
+    p.Ca = (int)Kp;
+    p.B = p.H = p.W = p.Ho = p.Wo = 1;
+    p.R = p.S = 1;
+    p.pad = 0;
+    p.stride = 1;
+    p.a_codes = (const uint8_t*)workspace;
+    p.w_prepared = w_prepared;
+    p.w_scale = w_scale;
+    p.x_scale = x_scale;
+    p.bias = bias;
+    p.y = y;
+    return launch_gemm(p, st);
+}
+
+static fpq_status conv_shape(int B, int C, int H, int W, int C_out, int R, int S, int pad, int stride, int* Ho,
+                             int* Wo)
+{
+    if (B < 0 || C < 1 || H < 1 || W < 1 || C_out < 0 || R < 1 || S < 1 || pad < 0 || stride < 1)
+        return FPQ_ERR_SHAPE;
+    if (H + 2 * pad < R || W + 2 * pad < S)
+        return FPQ_ERR_SHAPE;
+    *Ho = (H + 2 * pad - R) / stride + 1;
+    *Wo = (W + 2 * pad - S) / stride + 1;
+    if ((int64_t)B * C * H * W > ((int64_t)1 << 40) || (int64_t)B * C_out * *Ho * *Wo > ((int64_t)1 << 40))
+        return FPQ_ERR_SHAPE;
+    return FPQ_OK;
+}
+
+size_t fpq_conv2d_workspace_size(int B, int C, int H, int W, int C_out, int R, int S, int pad, int stride,
+                                 fpq_format fx, fpq_format fw)
+{
+    int Ho, Wo;
+    if (check_pair(fx, fw) != FPQ_OK || conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo) != FPQ_OK)
+        return 0;
+    return (size_t)B * H * W * (size_t)round_up(C, 16);
+}
+
+fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_scale, float x_scale, fpq_format fx,
+                      fpq_format fw, const float* bias, float* y, int B, int C, int H, int W, int C_out, int R, int S,
+                      int pad, int stride, void* workspace, size_t ws_bytes, void* stream)
+{
+    fpq_status s = check_pair(fx, fw);
+    if (s != FPQ_OK)
+        return s;
+    int Ho, Wo;
+    s = conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo);
+    if (s != FPQ_OK)
+        return s;
+    if (B == 0 || C_out == 0)
+        return FPQ_OK;
+    if (B > 65535)
+        return FPQ_ERR_SHAPE;
+    if (!x || !w_prepared || !w_scale || !y)
+        return FPQ_ERR_NULL;
+    if (!aligned(x, 4) || !aligned(y, 4) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
+        (bias && !aligned(bias, 4)))
+        return FPQ_ERR_ALIGN;
+    const int Ca = (int)round_up(C, 16);
+    if (!workspace || ws_bytes < (size_t)B * H * W * (size_t)Ca)
+        return FPQ_ERR_WORKSPACE;
+    if (!aligned(workspace, 128))
+        return FPQ_ERR_ALIGN;
+    if (!status_word())
+        return FPQ_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H * W, Ca, x_scale, (uint8_t*)workspace, st) != cudaSuccess)
+        return FPQ_ERR_CUDA;
+    GemmProblem p{};
+    p.conv = 1;
+    p.w4 = is_e2m1(fw) ? 1 : 0;
+    p.M = (int64_t)B * Ho * Wo;
+    p.N = C_out;
+    p.Cp = (int)padded_c(C);
+    p.Ca = Ca;
+    p.B = B;
+    p.H = H;
+    p.W = W;
+    p.Ho = Ho;
+    p.Wo = Wo;
+    p.R = R;
+    p.S = S;
+    p.pad = pad;
+    p.stride = stride;
+    p.a_codes = (const uint8_t*)workspace;
+    p.w_prepared = w_prepared;
+    p.w_scale = w_scale;
+    p.x_scale = x_scale;
+    p.bias = bias;
+    p.y = y;
+    return launch_gemm(p, st);
+}
+
+fpq_status fpq_linear_host(const float* x_host, float* x_dev, const void* w_prepared, const float* w_scale,
+                           float x_scale, fpq_format fx, fpq_format fw, const float* bias, float* y_dev,
+                           float* y_host, int64_t M, int64_t N, int64_t K, void* workspace, size_t ws_bytes,
+                           void* stream)
+{
+    if (!x_host || !x_dev || !y_dev || !y_host)
+        return FPQ_ERR_NULL;
+    if (M < 0 || N < 0 || K < 0)
+        return FPQ_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(x_dev, x_host, sizeof(float) * (size_t)M * K, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return FPQ_ERR_CUDA;
+    fpq_status s = fpq_linear(x_dev, w_prepared, w_scale, x_scale, fx, fw, bias, y_dev, M, N, K, workspace, ws_bytes,
+                              stream);
+    if (s != FPQ_OK)
+        return s;
+    if (cudaMemcpyAsync(y_host, y_dev, sizeof(float) * (size_t)M * N, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return FPQ_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
+}
+
+fpq_status fpq_conv2d_host(const float* x_host, float* x_dev, const void* w_prepared, const float* w_scale,
+                           float x_scale, fpq_format fx, fpq_format fw, const float* bias, float* y_dev,
+                           float* y_host, int B, int C, int H, int W, int C_out, int R, int S, int pad, int stride,
+                           void* workspace, size_t ws_bytes, void* stream)
+{
+    if (!x_host || !x_dev || !y_dev || !y_host)
+        return FPQ_ERR_NULL;
+    int Ho, Wo;
+    fpq_status s = conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo);
+    if (s != FPQ_OK)
+        return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(x_dev, x_host, sizeof(float) * (size_t)B * C * H * W, cudaMemcpyHostToDevice, st) !=
+        cudaSuccess)
+        return FPQ_ERR_CUDA;
+    s = fpq_conv2d(x_dev, w_prepared, w_scale, x_scale, fx, fw, bias, y_dev, B, C, H, W, C_out, R, S, pad, stride,
+                   workspace, ws_bytes, stream);
+    if (s != FPQ_OK)
+        return s;
+    if (cudaMemcpyAsync(y_host, y_dev, sizeof(float) * (size_t)B * C_out * Ho * Wo, cudaMemcpyDeviceToHost, st) !=
+        cudaSuccess)
+        return FPQ_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
+}
+
+fpq_status fpq_read_status(void* stream)
+{
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess)
+        return FPQ_ERR_CUDA;
+    int* sw = status_word();
+    if (!sw)
+        return FPQ_ERR_CUDA;
+    int v = 0, zero = 0;
+    if (cudaMemcpy(&v, sw, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return FPQ_ERR_CUDA;
+    if (v != 0 && cudaMemcpy(sw, &zero, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess)
+        return FPQ_ERR_CUDA;
+    return (fpq_status)v;
+}
+
+const char* fpq_status_string(fpq_status s)
+{
+    switch (s) {
+    case FPQ_OK: return "ok";
+    case FPQ_ERR_NULL: return "null pointer";
+    case FPQ_ERR_FORMAT: return "invalid number format";
+    case FPQ_ERR_SHAPE: return "invalid shape";
+    case FPQ_ERR_ALIGN: return "misaligned pointer";
+    case FPQ_ERR_UNSUPPORTED: return "unsupported operand formats or geometry";
+    case FPQ_ERR_WORKSPACE: return "workspace missing or too small";
+    case FPQ_ERR_CUDA: return "CUDA call failed";
+    case FPQ_ERR_TIMEOUT: return "device-side wait timed out";
+    case FPQ_ERR_NAN_INPUT: return "NaN input quantized to zero";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,91 @@
+"""Shared plumbing of the GPU parity tests: run a layer through the C-ABI binding and
+through the CPU oracle on the same seeded tensors."""
+import numpy as np
+import torch
+
+import oracle as O
+import paper_2408_06995_b200 as fpq
+from paper_2408_06995_b200 import build as fpq_build
+
+fpq_build.build()
+
+FMT = {"e4m3": (fpq.E4M3, O.E4M3), "e2m1": (fpq.E2M1, O.E2M1)}
+
+
+def to_oracle(f: fpq.Format) -> O.Format:
+    return O.Format(f.exp_bits, f.man_bits, f.exp_bias, f.sat_mode)
+
+
+def layer_scales(L):
+    """max-scaling per output channel / per tensor; each side divides with its own routine."""
+    gfw, ofw = FMT[L.wfmt]
+    w2 = L.w.reshape(L.N, -1)
+    wmax = np.abs(w2).max(axis=1)
+    xmax = float(np.abs(L.x).max())
+    ws_o = np.array([O.scale_from_max(v, ofw) for v in wmax], dtype=np.float32)
+    xs_o = O.scale_from_max(xmax, O.E4M3)
+    ws_g = np.array([fpq.fpq_scale_from_max(float(v), gfw) for v in wmax], dtype=np.float32)
+    xs_g = fpq.fpq_scale_from_max(xmax, fpq.E4M3)
+    assert np.array_equal(ws_o, ws_g) and np.float32(xs_o) == np.float32(xs_g)
+    return ws_g, xs_g
+
+
+def gpu_prepare(L, ws):
+    """Weight encode + contraction-ready copy on the GPU; returns (codes, prepared)."""
+    gfw, _ = FMT[L.wfmt]
+    dev = "cuda"
+    w2 = torch.from_numpy(L.w.reshape(L.N, -1)).to(dev)
+    rb = None
+    if L.bits is not None:
+        rb = torch.from_numpy(O.pack_bits(L.bits)).to(dev)
+    codes = fpq.fpq_quantize_weight(w2, torch.from_numpy(ws).to(dev), gfw, rb)
+    if L.kind == "linear":
+        prep = fpq.fpq_prepare_weight(codes, gfw, fpq.LINEAR, L.N, L.K)
+    else:
+        prep = fpq.fpq_prepare_weight(codes, gfw, fpq.CONV2D, L.N, L.C, L.R, L.S)
+    return codes, prep
+
+
+def gpu_layer(L, ws, xs, use_bias=True):
+    gfw, _ = FMT[L.wfmt]
+    dev = "cuda"
+    _, prep = gpu_prepare(L, ws)
+    x = torch.from_numpy(L.x).to(dev)
+    bias = torch.from_numpy(L.bias).to(dev) if use_bias else None
+    wsd = torch.from_numpy(ws).to(dev)
+    if L.kind == "linear":
+        y = fpq.fpq_linear(x, prep, wsd, xs, fpq.E4M3, gfw, bias, L.N)
+    else:
+        y = fpq.fpq_conv2d(x, prep, wsd, xs, fpq.E4M3, gfw, bias, L.N, L.R, L.S, L.pad, L.stride)
+    st = fpq.fpq_read_status()
+    assert st == fpq.OK, fpq.status_string(st)
+    return y.cpu().numpy()
+
+
+def oracle_layer(L, ws, xs, idx=None, use_bias=True):
+    _, ofw = FMT[L.wfmt]
+    rb = O.pack_bits(L.bits) if L.bits is not None else None
+    bias = L.bias if use_bias else None
+    if L.kind == "linear":
+        return O.linear(L.x, L.w, ws, xs, O.E4M3, ofw, bias, rb, idx)
+    return O.conv2d(L.x, L.w, ws, xs, O.E4M3, ofw, bias, rb, L.pad, L.stride, idx)
+
+
+def assert_close(y_gpu, y_ref, absum):
+    """|err| <= 1e-3 * sum_k |a_k b_k| per output element, plus two FP32 ulps of |y|
+    for the final scale-and-bias rounding."""
+    y_gpu = np.asarray(y_gpu, dtype=np.float64).reshape(-1)
+    y_ref = np.asarray(y_ref).reshape(-1)
+    absum = np.asarray(absum).reshape(-1)
+    tol = 1e-3 * absum + 2.0 * np.spacing(np.abs(y_ref).astype(np.float32)).astype(np.float64)
+    err = np.abs(y_gpu - y_ref)
+    worst = int(np.argmax(err - tol))
+    assert np.all(err <= tol), (worst, y_gpu[worst], y_ref[worst], err[worst], tol[worst])
+    return float((err / np.maximum(absum, 1e-30)).max())
+
+
+def sample_indices(total, n, seed, extra=()):
+    rng = np.random.default_rng(seed)
+    idx = rng.integers(0, total, size=n, dtype=np.int64)
+    idx = np.unique(np.concatenate([idx, np.asarray(extra, dtype=np.int64)]))
+    return idx

@@ -1,0 +1,83 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every declared symbol,
+and rejects what the host can detect before touching the GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2408_06995_b200 as fpq
+from paper_2408_06995_b200 import build as fpq_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    fpq_build.build()
+    return fpq.lib()
+
+
+def test_exports_every_declared_symbol(L):
+    header = open(os.path.join(ROOT, "include", "fpq.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(fpq_[a-z0-9_]+)\s*\(", header))
+    assert declared, "no declarations found"
+    assert declared == set(fpq.EXPORTS)
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_format_max_and_scale(L):
+    assert fpq.fpq_format_max(fpq.E4M3) == 448.0
+    assert fpq.fpq_format_max(fpq.Format(4, 3, 7, fpq.SAT_PAPER)) == 480.0
+    assert fpq.fpq_format_max(fpq.E2M1) == 6.0
+    assert fpq.fpq_format_max(fpq.E5M2) == 57344.0
+    assert fpq.fpq_format_max(fpq.Format(5, 2, 15, 0)) == 114688.0
+    assert fpq.fpq_format_max(fpq.E1M2) == 1.75
+    assert fpq.fpq_format_max(fpq.E3M4) == 15.5
+    assert fpq.fpq_format_max(fpq.E2M5) == 3.9375
+    assert fpq.fpq_format_max(fpq.Format(5, 3, 7)) == 0.0          # 9 bits
+    assert fpq.fpq_format_max(fpq.Format(4, 3, 7, 5)) == 0.0        # unknown saturation mode
+    import numpy as np
+    assert fpq.fpq_scale_from_max(3.0, fpq.E4M3) == float(np.float32(3.0) / np.float32(448.0))
+
+
+def test_host_side_rejections(L):
+    F = fpq.E4M3.c()
+    bad = fpq.Format(6, 3, 7).c()
+    one = ctypes.c_void_p(16)   # never dereferenced: rejected first
+    assert L.fpq_quantize_act(one, 16, 1.0, bad, one, None) == fpq.ERR_FORMAT
+    assert L.fpq_quantize_act(one, -1, 1.0, F, one, None) == fpq.ERR_SHAPE
+    assert L.fpq_quantize_act(None, 16, 1.0, F, one, None) == fpq.ERR_NULL
+    assert L.fpq_quantize_act(one, 0, 1.0, F, one, None) == fpq.OK
+    assert L.fpq_quantize_act(ctypes.c_void_p(18), 16, 1.0, F, one, None) == fpq.ERR_ALIGN
+    assert L.fpq_quantize_weight(None, 4, 4, one, F, None, one, None) == fpq.ERR_NULL
+    assert L.fpq_quantize_weight(one, -4, 4, one, F, None, one, None) == fpq.ERR_SHAPE
+    # contraction: operand pairs
+    e2m1, e3m4 = fpq.E2M1.c(), fpq.E3M4.c()
+    big = ctypes.c_void_p(1024)
+    assert L.fpq_linear(big, big, big, 1.0, e3m4, F, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_UNSUPPORTED
+    assert L.fpq_linear(big, big, big, 1.0, F, e3m4, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_UNSUPPORTED
+    paper_sat = fpq.Format(4, 3, 7, fpq.SAT_PAPER).c()
+    assert L.fpq_linear(big, big, big, 1.0, paper_sat, F, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_UNSUPPORTED
+    assert L.fpq_linear(big, big, big, 1.0, F, e2m1, None, big, -1, 8, 8, big, 1 << 20, None) == fpq.ERR_SHAPE
+    assert L.fpq_linear(None, big, big, 1.0, F, F, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_NULL
+    assert L.fpq_linear(ctypes.c_void_p(1028), big, big, 1.0, F, F, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_ALIGN
+    assert L.fpq_linear(big, big, big, 1.0, F, F, None, big, 8, 8, 8, big, 8, None) == fpq.ERR_WORKSPACE
+    assert L.fpq_linear(big, big, big, 1.0, F, F, None, big, 8, 8, 8, None, 0, None) == fpq.ERR_WORKSPACE
+    assert L.fpq_linear(big, big, big, 1.0, F, F, None, big, 0, 8, 8, None, 0, None) == fpq.OK
+    assert L.fpq_conv2d(big, big, big, 1.0, F, F, None, big, 1, 8, 2, 2, 8, 3, 3, 0, 1, big, 1 << 20, None) == fpq.ERR_SHAPE
+    assert L.fpq_conv2d(big, big, big, 1.0, F, F, None, big, 1, 8, 4, 4, 8, 3, 3, 1, 0, big, 1 << 20, None) == fpq.ERR_SHAPE
+    assert L.fpq_conv2d(big, big, big, 1.0, F, F, None, big, 1, 8, 4, 4, 8, 3, 3, 1, 1, big, 16, None) == fpq.ERR_WORKSPACE
+
+
+def test_sizes(L):
+    assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E4M3, fpq.E4M3) == 100 * 320
+    assert fpq.fpq_linear_workspace_size(100, 64, 321, fpq.E4M3, fpq.E2M1) == 100 * 336
+    assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E3M4, fpq.E4M3) == 0
+    assert fpq.fpq_conv2d_workspace_size(2, 4, 8, 8, 16, 3, 3, 1, 1, fpq.E4M3, fpq.E2M1) == 2 * 64 * 16
+    assert fpq.fpq_prepared_size(fpq.E4M3, fpq.LINEAR, 10, 320) == 10 * 384
+    assert fpq.fpq_prepared_size(fpq.E2M1, fpq.CONV2D, 10, 320, 3, 3) == 10 * 9 * 384 // 2
+    assert fpq.fpq_prepared_size(fpq.E2M1, fpq.LINEAR, 10, 320, 3, 3) == 0
+    assert fpq.status_string(fpq.ERR_TIMEOUT) == "device-side wait timed out"

@@ -1,0 +1,171 @@
+"""Parity of the quantized linear / conv layers (CUDA, through the C ABI) with the CPU oracle.
+
+Acceptance per output element: |err| <= 1e-3 * sum_k |a_k b_k| (+ 2 FP32 ulps of |y|
+for the final scale-and-bias rounding); the weight codes must match bit for bit.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2408_06995_b200 as fpq
+from paper_2408_06995_b200 import inputs as I
+from _helpers import FMT, assert_close, gpu_layer, gpu_prepare, layer_scales, oracle_layer, sample_indices
+
+pytestmark = pytest.mark.gpu
+
+
+def _check_full(L, use_bias=True):
+    ws, xs = layer_scales(L)
+    y = gpu_layer(L, ws, xs, use_bias)
+    yr, ab = oracle_layer(L, ws, xs, None, use_bias)
+    assert y.shape == yr.shape
+    return assert_close(y, yr, ab)
+
+
+def _check_sampled(L, nsamp, seed):
+    ws, xs = layer_scales(L)
+    y = gpu_layer(L, ws, xs)
+    total = y.size
+    if L.kind == "linear":
+        edge = [0, L.N - 1, total - L.N, total - 1]
+    else:
+        edge = [0, L.Wo - 1, total - 1, total - L.Ho * L.Wo]
+    idx = sample_indices(total, nsamp, seed, edge)
+    yr, ab = oracle_layer(L, ws, xs, idx)
+    assert np.all(np.isfinite(y))
+    return assert_close(y.reshape(-1)[idx], yr, ab)
+
+
+# ---- linear ------------------------------------------------------------------------------
+
+def test_config1_linear_w8a8_every_element():
+    (L,) = I.config1()
+    _check_full(L)
+
+
+@pytest.mark.parametrize("wfmt", ["e4m3", "e2m1"])
+@pytest.mark.parametrize("M,K,N", [(1, 16, 1), (2, 1280, 320), (127, 128, 64), (128, 128, 128), (129, 129, 129),
+                                   (130, 200, 72), (154, 768, 640), (300, 320, 960), (257, 1000, 4), (64, 48, 260)])
+def test_linear_ragged_shapes(wfmt, M, K, N):
+    L = I.linear_layer("t", M, K, N, wfmt, rounding=(wfmt == "e2m1"))
+    I.draw(L, 7, M + K + N, "normal", 0.02, True, 0.01, (0.001, 20.0))
+    _check_full(L)
+    _check_full(L, use_bias=False)
+
+
+@pytest.mark.parametrize("wfmt", ["e4m3", "e2m1"])
+def test_linear_small_integers_are_exact(wfmt):
+    rng = np.random.default_rng(3)
+    M, K, N = 200, 384, 136
+    ints = np.array([0, 1, 2, -1, -2, 4, -4], dtype=np.float32)
+    L = I.linear_layer("ints", M, K, N, wfmt)
+    L.x = ints[rng.integers(0, 7, (M, K))]
+    L.w = ints[rng.integers(0, 7, (N, K))]
+    L.bias = np.zeros(N, np.float32)
+    ws = np.ones(N, np.float32)
+    y = gpu_layer(L, ws, 1.0)
+    assert np.array_equal(y.astype(np.float64), L.x.astype(np.float64) @ L.w.astype(np.float64).T)
+
+
+def test_weight_codes_and_prepared_copy_are_bit_exact():
+    for wfmt, C, R in (("e4m3", 20, 3), ("e2m1", 20, 3), ("e2m1", 130, 1), ("e4m3", 7, 3), ("e2m1", 7, 3)):
+        L = I.conv_layer("w", 1, C, 8, 8, 10, R, wfmt=wfmt, rounding=True)
+        I.draw(L, 8, C + R, "normal", 0.05, True)
+        ws, xs = layer_scales(L)
+        gfw, ofw = FMT[wfmt]
+        codes, prep = gpu_prepare(L, ws)
+        want = O.quantize_weight(L.w.reshape(L.N, -1), ws, ofw, O.pack_bits(L.bits))
+        assert np.array_equal(codes.cpu().numpy(), want)
+        # prepared copy: [N][R*S][C_pad], taps outermost, zero padded
+        K = C * R * R
+        flat = want if ofw.bits == 8 else np.stack([want & 15, want >> 4], -1).reshape(L.N, -1)[:, :K]
+        Cp = (C + 127) // 128 * 128
+        exp = np.zeros((L.N, R * R, Cp), np.uint8)
+        exp[:, :, :C] = flat.reshape(L.N, C, R * R).transpose(0, 2, 1)
+        if ofw.bits == 4:
+            e2 = exp.reshape(L.N, -1)
+            exp = (e2[:, 0::2] | (e2[:, 1::2] << 4)).astype(np.uint8)
+        assert np.array_equal(prep.cpu().numpy().reshape(L.N, -1), exp.reshape(L.N, -1))
+
+
+# ---- conv ---------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("wfmt", ["e4m3", "e2m1"])
+@pytest.mark.parametrize("B,C,H,W,Co,R,pad,stride", [
+    (1, 16, 8, 8, 16, 3, 1, 1),
+    (2, 4, 16, 16, 8, 3, 1, 1),        # fewer channels than one 16-byte row
+    (3, 20, 9, 7, 5, 3, 1, 1),         # odd extents, ragged everything
+    (2, 32, 16, 16, 24, 3, 1, 2),      # stride 2
+    (1, 8, 11, 13, 6, 3, 1, 2),
+    (2, 130, 8, 8, 140, 1, 0, 1),      # 1x1, channels just past a chunk
+    (1, 64, 32, 32, 64, 3, 1, 1),
+    (2, 16, 64, 64, 4, 3, 1, 1),       # conv_out-like
+    (1, 8, 5, 5, 8, 3, 0, 1),          # no padding
+    (5, 12, 4, 4, 260, 3, 1, 1),       # several images per tile, three N tiles
+])
+def test_conv_ragged_shapes(wfmt, B, C, H, W, Co, R, pad, stride):
+    L = I.conv_layer("t", B, C, H, W, Co, R, pad=pad, stride=stride, wfmt=wfmt, rounding=True)
+    I.draw(L, 9, B + C + H + Co, "silu", 0.03, True)
+    _check_full(L)
+
+
+def test_conv_1x1_matches_linear_on_the_gpu():
+    L = I.conv_layer("c", 2, 96, 8, 8, 80, 1, wfmt="e4m3")
+    I.draw(L, 10, 0, "normal", 0.02, True)
+    ws, xs = layer_scales(L)
+    yc = gpu_layer(L, ws, xs)
+    Ll = I.linear_layer("l", 2 * 64, 96, 80, "e4m3")
+    Ll.x = np.ascontiguousarray(L.x.transpose(0, 2, 3, 1).reshape(-1, 96))
+    Ll.w = L.w.reshape(80, 96)
+    Ll.bias = L.bias
+    yl = gpu_layer(Ll, ws, xs)
+    assert np.array_equal(yc.transpose(0, 2, 3, 1).reshape(-1, 80), yl)
+
+
+def test_conv_one_hot_tap_is_a_shift():
+    B, C, H, W = 2, 16, 8, 8
+    L = I.conv_layer("s", B, C, H, W, 1, 3, wfmt="e4m3")
+    I.draw(L, 11, 0, "normal", 0.02)
+    L.bias[:] = 0
+    xs = O.scale_from_max(np.abs(L.x).max(), O.E4M3)
+    xq = O.decode_table(O.E4M3)[O.quantize_act(L.x, xs, O.E4M3)] * np.float64(xs)
+    for r, s in [(0, 0), (1, 2), (2, 1), (1, 1)]:
+        L.w[:] = 0
+        L.w[0, 5, r, s] = 1.0
+        y = gpu_layer(L, np.ones(1, np.float32), float(xs))
+        want = np.zeros((B, H, W))
+        ys, xsl = slice(max(0, 1 - r), min(H, H + 1 - r)), slice(max(0, 1 - s), min(W, W + 1 - s))
+        for oy in range(H):
+            for ox in range(W):
+                iy, ix = oy + r - 1, ox + s - 1
+                if 0 <= iy < H and 0 <= ix < W:
+                    want[:, oy, ox] = xq[:, 5, iy, ix]
+        assert np.allclose(y[:, 0], want, rtol=3e-7, atol=0)
+
+
+def test_config2_conv_w8a8_reduced_batch_every_element():
+    (L,) = I.config2(batch=4)
+    _check_full(L)
+
+
+def test_config3_pair_w4a8_reduced_batch_every_element():
+    for L in I.config3(batch=2):
+        _check_full(L)
+
+
+# ---- full sizes, sampled outputs ---------------------------------------------------------
+
+def test_config2_full_size_sampled():
+    (L,) = I.config2()
+    _check_sampled(L, 1 << 14, 1)
+
+
+def test_config3_full_size_sampled():
+    for j, L in enumerate(I.config3()):
+        _check_sampled(L, 1 << 13, 2 + j)
+
+
+def test_config4_full_size_sampled():
+    for j, L in enumerate(I.config4()):
+        _check_sampled(L, 1 << 12, 10 + j)
