@@ -151,6 +151,32 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
                       size_t ws_bytes, void* stream);
 
 /*
+ * The two stages of fpq_linear / fpq_conv2d as separate calls (the layer call
+ * is exactly stage 1 followed by stage 2 on the same stream):
+ *   stage 1, *_quantize_input: activation quantize (Sec. IV-B rounding equation,
+ *            static per-tensor scale) written to `workspace` in the operand
+ *            layout of the contraction (linear: [M][K rounded up to 16] codes;
+ *            conv: channels-last [B][H][W][C rounded up to 16] codes, zero padded);
+ *   stage 2, *_contract: the low-bit contraction on those codes and the
+ *            dequantize + bias epilogue (Sec. V-B, Y = W A; Sec. VI-A).
+ * Arguments, alignment rules and errors are those of the layer calls.
+ */
+fpq_status fpq_linear_quantize_input(const float* x, float x_scale, fpq_format fx, fpq_format fw,
+                                     int64_t M, int64_t N, int64_t K, void* workspace,
+                                     size_t ws_bytes, void* stream);
+fpq_status fpq_linear_contract(const void* workspace, size_t ws_bytes, const void* w_prepared,
+                               const float* w_scale, float x_scale, fpq_format fx, fpq_format fw,
+                               const float* bias, float* y, int64_t M, int64_t N, int64_t K,
+                               void* stream);
+fpq_status fpq_conv2d_quantize_input(const float* x, float x_scale, fpq_format fx, fpq_format fw,
+                                     int B, int C, int H, int W, int C_out, int R, int S, int pad,
+                                     int stride, void* workspace, size_t ws_bytes, void* stream);
+fpq_status fpq_conv2d_contract(const void* workspace, size_t ws_bytes, const void* w_prepared,
+                               const float* w_scale, float x_scale, fpq_format fx, fpq_format fw,
+                               const float* bias, float* y, int B, int C, int H, int W, int C_out,
+                               int R, int S, int pad, int stride, void* stream);
+
+/*
  * Host-buffer forms of the two layers: x_host / y_host are host pointers
  * (pinned memory for asynchronous copies), x_dev / y_dev are device staging
  * buffers of the same sizes owned by the caller.  The call copies x in, runs the

@@ -65,6 +65,7 @@ EXPORTS = [
     "fpq_scale_from_max", "fpq_format_max", "fpq_quantize_weight", "fpq_quantize_act",
     "fpq_prepared_size", "fpq_prepare_weight", "fpq_linear_workspace_size", "fpq_linear",
     "fpq_conv2d_workspace_size", "fpq_conv2d", "fpq_linear_host", "fpq_conv2d_host",
+    "fpq_linear_quantize_input", "fpq_linear_contract", "fpq_conv2d_quantize_input", "fpq_conv2d_contract",
     "fpq_read_status", "fpq_status_string",
 ]
 
@@ -107,6 +108,14 @@ def lib() -> ctypes.CDLL:
         L.fpq_linear_host.argtypes = [vp, vp, vp, vp, f32, F, F, vp, vp, vp, i64, i64, i64, vp, sz, vp]
         L.fpq_conv2d_host.restype = i32
         L.fpq_conv2d_host.argtypes = [vp, vp, vp, vp, f32, F, F, vp, vp, vp] + [i32] * 9 + [vp, sz, vp]
+        L.fpq_linear_quantize_input.restype = i32
+        L.fpq_linear_quantize_input.argtypes = [vp, f32, F, F, i64, i64, i64, vp, sz, vp]
+        L.fpq_linear_contract.restype = i32
+        L.fpq_linear_contract.argtypes = [vp, sz, vp, vp, f32, F, F, vp, vp, i64, i64, i64, vp]
+        L.fpq_conv2d_quantize_input.restype = i32
+        L.fpq_conv2d_quantize_input.argtypes = [vp, f32, F, F] + [i32] * 9 + [vp, sz, vp]
+        L.fpq_conv2d_contract.restype = i32
+        L.fpq_conv2d_contract.argtypes = [vp, sz, vp, vp, f32, F, F, vp, vp] + [i32] * 9 + [vp]
         L.fpq_read_status.restype = i32
         L.fpq_read_status.argtypes = [vp]
         L.fpq_status_string.restype = ctypes.c_char_p
@@ -219,6 +228,39 @@ def fpq_conv2d(x, w_prepared, w_scale, x_scale, fx: Format, fw: Format, bias, C_
     _check(lib().fpq_conv2d(_ptr(x), _ptr(w_prepared), _ptr(w_scale), float(x_scale), fx.c(), fw.c(), _ptr(bias),
                             _ptr(y), B, C, H, W, C_out, R, S, pad, stride, _ptr(workspace), workspace.numel(),
                             _stream()), "fpq_conv2d")
+    return y
+
+
+def fpq_linear_quantize_input(x, x_scale, fx: Format, fw: Format, N: int, workspace):
+    M, K = x.shape
+    _check(lib().fpq_linear_quantize_input(_ptr(x), float(x_scale), fx.c(), fw.c(), M, N, K, _ptr(workspace),
+                                           workspace.numel(), _stream()), "fpq_linear_quantize_input")
+    return workspace
+
+
+def fpq_linear_contract(workspace, w_prepared, w_scale, x_scale, fx: Format, fw: Format, bias, y, K: int):
+    M, N = y.shape
+    _check(lib().fpq_linear_contract(_ptr(workspace), workspace.numel(), _ptr(w_prepared), _ptr(w_scale),
+                                     float(x_scale), fx.c(), fw.c(), _ptr(bias), _ptr(y), M, N, K, _stream()),
+           "fpq_linear_contract")
+    return y
+
+
+def fpq_conv2d_quantize_input(x, x_scale, fx: Format, fw: Format, C_out, R, S, pad, stride, workspace):
+    B, C, H, W = x.shape
+    _check(lib().fpq_conv2d_quantize_input(_ptr(x), float(x_scale), fx.c(), fw.c(), B, C, H, W, C_out, R, S, pad,
+                                           stride, _ptr(workspace), workspace.numel(), _stream()),
+           "fpq_conv2d_quantize_input")
+    return workspace
+
+
+def fpq_conv2d_contract(workspace, w_prepared, w_scale, x_scale, fx: Format, fw: Format, bias, y, in_shape, R, S,
+                        pad, stride):
+    B, C, H, W = in_shape
+    C_out = y.shape[1]
+    _check(lib().fpq_conv2d_contract(_ptr(workspace), workspace.numel(), _ptr(w_prepared), _ptr(w_scale),
+                                     float(x_scale), fx.c(), fw.c(), _ptr(bias), _ptr(y), B, C, H, W, C_out, R, S,
+                                     pad, stride, _stream()), "fpq_conv2d_contract")
     return y
 
 

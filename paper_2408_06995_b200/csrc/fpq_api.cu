@@ -199,33 +199,58 @@ size_t fpq_linear_workspace_size(int64_t M, int64_t N, int64_t K, fpq_format fx,
     return (size_t)(M * round_up(K, 16));
 }
 
-fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_scale, float x_scale, fpq_format fx,
-                      fpq_format fw, const float* bias, float* y, int64_t M, int64_t N, int64_t K, void* workspace,
-                      size_t ws_bytes, void* stream)
+static fpq_status linear_checks(fpq_format fx, fpq_format fw, int64_t M, int64_t N, int64_t K, const void* workspace,
+                                size_t ws_bytes, bool* empty)
 {
     fpq_status s = check_pair(fx, fw);
     if (s != FPQ_OK)
         return s;
     if (M < 0 || N < 0 || K < 0 || M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff)
         return FPQ_ERR_SHAPE;
-    if (M == 0 || N == 0)
+    *empty = (M == 0 || N == 0);
+    if (*empty)
         return FPQ_OK;
     if (K == 0)
         return FPQ_ERR_SHAPE;
-    if (!x || !w_prepared || !w_scale || !y)
-        return FPQ_ERR_NULL;
-    if (!aligned(x, 16) || !aligned(y, 16) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
-        (bias && !aligned(bias, 4)))
-        return FPQ_ERR_ALIGN;
-    const int64_t Kp = round_up(K, 16);
-    if (!workspace || ws_bytes < (size_t)(M * Kp))
+    if (!workspace || ws_bytes < (size_t)(M * round_up(K, 16)))
         return FPQ_ERR_WORKSPACE;
     if (!aligned(workspace, 128))
         return FPQ_ERR_ALIGN;
+    return FPQ_OK;
+}
+
+fpq_status fpq_linear_quantize_input(const float* x, float x_scale, fpq_format fx, fpq_format fw, int64_t M, int64_t N,
+                                     int64_t K, void* workspace, size_t ws_bytes, void* stream)
+{
+    bool empty = false;
+    fpq_status s = linear_checks(fx, fw, M, N, K, workspace, ws_bytes, &empty);
+    if (s != FPQ_OK || empty)
+        return s;
+    if (!x)
+        return FPQ_ERR_NULL;
+    if (!aligned(x, 16))
+        return FPQ_ERR_ALIGN;
     if (!status_word())
         return FPQ_ERR_CUDA;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (launch_quantize_rows_e4m3(x, M, K, Kp, x_scale, (uint8_t*)workspace, st) != cudaSuccess)
+    return launch_quantize_rows_e4m3(x, M, K, round_up(K, 16), x_scale, (uint8_t*)workspace, (cudaStream_t)stream) ==
+                   cudaSuccess
+               ? FPQ_OK
+               : FPQ_ERR_CUDA;
+}
+
+fpq_status fpq_linear_contract(const void* workspace, size_t ws_bytes, const void* w_prepared, const float* w_scale,
+                               float x_scale, fpq_format fx, fpq_format fw, const float* bias, float* y, int64_t M,
+                               int64_t N, int64_t K, void* stream)
+{
+    bool empty = false;
+    fpq_status s = linear_checks(fx, fw, M, N, K, workspace, ws_bytes, &empty);
+    if (s != FPQ_OK || empty)
+        return s;
+    if (!w_prepared || !w_scale || !y)
+        return FPQ_ERR_NULL;
+    if (!aligned(y, 16) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) || (bias && !aligned(bias, 4)))
+        return FPQ_ERR_ALIGN;
+    if (!status_word())
         return FPQ_ERR_CUDA;
     GemmProblem p{};
     p.conv = 0;
@@ -233,7 +258,7 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
     p.M = M;
     p.N = (int)N;
     p.Cp = (int)padded_c(K);
-    p.Ca = (int)Kp;
+    p.Ca = (int)round_up(K, 16);
     p.B = p.H = p.W = p.Ho = p.Wo = 1;
     p.R = p.S = 1;
     p.pad = 0;
@@ -244,7 +269,27 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
     p.x_scale = x_scale;
     p.bias = bias;
     p.y = y;
-    return launch_gemm(p, st);
+    return launch_gemm(p, (cudaStream_t)stream);
+}
+
+fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_scale, float x_scale, fpq_format fx,
+                      fpq_format fw, const float* bias, float* y, int64_t M, int64_t N, int64_t K, void* workspace,
+                      size_t ws_bytes, void* stream)
+{
+    bool empty = false;
+    fpq_status s = linear_checks(fx, fw, M, N, K, workspace, ws_bytes, &empty);
+    if (s != FPQ_OK || empty)
+        return s;
+    // reject everything the second stage would reject before the first stage runs
+    if (!x || !w_prepared || !w_scale || !y)
+        return FPQ_ERR_NULL;
+    if (!aligned(x, 16) || !aligned(y, 16) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
+        (bias && !aligned(bias, 4)))
+        return FPQ_ERR_ALIGN;
+    s = fpq_linear_quantize_input(x, x_scale, fx, fw, M, N, K, workspace, ws_bytes, stream);
+    if (s != FPQ_OK)
+        return s;
+    return fpq_linear_contract(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream);
 }
 
 static fpq_status conv_shape(int B, int C, int H, int W, int C_out, int R, int S, int pad, int stride, int* Ho,
@@ -270,35 +315,63 @@ size_t fpq_conv2d_workspace_size(int B, int C, int H, int W, int C_out, int R, i
     return (size_t)B * H * W * (size_t)round_up(C, 16);
 }
 
-fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_scale, float x_scale, fpq_format fx,
-                      fpq_format fw, const float* bias, float* y, int B, int C, int H, int W, int C_out, int R, int S,
-                      int pad, int stride, void* workspace, size_t ws_bytes, void* stream)
+static fpq_status conv_checks(fpq_format fx, fpq_format fw, int B, int C, int H, int W, int C_out, int R, int S,
+                              int pad, int stride, const void* workspace, size_t ws_bytes, int* Ho, int* Wo,
+                              bool* empty)
 {
     fpq_status s = check_pair(fx, fw);
     if (s != FPQ_OK)
         return s;
-    int Ho, Wo;
-    s = conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo);
+    s = conv_shape(B, C, H, W, C_out, R, S, pad, stride, Ho, Wo);
     if (s != FPQ_OK)
         return s;
-    if (B == 0 || C_out == 0)
+    *empty = (B == 0 || C_out == 0);
+    if (*empty)
         return FPQ_OK;
     if (B > 65535)
         return FPQ_ERR_SHAPE;
-    if (!x || !w_prepared || !w_scale || !y)
-        return FPQ_ERR_NULL;
-    if (!aligned(x, 4) || !aligned(y, 4) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
-        (bias && !aligned(bias, 4)))
-        return FPQ_ERR_ALIGN;
-    const int Ca = (int)round_up(C, 16);
-    if (!workspace || ws_bytes < (size_t)B * H * W * (size_t)Ca)
+    if (!workspace || ws_bytes < (size_t)B * H * W * (size_t)round_up(C, 16))
         return FPQ_ERR_WORKSPACE;
     if (!aligned(workspace, 128))
         return FPQ_ERR_ALIGN;
+    return FPQ_OK;
+}
+
+fpq_status fpq_conv2d_quantize_input(const float* x, float x_scale, fpq_format fx, fpq_format fw, int B, int C, int H,
+                                     int W, int C_out, int R, int S, int pad, int stride, void* workspace,
+                                     size_t ws_bytes, void* stream)
+{
+    int Ho, Wo;
+    bool empty = false;
+    fpq_status s = conv_checks(fx, fw, B, C, H, W, C_out, R, S, pad, stride, workspace, ws_bytes, &Ho, &Wo, &empty);
+    if (s != FPQ_OK || empty)
+        return s;
+    if (!x)
+        return FPQ_ERR_NULL;
+    if (!aligned(x, 4))
+        return FPQ_ERR_ALIGN;
     if (!status_word())
         return FPQ_ERR_CUDA;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H * W, Ca, x_scale, (uint8_t*)workspace, st) != cudaSuccess)
+    return launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H * W, (int)round_up(C, 16), x_scale, (uint8_t*)workspace,
+                                             (cudaStream_t)stream) == cudaSuccess
+               ? FPQ_OK
+               : FPQ_ERR_CUDA;
+}
+
+fpq_status fpq_conv2d_contract(const void* workspace, size_t ws_bytes, const void* w_prepared, const float* w_scale,
+                               float x_scale, fpq_format fx, fpq_format fw, const float* bias, float* y, int B, int C,
+                               int H, int W, int C_out, int R, int S, int pad, int stride, void* stream)
+{
+    int Ho, Wo;
+    bool empty = false;
+    fpq_status s = conv_checks(fx, fw, B, C, H, W, C_out, R, S, pad, stride, workspace, ws_bytes, &Ho, &Wo, &empty);
+    if (s != FPQ_OK || empty)
+        return s;
+    if (!w_prepared || !w_scale || !y)
+        return FPQ_ERR_NULL;
+    if (!aligned(y, 4) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) || (bias && !aligned(bias, 4)))
+        return FPQ_ERR_ALIGN;
+    if (!status_word())
         return FPQ_ERR_CUDA;
     GemmProblem p{};
     p.conv = 1;
@@ -306,7 +379,7 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
     p.M = (int64_t)B * Ho * Wo;
     p.N = C_out;
     p.Cp = (int)padded_c(C);
-    p.Ca = Ca;
+    p.Ca = (int)round_up(C, 16);
     p.B = B;
     p.H = H;
     p.W = W;
@@ -322,7 +395,29 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
     p.x_scale = x_scale;
     p.bias = bias;
     p.y = y;
-    return launch_gemm(p, st);
+    return launch_gemm(p, (cudaStream_t)stream);
+}
+
+fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_scale, float x_scale, fpq_format fx,
+                      fpq_format fw, const float* bias, float* y, int B, int C, int H, int W, int C_out, int R, int S,
+                      int pad, int stride, void* workspace, size_t ws_bytes, void* stream)
+{
+    int Ho, Wo;
+    bool empty = false;
+    fpq_status s = conv_checks(fx, fw, B, C, H, W, C_out, R, S, pad, stride, workspace, ws_bytes, &Ho, &Wo, &empty);
+    if (s != FPQ_OK || empty)
+        return s;
+    if (!x || !w_prepared || !w_scale || !y)
+        return FPQ_ERR_NULL;
+    if (!aligned(x, 4) || !aligned(y, 4) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
+        (bias && !aligned(bias, 4)))
+        return FPQ_ERR_ALIGN;
+    s = fpq_conv2d_quantize_input(x, x_scale, fx, fw, B, C, H, W, C_out, R, S, pad, stride, workspace, ws_bytes,
+                                  stream);
+    if (s != FPQ_OK)
+        return s;
+    return fpq_conv2d_contract(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out, R,
+                               S, pad, stride, stream);
 }
 
 fpq_status fpq_linear_host(const float* x_host, float* x_dev, const void* w_prepared, const float* w_scale,
