@@ -1,0 +1,385 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized layer: prints ONE JSON line.
+
+Own arm (default): the DDIM-CIFAR-style 3x3 convolution, W8A8 (E4M3 weights with
+rounding decisions, E4M3 activations), input FP32 NCHW [64,128,32,32] -> 128
+channels, through the C-ABI library on the GPU.  A step is one fpq_conv2d call
+(activation quantize + contraction + dequantize/bias); weights are encoded once
+before the timed region (the encode's own time is reported separately).  Between
+timed steps a 256 MiB buffer is written so that every step starts with a cold
+L2.  With N > 1 (torchrun) every rank runs its own copy of the layer on its own
+batch: weak scaling, no collective on the data path.
+
+Reference arm (--impl reference): the CPU oracle, as it stands, on a bounded
+sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "W8A8 and W4A8 quantized-layer TFLOP/s on 1 B200 and % of dense FP8/FP4 peak"
+WORKLOAD = "ddim_cifar_conv3x3_w8a8: x fp32 NCHW [64,128,32,32] SiLU(N(0,1)), w [128,128,3,3] e4m3 + rounding bits, pad 1"
+NOMINAL_FP8_TFLOPS = 4500.0
+NOMINAL_FP4_TFLOPS = 9000.0
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle
+# ---------------------------------------------------------------------------------------------
+def oracle_sample_run(batch: int):
+    """One pass of the oracle layer (quantize weights and activations, FP64 conv) on the
+    first `batch` images of the workload.  Returns (seconds, flops, threads)."""
+    import numpy as np
+    import oracle as O
+    from paper_2408_06995_b200 import inputs as I
+
+    (L,) = I.config2(batch=batch)
+    w2 = L.w.reshape(L.N, -1)
+    ws = np.array([O.scale_from_max(v, O.E4M3) for v in np.abs(w2).max(axis=1)], dtype=np.float32)
+    xs = O.scale_from_max(float(np.abs(L.x).max()), O.E4M3)
+    rb = O.pack_bits(L.bits)
+    O.lib()
+    t0 = time.perf_counter()
+    O.conv2d(L.x, L.w, ws, xs, O.E4M3, O.E4M3, L.bias, rb, L.pad, L.stride)
+    dt = time.perf_counter() - t0
+    return dt, L.flops, os.cpu_count()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    batch = 4
+    for _ in range(args.warmup):
+        oracle_sample_run(batch)
+    total, flops = 0.0, 0
+    for _ in range(args.steps):
+        dt, fl, cores = oracle_sample_run(batch)
+        total += dt
+        flops += fl
+    value = flops / total / 1e12
+    sample = f"first {batch} of 64 images of the workload per step, whole oracle layer"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+# clock sampling during the timed region (NVML, read-only)
+# ---------------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+# ---------------------------------------------------------------------------------------------
+# own arm
+# ---------------------------------------------------------------------------------------------
+class ConvLayerOnGpu:
+    """Device-resident tensors of one conv layer, weights already encoded."""
+
+    def __init__(self, L, fpq, torch, dev):
+        import numpy as np
+        self.L, self.fpq, self.torch = L, fpq, torch
+        self.fw = fpq.E4M3 if L.wfmt == "e4m3" else fpq.E2M1
+        w2 = np.abs(L.w.reshape(L.N, -1)).max(axis=1)
+        self.ws = torch.tensor([fpq.fpq_scale_from_max(float(v), self.fw) for v in w2], dtype=torch.float32, device=dev)
+        self.xs = fpq.fpq_scale_from_max(float(np.abs(L.x).max()), fpq.E4M3)
+        self.w = torch.from_numpy(L.w.reshape(L.N, -1)).to(dev)
+        self.rb = None
+        if L.bits is not None:
+            self.rb = torch.from_numpy(np.packbits(L.bits, axis=1, bitorder="little")).to(dev)
+        self.x = torch.from_numpy(L.x).to(dev)
+        self.bias = torch.from_numpy(L.bias).to(dev)
+        self.y = torch.empty((L.B, L.N, L.Ho, L.Wo), dtype=torch.float32, device=dev)
+        self.ws_bytes = fpq.fpq_conv2d_workspace_size(L.B, L.C, L.H, L.W, L.N, L.R, L.S, L.pad, L.stride, fpq.E4M3, self.fw)
+        self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
+        self.encode()
+
+    def encode(self):
+        f, L = self.fpq, self.L
+        self.codes = f.fpq_quantize_weight(self.w, self.ws, self.fw, self.rb)
+        self.prep = f.fpq_prepare_weight(self.codes, self.fw, f.CONV2D, L.N, L.C, L.R, L.S)
+
+    def step(self):
+        f, L = self.fpq, self.L
+        f.fpq_conv2d(self.x, self.prep, self.ws, self.xs, f.E4M3, self.fw, self.bias, L.N, L.R, L.S, L.pad, L.stride,
+                     y=self.y, workspace=self.workspace)
+
+    def stage1(self):
+        f, L = self.fpq, self.L
+        f.fpq_conv2d_quantize_input(self.x, self.xs, f.E4M3, self.fw, L.N, L.R, L.S, L.pad, L.stride, self.workspace)
+
+    def stage2(self):
+        f, L = self.fpq, self.L
+        f.fpq_conv2d_contract(self.workspace, self.prep, self.ws, self.xs, f.E4M3, self.fw, self.bias, self.y,
+                              (L.B, L.C, L.H, L.W), L.R, L.S, L.pad, L.stride)
+
+    # algorithmic bytes (FP32 activations in, FP32 out, encoded weights, scales + bias)
+    def layer_bytes(self):
+        L = self.L
+        wbytes = L.N * L.K * (1 if L.wfmt == "e4m3" else 0.5)
+        return 4 * L.x.size + wbytes + 4 * L.M * L.N + 8 * L.N
+
+    def stage1_bytes(self):
+        L = self.L
+        return 4 * L.x.size + L.B * L.H * L.W * ((L.C + 15) // 16 * 16)
+
+    def stage2_bytes(self):
+        L = self.L
+        wbytes = L.N * L.K * (1 if L.wfmt == "e4m3" else 0.5)
+        return L.B * L.H * L.W * ((L.C + 15) // 16 * 16) + wbytes + 4 * L.M * L.N + 8 * L.N
+
+
+def timed_steps(torch, fn, flush, n, pre=None):
+    """n calls of fn, each after an L2 flush (and an untimed `pre`), each bracketed by CUDA events
+    on the current stream.  Returns the list of per-call milliseconds."""
+    evs = []
+    for _ in range(n):
+        flush.zero_()
+        if pre is not None:
+            pre()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in evs]
+
+
+def run_own(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the quantized layer has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2408_06995_b200 import build as fpq_build
+    fpq_build.build()
+    import paper_2408_06995_b200 as fpq
+    from paper_2408_06995_b200 import inputs as I
+
+    peaks = load_peaks()
+    (L,) = I.config2()
+    if world > 1:                       # every rank its own batch of the same law
+        L = I.draw(L, 2, 100 * rank, "silu", 0.03, True)
+    layer = ConvLayerOnGpu(L, fpq, torch, dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region: K steps, device time per step, max over ranks
+    timed_steps(torch, layer.step, flush, args.warmup)
+    sampler = ClockSampler(physical_gpu_index(local))
+    barrier()
+    sampler.start()
+    ms = timed_steps(torch, layer.step, flush, args.steps)
+    barrier()
+    clocks = sampler.stop()
+    st = fpq.fpq_read_status()
+    if st != fpq.OK:
+        raise SystemExit(f"device status after the timed region: {fpq.status_string(st)}")
+    total_ms = sum(ms)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    flops_step = L.flops
+    value = world * flops_step * args.steps / (total_ms * 1e-3) / 1e12
+    launches_per_step = 2
+
+    # ---- per-kernel durations in place (stage 2 right after stage 1, as in the layer call)
+    k = max(10, min(args.steps, 100))
+    ms_q = timed_steps(torch, layer.stage1, flush, k)
+    ms_c = timed_steps(torch, layer.stage2, flush, k, pre=layer.stage1)
+    t_q, t_c = statistics.mean(ms_q) * 1e-3, statistics.mean(ms_c) * 1e-3
+    if t_c >= t_q:
+        dom, t_dom, b_dom = "fpq_gemm_kernel (contraction + epilogue)", t_c, layer.stage2_bytes()
+    else:
+        dom, t_dom, b_dom = "quantize_nchw_to_nhwc_e4m3_kernel (activation quantize)", t_q, layer.stage1_bytes()
+    achieved = b_dom / t_dom / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
+                "algorithmic_bytes_per_launch": b_dom, "us_per_launch": t_dom * 1e6,
+                "kernels_us": {"activation_quantize": t_q * 1e6, "contraction": t_c * 1e6}}
+    t_layer = statistics.mean(ms) * 1e-3
+    layer_roof = {"algorithmic_bytes": layer.layer_bytes(), "achieved_gbs": layer.layer_bytes() / t_layer / 1e9,
+                  "frac_of_hbm_peak": layer.layer_bytes() / t_layer / 1e9 / peaks["hbm_gbs"],
+                  "t_hbm_us": layer.layer_bytes() / (peaks["hbm_gbs"] * 1e9) * 1e6,
+                  "t_tensor_us_nominal_fp8": flops_step / (NOMINAL_FP8_TFLOPS * 1e12) * 1e6}
+
+    # ---- weight encode (offline step), reported beside the metric
+    ms_enc = timed_steps(torch, layer.encode, flush, 10)
+
+    # ---- end to end through the host-buffer C-ABI call
+    xh = torch.from_numpy(L.x).pin_memory()
+    yh = torch.empty(layer.y.shape, dtype=torch.float32).pin_memory()
+    n_e2e = max(3, min(args.steps, 20))
+
+    def e2e_call():
+        fpq.fpq_conv2d_host(xh, layer.x, layer.prep, layer.ws, layer.xs, fpq.E4M3, layer.fw, layer.bias, layer.y, yh,
+                            L.R, L.S, L.pad, L.stride, layer.workspace)
+
+    for _ in range(3):
+        e2e_call()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(n_e2e):
+        e2e_call()
+    t_e2e = time.perf_counter() - t0
+    barrier()
+    if world > 1:
+        t = torch.tensor([t_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        t_e2e = float(t.item())
+    e2e = {"value": world * flops_step * n_e2e / t_e2e / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": xh.numel() * 4,
+           "d2h_bytes_per_step": yh.numel() * 4, "steps": n_e2e, "ms_per_step": 1e3 * t_e2e / n_e2e}
+
+    # ---- W4A8 (the LDM-4-style pair), same protocol, reported beside the headline
+    w4 = None
+    if rank == 0 and not args.skip_w4:
+        w4 = {}
+        for L4 in I.config3():
+            l4 = ConvLayerOnGpu(L4, fpq, torch, dev)
+            timed_steps(torch, l4.step, flush, 3)
+            m4 = timed_steps(torch, l4.step, flush, max(10, min(args.steps, 50)))
+            t4 = statistics.mean(m4) * 1e-3
+            w4[L4.name] = {"tflops": L4.flops / t4 / 1e12, "us": t4 * 1e6,
+                           "pct_dense_fp8_nominal": 100 * L4.flops / t4 / 1e12 / NOMINAL_FP8_TFLOPS,
+                           "pct_dense_fp4_nominal": 100 * L4.flops / t4 / 1e12 / NOMINAL_FP4_TFLOPS,
+                           "layer_frac_of_hbm_peak": l4.layer_bytes() / t4 / 1e9 / peaks["hbm_gbs"]}
+            del l4
+
+    # ---- CPU baseline: the oracle, as it stands, on the host cores (rank 0, N = 1 only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.skip_cpu:
+        dt, fl, cores = oracle_sample_run(64)
+        dt2, fl2, _ = oracle_sample_run(64)
+        cpu = {"value": (fl + fl2) / (dt + dt2) / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+               "sample": "the whole workload layer (64 images), two passes", "seconds": dt + dt2}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "e4m3 x e4m3 -> f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "l2": "flushed between steps (256 MiB write)",
+                       "path": "two kernels: activation quantize to channels-last codes, then TMA/tcgen05 implicit GEMM"},
+            "pct_dense_fp8_peak_nominal": 100 * value / world / NOMINAL_FP8_TFLOPS,
+            "pct_dense_fp8_peak_2x_measured_bf16": 100 * value / world / (2 * peaks["bf16_tflops"]),
+            "roofline": roofline, "layer_roofline": layer_roof, "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+            "weight_encode_us": statistics.mean(ms_enc) * 1e3, "w4a8": w4,
+            "step_us": {"median": statistics.median(ms) * 1e3, "min": min(ms) * 1e3},
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="own", choices=["own", "reference"])
+    ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline leg")
+    ap.add_argument("--skip-w4", action="store_true", help="leave out the W4A8 side measurement")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_own(args)
+
+
+if __name__ == "__main__":
+    main()
