@@ -50,7 +50,8 @@ enum {
     FPQ_ERR_WORKSPACE = -6,   /* workspace missing or too small */
     FPQ_ERR_CUDA = -7,        /* a CUDA runtime / driver call failed */
     FPQ_ERR_TIMEOUT = -8,     /* a bounded device-side wait expired (device status) */
-    FPQ_ERR_NAN_INPUT = -9    /* a NaN was quantized (to code 0) (device status) */
+    FPQ_ERR_NAN_INPUT = -9,   /* a NaN was quantized (to code 0) (device status) */
+    FPQ_ERR_TOO_LARGE = -10   /* problem exceeds a fixed built-in capacity */
 };
 
 enum { FPQ_SAT_PAPER = 0, FPQ_SAT_NATIVE = 1 };
@@ -191,6 +192,39 @@ fpq_status fpq_conv2d_host(const float* x_host, float* x_dev, const void* w_prep
                            const float* bias, float* y_dev, float* y_host, int B, int C, int H,
                            int W, int C_out, int R, int S, int pad, int stride, void* workspace,
                            size_t ws_bytes, void* stream);
+
+/*
+ * fpq_linear without a workspace argument.  (The paper has no counterpart: this
+ * entry point exists for integration reasons only.)
+ *
+ * Who it is for: code that runs where device memory cannot be requested - a
+ * plug-in called on someone else's stream that must not trigger the implicit
+ * device-wide synchronisation of cudaMalloc / cudaFree, a latency-critical
+ * serving loop whose memory was handed out once at start-up, or a host that
+ * gives the library no allocator at all.  Such a caller still owns x, y and the
+ * weights, but has nowhere to put the intermediate activation codes that
+ * fpq_linear writes to its `workspace`.
+ *
+ * Here those codes go to a fixed array inside the library image, of
+ * FPQ_STATIC_SCRATCH_BYTES bytes, which every GPU that loads the library keeps
+ * resident until the process ends.  The call makes no cudaMalloc, cudaFree or
+ * other allocating call.  Results are identical to fpq_linear's.
+ *
+ *   - Limit: M * (K rounded up to 16) <= FPQ_STATIC_SCRATCH_BYTES, otherwise
+ *     FPQ_ERR_TOO_LARGE and nothing is launched.  All other arguments, alignment
+ *     rules and errors are fpq_linear's.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the last call
+ *     left in it; each call overwrites every byte it later reads, so stale
+ *     contents are harmless, but two calls that overlap on the GPU (different
+ *     streams, or host threads launching concurrently) race on it.  Serialise
+ *     them on one stream.
+ */
+#define FPQ_STATIC_SCRATCH_BYTES (8u << 20)
+fpq_status fpq_linear_static(const float* x, const void* w_prepared, const float* w_scale,
+                             float x_scale, fpq_format fx, fpq_format fw, const float* bias,
+                             float* y, int64_t M, int64_t N, int64_t K, void* stream);
 
 /* Waits for `stream`, then returns and clears the sticky device status word:
  * FPQ_OK, FPQ_ERR_TIMEOUT, FPQ_ERR_NAN_INPUT, or FPQ_ERR_CUDA. */

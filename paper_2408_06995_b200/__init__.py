@@ -18,7 +18,8 @@ _SO = os.path.join(_HERE, "libfpq.so")
 
 OK = 0
 ERR_NULL, ERR_FORMAT, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED = -1, -2, -3, -4, -5
-ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NAN_INPUT = -6, -7, -8, -9
+ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NAN_INPUT, ERR_TOO_LARGE = -6, -7, -8, -9, -10
+STATIC_SCRATCH_BYTES = 8 << 20
 SAT_PAPER, SAT_NATIVE = 0, 1
 LINEAR, CONV2D = 0, 1
 
@@ -66,7 +67,7 @@ EXPORTS = [
     "fpq_prepared_size", "fpq_prepare_weight", "fpq_linear_workspace_size", "fpq_linear",
     "fpq_conv2d_workspace_size", "fpq_conv2d", "fpq_linear_host", "fpq_conv2d_host",
     "fpq_linear_quantize_input", "fpq_linear_contract", "fpq_conv2d_quantize_input", "fpq_conv2d_contract",
-    "fpq_read_status", "fpq_status_string",
+    "fpq_linear_static", "fpq_read_status", "fpq_status_string",
 ]
 
 _lib = None
@@ -116,6 +117,8 @@ def lib() -> ctypes.CDLL:
         L.fpq_conv2d_quantize_input.argtypes = [vp, f32, F, F] + [i32] * 9 + [vp, sz, vp]
         L.fpq_conv2d_contract.restype = i32
         L.fpq_conv2d_contract.argtypes = [vp, sz, vp, vp, f32, F, F, vp, vp] + [i32] * 9 + [vp]
+        L.fpq_linear_static.restype = i32
+        L.fpq_linear_static.argtypes = [vp, vp, vp, f32, F, F, vp, vp, i64, i64, i64, vp]
         L.fpq_read_status.restype = i32
         L.fpq_read_status.argtypes = [vp]
         L.fpq_status_string.restype = ctypes.c_char_p
@@ -261,6 +264,17 @@ def fpq_conv2d_contract(workspace, w_prepared, w_scale, x_scale, fx: Format, fw:
     _check(lib().fpq_conv2d_contract(_ptr(workspace), workspace.numel(), _ptr(w_prepared), _ptr(w_scale),
                                      float(x_scale), fx.c(), fw.c(), _ptr(bias), _ptr(y), B, C, H, W, C_out, R, S,
                                      pad, stride, _stream()), "fpq_conv2d_contract")
+    return y
+
+
+def fpq_linear_static(x, w_prepared, w_scale, x_scale, fx: Format, fw: Format, bias, y):
+    """fpq_linear for callers that cannot supply a workspace: the activation codes go to a
+    fixed STATIC_SCRATCH_BYTES array inside the library.  `y` is passed in, so the call itself
+    creates no tensor and allocates nothing.  Calls must not overlap on the GPU."""
+    M, K = x.shape
+    N = y.shape[1]
+    _check(lib().fpq_linear_static(_ptr(x), _ptr(w_prepared), _ptr(w_scale), float(x_scale), fx.c(), fw.c(),
+                                   _ptr(bias), _ptr(y), M, N, K, _stream()), "fpq_linear_static")
     return y
 
 

@@ -494,6 +494,7 @@ const char* fpq_status_string(fpq_status s)
     case FPQ_ERR_CUDA: return "CUDA call failed";
     case FPQ_ERR_TIMEOUT: return "device-side wait timed out";
     case FPQ_ERR_NAN_INPUT: return "NaN input quantized to zero";
+    case FPQ_ERR_TOO_LARGE: return "problem larger than the built-in scratch capacity";
     default: return "unknown status";
     }
 }
