@@ -157,7 +157,8 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
  *   stage 1, *_quantize_input: activation quantize (Sec. IV-B rounding equation,
  *            static per-tensor scale) written to `workspace` in the operand
  *            layout of the contraction (linear: [M][K rounded up to 16] codes;
- *            conv: channels-last [B][H][W][C rounded up to 16] codes, zero padded);
+ *            conv: channels-last codes with the zero padding frame materialised,
+ *            [B][H + 2 pad][W + 2 pad][C rounded up to 16]);
  *   stage 2, *_contract: the low-bit contraction on those codes and the
  *            dequantize + bias epilogue (Sec. V-B, Y = W A; Sec. VI-A).
  * Arguments, alignment rules and errors are those of the layer calls.

@@ -312,7 +312,7 @@ size_t fpq_conv2d_workspace_size(int B, int C, int H, int W, int C_out, int R, i
     int Ho, Wo;
     if (check_pair(fx, fw) != FPQ_OK || conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo) != FPQ_OK)
         return 0;
-    return (size_t)B * H * W * (size_t)round_up(C, 16);
+    return (size_t)B * (H + 2 * pad) * (W + 2 * pad) * (size_t)round_up(C, 16);
 }
 
 static fpq_status conv_checks(fpq_format fx, fpq_format fw, int B, int C, int H, int W, int C_out, int R, int S,
@@ -330,7 +330,7 @@ static fpq_status conv_checks(fpq_format fx, fpq_format fw, int B, int C, int H,
         return FPQ_OK;
     if (B > 65535)
         return FPQ_ERR_SHAPE;
-    if (!workspace || ws_bytes < (size_t)B * H * W * (size_t)round_up(C, 16))
+    if (!workspace || ws_bytes < (size_t)B * (H + 2 * pad) * (W + 2 * pad) * (size_t)round_up(C, 16))
         return FPQ_ERR_WORKSPACE;
     if (!aligned(workspace, 128))
         return FPQ_ERR_ALIGN;
@@ -352,7 +352,7 @@ fpq_status fpq_conv2d_quantize_input(const float* x, float x_scale, fpq_format f
         return FPQ_ERR_ALIGN;
     if (!status_word())
         return FPQ_ERR_CUDA;
-    return launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H * W, (int)round_up(C, 16), x_scale, (uint8_t*)workspace,
+    return launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H, W, pad, (int)round_up(C, 16), x_scale, (uint8_t*)workspace,
                                              (cudaStream_t)stream) == cudaSuccess
                ? FPQ_OK
                : FPQ_ERR_CUDA;

@@ -165,45 +165,73 @@ __global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const float* __
 }
 
 // ---------------------------------------------------------------------------------
-// NCHW FP32 -> NHWC codes [B][H*W][Cp] (Cp = C rounded up to 16, pad = 0), the A
-// operand of the implicit-GEMM convolution.  A block transposes a tile of
-// 64 channels x 32 pixels through shared memory: loads are coalesced along
-// pixels, stores along channels.
+// NCHW FP32 -> channels-last codes with a zero frame: [B][H+2p][W+2p][Cp] (Cp = C
+// rounded up to 16, channel padding and frame = code 0), the A operand of the
+// implicit-GEMM convolution.  A block transposes 128 channels x 32 pixels through
+// shared memory: loads are coalesced along pixels (16 in flight per thread), stores
+// are whole 128-byte channel rows.  The blocks also share out the frame pixels.
 // ---------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const float* __restrict__ x, int C, int HW,
-                                                                         int Cp, float rinv,
+__global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const float* __restrict__ x, int C, int H,
+                                                                         int W, int pad, int Cp, float rinv,
                                                                          uint8_t* __restrict__ codes, int* status)
 {
-    __shared__ __align__(16) uint8_t tile[32][64 + 16];
+    __shared__ __align__(16) uint8_t tile[32][128 + 16];
     bool nan = false;
+    const int HW = H * W, Wp = W + 2 * pad, Hp = H + 2 * pad;
     const int b = blockIdx.z;
-    const int c0 = blockIdx.y * 64;
+    const int c0 = blockIdx.y * 128;
     const int p0 = blockIdx.x * 32;
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 pixels x 8 channel groups of 16
     const float* xb = x + (int64_t)b * C * HW;
+    uint8_t* ob = codes + (int64_t)b * Hp * Wp * Cp;
     const int p = p0 + tx;
+    {
+        const int cl = ty * 16;
+        float a[16];
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-        // this thread converts 4 consecutive channels of one pixel
-        int cl = (ty + 8 * j) * 4;
-        float a[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            int c = c0 + cl + q;
+        for (int q = 0; q < 16; ++q) {
+            const int c = c0 + cl + q;
             a[q] = (c < C && p < HW) ? __ldg(xb + (int64_t)c * HW + p) : 0.f;
         }
-        uint32_t v = e4m3x4_from_scaled(__fmul_rn(a[0], rinv), __fmul_rn(a[1], rinv), __fmul_rn(a[2], rinv),
-                                        __fmul_rn(a[3], rinv), nan);
-        *reinterpret_cast<uint32_t*>(&tile[tx][cl]) = v;
+        uint4 v;
+        v.x = e4m3x4_from_scaled(__fmul_rn(a[0], rinv), __fmul_rn(a[1], rinv), __fmul_rn(a[2], rinv), __fmul_rn(a[3], rinv), nan);
+        v.y = e4m3x4_from_scaled(__fmul_rn(a[4], rinv), __fmul_rn(a[5], rinv), __fmul_rn(a[6], rinv), __fmul_rn(a[7], rinv), nan);
+        v.z = e4m3x4_from_scaled(__fmul_rn(a[8], rinv), __fmul_rn(a[9], rinv), __fmul_rn(a[10], rinv), __fmul_rn(a[11], rinv), nan);
+        v.w = e4m3x4_from_scaled(__fmul_rn(a[12], rinv), __fmul_rn(a[13], rinv), __fmul_rn(a[14], rinv), __fmul_rn(a[15], rinv), nan);
+        *reinterpret_cast<uint4*>(&tile[tx][cl]) = v;
     }
     __syncthreads();
-    // 32 pixels x 4 chunks of 16 channels
-    if (threadIdx.x < 128) {
-        int pl = threadIdx.x >> 2, ch = (threadIdx.x & 3) * 16;
-        int pp = p0 + pl, c = c0 + ch;
+    {
+        // 32 pixels x 8 chunks of 16 channels: 8 consecutive threads write one pixel's row
+        const int pl = threadIdx.x >> 3, ch = (threadIdx.x & 7) * 16;
+        const int pp = p0 + pl, c = c0 + ch;
         if (pp < HW && c < Cp) {
-            uint4 v = *reinterpret_cast<const uint4*>(&tile[pl][ch]);
-            *reinterpret_cast<uint4*>(codes + ((int64_t)b * HW + pp) * Cp + c) = v;
+            const int yy = pp / W, xx = pp - yy * W;
+            const uint4 v = *reinterpret_cast<const uint4*>(&tile[pl][ch]);
+            *reinterpret_cast<uint4*>(ob + ((int64_t)(yy + pad) * Wp + (xx + pad)) * Cp + c) = v;
+        }
+    }
+    // frame pixels of this image, shared out over the blocks of the image's pixel axis
+    if (pad > 0) {
+        const int nframe = Hp * Wp - HW;
+        const int chunks = (min(Cp - c0, 128)) / 16;
+        const int total = nframe * chunks;
+        for (int t = blockIdx.x * 256 + threadIdx.x; t < total; t += gridDim.x * 256) {
+            const int j = t / chunks, ch = (t - j * chunks) * 16;
+            int yp, xp;
+            const int top = pad * Wp;
+            if (j < top) {
+                yp = j / Wp; xp = j - yp * Wp;
+            } else if (j < 2 * top) {
+                const int k = j - top;
+                yp = H + pad + k / Wp; xp = k % Wp;
+            } else {
+                const int k = j - 2 * top;             // 2*pad frame pixels per interior row
+                yp = pad + k / (2 * pad);
+                const int e = k % (2 * pad);
+                xp = (e < pad) ? e : W + e;
+            }
+            *reinterpret_cast<uint4*>(ob + ((int64_t)yp * Wp + xp) * Cp + c0 + ch) = make_uint4(0, 0, 0, 0);
         }
     }
     if (nan)
@@ -292,11 +320,11 @@ cudaError_t launch_quantize_rows_e4m3(const float* x, int64_t M, int64_t K, int6
     return cudaGetLastError();
 }
 
-cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int HW, int Cp, float scale,
+cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int H, int W, int pad, int Cp, float scale,
                                               uint8_t* codes, cudaStream_t st)
 {
-    dim3 grid((HW + 31) / 32, (Cp + 63) / 64, B);
-    quantize_nchw_to_nhwc_e4m3_kernel<<<grid, 256, 0, st>>>(x, C, HW, Cp, 1.0f / scale, codes, status_word());
+    dim3 grid((H * W + 31) / 32, (Cp + 127) / 128, B);
+    quantize_nchw_to_nhwc_e4m3_kernel<<<grid, 256, 0, st>>>(x, C, H, W, pad, Cp, 1.0f / scale, codes, status_word());
     return cudaGetLastError();
 }
 
