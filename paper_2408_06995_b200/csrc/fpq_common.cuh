@@ -82,13 +82,18 @@ __device__ __forceinline__ uint32_t e4m3x4_from_scaled(float t0, float t1, float
     uint16_t lo, hi;
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(t1), "f"(t0));
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(t3), "f"(t2));
-    uint32_t v = (uint32_t)lo | ((uint32_t)hi << 16);
-    uint32_t mag = v & 0x7f7f7f7fu;
-    uint32_t is_nan = __vcmpeq4(mag, 0x7f7f7f7fu);
-    uint32_t is_zero = __vcmpeq4(mag, 0u);
-    if (is_nan)
+    const uint32_t v = (uint32_t)lo | ((uint32_t)hi << 16);
+    const uint32_t mag = v & 0x7f7f7f7fu;
+    // bytes whose magnitude is not zero keep their sign bit (so -0 becomes +0)
+    const uint32_t nonzero = (mag + 0x7f7f7f7fu) & 0x80808080u;
+    // a magnitude of 0x7f can only come from a NaN input (finite values saturate at 0x7e)
+    const uint32_t nan_bytes = (mag + 0x01010101u) & 0x80808080u;
+    if (nan_bytes) {
         nan = true;
-    return v & ~is_nan & ~(is_zero & 0x80808080u);
+        const uint32_t full = (nan_bytes >> 7) * 0xffu;
+        return (mag | (v & nonzero)) & ~full;
+    }
+    return mag | (v & nonzero);
 }
 
 // ---- PTX wrappers ----------------------------------------------------------------
@@ -125,21 +130,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait: gives up after about two seconds and reports false.
+// Bounded wait: gives up after about two seconds (4e9 SM cycles) and reports false.
+// The cycle counter is only consulted every 1024 unsuccessful polls.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
-    for (int i = 0; i < 64; ++i)
-        if (mbar_try_wait(bar, parity))
-            return true;
-    uint64_t t0;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    if (mbar_try_wait(bar, parity))
+        return true;
+    const long long t0 = clock64();
     for (;;) {
-        for (int i = 0; i < 256; ++i)
+        for (int i = 0; i < 1024; ++i)
             if (mbar_try_wait(bar, parity))
                 return true;
-        uint64_t t1;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-        if (t1 - t0 > 2000000000ull)
+        if (clock64() - t0 > 4000000000ll)
             return false;
     }
 }
@@ -201,15 +203,32 @@ __device__ __forceinline__ void tc_fence_after()
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 
-// D[tmem] (+)= A[smem] * B[smem], 8-bit / 4-bit floating operands, FP32 accumulate
-__device__ __forceinline__ void mma_f8f6f4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+// D[tmem] (+)= A[smem] * B[smem], 8-bit / 4-bit floating operands, FP32 accumulate.
+// The matrix descriptors are passed as their two 32-bit halves (the low half holds the
+// start address in 16-byte units and is the only part that moves), so advancing an
+// operand costs one 32-bit add in the issuing thread.  ACC = false overwrites D.
+template <bool ACC>
+__device__ __forceinline__ void mma_f8f6f4(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc)
 {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if (ACC) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "setp.eq.u32 p, 1, 1;\n\t"
+            "mov.b64 da, {%1, %3};\n\t"
+            "mov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %4, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "setp.eq.u32 p, 1, 0;\n\t"
+            "mov.b64 da, {%1, %3};\n\t"
+            "mov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %4, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc)
+            : "memory");
+    }
 }
 
 // the barrier gets one arrival once all MMAs issued so far by this thread are done
@@ -239,11 +258,16 @@ __device__ __forceinline__ void tmem_ld_wait()
 }
 
 // Shared-memory matrix descriptor: K-major rows of 128 bytes, 128-byte swizzle,
-// groups of 8 rows 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr)
+// groups of 8 rows 1024 bytes apart.  Low half: start address in 16-byte units (14 bits)
+// and the (ignored) leading byte offset 1; high half: stride byte offset 1024 >> 4,
+// descriptor version 1 (bit 46), layout type 2 = 128-byte swizzle (bits 61-63).
+// The swizzle is a function of the shared-memory address itself, so a start address
+// moved by whole 128-byte rows stays consistent with TMA-written data (base offset 0).
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t addr)
 {
-    return (uint64_t)((addr >> 4) & 0x3fffu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+    return ((addr >> 4) & 0x3fffu) | (1u << 16);
 }
+constexpr uint32_t SMEM_DESC_HI_K_SW128 = 64u | (1u << 14) | (2u << 29);
 
 // Instruction descriptor: FP32 accumulator, operand formats (0 = E4M3, 5 = E2M1),
 // both operands K-major, M = 128, N = n.

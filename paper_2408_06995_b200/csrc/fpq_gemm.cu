@@ -5,19 +5,20 @@
 //
 // A CTA (one per SM) walks 128 x BN output tiles.  Warp 0 issues TMA loads into two
 // shared-memory rings (activations, weights), warp 1 owns tensor memory and issues
-// the MMAs into one of two accumulators, warps 2-5 drain the other accumulator
+// the MMAs into one of two accumulators, warps 2-9 drain the other accumulator
 // (scale, bias, FP32 stores), so a tile's epilogue overlaps the next tile's main loop.
 //
-// Activation operand, three addressing modes:
-//   ROWS  linear: 128 rows of [M][Ca] codes per 128-wide reduction chunk;
+// The reduction of a tile is a list of blocks, block j = (128-wide chunk cc, tap), each
+// 4 MMAs of K = 32.  Activation operand, three addressing modes:
+//   ROWS  linear: 128 rows of [M][Ca] codes per chunk;
 //   FLAT  stride-1 convolution on the zero-framed channels-last codes
 //         [B][Hp][Wp][Ca] seen as one list of pixels: output position q reads input
-//         positions q + r*Wp + s, so one load of 128 + (R-1)*Wp + (S-1) pixel rows
-//         serves all R*S taps through matrix descriptors whose start address is moved
-//         by whole 128-byte rows (the 128-byte swizzle is a function of the shared-memory
-//         address itself, so TMA-written data and a shifted descriptor stay consistent;
-//         the descriptor's base-offset field stays 0);
-//   TAPS  any stride: one 4-D box (channels, x, y, image) per tap.
+//         positions q + r*Wp + s, so one load of 128 + (R-1)*Wp + (S-1) pixel rows per
+//         chunk serves all R*S taps through matrix descriptors whose start address is
+//         moved by whole 128-byte rows;
+//   TAPS  any stride: one 4-D box (channels, x, y, image) per block.
+// A ring stage carries the data of several blocks (one barrier handshake per stage);
+// weights whose whole reduction fits in shared memory stay resident across row tiles.
 #include <cuda.h>
 
 #include "fpq_common.cuh"
@@ -26,12 +27,36 @@
 namespace fpq {
 
 constexpr int BM = 128;        // output rows per tile (TMEM lanes)
-constexpr int BK = 128;        // reduction elements per chunk (one 128-byte swizzled row)
-constexpr int UMMA_K = 32;     // reduction elements per MMA instruction
-constexpr int NUM_THREADS = 192;
+constexpr int BK = 128;        // reduction elements per block (one 128-byte swizzled row)
+constexpr int NUM_EPI_WARPS = 8;   // two per TMEM lane quarter, each takes half of the columns
+constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
 constexpr int SMEM_BUDGET = 220 * 1024;
 
 enum { MODE_ROWS = 0, MODE_FLAT = 1, MODE_TAPS = 2 };
+
+// Division of a 31-bit unsigned number by a constant known on the host:
+// n / d = (umulhi(n, mul) + n) >> shift.
+struct FastDiv {
+    uint32_t mul, shift;
+};
+
+static FastDiv make_fastdiv(uint32_t d)
+{
+    FastDiv f{0, 0};
+    if (d > 1) {
+        uint32_t s = 0;
+        while ((1ull << s) < d)
+            ++s;
+        f.shift = s;
+        f.mul = (uint32_t)((((1ull << 32) * ((1ull << s) - d)) / d) + 1);
+    }
+    return f;
+}
+
+__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f)
+{
+    return (uint32_t)(((uint64_t)__umulhi(n, f.mul) + n) >> f.shift);
+}
 
 struct GemmArgs {
     int mode;
@@ -39,21 +64,27 @@ struct GemmArgs {
     int N;
     int cchunks;               // 128-wide chunks of the reduction per tap
     int taps, S, stride;
+    int nblk;                  // blocks per tile = cchunks * taps
     int Wp, HpWp;              // framed geometry
+    FastDiv div_HpWp, div_Wp, div_tiles, div_Wt, div_Ht, div_tx, div_ty;
     int Wt, Ht, Bt;            // TAPS: tile of Wt * Ht * Bt = 128 output pixels
     int tiles_x, tiles_y;
     int Ho, Wo, B;
     int m_tiles, n_tiles;
-    int a_boxes, a_box_rows;   // activation stage = a_boxes TMA boxes of a_box_rows pixel rows
-    int a_stage_bytes, b_stage_bytes;
-    int a_stages, b_stages;
+    int m_fastest;             // tile order: consecutive tiles share the column tile
+    // activation ring: a stage holds the data of a_span consecutive blocks
+    int a_boxes, a_box_rows;   // one chunk load = a_boxes TMA boxes of a_box_rows pixel rows
+    int a_chunk_bytes, a_span, a_stage_bytes, a_stages;
+    // weight ring: a stage holds b_span consecutive blocks; resident = the whole reduction,
+    // reloaded only when the column tile changes
+    int b_span, b_stage_bytes, b_stages, b_resident;
+    uint32_t a_chunk_tx, b_block_tx;   // bytes one load reports to its barrier
     const float* w_scale;
     float x_scale;
     const float* bias;
     float* y;
     int* status;
     uint32_t idesc;
-    uint32_t a_stage_tx, b_stage_tx;   // bytes one stage's loads report to its barrier
 };
 
 template <int BN>
@@ -61,6 +92,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
                                                                   const __grid_constant__ CUtensorMap tmB,
                                                                   const GemmArgs g)
 {
+    constexpr uint32_t B_BLOCK_BYTES = BN * BK;          // smem footprint (4-bit codes sit in 16-byte containers)
+    constexpr uint32_t BSTEP = B_BLOCK_BYTES / 16;       // the same in descriptor units
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -74,7 +107,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
     const uint32_t a_full = bars, a_empty = bars + 64, b_full = bars + 128, b_empty = bars + 192;
     const uint32_t acc_full = bars + 256, acc_empty = bars + 272;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + ctl_off + 288);
-    volatile uint32_t* abort_flag = tmem_slot + 1;
     float* s_scale = reinterpret_cast<float*>(smem + ctl_off + 320);   // [2][BN]
     float* s_bias = s_scale + 2 * BN;                                   // [2][BN]
 
@@ -91,9 +123,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(acc_full + 8 * s, 1);
-            mbar_init(acc_empty + 8 * s, 4);      // one arrival per epilogue warp
+            mbar_init(acc_empty + 8 * s, NUM_EPI_WARPS);      // one arrival per epilogue warp
         }
-        *abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
@@ -107,126 +138,283 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // tile index -> (row tile, column tile)
+    auto decode_tile = [&](int t, int& mt, int& nt) {
+        const int q = (int)fdiv((uint32_t)t, g.div_tiles);
+        if (g.m_fastest) { nt = q; mt = t - q * g.m_tiles; }
+        else             { mt = q; nt = t - q * g.n_tiles; }
+    };
+
+    // Every wait below is bounded; a role whose wait expires records FPQ_ERR_TIMEOUT and
+    // leaves its loop, the other roles then run into their own limits and follow.
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
+        // ---------------- TMA producer (one thread; its loops never divide) ----------------
         if (lane == 0) {
-            uint32_t ia = 0, ib = 0;              // loads issued so far into each ring
+            uint32_t sa = 0, pa = 0, sb = 0, pb = 0;   // stage and phase of the next load per ring
+            uint32_t na = 0, nb = 0;                   // stages issued (for the abort path)
+            int resident_nt = -1;
             bool dead = false;
             for (int t = blockIdx.x; t < total_tiles && !dead; t += gridDim.x) {
-                const int mt = t / g.n_tiles, nt = t - mt * g.n_tiles;
+                int mt, nt;
+                decode_tile(t, mt, nt);
                 const int n0 = nt * BN;
                 int x0 = 0, y0 = 0, b0 = 0;
                 if (g.mode == MODE_TAPS) {
-                    int r = mt;
-                    x0 = (r % g.tiles_x) * g.Wt;
-                    r /= g.tiles_x;
-                    y0 = (r % g.tiles_y) * g.Ht;
-                    b0 = (r / g.tiles_y) * g.Bt;
+                    const uint32_t r1 = fdiv((uint32_t)mt, g.div_tx);
+                    x0 = (mt - (int)r1 * g.tiles_x) * g.Wt * g.stride;
+                    const uint32_t r2 = fdiv(r1, g.div_ty);
+                    y0 = ((int)r1 - (int)r2 * g.tiles_y) * g.Ht * g.stride;
+                    b0 = (int)r2 * g.Bt;
                 }
-                for (int cc = 0; cc < g.cchunks && !dead; ++cc) {
-                    for (int tap = 0; tap < g.taps; ++tap) {
-                        if (g.mode == MODE_TAPS || tap == 0) {
-                            const uint32_t s = ia % g.a_stages, ph = (ia / g.a_stages) & 1;
-                            if (!mbar_wait(a_empty + 8 * s, ph ^ 1) || *abort_flag) { dead = true; break; }
-                            const uint32_t dst = a_ring + s * g.a_stage_bytes;
-                            mbar_expect_tx(a_full + 8 * s, g.a_stage_tx);
-                            if (g.mode == MODE_TAPS) {
-                                const int r = tap / g.S, sx = tap - r * g.S;
-                                tma_load_4d(dst, &tmA, a_full + 8 * s, cc * BK, x0 * g.stride + sx, y0 * g.stride + r, b0);
-                            } else {
-                                for (int bx = 0; bx < g.a_boxes; ++bx)
-                                    tma_load_4d(dst + bx * g.a_box_rows * 128, &tmA, a_full + 8 * s, cc * BK,
-                                                mt * BM + bx * g.a_box_rows, 0, 0);
+                const bool load_b = !(g.b_resident && resident_nt == nt);
+                resident_nt = nt;
+                int cc = 0, tap = 0, r = 0, sx = 0;    // block j = (cc, tap), tap = (r, sx)
+                int ja = 0, jb = 0;                    // position inside the current A / B stage
+                for (int j = 0; j < g.nblk; ++j) {
+                    if (ja == 0) {
+                        // activation stage: the data of the next a_span blocks
+                        if (!mbar_wait(a_empty + 8 * sa, pa ^ 1)) { dead = true; break; }
+                        const int nblocks = min(g.a_span, g.nblk - j);
+                        const int nloads = (g.mode == MODE_TAPS) ? nblocks : nblocks / g.taps;
+                        mbar_expect_tx(a_full + 8 * sa, (uint32_t)nloads * g.a_chunk_tx);
+                        uint32_t dst = a_ring + sa * g.a_stage_bytes;
+                        if (g.mode == MODE_TAPS) {
+                            int c2 = cc, t2 = tap, r2 = r, s2 = sx;
+                            for (int l = 0; l < nloads; ++l, dst += g.a_chunk_bytes) {
+                                tma_load_4d(dst, &tmA, a_full + 8 * sa, c2 * BK, x0 + s2, y0 + r2, b0);
+                                if (++s2 == g.S) { s2 = 0; ++r2; }
+                                if (++t2 == g.taps) { t2 = 0; r2 = 0; s2 = 0; ++c2; }
                             }
-                            ++ia;
+                        } else {
+                            for (int l = 0; l < nloads; ++l, dst += g.a_chunk_bytes)
+                                for (int bx = 0; bx < g.a_boxes; ++bx)
+                                    tma_load_4d(dst + bx * g.a_box_rows * 128, &tmA, a_full + 8 * sa, (cc + l) * BK,
+                                                mt * BM + bx * g.a_box_rows, 0, 0);
                         }
-                        const uint32_t s = ib % g.b_stages, ph = (ib / g.b_stages) & 1;
-                        if (!mbar_wait(b_empty + 8 * s, ph ^ 1) || *abort_flag) { dead = true; break; }
-                        mbar_expect_tx(b_full + 8 * s, g.b_stage_tx);
-                        tma_load_3d(b_ring + s * g.b_stage_bytes, &tmB, b_full + 8 * s, cc * BK, tap, n0);
-                        ++ib;
+                        ++na;
+                        if (++sa == (uint32_t)g.a_stages) { sa = 0; pa ^= 1; }
                     }
+                    if (jb == 0 && load_b) {
+                        if (!mbar_wait(b_empty + 8 * sb, pb ^ 1)) { dead = true; break; }
+                        const int nblocks = min(g.b_span, g.nblk - j);
+                        mbar_expect_tx(b_full + 8 * sb, (uint32_t)nblocks * g.b_block_tx);
+                        uint32_t dst = b_ring + sb * g.b_stage_bytes;
+                        int c2 = cc, t2 = tap;
+                        for (int l = 0; l < nblocks; ++l, dst += B_BLOCK_BYTES) {
+                            tma_load_3d(dst, &tmB, b_full + 8 * sb, c2 * BK, t2, n0);
+                            if (++t2 == g.taps) { t2 = 0; ++c2; }
+                        }
+                        ++nb;
+                        if (++sb == (uint32_t)g.b_stages) { sb = 0; pb ^= 1; }
+                    }
+                    if (++ja == g.a_span) ja = 0;
+                    if (++jb == g.b_span) jb = 0;
+                    if (++sx == g.S) { sx = 0; ++r; }
+                    if (++tap == g.taps) { tap = 0; r = 0; sx = 0; ++cc; }
                 }
             }
             if (dead) {
-                *abort_flag = 1;
                 atomicMin(g.status, FPQ_ERR_TIMEOUT);
                 // let the copies still in flight land before the CTA's shared memory is released
-                for (uint32_t i = (ia > (uint32_t)g.a_stages ? ia - g.a_stages : 0); i < ia; ++i)
+                for (uint32_t i = (na > (uint32_t)g.a_stages ? na - g.a_stages : 0); i < na; ++i)
                     (void)mbar_wait(a_full + 8 * (i % g.a_stages), (i / g.a_stages) & 1);
-                for (uint32_t i = (ib > (uint32_t)g.b_stages ? ib - g.b_stages : 0); i < ib; ++i)
+                for (uint32_t i = (nb > (uint32_t)g.b_stages ? nb - g.b_stages : 0); i < nb; ++i)
                     (void)mbar_wait(b_full + 8 * (i % g.b_stages), (i / g.b_stages) & 1);
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
+        // ---------------- MMA issuer (one thread) ----------------
+        // The tensor pipe retires one 128 x BN x 32 MMA every BN/2 cycles and its queue is
+        // shallow, so this thread has only a few hundred cycles per block of 4: operand
+        // positions are kept as descriptor low words (16-byte units) and the two common
+        // loop shapes (3x3 taps over one loaded chunk; one block per chunk) are
+        // straight-line code.
         if (lane == 0) {
-            uint32_t ia = 0, ib = 0, it = 0;
+            uint32_t sa = 0, pa = 0, sb = 0, pb = 0, it = 0;
+            int resident_nt = -1;
             bool dead = false;
+            const uint32_t a_chunk_step = (uint32_t)g.a_chunk_bytes >> 4;
+            const uint32_t b_res = smem_desc_lo(b_ring);           // resident weights start here
+            const uint32_t HI = SMEM_DESC_HI_K_SW128;
             for (int t = blockIdx.x; t < total_tiles && !dead; t += gridDim.x, ++it) {
+                int mt, nt;
+                decode_tile(t, mt, nt);
+                const bool new_b = !(g.b_resident && resident_nt == nt);
+                if (g.b_resident && new_b && resident_nt >= 0) {
+                    // the resident weights are done with once everything issued so far has run
+                    mma_commit(b_empty + 8 * sb);
+                    if (++sb == (uint32_t)g.b_stages) { sb = 0; pb ^= 1; }
+                }
+                resident_nt = nt;
                 const uint32_t buf = it & 1, aph = (it >> 1) & 1;
-                if (!mbar_wait(acc_empty + 8 * buf, aph ^ 1) || *abort_flag) { dead = true; break; }
+                if (!mbar_wait(acc_empty + 8 * buf, aph ^ 1)) { dead = true; break; }
+                if (g.b_resident && new_b)
+                    if (!mbar_wait(b_full + 8 * sb, pb)) { dead = true; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                uint32_t first = 1;
-                for (int cc = 0; cc < g.cchunks && !dead; ++cc) {
-                    uint32_t a_addr = 0;
-                    for (int tap = 0; tap < g.taps; ++tap) {
-                        if (g.mode == MODE_TAPS || tap == 0) {
-                            const uint32_t s = ia % g.a_stages, ph = (ia / g.a_stages) & 1;
-                            if (!mbar_wait(a_full + 8 * s, ph) || *abort_flag) { dead = true; break; }
-                            a_addr = a_ring + s * g.a_stage_bytes;
-                        }
-                        const uint32_t sb = ib % g.b_stages, phb = (ib / g.b_stages) & 1;
-                        if (!mbar_wait(b_full + 8 * sb, phb) || *abort_flag) { dead = true; break; }
+
+                if (g.mode == MODE_FLAT && g.taps == 9 && g.S == 3) {
+                    const uint32_t Wp8 = (uint32_t)g.Wp * 8u;
+                    const int chunks_per_stage = g.a_span / 9;
+                    for (int cc = 0; cc < g.cchunks && !dead;) {
+                        if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
                         tc_fence_after();
-                        uint32_t a_tap = a_addr;
-                        if (g.mode == MODE_FLAT) {
-                            const int r = tap / g.S, sx = tap - r * g.S;
-                            a_tap += (uint32_t)(r * g.Wp + sx) * 128u;
-                        }
-                        const uint64_t adesc = smem_desc_k_sw128(a_tap);
-                        const uint64_t bdesc = smem_desc_k_sw128(b_ring + sb * g.b_stage_bytes);
+                        const uint32_t abase = smem_desc_lo(a_ring + sa * g.a_stage_bytes);
+                        const int nch = min(chunks_per_stage, g.cchunks - cc);
+                        for (int c = 0; c < nch && !dead; ++c, ++cc) {
+                            const uint32_t ac = abase + c * a_chunk_step;
+                            const uint32_t bres = b_res + (uint32_t)cc * 9u * BSTEP;
+                            uint32_t bst = 0;
 #pragma unroll
-                        for (int kk = 0; kk < BK / UMMA_K; ++kk) {
-                            // 32 reduction elements = 32 bytes inside the swizzled row: +2 in 16-byte units
-                            mma_f8f6f4(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, g.idesc, first ? 0u : 1u);
-                            first = 0;
+                            for (int tap = 0; tap < 9; ++tap) {
+                                if (!g.b_resident && tap % 3 == 0) {
+                                    if (!mbar_wait(b_full + 8 * sb, pb)) { dead = true; break; }
+                                    tc_fence_after();
+                                    bst = smem_desc_lo(b_ring + sb * g.b_stage_bytes);
+                                }
+                                // tap (r, s) reads the chunk r * Wp + s pixel rows (128 B each) further down
+                                const uint32_t al = ac + (tap / 3) * Wp8 + (tap % 3) * 8u;
+                                const uint32_t bl = g.b_resident ? bres + tap * BSTEP : bst + (tap % 3) * BSTEP;
+                                // 32 reduction elements = 32 bytes inside the swizzled row: +2 units
+                                if (tap == 0 && cc == 0)
+                                    mma_f8f6f4<false>(d_tmem, al, bl, HI, g.idesc);
+                                else
+                                    mma_f8f6f4<true>(d_tmem, al, bl, HI, g.idesc);
+                                mma_f8f6f4<true>(d_tmem, al + 2, bl + 2, HI, g.idesc);
+                                mma_f8f6f4<true>(d_tmem, al + 4, bl + 4, HI, g.idesc);
+                                mma_f8f6f4<true>(d_tmem, al + 6, bl + 6, HI, g.idesc);
+                                if (!g.b_resident && tap % 3 == 2) {
+                                    mma_commit(b_empty + 8 * sb);
+                                    if (++sb == (uint32_t)g.b_stages) { sb = 0; pb ^= 1; }
+                                }
+                            }
                         }
-                        mma_commit(b_empty + 8 * sb);
-                        ++ib;
-                        if (g.mode == MODE_TAPS || tap == g.taps - 1) {
-                            mma_commit(a_empty + 8 * (ia % g.a_stages));
-                            ++ia;
+                        mma_commit(a_empty + 8 * sa);
+                        if (++sa == (uint32_t)g.a_stages) { sa = 0; pa ^= 1; }
+                    }
+                } else if (g.taps == 1 && g.mode != MODE_TAPS && g.a_span <= 4 &&
+                           (g.b_resident || g.b_span == g.a_span)) {
+                    // one block per 128-wide chunk; a stage carries up to 4 chunks of both operands
+                    for (int cc = 0; cc < g.cchunks && !dead;) {
+                        if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
+                        uint32_t bbase = b_res + (uint32_t)cc * BSTEP;
+                        if (!g.b_resident) {
+                            if (!mbar_wait(b_full + 8 * sb, pb)) { dead = true; break; }
+                            bbase = smem_desc_lo(b_ring + sb * g.b_stage_bytes);
+                        }
+                        tc_fence_after();
+                        const uint32_t abase = smem_desc_lo(a_ring + sa * g.a_stage_bytes);
+                        const int n = min(g.a_span, g.cchunks - cc);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            if (c < n) {
+                                const uint32_t al = abase + c * (BM * BK / 16), bl = bbase + c * BSTEP;
+                                if (c == 0 && cc == 0)
+                                    mma_f8f6f4<false>(d_tmem, al, bl, HI, g.idesc);
+                                else
+                                    mma_f8f6f4<true>(d_tmem, al, bl, HI, g.idesc);
+                                mma_f8f6f4<true>(d_tmem, al + 2, bl + 2, HI, g.idesc);
+                                mma_f8f6f4<true>(d_tmem, al + 4, bl + 4, HI, g.idesc);
+                                mma_f8f6f4<true>(d_tmem, al + 6, bl + 6, HI, g.idesc);
+                            }
+                        }
+                        if (!g.b_resident) {
+                            mma_commit(b_empty + 8 * sb);
+                            if (++sb == (uint32_t)g.b_stages) { sb = 0; pb ^= 1; }
+                        }
+                        mma_commit(a_empty + 8 * sa);
+                        if (++sa == (uint32_t)g.a_stages) { sa = 0; pa ^= 1; }
+                        cc += n;
+                    }
+                } else {
+                    // general shape: block by block
+                    uint32_t a_lo = 0, b_lo = b_res;       // operands of the current block
+                    uint32_t a_chunk_lo = 0;               // FLAT/ROWS: current chunk in its stage
+                    uint32_t row_off8 = 0;                 // FLAT: (r * Wp + s) * 8 of the current tap
+                    const uint32_t row_wrap8 = (uint32_t)(g.Wp - g.S) * 8u;
+                    const bool flat = g.mode == MODE_FLAT, taps_mode = g.mode == MODE_TAPS;
+                    int tap = 0, sx = 0, ja = 0, jb = 0;
+                    for (int j = 0; j < g.nblk; ++j) {
+                        if (ja == 0) {
+                            if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
+                            a_chunk_lo = smem_desc_lo(a_ring + sa * g.a_stage_bytes);
+                            a_lo = a_chunk_lo;
+                            tc_fence_after();
+                        }
+                        if (jb == 0 && !g.b_resident) {
+                            if (!mbar_wait(b_full + 8 * sb, pb)) { dead = true; break; }
+                            tc_fence_after();
+                            b_lo = smem_desc_lo(b_ring + sb * g.b_stage_bytes);
+                        }
+                        const uint32_t al = flat ? a_chunk_lo + row_off8 : a_lo;
+                        if (j == 0)
+                            mma_f8f6f4<false>(d_tmem, al, b_lo, HI, g.idesc);
+                        else
+                            mma_f8f6f4<true>(d_tmem, al, b_lo, HI, g.idesc);
+                        mma_f8f6f4<true>(d_tmem, al + 2, b_lo + 2, HI, g.idesc);
+                        mma_f8f6f4<true>(d_tmem, al + 4, b_lo + 4, HI, g.idesc);
+                        mma_f8f6f4<true>(d_tmem, al + 6, b_lo + 6, HI, g.idesc);
+                        const bool last = (j == g.nblk - 1);
+                        b_lo += BSTEP;
+                        if (++jb == g.b_span || last) {
+                            jb = 0;
+                            if (!g.b_resident) {
+                                mma_commit(b_empty + 8 * sb);
+                                if (++sb == (uint32_t)g.b_stages) { sb = 0; pb ^= 1; }
+                            }
+                        }
+                        // next block's activation operand
+                        row_off8 += 8;
+                        if (++sx == g.S) { sx = 0; row_off8 += row_wrap8; }
+                        if (taps_mode) a_lo += a_chunk_step;
+                        if (++tap == g.taps) {
+                            tap = 0; sx = 0; row_off8 = 0;
+                            a_chunk_lo += a_chunk_step;
+                            if (!taps_mode) a_lo = a_chunk_lo;
+                        }
+                        if (++ja == g.a_span || last) {
+                            ja = 0;
+                            mma_commit(a_empty + 8 * sa);
+                            if (++sa == (uint32_t)g.a_stages) { sa = 0; pa ^= 1; }
                         }
                     }
                 }
+                if (dead)
+                    break;
                 mma_commit(acc_full + 8 * buf);
             }
-            if (dead) {
-                *abort_flag = 1;
+            if (dead)
                 atomicMin(g.status, FPQ_ERR_TIMEOUT);
-            }
         }
     } else {
-        // ---------------- epilogue: 4 warps, one TMEM lane quarter each ----------------
-        const int et = threadIdx.x - 64;           // 0..127
-        const int quarter = warp & 3;              // TMEM lanes this warp may read
+        // ---------------- epilogue: 8 warps; warp w reads TMEM lane quarter w % 4 and the
+        // column half (w - 2) / 4 of the accumulator ----------------
+        constexpr int EPI_THREADS = 32 * NUM_EPI_WARPS;
+        constexpr int HALF = BN / 2;               // columns per warp
+        constexpr int CHUNKS = HALF / 32;          // 32-column TMEM loads per warp (1 or 2)
+        const int et = threadIdx.x - 64;
+        const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;       // row of the tile held by this thread
         uint32_t it = 0;
         bool dead = false;
+        int loaded_nt[2] = {-1, -1};               // which column tile each scale/bias buffer holds
         for (int t = blockIdx.x; t < total_tiles && !dead; t += gridDim.x, ++it) {
-            const int mt = t / g.n_tiles, nt = t - mt * g.n_tiles;
+            int mt, nt;
+            decode_tile(t, mt, nt);
             const int n0 = nt * BN;
             const uint32_t buf = it & 1, aph = (it >> 1) & 1;
             float* sc = s_scale + buf * BN;
             float* bi = s_bias + buf * BN;
-            for (int i = et; i < BN; i += 128) {
-                const int n = n0 + i;
-                sc[i] = (n < g.N) ? g.x_scale * __ldg(g.w_scale + n) : 0.f;
-                bi[i] = (g.bias && n < g.N) ? __ldg(g.bias + n) : 0.f;
+            if (loaded_nt[buf] != nt) {            // same decision in every epilogue thread
+                for (int i = et; i < BN; i += EPI_THREADS) {
+                    const int n = n0 + i;
+                    sc[i] = (n < g.N) ? g.x_scale * __ldg(g.w_scale + n) : 0.f;
+                    bi[i] = (g.bias && n < g.N) ? __ldg(g.bias + n) : 0.f;
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+                loaded_nt[buf] = nt;
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
 
             // where this thread's row goes
             bool row_valid;
@@ -240,58 +428,83 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
             } else {
                 int ox, oy, b;
                 if (g.mode == MODE_FLAT) {
-                    const int64_t q = (int64_t)mt * BM + row;
-                    b = (int)(q / g.HpWp);
-                    const int rem = (int)(q - (int64_t)b * g.HpWp);
-                    oy = rem / g.Wp;
-                    ox = rem - oy * g.Wp;
+                    const uint32_t q = (uint32_t)mt * BM + row;
+                    b = (int)fdiv(q, g.div_HpWp);
+                    const uint32_t rem = q - (uint32_t)b * g.HpWp;
+                    oy = (int)fdiv(rem, g.div_Wp);
+                    ox = (int)rem - oy * g.Wp;
                 } else {
-                    int r = mt;
-                    const int x0 = (r % g.tiles_x) * g.Wt;
-                    r /= g.tiles_x;
-                    const int y0 = (r % g.tiles_y) * g.Ht;
-                    const int b0 = (r / g.tiles_y) * g.Bt;
-                    ox = x0 + row % g.Wt;
-                    oy = y0 + (row / g.Wt) % g.Ht;
-                    b = b0 + row / (g.Wt * g.Ht);
+                    const uint32_t r1 = fdiv((uint32_t)mt, g.div_tx);
+                    const int x0 = (mt - (int)r1 * g.tiles_x) * g.Wt;
+                    const uint32_t r2 = fdiv(r1, g.div_ty);
+                    const int y0 = ((int)r1 - (int)r2 * g.tiles_y) * g.Ht;
+                    const int b0 = (int)r2 * g.Bt;
+                    const uint32_t q1 = fdiv((uint32_t)row, g.div_Wt);
+                    ox = x0 + (row - (int)q1 * g.Wt);
+                    const uint32_t q2 = fdiv(q1, g.div_Ht);
+                    oy = y0 + ((int)q1 - (int)q2 * g.Ht);
+                    b = b0 + (int)q2;
                 }
                 row_valid = ox < g.Wo && oy < g.Ho && b < g.B;
                 nstride = (int64_t)g.Ho * g.Wo;
                 yrow = g.y + ((int64_t)b * g.N * g.Ho + oy) * g.Wo + ox;   // + n * Ho * Wo
             }
 
-            bool ok = mbar_wait(acc_full + 8 * buf, aph);
-            if (!ok || *abort_flag) { dead = true; }
+            if (!mbar_wait(acc_full + 8 * buf, aph)) { dead = true; }
             tc_fence_after();
-            if (!dead) {
-                const bool vec_ok = (g.mode == MODE_ROWS) && (g.N % 4 == 0);
-                const uint32_t t_addr = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
-#pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
-                    if (n0 + c * 32 >= g.N)
-                        break;                                  // whole chunk past the last column
-                    uint32_t r[32];
-                    tmem_ld32(t_addr + c * 32, r);
-                    tmem_ld_wait();
-                    if (!row_valid)
-                        continue;
-                    const int nb = n0 + c * 32;
-                    if (vec_ok && nb + 32 <= g.N) {
+            const int ncol0 = n0 + half * HALF;    // first output column of this warp
+            if (!dead && ncol0 < g.N) {
+                const uint32_t t_addr = tmem_base + buf * BN + half * HALF + ((uint32_t)(quarter * 32) << 16);
+                uint32_t r[CHUNKS][32];
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            float4 v;
-                            v.x = fmaf(__uint_as_float(r[j + 0]), sc[c * 32 + j + 0], bi[c * 32 + j + 0]);
-                            v.y = fmaf(__uint_as_float(r[j + 1]), sc[c * 32 + j + 1], bi[c * 32 + j + 1]);
-                            v.z = fmaf(__uint_as_float(r[j + 2]), sc[c * 32 + j + 2], bi[c * 32 + j + 2]);
-                            v.w = fmaf(__uint_as_float(r[j + 3]), sc[c * 32 + j + 3], bi[c * 32 + j + 3]);
-                            *reinterpret_cast<float4*>(yrow + nb + j) = v;
-                        }
-                    } else {
+                for (int c = 0; c < CHUNKS; ++c)
+                    tmem_ld32(t_addr + c * 32, r[c]);
+                tmem_ld_wait();
+                if (row_valid) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (nb + j < g.N)
-                                yrow[(int64_t)(nb + j) * nstride] =
-                                    fmaf(__uint_as_float(r[j]), sc[c * 32 + j], bi[c * 32 + j]);
+                    for (int c = 0; c < CHUNKS; ++c) {
+                        const int nb = ncol0 + c * 32;
+                        const float* scc = sc + half * HALF + c * 32;
+                        const float* bic = bi + half * HALF + c * 32;
+                        const float4* sc4 = reinterpret_cast<const float4*>(scc);
+                        const float4* bi4 = reinterpret_cast<const float4*>(bic);
+                        if (nb + 32 <= g.N) {
+                            if (g.mode == MODE_ROWS) {
+                                if (g.N % 4 == 0) {
+                                    float4* dst = reinterpret_cast<float4*>(yrow + nb);
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) {
+                                        const float4 s4 = sc4[j], b4 = bi4[j];
+                                        float4 v;
+                                        v.x = fmaf(__uint_as_float(r[c][4 * j + 0]), s4.x, b4.x);
+                                        v.y = fmaf(__uint_as_float(r[c][4 * j + 1]), s4.y, b4.y);
+                                        v.z = fmaf(__uint_as_float(r[c][4 * j + 2]), s4.z, b4.z);
+                                        v.w = fmaf(__uint_as_float(r[c][4 * j + 3]), s4.w, b4.w);
+                                        dst[j] = v;
+                                    }
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j)
+                                        yrow[nb + j] = fmaf(__uint_as_float(r[c][j]), scc[j], bic[j]);
+                                }
+                            } else {
+                                float* dst = yrow + (int64_t)nb * nstride;
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    const float4 s4 = sc4[j], b4 = bi4[j];
+                                    dst[0] = fmaf(__uint_as_float(r[c][4 * j + 0]), s4.x, b4.x);
+                                    dst[nstride] = fmaf(__uint_as_float(r[c][4 * j + 1]), s4.y, b4.y);
+                                    dst[2 * nstride] = fmaf(__uint_as_float(r[c][4 * j + 2]), s4.z, b4.z);
+                                    dst[3 * nstride] = fmaf(__uint_as_float(r[c][4 * j + 3]), s4.w, b4.w);
+                                    dst += 4 * nstride;
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                if (nb + j < g.N)
+                                    yrow[(int64_t)(nb + j) * nstride] = fmaf(__uint_as_float(r[c][j]), scc[j], bic[j]);
+                            }
                         }
                     }
                 }
@@ -302,10 +515,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
             if (lane == 0)
                 mbar_arrive(acc_empty + 8 * buf);
         }
-        if (dead) {
-            *abort_flag = 1;
+        if (dead)
             atomicMin(g.status, FPQ_ERR_TIMEOUT);
-        }
     }
 
     tc_fence_before();
@@ -342,45 +553,94 @@ static int pow2_at_least(int v)
     return p;
 }
 
-static int sm_count()
+struct DeviceInfo {
+    int sms;
+    bool smem_set[3];
+};
+
+static DeviceInfo* device_info()
 {
-    static int n[64] = {0};
+    static DeviceInfo info[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
-        return 148;
-    if (!n[dev]) {
+        return nullptr;
+    if (!info[dev].sms) {
         int v = 0;
         if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v < 1)
             v = 148;
-        n[dev] = v;
+        info[dev].sms = v;
     }
-    return n[dev];
+    return &info[dev];
 }
 
 template <int BN>
 static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs& g, cudaStream_t st)
 {
-    g.b_stage_bytes = BN * BK;
-    // split the shared-memory budget between the two rings
-    const int ctl = 320 + 4 * BN * 4 + 1024;
-    int a_stages = (g.mode == MODE_TAPS) ? 4 : 2;
-    int b_stages = (SMEM_BUDGET - ctl - a_stages * g.a_stage_bytes) / g.b_stage_bytes;
-    if (g.mode != MODE_TAPS && b_stages > 6 && SMEM_BUDGET - ctl - 3 * g.a_stage_bytes >= 4 * g.b_stage_bytes) {
-        a_stages = 3;
-        b_stages = (SMEM_BUDGET - ctl - a_stages * g.a_stage_bytes) / g.b_stage_bytes;
-    }
-    if (b_stages > 8)
-        b_stages = 8;
-    if (b_stages < 2)
-        return FPQ_ERR_UNSUPPORTED;
-    g.a_stages = a_stages;
-    g.b_stages = b_stages;
-    const int dyn = a_stages * g.a_stage_bytes + b_stages * g.b_stage_bytes + ctl;
-    if (cudaFuncSetAttribute(fpq_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) !=
-        cudaSuccess)
+    // Split the shared-memory budget between the two rings.  A barrier handshake costs the
+    // single issuing thread a few hundred cycles, so every stage is made to carry 8-36 MMAs;
+    // weights that fit stay resident for all row tiles of a column tile.
+    DeviceInfo* di = device_info();
+    if (!di)
         return FPQ_ERR_CUDA;
+    const int ctl = 320 + 4 * BN * 4 + 1024;
+    const int budget = SMEM_BUDGET - ctl;
+    const int b_block = BN * BK;
+    const int a_min_span = (g.mode == MODE_FLAT) ? g.taps : 1;
+    const int64_t b_all = (int64_t)g.nblk * b_block;
+    if (b_all + 2 * g.a_chunk_bytes <= budget) {
+        g.b_resident = 1;
+        g.b_span = g.nblk;
+        g.b_stages = 1;
+        g.m_fastest = 1;
+        const int room = budget - (int)b_all;
+        int chunks = room / (2 * g.a_chunk_bytes);            // chunks (TAPS: boxes) per stage
+        const int want = (g.mode == MODE_FLAT && g.taps >= 4) ? 1 : 4;
+        if (chunks > want) chunks = want;
+        const int avail = (g.mode == MODE_TAPS) ? g.nblk : g.cchunks;
+        if (chunks > avail) chunks = avail;
+        if (chunks < 1) chunks = 1;
+        g.a_span = chunks * a_min_span;
+        g.a_stage_bytes = chunks * g.a_chunk_bytes;
+        g.a_stages = room / g.a_stage_bytes;
+        if (g.a_stages > 4) g.a_stages = 4;
+    } else {
+        g.b_resident = 0;
+        g.m_fastest = 0;
+        int chunks;
+        if (g.mode == MODE_FLAT && g.taps > 1) {
+            g.b_span = (g.taps == 9 && g.S == 3) ? 3 : 1;
+            g.a_span = g.taps;                                // one chunk per stage serves all taps
+            chunks = 1;
+            g.a_stages = 2;
+        } else {
+            g.b_span = (g.mode == MODE_TAPS && g.taps % 3 == 0) ? 3 : 2;
+            if (g.b_span > g.nblk) g.b_span = g.nblk;
+            g.a_span = g.b_span;
+            chunks = g.a_span;
+            g.a_stages = 3;
+        }
+        g.a_stage_bytes = chunks * g.a_chunk_bytes;
+        g.b_stages = (budget - g.a_stages * g.a_stage_bytes) / (g.b_span * b_block);
+        if (g.b_stages < 2 && g.a_stages > 2) {
+            g.a_stages = 2;
+            g.b_stages = (budget - g.a_stages * g.a_stage_bytes) / (g.b_span * b_block);
+        }
+        if (g.b_stages > 8) g.b_stages = 8;
+    }
+    g.b_stage_bytes = g.b_span * b_block;
+    if (g.a_stages < 1 || g.b_stages < 1 || (!g.b_resident && g.b_stages < 2))
+        return FPQ_ERR_UNSUPPORTED;
+    g.div_tiles = make_fastdiv((uint32_t)(g.m_fastest ? g.m_tiles : g.n_tiles));
+    const int dyn = g.a_stages * g.a_stage_bytes + g.b_stages * g.b_stage_bytes + ctl;
+    const int slot = BN == 64 ? 0 : (BN == 128 ? 1 : 2);
+    if (!di->smem_set[slot]) {
+        if (cudaFuncSetAttribute(fpq_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) !=
+            cudaSuccess)
+            return FPQ_ERR_CUDA;
+        di->smem_set[slot] = true;
+    }
     const int64_t tiles = (int64_t)g.m_tiles * g.n_tiles;
-    const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+    const int grid = (int)(tiles < di->sms ? tiles : di->sms);
     fpq_gemm_kernel<BN><<<grid, NUM_THREADS, dyn, st>>>(tmA, tmB, g);
     return cudaGetLastError() == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
 }
@@ -395,6 +655,7 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
     g.N = p.N;
     g.cchunks = p.Cp / BK;
     g.taps = p.R * p.S;
+    g.nblk = g.cchunks * g.taps;
     g.S = p.S;
     g.stride = p.stride;
     g.Ho = p.Ho;
@@ -409,13 +670,16 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
     const int BN = (p.N <= 64) ? 64 : 128;
     g.n_tiles = (p.N + BN - 1) / BN;
     g.idesc = idesc_f8f6f4(0u, p.w4 ? 5u : 0u, (uint32_t)BN);
-    g.b_stage_tx = (uint32_t)(BN * BK) / (p.w4 ? 2 : 1);
+    g.b_block_tx = (uint32_t)(BN * BK) / (p.w4 ? 2 : 1);
 
     CUtensorMap tmA, tmB;
     cuuint64_t dimsA[4], stridesA[3];
     cuuint32_t boxA[4], estrA[4] = {1, 1, 1, 1};
     const int Hp = p.H + 2 * p.pad, Wp = p.W + 2 * p.pad;
     int64_t mtiles;
+    g.Wp = 1;
+    g.HpWp = 1;
+    g.Wt = g.Ht = g.Bt = g.tiles_x = g.tiles_y = 1;
     if (!p.conv) {
         g.mode = MODE_ROWS;
         g.M = p.M;
@@ -431,7 +695,8 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
         // FLAT wastes the frame positions; take it when that costs little more than TAPS' exact tiles
         const int64_t flat_tiles = (framed + BM - 1) / BM;
         const int64_t exact_tiles = ((int64_t)p.B * p.Ho * p.Wo + BM - 1) / BM;
-        const bool flat_ok = p.stride == 1 && halo_rows <= 2 * 256 - 16 && flat_tiles * 4 <= exact_tiles * 5 + 4;
+        const bool flat_ok = p.stride == 1 && halo_rows <= 2 * 256 - 16 && flat_tiles * 4 <= exact_tiles * 5 + 4 &&
+                             framed < 0x7fffff00ll;
         if (flat_ok) {
             g.mode = MODE_FLAT;
             g.M = framed;
@@ -472,11 +737,17 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
             estrA[1] = estrA[2] = (cuuint32_t)p.stride;
         }
     }
-    if (mtiles <= 0 || mtiles * g.n_tiles > 0x7fffffff)
+    if (mtiles <= 0 || mtiles * g.n_tiles > 0x7fffff00ll)
         return FPQ_ERR_SHAPE;
     g.m_tiles = (int)mtiles;
-    g.a_stage_bytes = g.a_boxes * g.a_box_rows * 128;
-    g.a_stage_tx = (uint32_t)g.a_stage_bytes;
+    g.div_HpWp = make_fastdiv((uint32_t)g.HpWp);
+    g.div_Wp = make_fastdiv((uint32_t)g.Wp);
+    g.div_Wt = make_fastdiv((uint32_t)g.Wt);
+    g.div_Ht = make_fastdiv((uint32_t)g.Ht);
+    g.div_tx = make_fastdiv((uint32_t)g.tiles_x);
+    g.div_ty = make_fastdiv((uint32_t)g.tiles_y);
+    g.a_chunk_bytes = g.a_boxes * g.a_box_rows * 128;
+    g.a_chunk_tx = (uint32_t)g.a_chunk_bytes;
     if (enc(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, (void*)p.a_codes, dimsA, stridesA, boxA, estrA,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)

@@ -188,10 +188,15 @@ __global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const f
     {
         const int cl = ty * 16;
         float a[16];
+        const float* px = xb + (int64_t)(c0 + cl) * HW + p;
+        if (c0 + 128 <= C && p0 + 32 <= HW) {            // interior tile: no predicates
 #pragma unroll
-        for (int q = 0; q < 16; ++q) {
-            const int c = c0 + cl + q;
-            a[q] = (c < C && p < HW) ? __ldg(xb + (int64_t)c * HW + p) : 0.f;
+            for (int q = 0; q < 16; ++q)
+                a[q] = __ldg(px + (int64_t)q * HW);
+        } else {
+#pragma unroll
+            for (int q = 0; q < 16; ++q)
+                a[q] = (c0 + cl + q < C && p < HW) ? __ldg(px + (int64_t)q * HW) : 0.f;
         }
         uint4 v;
         v.x = e4m3x4_from_scaled(__fmul_rn(a[0], rinv), __fmul_rn(a[1], rinv), __fmul_rn(a[2], rinv), __fmul_rn(a[3], rinv), nan);
