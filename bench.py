@@ -5,9 +5,12 @@ Own arm (default): the DDIM-CIFAR-style 3x3 convolution, W8A8 (E4M3 weights with
 rounding decisions, E4M3 activations), input FP32 NCHW [64,128,32,32] -> 128
 channels, through the C-ABI library on the GPU.  A step is one fpq_conv2d call
 (activation quantize + contraction + dequantize/bias); weights are encoded once
-before the timed region (the encode's own time is reported separately).  Between
-timed steps a 256 MiB buffer is written so that every step starts with a cold
-L2.  With N > 1 (torchrun) every rank runs its own copy of the layer on its own
+before the timed region (the encode's own time is reported separately).  The
+steps rotate over several resident copies of (input, scratch, output) whose total
+size is a multiple of the L2, so every step reads its input from HBM and its
+writes push earlier steps' outputs out to HBM (inputs larger than L2); the K
+timed steps are replayed as one CUDA graph so that host launch time is not part
+of the number.  With N > 1 (torchrun) every rank runs its own copy of the layer on its own
 batch: weak scaling, no collective on the data path.
 
 Reference arm (--impl reference): the CPU oracle, as it stands, on a bounded
@@ -30,6 +33,9 @@ METRIC = "W8A8 and W4A8 quantized-layer TFLOP/s on 1 B200 and % of dense FP8/FP4
 WORKLOAD = "ddim_cifar_conv3x3_w8a8: x fp32 NCHW [64,128,32,32] SiLU(N(0,1)), w [128,128,3,3] e4m3 + rounding bits, pad 1"
 NOMINAL_FP8_TFLOPS = 4500.0
 NOMINAL_FP4_TFLOPS = 9000.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
+# profiles/ (None until a capture of the current kernel exists)
+TRAFFIC = {}
 
 
 def load_peaks():
@@ -128,7 +134,7 @@ class ClockSampler(threading.Thread):
                         self.reasons.add(name)
             except Exception:
                 pass
-            time.sleep(0.002)
+            time.sleep(0.0005)
 
     def stop(self):
         self._stop_evt.set()
@@ -152,9 +158,11 @@ def physical_gpu_index(local: int) -> int:
 # own arm
 # ---------------------------------------------------------------------------------------------
 class ConvLayerOnGpu:
-    """Device-resident tensors of one conv layer, weights already encoded."""
+    """Device-resident tensors of one conv layer, weights already encoded.  Activations,
+    scratch and outputs exist in several copies whose total size is a multiple of the L2;
+    every call moves on to the next copy."""
 
-    def __init__(self, L, fpq, torch, dev):
+    def __init__(self, L, fpq, torch, dev, l2_bytes=128 << 20):
         import numpy as np
         self.L, self.fpq, self.torch = L, fpq, torch
         self.fw = fpq.E4M3 if L.wfmt == "e4m3" else fpq.E2M1
@@ -165,12 +173,21 @@ class ConvLayerOnGpu:
         self.rb = None
         if L.bits is not None:
             self.rb = torch.from_numpy(np.packbits(L.bits, axis=1, bitorder="little")).to(dev)
-        self.x = torch.from_numpy(L.x).to(dev)
         self.bias = torch.from_numpy(L.bias).to(dev)
-        self.y = torch.empty((L.B, L.N, L.Ho, L.Wo), dtype=torch.float32, device=dev)
         self.ws_bytes = fpq.fpq_conv2d_workspace_size(L.B, L.C, L.H, L.W, L.N, L.R, L.S, L.pad, L.stride, fpq.E4M3, self.fw)
-        self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
+        self.set_bytes = 4 * L.x.size + 4 * L.M * L.N + self.ws_bytes
+        self.nsets = max(2, -(-3 * l2_bytes // self.set_bytes))        # >= 3 x L2 in rotation
+        x0 = torch.from_numpy(L.x).to(dev)
+        self.xs_ = [x0] + [x0.clone() for _ in range(self.nsets - 1)]
+        self.ys_ = [torch.empty((L.B, L.N, L.Ho, L.Wo), dtype=torch.float32, device=dev) for _ in range(self.nsets)]
+        self.wss_ = [torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev) for _ in range(self.nsets)]
+        self.i = 0
+        self._rot()
         self.encode()
+
+    def _rot(self):
+        self.i = (self.i + 1) % self.nsets
+        self.x, self.y, self.workspace = self.xs_[self.i], self.ys_[self.i], self.wss_[self.i]
 
     def encode(self):
         f, L = self.fpq, self.L
@@ -179,15 +196,18 @@ class ConvLayerOnGpu:
 
     def step(self):
         f, L = self.fpq, self.L
+        self._rot()
         f.fpq_conv2d(self.x, self.prep, self.ws, self.xs, f.E4M3, self.fw, self.bias, L.N, L.R, L.S, L.pad, L.stride,
                      y=self.y, workspace=self.workspace)
 
     def stage1(self):
         f, L = self.fpq, self.L
+        self._rot()
         f.fpq_conv2d_quantize_input(self.x, self.xs, f.E4M3, self.fw, L.N, L.R, L.S, L.pad, L.stride, self.workspace)
 
     def stage2(self):
         f, L = self.fpq, self.L
+        self._rot()
         f.fpq_conv2d_contract(self.workspace, self.prep, self.ws, self.xs, f.E4M3, self.fw, self.bias, self.y,
                               (L.B, L.C, L.H, L.W), L.R, L.S, L.pad, L.stride)
 
@@ -198,30 +218,47 @@ class ConvLayerOnGpu:
         return 4 * L.x.size + wbytes + 4 * L.M * L.N + 8 * L.N
 
     def stage1_bytes(self):
-        L = self.L
-        return 4 * L.x.size + L.B * L.H * L.W * ((L.C + 15) // 16 * 16)
+        return 4 * self.L.x.size + self.ws_bytes
 
     def stage2_bytes(self):
         L = self.L
         wbytes = L.N * L.K * (1 if L.wfmt == "e4m3" else 0.5)
-        return L.B * L.H * L.W * ((L.C + 15) // 16 * 16) + wbytes + 4 * L.M * L.N + 8 * L.N
+        return self.ws_bytes + wbytes + 4 * L.M * L.N + 8 * L.N
 
 
-def timed_steps(torch, fn, flush, n, pre=None):
-    """n calls of fn, each after an L2 flush (and an untimed `pre`), each bracketed by CUDA events
-    on the current stream.  Returns the list of per-call milliseconds."""
-    evs = []
-    for _ in range(n):
-        flush.zero_()
-        if pre is not None:
-            pre()
+class GraphOf:
+    """n calls of fn captured once into a CUDA graph (the library only enqueues kernels, so the
+    capture sees every launch); replay() then costs no per-launch host time."""
+
+    def __init__(self, torch, fn, n):
+        self.torch, self.n = torch, n
+        self.g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()                                   # first call outside the capture (one-time set-up)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(self.g, stream=side):
+                for _ in range(n):
+                    fn()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+
+    def timed_replay(self):
+        """Milliseconds of one replay, CUDA events on the launching stream."""
+        torch = self.torch
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        fn()
+        self.g.replay()
         e1.record()
-        evs.append((e0, e1))
-    torch.cuda.synchronize()
-    return [a.elapsed_time(b) for a, b in evs]
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+
+def per_launch_us(torch, fn, n, reps=3):
+    g = GraphOf(torch, fn, n)
+    g.timed_replay()
+    return min(g.timed_replay() for _ in range(reps)) * 1e3 / n
 
 
 def run_own(args):
@@ -250,25 +287,27 @@ def run_own(args):
     if world > 1:                       # every rank its own batch of the same law
         L = I.draw(L, 2, 100 * rank, "silu", 0.03, True)
     layer = ConvLayerOnGpu(L, fpq, torch, dev)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- timed region: K steps, device time per step, max over ranks
-    timed_steps(torch, layer.step, flush, args.warmup)
+    # ---- timed region: W warm-up steps, then exactly K steps replayed as one CUDA graph
+    for _ in range(args.warmup):
+        layer.step()
+    torch.cuda.synchronize()
+    steps_graph = GraphOf(torch, layer.step, args.steps)
+    steps_graph.timed_replay()                         # untimed: graph upload, clocks, L2 turnover
     sampler = ClockSampler(physical_gpu_index(local))
     barrier()
     sampler.start()
-    ms = timed_steps(torch, layer.step, flush, args.steps)
+    total_ms = steps_graph.timed_replay()
     barrier()
     clocks = sampler.stop()
     st = fpq.fpq_read_status()
     if st != fpq.OK:
         raise SystemExit(f"device status after the timed region: {fpq.status_string(st)}")
-    total_ms = sum(ms)
     if world > 1:
         t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -276,36 +315,48 @@ def run_own(args):
     flops_step = L.flops
     value = world * flops_step * args.steps / (total_ms * 1e-3) / 1e12
     launches_per_step = 2
+    t_layer = total_ms * 1e-3 / args.steps
 
-    # ---- per-kernel durations in place (stage 2 right after stage 1, as in the layer call)
-    k = max(10, min(args.steps, 100))
-    ms_q = timed_steps(torch, layer.stage1, flush, k)
-    ms_c = timed_steps(torch, layer.stage2, flush, k, pre=layer.stage1)
-    t_q, t_c = statistics.mean(ms_q) * 1e-3, statistics.mean(ms_c) * 1e-3
+    # ---- per-kernel durations: each kernel alone, n launches rotating over the same buffer sets
+    n_k = 10 * layer.nsets
+    t_q = per_launch_us(torch, layer.stage1, n_k) * 1e-6
+    t_c = per_launch_us(torch, layer.stage2, n_k) * 1e-6
     if t_c >= t_q:
         dom, t_dom, b_dom = "fpq_gemm_kernel (contraction + epilogue)", t_c, layer.stage2_bytes()
     else:
         dom, t_dom, b_dom = "quantize_nchw_to_nhwc_e4m3_kernel (activation quantize)", t_q, layer.stage1_bytes()
     achieved = b_dom / t_dom / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
+                "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": TRAFFIC.get(dom),
                 "algorithmic_bytes_per_launch": b_dom, "us_per_launch": t_dom * 1e6,
-                "kernels_us": {"activation_quantize": t_q * 1e6, "contraction": t_c * 1e6}}
-    t_layer = statistics.mean(ms) * 1e-3
+                "kernels_us": {"activation_quantize": t_q * 1e6, "contraction": t_c * 1e6},
+                "how": "each kernel replayed alone from a CUDA graph over the rotating buffer sets"}
     layer_roof = {"algorithmic_bytes": layer.layer_bytes(), "achieved_gbs": layer.layer_bytes() / t_layer / 1e9,
                   "frac_of_hbm_peak": layer.layer_bytes() / t_layer / 1e9 / peaks["hbm_gbs"],
                   "t_hbm_us": layer.layer_bytes() / (peaks["hbm_gbs"] * 1e9) * 1e6,
                   "t_tensor_us_nominal_fp8": flops_step / (NOMINAL_FP8_TFLOPS * 1e12) * 1e6}
 
+    # ---- the same K steps launched one by one from the host (launch-bound), for comparison
+    evs = []
+    for _ in range(min(args.steps, 200)):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        layer.step()
+        e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    eager_us = statistics.median(a.elapsed_time(b) for a, b in evs) * 1e3
+
     # ---- weight encode (offline step), reported beside the metric
-    ms_enc = timed_steps(torch, layer.encode, flush, 10)
+    enc_us = per_launch_us(torch, layer.encode, 20)
 
     # ---- end to end through the host-buffer C-ABI call
     xh = torch.from_numpy(L.x).pin_memory()
-    yh = torch.empty(layer.y.shape, dtype=torch.float32).pin_memory()
+    yh = torch.empty(layer.ys_[0].shape, dtype=torch.float32).pin_memory()
     n_e2e = max(3, min(args.steps, 20))
 
     def e2e_call():
+        layer._rot()
         fpq.fpq_conv2d_host(xh, layer.x, layer.prep, layer.ws, layer.xs, fpq.E4M3, layer.fw, layer.bias, layer.y, yh,
                             L.R, L.S, L.pad, L.stride, layer.workspace)
 
@@ -330,14 +381,15 @@ def run_own(args):
         w4 = {}
         for L4 in I.config3():
             l4 = ConvLayerOnGpu(L4, fpq, torch, dev)
-            timed_steps(torch, l4.step, flush, 3)
-            m4 = timed_steps(torch, l4.step, flush, max(10, min(args.steps, 50)))
-            t4 = statistics.mean(m4) * 1e-3
+            for _ in range(3):
+                l4.step()
+            t4 = per_launch_us(torch, l4.step, 5 * l4.nsets) * 1e-6
             w4[L4.name] = {"tflops": L4.flops / t4 / 1e12, "us": t4 * 1e6,
                            "pct_dense_fp8_nominal": 100 * L4.flops / t4 / 1e12 / NOMINAL_FP8_TFLOPS,
                            "pct_dense_fp4_nominal": 100 * L4.flops / t4 / 1e12 / NOMINAL_FP4_TFLOPS,
                            "layer_frac_of_hbm_peak": l4.layer_bytes() / t4 / 1e9 / peaks["hbm_gbs"]}
             del l4
+            torch.cuda.empty_cache()
 
     # ---- CPU baseline: the oracle, as it stands, on the host cores (rank 0, N = 1 only)
     cpu = None
@@ -352,14 +404,17 @@ def run_own(args):
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "e4m3 x e4m3 -> f32", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "l2": "flushed between steps (256 MiB write)",
-                       "path": "two kernels: activation quantize to channels-last codes, then TMA/tcgen05 implicit GEMM"},
+            "config": {"workload": WORKLOAD,
+                       "l2": f"inputs larger than L2: steps rotate over {layer.nsets} resident (x, scratch, y) sets, "
+                             f"{layer.nsets * layer.set_bytes >> 20} MiB",
+                       "launch": "the K timed steps are one CUDA graph replay",
+                       "path": "two kernels per step: activation quantize to framed channels-last codes, "
+                               "then the persistent TMA/tcgen05 implicit GEMM with fused dequantize + bias"},
             "pct_dense_fp8_peak_nominal": 100 * value / world / NOMINAL_FP8_TFLOPS,
             "pct_dense_fp8_peak_2x_measured_bf16": 100 * value / world / (2 * peaks["bf16_tflops"]),
             "roofline": roofline, "layer_roofline": layer_roof, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
-            "weight_encode_us": statistics.mean(ms_enc) * 1e3, "w4a8": w4,
-            "step_us": {"median": statistics.median(ms) * 1e3, "min": min(ms) * 1e3},
+            "weight_encode_us": enc_us, "w4a8": w4, "eager_step_us": eager_us,
         }
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -369,7 +424,7 @@ def run_own(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline leg")
