@@ -238,9 +238,10 @@ fpq_status fpq_linear_quantize_input(const float* x, float x_scale, fpq_format f
                : FPQ_ERR_CUDA;
 }
 
-fpq_status fpq_linear_contract(const void* workspace, size_t ws_bytes, const void* w_prepared, const float* w_scale,
-                               float x_scale, fpq_format fx, fpq_format fw, const float* bias, float* y, int64_t M,
-                               int64_t N, int64_t K, void* stream)
+static fpq_status linear_contract_impl(const void* workspace, size_t ws_bytes, const void* w_prepared,
+                                       const float* w_scale, float x_scale, fpq_format fx, fpq_format fw,
+                                       const float* bias, float* y, int64_t M, int64_t N, int64_t K, void* stream,
+                                       int after_stage1)
 {
     bool empty = false;
     fpq_status s = linear_checks(fx, fw, M, N, K, workspace, ws_bytes, &empty);
@@ -254,6 +255,7 @@ fpq_status fpq_linear_contract(const void* workspace, size_t ws_bytes, const voi
         return FPQ_ERR_CUDA;
     GemmProblem p{};
     p.conv = 0;
+    p.after_stage1 = after_stage1;
     p.w4 = is_e2m1(fw) ? 1 : 0;
     p.M = M;
     p.N = (int)N;
@@ -270,6 +272,13 @@ fpq_status fpq_linear_contract(const void* workspace, size_t ws_bytes, const voi
     p.bias = bias;
     p.y = y;
     return launch_gemm(p, (cudaStream_t)stream);
+}
+
+fpq_status fpq_linear_contract(const void* workspace, size_t ws_bytes, const void* w_prepared, const float* w_scale,
+                               float x_scale, fpq_format fx, fpq_format fw, const float* bias, float* y, int64_t M,
+                               int64_t N, int64_t K, void* stream)
+{
+    return linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream, 0);
 }
 
 fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_scale, float x_scale, fpq_format fx,
@@ -289,7 +298,7 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
     s = fpq_linear_quantize_input(x, x_scale, fx, fw, M, N, K, workspace, ws_bytes, stream);
     if (s != FPQ_OK)
         return s;
-    return fpq_linear_contract(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream);
+    return linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream, 1);
 }
 
 static fpq_status conv_shape(int B, int C, int H, int W, int C_out, int R, int S, int pad, int stride, int* Ho,
@@ -358,9 +367,10 @@ fpq_status fpq_conv2d_quantize_input(const float* x, float x_scale, fpq_format f
                : FPQ_ERR_CUDA;
 }
 
-fpq_status fpq_conv2d_contract(const void* workspace, size_t ws_bytes, const void* w_prepared, const float* w_scale,
-                               float x_scale, fpq_format fx, fpq_format fw, const float* bias, float* y, int B, int C,
-                               int H, int W, int C_out, int R, int S, int pad, int stride, void* stream)
+static fpq_status conv2d_contract_impl(const void* workspace, size_t ws_bytes, const void* w_prepared,
+                                       const float* w_scale, float x_scale, fpq_format fx, fpq_format fw,
+                                       const float* bias, float* y, int B, int C, int H, int W, int C_out, int R,
+                                       int S, int pad, int stride, void* stream, int after_stage1)
 {
     int Ho, Wo;
     bool empty = false;
@@ -375,6 +385,7 @@ fpq_status fpq_conv2d_contract(const void* workspace, size_t ws_bytes, const voi
         return FPQ_ERR_CUDA;
     GemmProblem p{};
     p.conv = 1;
+    p.after_stage1 = after_stage1;
     p.w4 = is_e2m1(fw) ? 1 : 0;
     p.M = (int64_t)B * Ho * Wo;
     p.N = C_out;
@@ -398,6 +409,14 @@ fpq_status fpq_conv2d_contract(const void* workspace, size_t ws_bytes, const voi
     return launch_gemm(p, (cudaStream_t)stream);
 }
 
+fpq_status fpq_conv2d_contract(const void* workspace, size_t ws_bytes, const void* w_prepared, const float* w_scale,
+                               float x_scale, fpq_format fx, fpq_format fw, const float* bias, float* y, int B, int C,
+                               int H, int W, int C_out, int R, int S, int pad, int stride, void* stream)
+{
+    return conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out,
+                                R, S, pad, stride, stream, 0);
+}
+
 fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_scale, float x_scale, fpq_format fx,
                       fpq_format fw, const float* bias, float* y, int B, int C, int H, int W, int C_out, int R, int S,
                       int pad, int stride, void* workspace, size_t ws_bytes, void* stream)
@@ -416,8 +435,8 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
                                   stream);
     if (s != FPQ_OK)
         return s;
-    return fpq_conv2d_contract(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out, R,
-                               S, pad, stride, stream);
+    return conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out,
+                                R, S, pad, stride, stream, 1);
 }
 
 fpq_status fpq_linear_host(const float* x_host, float* x_dev, const void* w_prepared, const float* w_scale,

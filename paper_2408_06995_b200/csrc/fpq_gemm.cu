@@ -85,6 +85,7 @@ struct GemmArgs {
     float* y;
     int* status;
     uint32_t idesc;
+    int wait_prior_grid;       // launched with programmatic stream serialization behind the quantize kernel
 };
 
 template <int BN>
@@ -154,6 +155,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
             uint32_t na = 0, nb = 0;                   // stages issued (for the abort path)
             int resident_nt = -1;
             bool dead = false;
+            bool prior_done = !g.wait_prior_grid;
             for (int t = blockIdx.x; t < total_tiles && !dead; t += gridDim.x) {
                 int mt, nt;
                 decode_tile(t, mt, nt);
@@ -170,7 +172,27 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
                 resident_nt = nt;
                 int cc = 0, tap = 0, r = 0, sx = 0;    // block j = (cc, tap), tap = (r, sx)
                 int ja = 0, jb = 0;                    // position inside the current A / B stage
+                bool early_b = false;
                 for (int j = 0; j < g.nblk; ++j) {
+                    if (jb == 0 && load_b && !prior_done && g.b_resident) {
+                        // the weights do not depend on the kernel in front: fetch them before waiting for it
+                        if (!mbar_wait(b_empty + 8 * sb, pb ^ 1)) { dead = true; break; }
+                        mbar_expect_tx(b_full + 8 * sb, (uint32_t)g.nblk * g.b_block_tx);
+                        uint32_t dst = b_ring + sb * g.b_stage_bytes;
+                        int c2 = 0, t2 = 0;
+                        for (int l = 0; l < g.nblk; ++l, dst += B_BLOCK_BYTES) {
+                            tma_load_3d(dst, &tmB, b_full + 8 * sb, c2 * BK, t2, n0);
+                            if (++t2 == g.taps) { t2 = 0; ++c2; }
+                        }
+                        ++nb;
+                        if (++sb == (uint32_t)g.b_stages) { sb = 0; pb ^= 1; }
+                        early_b = true;
+                    }
+                    if (!prior_done) {
+                        // the activation codes are written by the preceding grid
+                        asm volatile("griddepcontrol.wait;" ::: "memory");
+                        prior_done = true;
+                    }
                     if (ja == 0) {
                         // activation stage: the data of the next a_span blocks
                         if (!mbar_wait(a_empty + 8 * sa, pa ^ 1)) { dead = true; break; }
@@ -194,7 +216,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
                         ++na;
                         if (++sa == (uint32_t)g.a_stages) { sa = 0; pa ^= 1; }
                     }
-                    if (jb == 0 && load_b) {
+                    if (jb == 0 && load_b && !early_b) {
                         if (!mbar_wait(b_empty + 8 * sb, pb ^ 1)) { dead = true; break; }
                         const int nblocks = min(g.b_span, g.nblk - j);
                         mbar_expect_tx(b_full + 8 * sb, (uint32_t)nblocks * g.b_block_tx);
@@ -641,8 +663,18 @@ static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB,
     }
     const int64_t tiles = (int64_t)g.m_tiles * g.n_tiles;
     const int grid = (int)(tiles < di->sms ? tiles : di->sms);
-    fpq_gemm_kernel<BN><<<grid, NUM_THREADS, dyn, st>>>(tmA, tmB, g);
-    return cudaGetLastError() == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = (size_t)dyn;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g.wait_prior_grid ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, fpq_gemm_kernel<BN>, tmA, tmB, (const GemmArgs)g) == cudaSuccess ? FPQ_OK
+                                                                                                      : FPQ_ERR_CUDA;
 }
 
 fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
@@ -666,6 +698,7 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
     g.bias = p.bias;
     g.y = p.y;
     g.status = status_word();
+    g.wait_prior_grid = p.after_stage1;
 
     const int BN = (p.N <= 64) ? 64 : 128;
     g.n_tiles = (p.N + BN - 1) / BN;

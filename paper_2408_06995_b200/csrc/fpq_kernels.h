@@ -22,6 +22,7 @@ cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, in
 // Geometry of one contraction launch (linear: taps = 1, rows of Ca codes).
 struct GemmProblem {
     int conv;            // 0 linear, 1 conv
+    int after_stage1;    // launched right behind this library's own activation-quantize kernel
     int w4;              // weights are E2M1
     int64_t M;           // linear rows
     int N;               // outputs / out channels

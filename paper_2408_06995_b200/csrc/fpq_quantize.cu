@@ -133,6 +133,7 @@ __global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const float* __
                                                                  int64_t Kp, float rinv, uint8_t* __restrict__ codes,
                                                                  int* status)
 {
+    asm volatile("griddepcontrol.launch_dependents;");
     bool nan = false;
     int64_t vec_per_row = Kp / 16;
     int64_t total = M * vec_per_row;
@@ -176,6 +177,9 @@ __global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const f
                                                                          uint8_t* __restrict__ codes, int* status)
 {
     __shared__ __align__(16) uint8_t tile[32][128 + 16];
+    // the contraction queued behind this kernel may start its set-up (it waits for this grid
+    // to finish before it reads the codes)
+    asm volatile("griddepcontrol.launch_dependents;");
     bool nan = false;
     const int HW = H * W, Wp = W + 2 * pad, Hp = H + 2 * pad;
     const int b = blockIdx.z;
