@@ -241,7 +241,7 @@ fpq_status fpq_linear_quantize_input(const float* x, float x_scale, fpq_format f
 static fpq_status linear_contract_impl(const void* workspace, size_t ws_bytes, const void* w_prepared,
                                        const float* w_scale, float x_scale, fpq_format fx, fpq_format fw,
                                        const float* bias, float* y, int64_t M, int64_t N, int64_t K, void* stream,
-                                       int after_stage1)
+                                       int after_stage1, const float* x_fused)
 {
     bool empty = false;
     fpq_status s = linear_checks(fx, fw, M, N, K, workspace, ws_bytes, &empty);
@@ -255,6 +255,8 @@ static fpq_status linear_contract_impl(const void* workspace, size_t ws_bytes, c
         return FPQ_ERR_CUDA;
     GemmProblem p{};
     p.conv = 0;
+    p.x = x_fused;
+    p.C = (int)K;
     p.after_stage1 = after_stage1;
     p.w4 = is_e2m1(fw) ? 1 : 0;
     p.M = M;
@@ -278,7 +280,8 @@ fpq_status fpq_linear_contract(const void* workspace, size_t ws_bytes, const voi
                                float x_scale, fpq_format fx, fpq_format fw, const float* bias, float* y, int64_t M,
                                int64_t N, int64_t K, void* stream)
 {
-    return linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream, 0);
+    return linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream, 0,
+                                nullptr);
 }
 
 fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_scale, float x_scale, fpq_format fx,
@@ -295,10 +298,15 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
     if (!aligned(x, 16) || !aligned(y, 16) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
         (bias && !aligned(bias, 4)))
         return FPQ_ERR_ALIGN;
+    // one kernel: the activations are quantized inside the contraction's operand staging
+    s = linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream, 0, x);
+    if (s != FPQ_ERR_UNSUPPORTED)
+        return s;
     s = fpq_linear_quantize_input(x, x_scale, fx, fw, M, N, K, workspace, ws_bytes, stream);
     if (s != FPQ_OK)
         return s;
-    return linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream, 1);
+    return linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream, 1,
+                                nullptr);
 }
 
 static fpq_status conv_shape(int B, int C, int H, int W, int C_out, int R, int S, int pad, int stride, int* Ho,
@@ -370,7 +378,8 @@ fpq_status fpq_conv2d_quantize_input(const float* x, float x_scale, fpq_format f
 static fpq_status conv2d_contract_impl(const void* workspace, size_t ws_bytes, const void* w_prepared,
                                        const float* w_scale, float x_scale, fpq_format fx, fpq_format fw,
                                        const float* bias, float* y, int B, int C, int H, int W, int C_out, int R,
-                                       int S, int pad, int stride, void* stream, int after_stage1)
+                                       int S, int pad, int stride, void* stream, int after_stage1,
+                                       const float* x_fused)
 {
     int Ho, Wo;
     bool empty = false;
@@ -385,6 +394,8 @@ static fpq_status conv2d_contract_impl(const void* workspace, size_t ws_bytes, c
         return FPQ_ERR_CUDA;
     GemmProblem p{};
     p.conv = 1;
+    p.x = x_fused;
+    p.C = C;
     p.after_stage1 = after_stage1;
     p.w4 = is_e2m1(fw) ? 1 : 0;
     p.M = (int64_t)B * Ho * Wo;
@@ -414,7 +425,7 @@ fpq_status fpq_conv2d_contract(const void* workspace, size_t ws_bytes, const voi
                                int H, int W, int C_out, int R, int S, int pad, int stride, void* stream)
 {
     return conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out,
-                                R, S, pad, stride, stream, 0);
+                                R, S, pad, stride, stream, 0, nullptr);
 }
 
 fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_scale, float x_scale, fpq_format fx,
@@ -431,12 +442,18 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
     if (!aligned(x, 4) || !aligned(y, 4) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
         (bias && !aligned(bias, 4)))
         return FPQ_ERR_ALIGN;
+    // one kernel where the geometry allows it (stride 1): the activations are quantized inside the
+    // contraction's operand staging; otherwise quantize to codes first
+    s = conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out, R,
+                             S, pad, stride, stream, 0, x);
+    if (s != FPQ_ERR_UNSUPPORTED)
+        return s;
     s = fpq_conv2d_quantize_input(x, x_scale, fx, fw, B, C, H, W, C_out, R, S, pad, stride, workspace, ws_bytes,
                                   stream);
     if (s != FPQ_OK)
         return s;
     return conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out,
-                                R, S, pad, stride, stream, 1);
+                                R, S, pad, stride, stream, 1, nullptr);
 }
 
 fpq_status fpq_linear_host(const float* x_host, float* x_dev, const void* w_prepared, const float* w_scale,

@@ -29,7 +29,9 @@ namespace fpq {
 constexpr int BM = 128;        // output rows per tile (TMEM lanes)
 constexpr int BK = 128;        // reduction elements per block (one 128-byte swizzled row)
 constexpr int NUM_EPI_WARPS = 8;   // two per TMEM lane quarter, each takes half of the columns
+constexpr int NUM_XFORM_WARPS = 8; // fused form only: quantize FP32 activations into the A ring
 constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
+constexpr int NUM_THREADS_FUSED = NUM_THREADS + 32 * NUM_XFORM_WARPS;
 constexpr int SMEM_BUDGET = 220 * 1024;
 
 enum { MODE_ROWS = 0, MODE_FLAT = 1, MODE_TAPS = 2 };
@@ -86,10 +88,111 @@ struct GemmArgs {
     int* status;
     uint32_t idesc;
     int wait_prior_grid;       // launched with programmatic stream serialization behind the quantize kernel
+    // fused form: the FP32 activations themselves (NCHW for FLAT, [M][K] for ROWS)
+    const float* x;
+    float rinv;                // 1.0f / x_scale
+    int C, H, W, pad;          // channels (ROWS: K), image size, zero padding
 };
 
-template <int BN>
-__global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
+// Fused activation-quantize prologue, NCHW source: one 128-channel chunk of the rows
+// [q0, q0 + rows) of the framed pixel list, written as E4M3 codes in the K-major,
+// 128-byte-swizzled layout the MMA reads.  Warp tw owns channels [16 tw, 16 tw + 16); its
+// lanes walk the pixel rows, so global loads are coalesced along x and each thread ends
+// with one 16-byte store (8 consecutive rows hit 8 different 16-byte columns: no bank
+// conflicts).  Frame positions and channels past C are code 0.
+__device__ __forceinline__ void fill_chunk_nchw(const GemmArgs& g, uint8_t* dst, uint32_t q0, int rows, int c_base,
+                                                int tw, int lane, bool& nan)
+{
+    const int cg = c_base + tw * 16;
+    const int HW = g.H * g.W;
+    for (int i0 = lane; i0 < rows; i0 += 64) {
+        float a[2][16];
+        bool have[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int i = i0 + 32 * u;
+            have[u] = false;
+            const uint32_t f = q0 + (uint32_t)i;
+            if (i < rows && (int64_t)f < g.M && cg < g.C) {
+                const uint32_t b = fdiv(f, g.div_HpWp);
+                const uint32_t rem = f - b * (uint32_t)g.HpWp;
+                const uint32_t yp = fdiv(rem, g.div_Wp);
+                const int y = (int)yp - g.pad, x = (int)(rem - yp * (uint32_t)g.Wp) - g.pad;
+                if ((unsigned)y < (unsigned)g.H && (unsigned)x < (unsigned)g.W) {
+                    have[u] = true;
+                    const float* p = g.x + ((int64_t)(b * (uint32_t)g.C + (uint32_t)cg) * g.H + y) * g.W + x;
+                    if (cg + 16 <= g.C) {
+#pragma unroll
+                        for (int q = 0; q < 16; ++q)
+                            a[u][q] = __ldg(p + (int64_t)q * HW);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 16; ++q)
+                            a[u][q] = (cg + q < g.C) ? __ldg(p + (int64_t)q * HW) : 0.f;
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int i = i0 + 32 * u;
+            if (i < rows) {
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (have[u]) {
+                    const float r = g.rinv;
+                    v.x = e4m3x4_from_scaled(__fmul_rn(a[u][0], r), __fmul_rn(a[u][1], r), __fmul_rn(a[u][2], r), __fmul_rn(a[u][3], r), nan);
+                    v.y = e4m3x4_from_scaled(__fmul_rn(a[u][4], r), __fmul_rn(a[u][5], r), __fmul_rn(a[u][6], r), __fmul_rn(a[u][7], r), nan);
+                    v.z = e4m3x4_from_scaled(__fmul_rn(a[u][8], r), __fmul_rn(a[u][9], r), __fmul_rn(a[u][10], r), __fmul_rn(a[u][11], r), nan);
+                    v.w = e4m3x4_from_scaled(__fmul_rn(a[u][12], r), __fmul_rn(a[u][13], r), __fmul_rn(a[u][14], r), __fmul_rn(a[u][15], r), nan);
+                }
+                *reinterpret_cast<uint4*>(dst + i * 128 + ((tw ^ (i & 7)) << 4)) = v;
+            }
+        }
+    }
+}
+
+// The same for a row-major [M][K] source: 8 consecutive threads read the 128 reduction
+// elements of one row (512 contiguous bytes), a warp covers 4 rows per pass.
+__device__ __forceinline__ void fill_chunk_rows(const GemmArgs& g, uint8_t* dst, int64_t m0, int k_base, int tid,
+                                                bool& nan)
+{
+    const bool vec = (g.C % 4) == 0;
+#pragma unroll 2
+    for (int it = 0; it < (BM * 8) / (32 * NUM_XFORM_WARPS); ++it) {
+        const int idx = it * (32 * NUM_XFORM_WARPS) + tid;
+        const int i = idx >> 3, j = idx & 7;
+        const int64_t m = m0 + i;
+        const int k = k_base + 16 * j;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (m < g.M && k < g.C) {
+            const float* p = g.x + m * g.C + k;
+            float a[16];
+            if (vec && k + 16 <= g.C) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float4 t = __ldg(reinterpret_cast<const float4*>(p) + q);
+                    a[4 * q] = t.x; a[4 * q + 1] = t.y; a[4 * q + 2] = t.z; a[4 * q + 3] = t.w;
+                }
+            } else {
+#pragma unroll
+                for (int q = 0; q < 16; ++q)
+                    a[q] = (k + q < g.C) ? __ldg(p + q) : 0.f;
+            }
+            const float r = g.rinv;
+            v.x = e4m3x4_from_scaled(__fmul_rn(a[0], r), __fmul_rn(a[1], r), __fmul_rn(a[2], r), __fmul_rn(a[3], r), nan);
+            v.y = e4m3x4_from_scaled(__fmul_rn(a[4], r), __fmul_rn(a[5], r), __fmul_rn(a[6], r), __fmul_rn(a[7], r), nan);
+            v.z = e4m3x4_from_scaled(__fmul_rn(a[8], r), __fmul_rn(a[9], r), __fmul_rn(a[10], r), __fmul_rn(a[11], r), nan);
+            v.w = e4m3x4_from_scaled(__fmul_rn(a[12], r), __fmul_rn(a[13], r), __fmul_rn(a[14], r), __fmul_rn(a[15], r), nan);
+        }
+        *reinterpret_cast<uint4*>(dst + i * 128 + ((j ^ (i & 7)) << 4)) = v;
+    }
+}
+
+// FUSED = false: the activation operand is read as codes (TMA, written by a quantize kernel).
+// FUSED = true : 8 more warps read the FP32 activations and quantize them straight into the
+//                activation ring, so the codes never exist in global memory.
+template <int BN, bool FUSED>
+__global__ void __launch_bounds__(FUSED ? NUM_THREADS_FUSED : NUM_THREADS, 1) fpq_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                                   const __grid_constant__ CUtensorMap tmB,
                                                                   const GemmArgs g)
 {
@@ -117,7 +220,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 8; ++s) {
-            mbar_init(a_full + 8 * s, 1);
+            mbar_init(a_full + 8 * s, FUSED ? NUM_XFORM_WARPS : 1);
             mbar_init(a_empty + 8 * s, 1);
             mbar_init(b_full + 8 * s, 1);
             mbar_init(b_empty + 8 * s, 1);
@@ -193,7 +296,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
                         asm volatile("griddepcontrol.wait;" ::: "memory");
                         prior_done = true;
                     }
-                    if (ja == 0) {
+                    if (ja == 0 && !FUSED) {
                         // activation stage: the data of the next a_span blocks
                         if (!mbar_wait(a_empty + 8 * sa, pa ^ 1)) { dead = true; break; }
                         const int nblocks = min(g.a_span, g.nblk - j);
@@ -408,7 +511,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
             if (dead)
                 atomicMin(g.status, FPQ_ERR_TIMEOUT);
         }
-    } else {
+    } else if (warp < 2 + NUM_EPI_WARPS) {
         // ---------------- epilogue: 8 warps; warp w reads TMEM lane quarter w % 4 and the
         // column half (w - 2) / 4 of the accumulator ----------------
         constexpr int EPI_THREADS = 32 * NUM_EPI_WARPS;
@@ -539,6 +642,40 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) fpq_gemm_kernel(const __grid_c
         }
         if (dead)
             atomicMin(g.status, FPQ_ERR_TIMEOUT);
+    } else if (FUSED) {
+        // ---------------- activation-quantize prologue: 8 warps fill the A ring ----------------
+        const int tw = warp - (2 + NUM_EPI_WARPS);
+        const int tid = threadIdx.x - 32 * (2 + NUM_EPI_WARPS);
+        const int chunks_per_stage = g.a_span / g.taps;
+        const int rows = g.a_chunk_bytes >> 7;
+        uint32_t sa = 0, pa = 0;
+        bool dead = false, nan = false;
+        for (int t = blockIdx.x; t < total_tiles && !dead; t += gridDim.x) {
+            int mt, nt;
+            decode_tile(t, mt, nt);
+            for (int cc = 0; cc < g.cchunks;) {
+                if (!mbar_wait(a_empty + 8 * sa, pa ^ 1)) { dead = true; break; }
+                const int nch = min(chunks_per_stage, g.cchunks - cc);
+                uint8_t* dst = smem + sa * g.a_stage_bytes;
+                for (int l = 0; l < nch; ++l, dst += g.a_chunk_bytes) {
+                    if (g.mode == MODE_ROWS)
+                        fill_chunk_rows(g, dst, (int64_t)mt * BM, (cc + l) * BK, tid, nan);
+                    else
+                        fill_chunk_nchw(g, dst, (uint32_t)mt * BM, rows, (cc + l) * BK, tw, lane, nan);
+                }
+                // make the generic-proxy writes visible to the tensor core's reads, then signal
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0)
+                    mbar_arrive(a_full + 8 * sa);
+                if (++sa == (uint32_t)g.a_stages) { sa = 0; pa ^= 1; }
+                cc += nch;
+            }
+        }
+        if (nan)
+            atomicMin(g.status, FPQ_ERR_NAN_INPUT);
+        if (dead)
+            atomicMin(g.status, FPQ_ERR_TIMEOUT);
     }
 
     tc_fence_before();
@@ -577,7 +714,7 @@ static int pow2_at_least(int v)
 
 struct DeviceInfo {
     int sms;
-    bool smem_set[3];
+    bool smem_set[4];
 };
 
 static DeviceInfo* device_info()
@@ -595,7 +732,7 @@ static DeviceInfo* device_info()
     return &info[dev];
 }
 
-template <int BN>
+template <int BN, bool FUSED>
 static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs& g, cudaStream_t st)
 {
     // Split the shared-memory budget between the two rings.  A barrier handshake costs the
@@ -654,9 +791,9 @@ static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB,
         return FPQ_ERR_UNSUPPORTED;
     g.div_tiles = make_fastdiv((uint32_t)(g.m_fastest ? g.m_tiles : g.n_tiles));
     const int dyn = g.a_stages * g.a_stage_bytes + g.b_stages * g.b_stage_bytes + ctl;
-    const int slot = BN == 64 ? 0 : (BN == 128 ? 1 : 2);
+    const int slot = (BN == 64 ? 0 : 1) + (FUSED ? 2 : 0);
     if (!di->smem_set[slot]) {
-        if (cudaFuncSetAttribute(fpq_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) !=
+        if (cudaFuncSetAttribute(fpq_gemm_kernel<BN, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) !=
             cudaSuccess)
             return FPQ_ERR_CUDA;
         di->smem_set[slot] = true;
@@ -665,7 +802,7 @@ static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB,
     const int grid = (int)(tiles < di->sms ? tiles : di->sms);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.blockDim = dim3(FUSED ? NUM_THREADS_FUSED : NUM_THREADS);
     cfg.dynamicSmemBytes = (size_t)dyn;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -673,7 +810,7 @@ static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = g.wait_prior_grid ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, fpq_gemm_kernel<BN>, tmA, tmB, (const GemmArgs)g) == cudaSuccess ? FPQ_OK
+    return cudaLaunchKernelEx(&cfg, fpq_gemm_kernel<BN, FUSED>, tmA, tmB, (const GemmArgs)g) == cudaSuccess ? FPQ_OK
                                                                                                       : FPQ_ERR_CUDA;
 }
 
@@ -798,9 +935,20 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return FPQ_ERR_CUDA;
 
-    if (BN == 64)
-        return launch_variant<64>(tmA, tmB, g, st);
-    return launch_variant<128>(tmA, tmB, g, st);
+    const bool fused = p.x != nullptr && g.mode != MODE_TAPS;
+    if (fused) {
+        g.x = p.x;
+        g.rinv = 1.0f / p.x_scale;
+        g.C = p.C;
+        g.H = p.H;
+        g.W = p.W;
+        g.pad = p.pad;
+        g.wait_prior_grid = 0;
+        return BN == 64 ? launch_variant<64, true>(tmA, tmB, g, st) : launch_variant<128, true>(tmA, tmB, g, st);
+    }
+    if (p.x != nullptr)
+        return FPQ_ERR_UNSUPPORTED;     // the caller falls back to the two-kernel route
+    return BN == 64 ? launch_variant<64, false>(tmA, tmB, g, st) : launch_variant<128, false>(tmA, tmB, g, st);
 }
 
 }  // namespace fpq

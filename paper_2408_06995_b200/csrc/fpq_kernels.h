@@ -30,7 +30,9 @@ struct GemmProblem {
     int Ca;              // padded channels (row length) of the activation codes (multiple of 16)
     int B, H, W, Ho, Wo; // conv geometry
     int R, S, pad, stride;
-    const uint8_t* a_codes;   // [M][Ca] or [B][H][W][Ca]
+    const uint8_t* a_codes;   // [M][Ca] or framed [B][Hp][Wp][Ca]; unused by the fused form
+    const float* x;           // fused form: FP32 activations ([M][C] or NCHW); NULL = read a_codes
+    int C;                    // fused form: channels / reduction length of x
     const void* w_prepared;   // [N][R*S][Cp]
     const float* w_scale;
     float x_scale;

@@ -169,3 +169,56 @@ def test_config3_full_size_sampled():
 def test_config4_full_size_sampled():
     for j, L in enumerate(I.config4()):
         _check_sampled(L, 1 << 12, 10 + j)
+
+
+# ---- the two-kernel route (activation codes in a workspace, then the contraction) ---------------
+
+def _staged(L, ws, xs):
+    gfw, _ = FMT[L.wfmt]
+    _, prep = gpu_prepare(L, ws)
+    x = torch.from_numpy(L.x).cuda()
+    bias = torch.from_numpy(L.bias).cuda()
+    wsd = torch.from_numpy(ws).cuda()
+    if L.kind == "linear":
+        wk = torch.empty(max(1, fpq.fpq_linear_workspace_size(L.M, L.N, L.K, fpq.E4M3, gfw)), dtype=torch.uint8, device="cuda")
+        y = torch.empty((L.M, L.N), dtype=torch.float32, device="cuda")
+        fpq.fpq_linear_quantize_input(x, xs, fpq.E4M3, gfw, L.N, wk)
+        fpq.fpq_linear_contract(wk, prep, wsd, xs, fpq.E4M3, gfw, bias, y, L.K)
+    else:
+        wk = torch.empty(max(1, fpq.fpq_conv2d_workspace_size(L.B, L.C, L.H, L.W, L.N, L.R, L.S, L.pad, L.stride,
+                                                               fpq.E4M3, gfw)), dtype=torch.uint8, device="cuda")
+        y = torch.empty((L.B, L.N, L.Ho, L.Wo), dtype=torch.float32, device="cuda")
+        fpq.fpq_conv2d_quantize_input(x, xs, fpq.E4M3, gfw, L.N, L.R, L.S, L.pad, L.stride, wk)
+        fpq.fpq_conv2d_contract(wk, prep, wsd, xs, fpq.E4M3, gfw, bias, y, (L.B, L.C, L.H, L.W), L.R, L.S, L.pad, L.stride)
+    assert fpq.fpq_read_status() == fpq.OK
+    return y.cpu().numpy(), wk.cpu().numpy()
+
+
+@pytest.mark.parametrize("wfmt", ["e4m3", "e2m1"])
+def test_two_kernel_route_matches_the_oracle_and_the_fused_call(wfmt):
+    layers = [
+        I.draw(I.linear_layer("l", 300, 320, 200, wfmt, rounding=True), 13, 0, "normal", 0.02, True),
+        I.draw(I.linear_layer("l2", 130, 1000, 72, wfmt), 13, 10, "normal", 0.02, True),
+        I.draw(I.conv_layer("c", 3, 20, 9, 7, 37, 3, wfmt=wfmt, rounding=True), 13, 20, "silu", 0.03, True),
+        I.draw(I.conv_layer("c2", 2, 130, 16, 16, 140, 1, wfmt=wfmt), 13, 30, "silu", 0.03, True),
+        I.draw(I.conv_layer("c3", 2, 32, 16, 16, 24, 3, stride=2, wfmt=wfmt), 13, 40, "silu", 0.03, True),
+    ]
+    for L in layers:
+        ws, xs = layer_scales(L)
+        y2, codes = _staged(L, ws, xs)
+        yr, ab = oracle_layer(L, ws, xs)
+        assert_close(y2, yr, ab)
+        assert np.array_equal(y2, gpu_layer(L, ws, xs))      # same MMAs in the same order
+        # the codes in the workspace are the oracle's, in the operand layout
+        want = O.quantize_act(L.x, xs, O.E4M3)
+        if L.kind == "linear":
+            Kp = (L.K + 15) // 16 * 16
+            got = codes[: L.M * Kp].reshape(L.M, Kp)
+            assert np.array_equal(got[:, : L.K], want) and not got[:, L.K:].any()
+        else:
+            Cp = (L.C + 15) // 16 * 16
+            Hp, Wp = L.H + 2 * L.pad, L.W + 2 * L.pad
+            got = codes[: L.B * Hp * Wp * Cp].reshape(L.B, Hp, Wp, Cp)
+            inner = got[:, L.pad:L.pad + L.H, L.pad:L.pad + L.W, : L.C]
+            assert np.array_equal(inner, want.transpose(0, 2, 3, 1))
+            assert got.sum() == inner.sum()                    # frame and channel padding are code 0
