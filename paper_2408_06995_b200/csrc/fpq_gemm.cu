@@ -28,10 +28,16 @@ namespace fpq {
 
 constexpr int BM = 128;        // output rows per tile (TMEM lanes)
 constexpr int BK = 128;        // reduction elements per block (one 128-byte swizzled row)
-constexpr int NUM_EPI_WARPS = 8;   // two per TMEM lane quarter, each takes half of the columns
-constexpr int NUM_XFORM_WARPS = 8; // fused form only: quantize FP32 activations into the A ring
-constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
-constexpr int NUM_THREADS_FUSED = NUM_THREADS + 32 * NUM_XFORM_WARPS;
+// Warp roles.  Plain form: producer, MMA issuer, 8 epilogue warps (two per TMEM lane quarter,
+// each half of the columns).  Fused form: producer, MMA issuer, 4 epilogue warps and 16
+// transform warps that quantize FP32 activations into the A ring - the conversion is bound by
+// instruction issue, so it gets most of the SM's warps.
+constexpr int NUM_XFORM_WARPS = 16;
+__host__ __device__ constexpr int epi_warps(bool fused) { return fused ? 4 : 8; }
+__host__ __device__ constexpr int num_threads(bool fused)
+{
+    return 64 + 32 * epi_warps(fused) + (fused ? 32 * NUM_XFORM_WARPS + 32 : 0);   // + one L2-prefetch warp
+}
 constexpr int SMEM_BUDGET = 220 * 1024;
 
 enum { MODE_ROWS = 0, MODE_FLAT = 1, MODE_TAPS = 2 };
@@ -96,58 +102,92 @@ struct GemmArgs {
 
 // Fused activation-quantize prologue, NCHW source: one 128-channel chunk of the rows
 // [q0, q0 + rows) of the framed pixel list, written as E4M3 codes in the K-major,
-// 128-byte-swizzled layout the MMA reads.  Warp tw owns channels [16 tw, 16 tw + 16); its
+// 128-byte-swizzled layout the MMA reads.  Warp tw owns channels [16 (tw % 8), +16) of every other 32-row batch; its
 // lanes walk the pixel rows, so global loads are coalesced along x and each thread ends
-// with one 16-byte store (8 consecutive rows hit 8 different 16-byte columns: no bank
-// conflicts).  Frame positions and channels past C are code 0.
+// with one 16-byte store per row (8 consecutive rows hit 8 different 16-byte columns: no
+// bank conflicts).  Frame positions and channels past C are code 0.  The loads of the next
+// row are issued before the current one is converted.
+struct NchwRows {
+    const GemmArgs& g;
+    uint32_t q0;
+    int rows, cg, HW;
+    // source address of channel cg at pixel row i, or nullptr for a frame / out-of-range row
+    __device__ __forceinline__ const float* src(int i) const
+    {
+        const uint32_t f = q0 + (uint32_t)i;
+        if (i >= rows || (int64_t)f >= g.M || cg >= g.C)
+            return nullptr;
+        const uint32_t b = fdiv(f, g.div_HpWp);
+        const uint32_t rem = f - b * (uint32_t)g.HpWp;
+        const uint32_t yp = fdiv(rem, g.div_Wp);
+        const int y = (int)yp - g.pad, x = (int)(rem - yp * (uint32_t)g.Wp) - g.pad;
+        if ((unsigned)y >= (unsigned)g.H || (unsigned)x >= (unsigned)g.W)
+            return nullptr;
+        return g.x + ((int64_t)(b * (uint32_t)g.C + (uint32_t)cg) * g.H + y) * g.W + x;
+    }
+    __device__ __forceinline__ void load(float (&a)[16], const float* p) const
+    {
+        if (cg + 16 <= g.C) {
+#pragma unroll
+            for (int q = 0; q < 16; ++q)
+                a[q] = __ldcg(p + (int64_t)q * HW);
+        } else {
+#pragma unroll
+            for (int q = 0; q < 16; ++q)
+                a[q] = (cg + q < g.C) ? __ldcg(p + (int64_t)q * HW) : 0.f;
+        }
+    }
+};
+
+// Sixteen codes for the MMA operand.  Unlike codes that are stored, a minus zero may stay:
+// as an operand it only ever contributes a signed zero to the sum.  NaN still becomes code 0.
+__device__ __forceinline__ uint32_t e4m3x4_operand(float t0, float t1, float t2, float t3, bool& nan)
+{
+    uint16_t lo, hi;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(t1), "f"(t0));
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(t3), "f"(t2));
+    const uint32_t v = (uint32_t)lo | ((uint32_t)hi << 16);
+    const uint32_t nan_bytes = ((v & 0x7f7f7f7fu) + 0x01010101u) & 0x80808080u;
+    if (nan_bytes) {
+        nan = true;
+        return v & ~((nan_bytes >> 7) * 0xffu);
+    }
+    return v;
+}
+
+__device__ __forceinline__ uint4 e4m3x16(const float (&a)[16], float r, bool& nan)
+{
+    uint4 v;
+    v.x = e4m3x4_operand(__fmul_rn(a[0], r), __fmul_rn(a[1], r), __fmul_rn(a[2], r), __fmul_rn(a[3], r), nan);
+    v.y = e4m3x4_operand(__fmul_rn(a[4], r), __fmul_rn(a[5], r), __fmul_rn(a[6], r), __fmul_rn(a[7], r), nan);
+    v.z = e4m3x4_operand(__fmul_rn(a[8], r), __fmul_rn(a[9], r), __fmul_rn(a[10], r), __fmul_rn(a[11], r), nan);
+    v.w = e4m3x4_operand(__fmul_rn(a[12], r), __fmul_rn(a[13], r), __fmul_rn(a[14], r), __fmul_rn(a[15], r), nan);
+    return v;
+}
+
 __device__ __forceinline__ void fill_chunk_nchw(const GemmArgs& g, uint8_t* dst, uint32_t q0, int rows, int c_base,
                                                 int tw, int lane, bool& nan)
 {
-    const int cg = c_base + tw * 16;
-    const int HW = g.H * g.W;
-    for (int i0 = lane; i0 < rows; i0 += 64) {
-        float a[2][16];
-        bool have[2];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int i = i0 + 32 * u;
-            have[u] = false;
-            const uint32_t f = q0 + (uint32_t)i;
-            if (i < rows && (int64_t)f < g.M && cg < g.C) {
-                const uint32_t b = fdiv(f, g.div_HpWp);
-                const uint32_t rem = f - b * (uint32_t)g.HpWp;
-                const uint32_t yp = fdiv(rem, g.div_Wp);
-                const int y = (int)yp - g.pad, x = (int)(rem - yp * (uint32_t)g.Wp) - g.pad;
-                if ((unsigned)y < (unsigned)g.H && (unsigned)x < (unsigned)g.W) {
-                    have[u] = true;
-                    const float* p = g.x + ((int64_t)(b * (uint32_t)g.C + (uint32_t)cg) * g.H + y) * g.W + x;
-                    if (cg + 16 <= g.C) {
-#pragma unroll
-                        for (int q = 0; q < 16; ++q)
-                            a[u][q] = __ldg(p + (int64_t)q * HW);
-                    } else {
-#pragma unroll
-                        for (int q = 0; q < 16; ++q)
-                            a[u][q] = (cg + q < g.C) ? __ldg(p + (int64_t)q * HW) : 0.f;
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int i = i0 + 32 * u;
-            if (i < rows) {
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (have[u]) {
-                    const float r = g.rinv;
-                    v.x = e4m3x4_from_scaled(__fmul_rn(a[u][0], r), __fmul_rn(a[u][1], r), __fmul_rn(a[u][2], r), __fmul_rn(a[u][3], r), nan);
-                    v.y = e4m3x4_from_scaled(__fmul_rn(a[u][4], r), __fmul_rn(a[u][5], r), __fmul_rn(a[u][6], r), __fmul_rn(a[u][7], r), nan);
-                    v.z = e4m3x4_from_scaled(__fmul_rn(a[u][8], r), __fmul_rn(a[u][9], r), __fmul_rn(a[u][10], r), __fmul_rn(a[u][11], r), nan);
-                    v.w = e4m3x4_from_scaled(__fmul_rn(a[u][12], r), __fmul_rn(a[u][13], r), __fmul_rn(a[u][14], r), __fmul_rn(a[u][15], r), nan);
-                }
-                *reinterpret_cast<uint4*>(dst + i * 128 + ((tw ^ (i & 7)) << 4)) = v;
-            }
-        }
+    const int cgrp = tw & 7;
+    const NchwRows R{g, q0, rows, c_base + cgrp * 16, g.H * g.W};
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    float a[16], b[16];
+    int i = lane + 32 * (tw >> 3);
+    const float* pa = R.src(i);
+    if (pa)
+        R.load(a, pa);
+    while (i < rows) {
+        const int i2 = i + 64;
+        const float* pb = R.src(i2);
+        if (pb)
+            R.load(b, pb);
+        *reinterpret_cast<uint4*>(dst + i * 128 + ((cgrp ^ (i & 7)) << 4)) = pa ? e4m3x16(a, g.rinv, nan) : zero;
+        i = i2 + 64;
+        pa = R.src(i);
+        if (pa)
+            R.load(a, pa);
+        if (i2 < rows)
+            *reinterpret_cast<uint4*>(dst + i2 * 128 + ((cgrp ^ (i2 & 7)) << 4)) = pb ? e4m3x16(b, g.rinv, nan) : zero;
     }
 }
 
@@ -170,19 +210,15 @@ __device__ __forceinline__ void fill_chunk_rows(const GemmArgs& g, uint8_t* dst,
             if (vec && k + 16 <= g.C) {
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const float4 t = __ldg(reinterpret_cast<const float4*>(p) + q);
+                    const float4 t = __ldcg(reinterpret_cast<const float4*>(p) + q);
                     a[4 * q] = t.x; a[4 * q + 1] = t.y; a[4 * q + 2] = t.z; a[4 * q + 3] = t.w;
                 }
             } else {
 #pragma unroll
                 for (int q = 0; q < 16; ++q)
-                    a[q] = (k + q < g.C) ? __ldg(p + q) : 0.f;
+                    a[q] = (k + q < g.C) ? __ldcg(p + q) : 0.f;
             }
-            const float r = g.rinv;
-            v.x = e4m3x4_from_scaled(__fmul_rn(a[0], r), __fmul_rn(a[1], r), __fmul_rn(a[2], r), __fmul_rn(a[3], r), nan);
-            v.y = e4m3x4_from_scaled(__fmul_rn(a[4], r), __fmul_rn(a[5], r), __fmul_rn(a[6], r), __fmul_rn(a[7], r), nan);
-            v.z = e4m3x4_from_scaled(__fmul_rn(a[8], r), __fmul_rn(a[9], r), __fmul_rn(a[10], r), __fmul_rn(a[11], r), nan);
-            v.w = e4m3x4_from_scaled(__fmul_rn(a[12], r), __fmul_rn(a[13], r), __fmul_rn(a[14], r), __fmul_rn(a[15], r), nan);
+            v = e4m3x16(a, g.rinv, nan);
         }
         *reinterpret_cast<uint4*>(dst + i * 128 + ((j ^ (i & 7)) << 4)) = v;
     }
@@ -192,10 +228,11 @@ __device__ __forceinline__ void fill_chunk_rows(const GemmArgs& g, uint8_t* dst,
 // FUSED = true : 8 more warps read the FP32 activations and quantize them straight into the
 //                activation ring, so the codes never exist in global memory.
 template <int BN, bool FUSED>
-__global__ void __launch_bounds__(FUSED ? NUM_THREADS_FUSED : NUM_THREADS, 1) fpq_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
+__global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                                   const __grid_constant__ CUtensorMap tmB,
                                                                   const GemmArgs g)
 {
+    constexpr int NUM_EPI_WARPS = epi_warps(FUSED);
     constexpr uint32_t B_BLOCK_BYTES = BN * BK;          // smem footprint (4-bit codes sit in 16-byte containers)
     constexpr uint32_t BSTEP = B_BLOCK_BYTES / 16;       // the same in descriptor units
     extern __shared__ uint8_t smem_raw[];
@@ -512,11 +549,12 @@ __global__ void __launch_bounds__(FUSED ? NUM_THREADS_FUSED : NUM_THREADS, 1) fp
                 atomicMin(g.status, FPQ_ERR_TIMEOUT);
         }
     } else if (warp < 2 + NUM_EPI_WARPS) {
-        // ---------------- epilogue: 8 warps; warp w reads TMEM lane quarter w % 4 and the
-        // column half (w - 2) / 4 of the accumulator ----------------
+        // ---------------- epilogue: warp w reads TMEM lane quarter w % 4 and the column
+        // slice (w - 2) / 4 of the accumulator ----------------
         constexpr int EPI_THREADS = 32 * NUM_EPI_WARPS;
-        constexpr int HALF = BN / 2;               // columns per warp
-        constexpr int CHUNKS = HALF / 32;          // 32-column TMEM loads per warp (1 or 2)
+        constexpr int HALF = BN / (NUM_EPI_WARPS / 4);   // columns per warp
+        constexpr int CHUNKS = HALF / 32;                // 32-column TMEM loads per warp
+        constexpr int G = FUSED ? 1 : CHUNKS;            // chunks held in registers at a time
         const int et = threadIdx.x - 64;
         const int quarter = warp & 3;
         const int half = (warp - 2) >> 2;
@@ -580,14 +618,19 @@ __global__ void __launch_bounds__(FUSED ? NUM_THREADS_FUSED : NUM_THREADS, 1) fp
             const int ncol0 = n0 + half * HALF;    // first output column of this warp
             if (!dead && ncol0 < g.N) {
                 const uint32_t t_addr = tmem_base + buf * BN + half * HALF + ((uint32_t)(quarter * 32) << 16);
-                uint32_t r[CHUNKS][32];
 #pragma unroll
-                for (int c = 0; c < CHUNKS; ++c)
-                    tmem_ld32(t_addr + c * 32, r[c]);
+                for (int c0 = 0; c0 < CHUNKS; c0 += G) {
+                if (ncol0 + c0 * 32 >= g.N)
+                    break;
+                uint32_t r[G][32];
+#pragma unroll
+                for (int c = 0; c < G; ++c)
+                    tmem_ld32(t_addr + (c0 + c) * 32, r[c]);
                 tmem_ld_wait();
                 if (row_valid) {
 #pragma unroll
-                    for (int c = 0; c < CHUNKS; ++c) {
+                    for (int cl = 0; cl < G; ++cl) {
+                        const int c = c0 + cl;
                         const int nb = ncol0 + c * 32;
                         const float* scc = sc + half * HALF + c * 32;
                         const float* bic = bi + half * HALF + c * 32;
@@ -601,26 +644,26 @@ __global__ void __launch_bounds__(FUSED ? NUM_THREADS_FUSED : NUM_THREADS, 1) fp
                                     for (int j = 0; j < 8; ++j) {
                                         const float4 s4 = sc4[j], b4 = bi4[j];
                                         float4 v;
-                                        v.x = fmaf(__uint_as_float(r[c][4 * j + 0]), s4.x, b4.x);
-                                        v.y = fmaf(__uint_as_float(r[c][4 * j + 1]), s4.y, b4.y);
-                                        v.z = fmaf(__uint_as_float(r[c][4 * j + 2]), s4.z, b4.z);
-                                        v.w = fmaf(__uint_as_float(r[c][4 * j + 3]), s4.w, b4.w);
+                                        v.x = fmaf(__uint_as_float(r[cl][4 * j + 0]), s4.x, b4.x);
+                                        v.y = fmaf(__uint_as_float(r[cl][4 * j + 1]), s4.y, b4.y);
+                                        v.z = fmaf(__uint_as_float(r[cl][4 * j + 2]), s4.z, b4.z);
+                                        v.w = fmaf(__uint_as_float(r[cl][4 * j + 3]), s4.w, b4.w);
                                         dst[j] = v;
                                     }
                                 } else {
 #pragma unroll
                                     for (int j = 0; j < 32; ++j)
-                                        yrow[nb + j] = fmaf(__uint_as_float(r[c][j]), scc[j], bic[j]);
+                                        yrow[nb + j] = fmaf(__uint_as_float(r[cl][j]), scc[j], bic[j]);
                                 }
                             } else {
                                 float* dst = yrow + (int64_t)nb * nstride;
 #pragma unroll
                                 for (int j = 0; j < 8; ++j) {
                                     const float4 s4 = sc4[j], b4 = bi4[j];
-                                    dst[0] = fmaf(__uint_as_float(r[c][4 * j + 0]), s4.x, b4.x);
-                                    dst[nstride] = fmaf(__uint_as_float(r[c][4 * j + 1]), s4.y, b4.y);
-                                    dst[2 * nstride] = fmaf(__uint_as_float(r[c][4 * j + 2]), s4.z, b4.z);
-                                    dst[3 * nstride] = fmaf(__uint_as_float(r[c][4 * j + 3]), s4.w, b4.w);
+                                    dst[0] = fmaf(__uint_as_float(r[cl][4 * j + 0]), s4.x, b4.x);
+                                    dst[nstride] = fmaf(__uint_as_float(r[cl][4 * j + 1]), s4.y, b4.y);
+                                    dst[2 * nstride] = fmaf(__uint_as_float(r[cl][4 * j + 2]), s4.z, b4.z);
+                                    dst[3 * nstride] = fmaf(__uint_as_float(r[cl][4 * j + 3]), s4.w, b4.w);
                                     dst += 4 * nstride;
                                 }
                             }
@@ -628,10 +671,11 @@ __global__ void __launch_bounds__(FUSED ? NUM_THREADS_FUSED : NUM_THREADS, 1) fp
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
                                 if (nb + j < g.N)
-                                    yrow[(int64_t)(nb + j) * nstride] = fmaf(__uint_as_float(r[c][j]), scc[j], bic[j]);
+                                    yrow[(int64_t)(nb + j) * nstride] = fmaf(__uint_as_float(r[cl][j]), scc[j], bic[j]);
                             }
                         }
                     }
+                }
                 }
             }
             // hand the accumulator back to the MMA warp
@@ -642,9 +686,69 @@ __global__ void __launch_bounds__(FUSED ? NUM_THREADS_FUSED : NUM_THREADS, 1) fp
         }
         if (dead)
             atomicMin(g.status, FPQ_ERR_TIMEOUT);
+    } else if (FUSED && warp == 2 + NUM_EPI_WARPS + NUM_XFORM_WARPS) {
+        // ---------------- L2 prefetch warp ----------------
+        // A transform thread can keep only two rows of loads in flight, so it cannot hide DRAM
+        // latency.  This warp runs two tiles ahead and asks the L2 for every 128-byte line of
+        // FP32 activations those tiles will read; it synchronises with nobody.
+        const int rows = g.a_chunk_bytes >> 7;
+        const int ahead = 2 * (int)gridDim.x;
+        auto prefetch_tile = [&](int t) {
+            int mt, nt;
+            decode_tile(t, mt, nt);
+            if (g.mode == MODE_ROWS) {
+                // 128 rows of C floats: one contiguous span
+                const int64_t m0 = (int64_t)mt * BM;
+                const int64_t m1 = min(m0 + BM, g.M);
+                const char* p0 = reinterpret_cast<const char*>(g.x + m0 * g.C);
+                const int64_t bytes = (m1 - m0) * g.C * 4;
+                for (int64_t o = (int64_t)lane * 128; o < bytes; o += 32 * 128)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(p0 + o));
+                return;
+            }
+            const uint32_t f_lo = (uint32_t)mt * BM;
+            if ((int64_t)f_lo >= g.M)
+                return;
+            const uint32_t f_hi = (uint32_t)min((int64_t)f_lo + rows, g.M) - 1u;
+            const uint32_t b_lo = fdiv(f_lo, g.div_HpWp), b_hi = fdiv(f_hi, g.div_HpWp);
+            const int yp_lo = (int)fdiv(f_lo - b_lo * (uint32_t)g.HpWp, g.div_Wp);
+            const int yp_hi = (int)fdiv(f_hi - b_hi * (uint32_t)g.HpWp, g.div_Wp);
+            for (int part = 0; part < 2; ++part) {
+                if (part == 1 && b_hi == b_lo)
+                    break;
+                const uint32_t b = part ? b_hi : b_lo;
+                const int y0 = part ? 0 : max(yp_lo - g.pad, 0);
+                const int y1 = (part || b_hi == b_lo) ? min(yp_hi - g.pad, g.H - 1) : g.H - 1;
+                if ((int)b >= g.B || y1 < y0)
+                    continue;
+                const int bytes = (y1 - y0 + 1) * g.W * 4;        // contiguous per channel
+                for (int c = lane; c < g.C; c += 32) {
+                    const char* p0 = reinterpret_cast<const char*>(
+                        g.x + ((int64_t)(b * (uint32_t)g.C + (uint32_t)c) * g.H + y0) * g.W);
+                    for (int o = 0; o < bytes; o += 128)
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(p0 + o));
+                }
+            }
+        };
+        int last_mt = -1;
+        for (int t = blockIdx.x; t < total_tiles + ahead; t += gridDim.x) {
+            // tiles t (first two iterations) and t + ahead
+            const int tp = (t < (int)blockIdx.x + ahead) ? t : -1;
+            for (int k = 0; k < 2; ++k) {
+                const int tt = k == 0 ? tp : t + ahead;
+                if (tt < 0 || tt >= total_tiles)
+                    continue;
+                int mt, nt;
+                decode_tile(tt, mt, nt);
+                if (mt == last_mt)
+                    continue;
+                last_mt = mt;
+                prefetch_tile(tt);
+            }
+        }
     } else if (FUSED) {
         // ---------------- activation-quantize prologue: 8 warps fill the A ring ----------------
-        const int tw = warp - (2 + NUM_EPI_WARPS);
+        const int tw = warp - (2 + NUM_EPI_WARPS);      // channel group tw % 8, row phase tw / 8
         const int tid = threadIdx.x - 32 * (2 + NUM_EPI_WARPS);
         const int chunks_per_stage = g.a_span / g.taps;
         const int rows = g.a_chunk_bytes >> 7;
@@ -802,7 +906,7 @@ static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB,
     const int grid = (int)(tiles < di->sms ? tiles : di->sms);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(FUSED ? NUM_THREADS_FUSED : NUM_THREADS);
+    cfg.blockDim = dim3(num_threads(FUSED));
     cfg.dynamicSmemBytes = (size_t)dyn;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
