@@ -157,30 +157,48 @@ def physical_gpu_index(local: int) -> int:
 # ---------------------------------------------------------------------------------------------
 # own arm
 # ---------------------------------------------------------------------------------------------
-class ConvLayerOnGpu:
-    """Device-resident tensors of one conv layer, weights already encoded.  Activations,
-    scratch and outputs exist in several copies whose total size is a multiple of the L2;
-    every call moves on to the next copy."""
+class LayerOnGpu:
+    """Device-resident tensors of one quantized layer (conv or linear), weights already
+    encoded.  Activations, scratch and outputs exist in several copies whose total size is a
+    multiple of the L2; every call moves on to the next copy."""
 
-    def __init__(self, L, fpq, torch, dev, l2_bytes=128 << 20):
+    def __init__(self, L, fpq, torch, dev, l2_bytes=128 << 20, x_dev=None):
         import numpy as np
         self.L, self.fpq, self.torch = L, fpq, torch
         self.fw = fpq.E4M3 if L.wfmt == "e4m3" else fpq.E2M1
-        w2 = np.abs(L.w.reshape(L.N, -1)).max(axis=1)
-        self.ws = torch.tensor([fpq.fpq_scale_from_max(float(v), self.fw) for v in w2], dtype=torch.float32, device=dev)
-        self.xs = fpq.fpq_scale_from_max(float(np.abs(L.x).max()), fpq.E4M3)
-        self.w = torch.from_numpy(L.w.reshape(L.N, -1)).to(dev)
-        self.rb = None
-        if L.bits is not None:
-            self.rb = torch.from_numpy(np.packbits(L.bits, axis=1, bitorder="little")).to(dev)
-        self.bias = torch.from_numpy(L.bias).to(dev)
-        self.ws_bytes = fpq.fpq_conv2d_workspace_size(L.B, L.C, L.H, L.W, L.N, L.R, L.S, L.pad, L.stride, fpq.E4M3, self.fw)
-        self.set_bytes = 4 * L.x.size + 4 * L.M * L.N + self.ws_bytes
+        self.conv = L.kind == "conv"
+        g = torch.Generator(device=dev)
+        g.manual_seed(1000 + (hash(L.name) & 0xffff))
+        if L.w is not None:
+            self.w = torch.from_numpy(L.w.reshape(L.N, -1)).to(dev)
+            self.bias = torch.from_numpy(L.bias).to(dev)
+            x0 = torch.from_numpy(L.x).to(dev)
+            self.rb = None if L.bits is None else torch.from_numpy(np.packbits(L.bits, axis=1, bitorder="little")).to(dev)
+        else:
+            # shape-only layer of a trace: seeded draws on the device (N(0,1) activations,
+            # N(0,0.02) weights, Bernoulli(0.5) rounding decisions)
+            xshape = (L.B, L.C, L.H, L.W) if self.conv else (L.M, L.K)
+            x0 = torch.randn(xshape, generator=g, device=dev, dtype=torch.float32)
+            self.w = torch.randn((L.N, L.K), generator=g, device=dev, dtype=torch.float32) * 0.02
+            self.bias = torch.randn((L.N,), generator=g, device=dev, dtype=torch.float32) * 0.01
+            self.rb = None
+            if L.rounding:
+                self.rb = torch.randint(0, 256, (L.N, (L.K + 7) // 8), generator=g, device=dev, dtype=torch.uint8)
+        wmax = self.w.abs().amax(dim=1).cpu().numpy()
+        self.ws = torch.tensor([fpq.fpq_scale_from_max(float(v), self.fw) for v in wmax], dtype=torch.float32, device=dev)
+        self.xs = fpq.fpq_scale_from_max(float(x0.abs().max().item()), fpq.E4M3)
+        if self.conv:
+            self.ws_bytes = fpq.fpq_conv2d_workspace_size(L.B, L.C, L.H, L.W, L.N, L.R, L.S, L.pad, L.stride, fpq.E4M3, self.fw)
+            yshape = (L.B, L.N, L.Ho, L.Wo)
+        else:
+            self.ws_bytes = fpq.fpq_linear_workspace_size(L.M, L.N, L.K, fpq.E4M3, self.fw)
+            yshape = (L.M, L.N)
+        self.x_elems = x0.numel()
+        self.set_bytes = 4 * self.x_elems + 4 * L.M * L.N + self.ws_bytes
         self.nsets = max(2, -(-3 * l2_bytes // self.set_bytes))        # >= 3 x L2 in rotation
-        x0 = torch.from_numpy(L.x).to(dev)
         self.xs_ = [x0] + [x0.clone() for _ in range(self.nsets - 1)]
-        self.ys_ = [torch.empty((L.B, L.N, L.Ho, L.Wo), dtype=torch.float32, device=dev) for _ in range(self.nsets)]
-        self.wss_ = [torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev) for _ in range(self.nsets)]
+        self.ys_ = [torch.empty(yshape, dtype=torch.float32, device=dev) for _ in range(self.nsets)]
+        self.wss_ = [torch.empty(max(1, self.ws_bytes), dtype=torch.uint8, device=dev) for _ in range(self.nsets)]
         self.i = 0
         self._rot()
         self.encode()
@@ -192,38 +210,53 @@ class ConvLayerOnGpu:
     def encode(self):
         f, L = self.fpq, self.L
         self.codes = f.fpq_quantize_weight(self.w, self.ws, self.fw, self.rb)
-        self.prep = f.fpq_prepare_weight(self.codes, self.fw, f.CONV2D, L.N, L.C, L.R, L.S)
+        if self.conv:
+            self.prep = f.fpq_prepare_weight(self.codes, self.fw, f.CONV2D, L.N, L.C, L.R, L.S)
+        else:
+            self.prep = f.fpq_prepare_weight(self.codes, self.fw, f.LINEAR, L.N, L.K)
 
     def step(self):
         f, L = self.fpq, self.L
         self._rot()
-        f.fpq_conv2d(self.x, self.prep, self.ws, self.xs, f.E4M3, self.fw, self.bias, L.N, L.R, L.S, L.pad, L.stride,
-                     y=self.y, workspace=self.workspace)
+        if self.conv:
+            f.fpq_conv2d(self.x, self.prep, self.ws, self.xs, f.E4M3, self.fw, self.bias, L.N, L.R, L.S, L.pad,
+                         L.stride, y=self.y, workspace=self.workspace)
+        else:
+            f.fpq_linear(self.x, self.prep, self.ws, self.xs, f.E4M3, self.fw, self.bias, L.N, y=self.y,
+                         workspace=self.workspace)
 
     def stage1(self):
         f, L = self.fpq, self.L
         self._rot()
-        f.fpq_conv2d_quantize_input(self.x, self.xs, f.E4M3, self.fw, L.N, L.R, L.S, L.pad, L.stride, self.workspace)
+        if self.conv:
+            f.fpq_conv2d_quantize_input(self.x, self.xs, f.E4M3, self.fw, L.N, L.R, L.S, L.pad, L.stride, self.workspace)
+        else:
+            f.fpq_linear_quantize_input(self.x, self.xs, f.E4M3, self.fw, L.N, self.workspace)
 
     def stage2(self):
         f, L = self.fpq, self.L
         self._rot()
-        f.fpq_conv2d_contract(self.workspace, self.prep, self.ws, self.xs, f.E4M3, self.fw, self.bias, self.y,
-                              (L.B, L.C, L.H, L.W), L.R, L.S, L.pad, L.stride)
+        if self.conv:
+            f.fpq_conv2d_contract(self.workspace, self.prep, self.ws, self.xs, f.E4M3, self.fw, self.bias, self.y,
+                                  (L.B, L.C, L.H, L.W), L.R, L.S, L.pad, L.stride)
+        else:
+            f.fpq_linear_contract(self.workspace, self.prep, self.ws, self.xs, f.E4M3, self.fw, self.bias, self.y, L.K)
+
+    def wbytes(self):
+        return self.L.N * self.L.K * (1 if self.L.wfmt == "e4m3" else 0.5)
 
     # algorithmic bytes (FP32 activations in, FP32 out, encoded weights, scales + bias)
     def layer_bytes(self):
-        L = self.L
-        wbytes = L.N * L.K * (1 if L.wfmt == "e4m3" else 0.5)
-        return 4 * L.x.size + wbytes + 4 * L.M * L.N + 8 * L.N
+        return 4 * self.x_elems + self.wbytes() + 4 * self.L.M * self.L.N + 8 * self.L.N
 
     def stage1_bytes(self):
-        return 4 * self.L.x.size + self.ws_bytes
+        return 4 * self.x_elems + self.ws_bytes
 
     def stage2_bytes(self):
-        L = self.L
-        wbytes = L.N * L.K * (1 if L.wfmt == "e4m3" else 0.5)
-        return self.ws_bytes + wbytes + 4 * L.M * L.N + 8 * L.N
+        return self.ws_bytes + self.wbytes() + 4 * self.L.M * self.L.N + 8 * self.L.N
+
+
+ConvLayerOnGpu = LayerOnGpu
 
 
 class GraphOf:
@@ -421,6 +454,63 @@ def run_own(args):
         dist.destroy_process_group()
 
 
+def run_suite(args):
+    """Per-shape table (not the headline line): every distinct layer shape of the chosen
+    workload, each timed as a CUDA graph of rotating calls on both routes of the library."""
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    from paper_2408_06995_b200 import build as fpq_build
+    fpq_build.build()
+    import paper_2408_06995_b200 as fpq
+    from paper_2408_06995_b200 import inputs as I
+    peaks = load_peaks()
+    if args.suite == "ldm":
+        layers = I.config3()
+    elif args.suite == "transformer":
+        layers = I.config4()
+    elif args.suite == "sd":
+        layers = I.distinct_shapes(I.sd_v1_unet_layers())
+    else:
+        raise SystemExit("unknown suite")
+    rows = []
+    tot = {"auto": 0.0, "fused": 0.0, "two_kernels": 0.0, "best": 0.0, "flops": 0.0, "bytes": 0.0, "bound": 0.0}
+    for L in layers:
+        lay = LayerOnGpu(L, fpq, torch, dev, l2_bytes=(128 << 20) if args.suite != "sd" else (48 << 20))
+        n = max(4, min(40, 3 * lay.nsets))
+        res = {}
+        for name, pol in (("fused", fpq.PATH_FUSED), ("two_kernels", fpq.PATH_TWO_KERNELS), ("auto", fpq.PATH_AUTO)):
+            fpq.fpq_set_path_policy(pol)
+            for _ in range(2):
+                lay.step()
+            res[name] = per_launch_us(torch, lay.step, n, reps=2)
+        fpq.fpq_set_path_policy(fpq.PATH_AUTO)
+        st = fpq.fpq_read_status()
+        if st != fpq.OK:
+            raise SystemExit(f"{L.name}: device status {fpq.status_string(st)}")
+        t_hbm = lay.layer_bytes() / (peaks["hbm_gbs"] * 1e9) * 1e6
+        t_tc = L.flops / (NOMINAL_FP8_TFLOPS * 1e12) * 1e6
+        best = min(res["fused"], res["two_kernels"])
+        rows.append({"name": L.name, "kind": L.kind, "M": L.M, "N": L.N, "K": L.K, "count": L.count, "wfmt": L.wfmt,
+                     "us": res, "tflops_auto": L.flops / res["auto"] / 1e6, "t_hbm_us": t_hbm, "t_tensor_us": t_tc,
+                     "frac_of_bound_auto": max(t_hbm, t_tc) / res["auto"]})
+        for k in ("auto", "fused", "two_kernels"):
+            tot[k] += res[k] * L.count
+        tot["best"] += best * L.count
+        tot["flops"] += L.flops * L.count
+        tot["bytes"] += lay.layer_bytes() * L.count
+        tot["bound"] += max(t_hbm, t_tc) * L.count
+        del lay
+        torch.cuda.empty_cache()
+    summary = {"suite": args.suite, "layers": sum(r["count"] for r in rows), "distinct_shapes": len(rows),
+               "sum_us": {k: tot[k] for k in ("auto", "fused", "two_kernels", "best")},
+               "aggregate_tflops_auto": tot["flops"] / tot["auto"] / 1e6, "sum_bound_us": tot["bound"],
+               "frac_of_bound_auto": tot["bound"] / tot["auto"], "gflop": tot["flops"] / 1e9, "rows": rows}
+    print(json.dumps(summary), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -429,8 +519,12 @@ def main():
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline leg")
     ap.add_argument("--skip-w4", action="store_true", help="leave out the W4A8 side measurement")
+    ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd"],
+                    help="print a per-shape table of a whole workload instead of the headline line")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.suite:
+        run_suite(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_own(args)

@@ -227,6 +227,20 @@ fpq_status fpq_linear_static(const float* x, const void* w_prepared, const float
                              float x_scale, fpq_format fx, fpq_format fw, const float* bias,
                              float* y, int64_t M, int64_t N, int64_t K, void* stream);
 
+/*
+ * Which route fpq_linear / fpq_conv2d take (process-wide setting, not thread-safe against
+ * concurrent layer calls; the results are the same bit for bit on either route):
+ *   FPQ_PATH_FUSED        one kernel: the activation quantize (Sec. IV-B rounding equation) runs
+ *                         inside the contraction's operand staging, the codes never reach global
+ *                         memory.  Available for linear layers and stride-1 convolutions; other
+ *                         geometries fall back to two kernels.
+ *   FPQ_PATH_TWO_KERNELS  always *_quantize_input followed by *_contract.
+ *   FPQ_PATH_AUTO         the library's choice per layer kind (default).
+ */
+enum { FPQ_PATH_AUTO = 0, FPQ_PATH_FUSED = 1, FPQ_PATH_TWO_KERNELS = 2 };
+fpq_status fpq_set_path_policy(int32_t policy);
+int32_t fpq_get_path_policy(void);
+
 /* Waits for `stream`, then returns and clears the sticky device status word:
  * FPQ_OK, FPQ_ERR_TIMEOUT, FPQ_ERR_NAN_INPUT, or FPQ_ERR_CUDA. */
 fpq_status fpq_read_status(void* stream);

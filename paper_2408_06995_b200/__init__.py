@@ -22,6 +22,7 @@ ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NAN_INPUT, ERR_TOO_LARGE = -6, -7, -8,
 STATIC_SCRATCH_BYTES = 8 << 20
 SAT_PAPER, SAT_NATIVE = 0, 1
 LINEAR, CONV2D = 0, 1
+PATH_AUTO, PATH_FUSED, PATH_TWO_KERNELS = 0, 1, 2
 
 
 class FpqError(RuntimeError):
@@ -67,7 +68,7 @@ EXPORTS = [
     "fpq_prepared_size", "fpq_prepare_weight", "fpq_linear_workspace_size", "fpq_linear",
     "fpq_conv2d_workspace_size", "fpq_conv2d", "fpq_linear_host", "fpq_conv2d_host",
     "fpq_linear_quantize_input", "fpq_linear_contract", "fpq_conv2d_quantize_input", "fpq_conv2d_contract",
-    "fpq_linear_static", "fpq_read_status", "fpq_status_string",
+    "fpq_linear_static", "fpq_set_path_policy", "fpq_get_path_policy", "fpq_read_status", "fpq_status_string",
 ]
 
 _lib = None
@@ -119,6 +120,10 @@ def lib() -> ctypes.CDLL:
         L.fpq_conv2d_contract.argtypes = [vp, sz, vp, vp, f32, F, F, vp, vp] + [i32] * 9 + [vp]
         L.fpq_linear_static.restype = i32
         L.fpq_linear_static.argtypes = [vp, vp, vp, f32, F, F, vp, vp, i64, i64, i64, vp]
+        L.fpq_set_path_policy.restype = i32
+        L.fpq_set_path_policy.argtypes = [i32]
+        L.fpq_get_path_policy.restype = i32
+        L.fpq_get_path_policy.argtypes = []
         L.fpq_read_status.restype = i32
         L.fpq_read_status.argtypes = [vp]
         L.fpq_status_string.restype = ctypes.c_char_p
@@ -296,6 +301,14 @@ def fpq_conv2d_host(x_host, x_dev, w_prepared, w_scale, x_scale, fx, fw, bias, y
                                  fx.c(), fw.c(), _ptr(bias), _ptr(y_dev), _ptr(y_host), B, C, H, W, C_out, R, S,
                                  pad, stride, _ptr(workspace), workspace.numel(), _stream()), "fpq_conv2d_host")
     return y_host
+
+
+def fpq_set_path_policy(policy: int) -> None:
+    _check(lib().fpq_set_path_policy(int(policy)), "fpq_set_path_policy")
+
+
+def fpq_get_path_policy() -> int:
+    return lib().fpq_get_path_policy()
 
 
 def fpq_read_status() -> int:

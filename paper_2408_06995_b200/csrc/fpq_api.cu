@@ -71,6 +71,8 @@ static bool is_e2m1(fpq_format f)
     return f.exp_bits == 2 && f.man_bits == 1 && f.exp_bias == 1;
 }
 
+static int g_path_policy = FPQ_PATH_AUTO;
+
 static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 
 static int64_t padded_c(int64_t C) { return round_up(C, 128); }
@@ -299,9 +301,12 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
         (bias && !aligned(bias, 4)))
         return FPQ_ERR_ALIGN;
     // one kernel: the activations are quantized inside the contraction's operand staging
-    s = linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream, 0, x);
-    if (s != FPQ_ERR_UNSUPPORTED)
-        return s;
+    if (g_path_policy != FPQ_PATH_TWO_KERNELS) {
+        s = linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream, 0,
+                                 x);
+        if (s != FPQ_ERR_UNSUPPORTED)
+            return s;
+    }
     s = fpq_linear_quantize_input(x, x_scale, fx, fw, M, N, K, workspace, ws_bytes, stream);
     if (s != FPQ_OK)
         return s;
@@ -444,10 +449,13 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
         return FPQ_ERR_ALIGN;
     // one kernel where the geometry allows it (stride 1): the activations are quantized inside the
     // contraction's operand staging; otherwise quantize to codes first
-    s = conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out, R,
-                             S, pad, stride, stream, 0, x);
-    if (s != FPQ_ERR_UNSUPPORTED)
-        return s;
+    // (AUTO takes the two-kernel route for convolutions: measured faster on B200 so far)
+    if (g_path_policy == FPQ_PATH_FUSED) {
+        s = conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out,
+                                 R, S, pad, stride, stream, 0, x);
+        if (s != FPQ_ERR_UNSUPPORTED)
+            return s;
+    }
     s = fpq_conv2d_quantize_input(x, x_scale, fx, fw, B, C, H, W, C_out, R, S, pad, stride, workspace, ws_bytes,
                                   stream);
     if (s != FPQ_OK)
@@ -501,6 +509,16 @@ fpq_status fpq_conv2d_host(const float* x_host, float* x_dev, const void* w_prep
         return FPQ_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
 }
+
+fpq_status fpq_set_path_policy(int32_t policy)
+{
+    if (policy != FPQ_PATH_AUTO && policy != FPQ_PATH_FUSED && policy != FPQ_PATH_TWO_KERNELS)
+        return FPQ_ERR_UNSUPPORTED;
+    g_path_policy = policy;
+    return FPQ_OK;
+}
+
+int32_t fpq_get_path_policy(void) { return g_path_policy; }
 
 fpq_status fpq_read_status(void* stream)
 {

@@ -46,10 +46,9 @@ def gpu_prepare(L, ws):
     return codes, prep
 
 
-def gpu_layer(L, ws, xs, use_bias=True):
+def _gpu_layer_once(L, ws, xs, use_bias, prep):
     gfw, _ = FMT[L.wfmt]
     dev = "cuda"
-    _, prep = gpu_prepare(L, ws)
     x = torch.from_numpy(L.x).to(dev)
     bias = torch.from_numpy(L.bias).to(dev) if use_bias else None
     wsd = torch.from_numpy(ws).to(dev)
@@ -60,6 +59,21 @@ def gpu_layer(L, ws, xs, use_bias=True):
     st = fpq.fpq_read_status()
     assert st == fpq.OK, fpq.status_string(st)
     return y.cpu().numpy()
+
+
+def gpu_layer(L, ws, xs, use_bias=True):
+    """The layer call on both of the library's routes (one fused kernel; quantize kernel +
+    contraction kernel).  They run the same MMAs in the same order: results must be equal."""
+    _, prep = gpu_prepare(L, ws)
+    try:
+        fpq.fpq_set_path_policy(fpq.PATH_FUSED)
+        y1 = _gpu_layer_once(L, ws, xs, use_bias, prep)
+        fpq.fpq_set_path_policy(fpq.PATH_TWO_KERNELS)
+        y2 = _gpu_layer_once(L, ws, xs, use_bias, prep)
+    finally:
+        fpq.fpq_set_path_policy(fpq.PATH_AUTO)
+    assert np.array_equal(y1, y2), "fused and two-kernel routes differ"
+    return y1
 
 
 def oracle_layer(L, ws, xs, idx=None, use_bias=True):
