@@ -162,7 +162,7 @@ class LayerOnGpu:
     encoded.  Activations, scratch and outputs exist in several copies whose total size is a
     multiple of the L2; every call moves on to the next copy."""
 
-    def __init__(self, L, fpq, torch, dev, l2_bytes=128 << 20, x_dev=None):
+    def __init__(self, L, fpq, torch, dev, l2_bytes=128 << 20, nsets=None):
         import numpy as np
         self.L, self.fpq, self.torch = L, fpq, torch
         self.fw = fpq.E4M3 if L.wfmt == "e4m3" else fpq.E2M1
@@ -195,7 +195,7 @@ class LayerOnGpu:
             yshape = (L.M, L.N)
         self.x_elems = x0.numel()
         self.set_bytes = 4 * self.x_elems + 4 * L.M * L.N + self.ws_bytes
-        self.nsets = max(2, -(-3 * l2_bytes // self.set_bytes))        # >= 3 x L2 in rotation
+        self.nsets = nsets or max(2, -(-3 * l2_bytes // self.set_bytes))        # >= 3 x L2 in rotation
         self.xs_ = [x0] + [x0.clone() for _ in range(self.nsets - 1)]
         self.ys_ = [torch.empty(yshape, dtype=torch.float32, device=dev) for _ in range(self.nsets)]
         self.wss_ = [torch.empty(max(1, self.ws_bytes), dtype=torch.uint8, device=dev) for _ in range(self.nsets)]
@@ -294,6 +294,28 @@ def per_launch_us(torch, fn, n, reps=3):
     return min(g.timed_replay() for _ in range(reps)) * 1e3 / n
 
 
+def max_over_ranks(value: float, dist, device) -> float:
+    """The slowest rank's time: what a weak-scaling run of independent replicas is charged."""
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def rank_layer(I, rank: int, world: int):
+    """Rank r's copy of the workload layer: same law, its own draws (tensor seeds offset by
+    100 r), so that N ranks process N different batches with no exchange between them."""
+    (L,) = I.config2()
+    if world > 1:
+        L = I.draw(L, 2, 100 * rank, "silu", 0.03, True)
+    return L
+
+
+def whole_job_value(flops_per_step: float, steps: int, world: int, slowest_ms: float) -> float:
+    """TFLOP/s of the whole job: all ranks' work over the slowest rank's time."""
+    return world * flops_per_step * steps / (slowest_ms * 1e-3) / 1e12
+
+
 def run_own(args):
     import numpy as np
     import torch
@@ -316,9 +338,7 @@ def run_own(args):
     from paper_2408_06995_b200 import inputs as I
 
     peaks = load_peaks()
-    (L,) = I.config2()
-    if world > 1:                       # every rank its own batch of the same law
-        L = I.draw(L, 2, 100 * rank, "silu", 0.03, True)
+    L = rank_layer(I, rank, world)      # every rank its own batch of the same law
     layer = ConvLayerOnGpu(L, fpq, torch, dev)
 
     def barrier():
@@ -342,11 +362,9 @@ def run_own(args):
     if st != fpq.OK:
         raise SystemExit(f"device status after the timed region: {fpq.status_string(st)}")
     if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+        total_ms = max_over_ranks(total_ms, dist, dev)
     flops_step = L.flops
-    value = world * flops_step * args.steps / (total_ms * 1e-3) / 1e12
+    value = whole_job_value(flops_step, args.steps, world, total_ms)
     launches_per_step = 2
     t_layer = total_ms * 1e-3 / args.steps
 
@@ -402,9 +420,7 @@ def run_own(args):
     t_e2e = time.perf_counter() - t0
     barrier()
     if world > 1:
-        t = torch.tensor([t_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        t_e2e = float(t.item())
+        t_e2e = max_over_ranks(t_e2e, dist, dev)
     e2e = {"value": world * flops_step * n_e2e / t_e2e / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": xh.numel() * 4,
            "d2h_bytes_per_step": yh.numel() * 4, "steps": n_e2e, "ms_per_step": 1e3 * t_e2e / n_e2e}
 
@@ -452,6 +468,52 @@ def run_own(args):
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_trace(args):
+    """One denoising step of the SD-v1-style U-Net as a layer trace: all 234 conv / linear
+    layers (W4A8 with rounding decisions), each with its own buffers, launched back to back on one
+    stream and replayed as one CUDA graph.  The buffers of one pass total several GB, so every
+    layer finds its input in HBM."""
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    from paper_2408_06995_b200 import build as fpq_build
+    fpq_build.build()
+    import paper_2408_06995_b200 as fpq
+    from paper_2408_06995_b200 import inputs as I
+    peaks = load_peaks()
+    trace = I.sd_v1_unet_layers()
+    layers = [LayerOnGpu(L, fpq, torch, dev, nsets=1) for L in trace]
+    torch.cuda.synchronize()
+
+    def one_pass():
+        for lay in layers:
+            lay.step()
+
+    for _ in range(2):
+        one_pass()
+    torch.cuda.synchronize()
+    g = GraphOf(torch, one_pass, 1)
+    g.timed_replay()
+    ms = [g.timed_replay() for _ in range(max(3, min(args.steps, 20)))]
+    st = fpq.fpq_read_status()
+    if st != fpq.OK:
+        raise SystemExit(f"device status: {fpq.status_string(st)}")
+    flops = sum(L.flops for L in trace)
+    bytes_ = sum(lay.layer_bytes() for lay in layers)
+    bound_us = sum(max(lay.layer_bytes() / (peaks["hbm_gbs"] * 1e9), lay.L.flops / (NOMINAL_FP8_TFLOPS * 1e12)) * 1e6
+                   for lay in layers)
+    t = statistics.median(ms) * 1e-3
+    print(json.dumps({"suite": "sd_trace", "layers": len(layers), "gflop": flops / 1e9, "algorithmic_mb": bytes_ / 1e6,
+                      "ms_per_step": t * 1e3, "min_ms": min(ms), "aggregate_tflops": flops / t / 1e12,
+                      "pct_dense_fp8_peak_nominal": 100 * flops / t / 1e12 / NOMINAL_FP8_TFLOPS,
+                      "pct_dense_fp4_peak_nominal": 100 * flops / t / 1e12 / NOMINAL_FP4_TFLOPS,
+                      "sum_of_per_layer_bounds_us": bound_us, "frac_of_bound": bound_us * 1e-6 / t,
+                      "device_buffers_gb": sum(l.set_bytes for l in layers) / 1e9, "launch": "one CUDA graph replay"}),
+          flush=True)
 
 
 def run_suite(args):
@@ -519,10 +581,12 @@ def main():
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline leg")
     ap.add_argument("--skip-w4", action="store_true", help="leave out the W4A8 side measurement")
-    ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd"],
+    ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd", "sd_trace"],
                     help="print a per-shape table of a whole workload instead of the headline line")
     args = ap.parse_args()
-    if args.suite:
+    if args.suite == "sd_trace":
+        run_trace(args)
+    elif args.suite:
         run_suite(args)
     elif args.impl == "reference":
         run_reference(args)

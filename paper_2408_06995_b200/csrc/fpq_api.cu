@@ -301,7 +301,8 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
         (bias && !aligned(bias, 4)))
         return FPQ_ERR_ALIGN;
     // one kernel: the activations are quantized inside the contraction's operand staging
-    if (g_path_policy != FPQ_PATH_TWO_KERNELS) {
+    // (AUTO takes the two-kernel route: measured faster on B200 so far)
+    if (g_path_policy == FPQ_PATH_FUSED) {
         s = linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream, 0,
                                  x);
         if (s != FPQ_ERR_UNSUPPORTED)
@@ -449,7 +450,6 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
         return FPQ_ERR_ALIGN;
     // one kernel where the geometry allows it (stride 1): the activations are quantized inside the
     // contraction's operand staging; otherwise quantize to codes first
-    // (AUTO takes the two-kernel route for convolutions: measured faster on B200 so far)
     if (g_path_policy == FPQ_PATH_FUSED) {
         s = conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out,
                                  R, S, pad, stride, stream, 0, x);
