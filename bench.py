@@ -74,7 +74,8 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    batch = 4
+    # bounded sample per step, sized so that the whole run stays within a few minutes
+    batch = 4 if args.steps <= 100 else (2 if args.steps <= 300 else 1)
     for _ in range(args.warmup):
         oracle_sample_run(batch)
     total, flops = 0.0, 0
@@ -576,7 +577,7 @@ def run_suite(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline leg")
