@@ -86,6 +86,7 @@ struct GemmArgs {
     // weight ring: a stage holds b_span consecutive blocks; resident = the whole reduction,
     // reloaded only when the column tile changes
     int b_span, b_stage_bytes, b_stages, b_resident;
+    int a_resident;            // a row tile's whole activation panel stays in the ring while the CTA walks its column tiles
     uint32_t a_chunk_tx, b_block_tx;   // bytes one load reports to its barrier
     const float* w_scale;
     float x_scale;
@@ -254,6 +255,10 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int total_tiles = g.m_tiles * g.n_tiles;
+    // every CTA walks a contiguous range of the tile list, so consecutive tiles share the row tile
+    // (or, in column-tile-major order, the column tile) and its resident operand
+    const int t_lo = (int)((int64_t)blockIdx.x * total_tiles / gridDim.x);
+    const int t_hi = (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 8; ++s) {
@@ -293,10 +298,10 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         if (lane == 0) {
             uint32_t sa = 0, pa = 0, sb = 0, pb = 0;   // stage and phase of the next load per ring
             uint32_t na = 0, nb = 0;                   // stages issued (for the abort path)
-            int resident_nt = -1;
+            int resident_nt = -1, resident_mt = -1;
             bool dead = false;
             bool prior_done = !g.wait_prior_grid;
-            for (int t = blockIdx.x; t < total_tiles && !dead; t += gridDim.x) {
+            for (int t = t_lo; t < t_hi && !dead; ++t) {
                 int mt, nt;
                 decode_tile(t, mt, nt);
                 const int n0 = nt * BN;
@@ -310,6 +315,8 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                 }
                 const bool load_b = !(g.b_resident && resident_nt == nt);
                 resident_nt = nt;
+                const bool load_a = !(g.a_resident && resident_mt == mt);
+                resident_mt = mt;
                 int cc = 0, tap = 0, r = 0, sx = 0;    // block j = (cc, tap), tap = (r, sx)
                 int ja = 0, jb = 0;                    // position inside the current A / B stage
                 bool early_b = false;
@@ -333,7 +340,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                         asm volatile("griddepcontrol.wait;" ::: "memory");
                         prior_done = true;
                     }
-                    if (ja == 0 && !FUSED) {
+                    if (ja == 0 && !FUSED && load_a) {
                         // activation stage: the data of the next a_span blocks
                         if (!mbar_wait(a_empty + 8 * sa, pa ^ 1)) { dead = true; break; }
                         const int nblocks = min(g.a_span, g.nblk - j);
@@ -393,12 +400,13 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         // straight-line code.
         if (lane == 0) {
             uint32_t sa = 0, pa = 0, sb = 0, pb = 0, it = 0;
-            int resident_nt = -1;
+            uint32_t sa0 = 0, pa0 = 0;                 // ring position of the resident activation panel
+            int resident_nt = -1, resident_mt = -1;
             bool dead = false;
             const uint32_t a_chunk_step = (uint32_t)g.a_chunk_bytes >> 4;
             const uint32_t b_res = smem_desc_lo(b_ring);           // resident weights start here
             const uint32_t HI = SMEM_DESC_HI_K_SW128;
-            for (int t = blockIdx.x; t < total_tiles && !dead; t += gridDim.x, ++it) {
+            for (int t = t_lo; t < t_hi && !dead; ++t, ++it) {
                 int mt, nt;
                 decode_tile(t, mt, nt);
                 const bool new_b = !(g.b_resident && resident_nt == nt);
@@ -408,6 +416,17 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                     if (++sb == (uint32_t)g.b_stages) { sb = 0; pb ^= 1; }
                 }
                 resident_nt = nt;
+                // resident activation panel: a tile of the same row tile re-reads the stages already
+                // filled (no wait), and the stages are handed back only when the row tile changes
+                const bool reuse_a = g.a_resident && resident_mt == mt;
+                resident_mt = mt;
+                if (reuse_a) { sa = sa0; pa = pa0; } else { sa0 = sa; pa0 = pa; }
+                bool keep_a = false;
+                if (g.a_resident && t + 1 < t_hi) {
+                    int mt2, nt2;
+                    decode_tile(t + 1, mt2, nt2);
+                    keep_a = mt2 == mt;
+                }
                 const uint32_t buf = it & 1, aph = (it >> 1) & 1;
                 if (!mbar_wait(acc_empty + 8 * buf, aph ^ 1)) { dead = true; break; }
                 if (g.b_resident && new_b)
@@ -419,7 +438,8 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                     const uint32_t Wp8 = (uint32_t)g.Wp * 8u;
                     const int chunks_per_stage = g.a_span / 9;
                     for (int cc = 0; cc < g.cchunks && !dead;) {
-                        if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
+                        if (!reuse_a)
+                            if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
                         tc_fence_after();
                         const uint32_t abase = smem_desc_lo(a_ring + sa * g.a_stage_bytes);
                         const int nch = min(chunks_per_stage, g.cchunks - cc);
@@ -451,14 +471,16 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                                 }
                             }
                         }
-                        mma_commit(a_empty + 8 * sa);
+                        if (!keep_a)
+                            mma_commit(a_empty + 8 * sa);
                         if (++sa == (uint32_t)g.a_stages) { sa = 0; pa ^= 1; }
                     }
                 } else if (g.taps == 1 && g.mode != MODE_TAPS && g.a_span <= 4 &&
                            (g.b_resident || g.b_span == g.a_span)) {
                     // one block per 128-wide chunk; a stage carries up to 4 chunks of both operands
                     for (int cc = 0; cc < g.cchunks && !dead;) {
-                        if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
+                        if (!reuse_a)
+                            if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
                         uint32_t bbase = b_res + (uint32_t)cc * BSTEP;
                         if (!g.b_resident) {
                             if (!mbar_wait(b_full + 8 * sb, pb)) { dead = true; break; }
@@ -484,7 +506,8 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                             mma_commit(b_empty + 8 * sb);
                             if (++sb == (uint32_t)g.b_stages) { sb = 0; pb ^= 1; }
                         }
-                        mma_commit(a_empty + 8 * sa);
+                        if (!keep_a)
+                            mma_commit(a_empty + 8 * sa);
                         if (++sa == (uint32_t)g.a_stages) { sa = 0; pa ^= 1; }
                         cc += n;
                     }
@@ -498,7 +521,8 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                     int tap = 0, sx = 0, ja = 0, jb = 0;
                     for (int j = 0; j < g.nblk; ++j) {
                         if (ja == 0) {
-                            if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
+                            if (!reuse_a)
+                                if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
                             a_chunk_lo = smem_desc_lo(a_ring + sa * g.a_stage_bytes);
                             a_lo = a_chunk_lo;
                             tc_fence_after();
@@ -536,7 +560,8 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                         }
                         if (++ja == g.a_span || last) {
                             ja = 0;
-                            mma_commit(a_empty + 8 * sa);
+                            if (!keep_a)
+                                mma_commit(a_empty + 8 * sa);
                             if (++sa == (uint32_t)g.a_stages) { sa = 0; pa ^= 1; }
                         }
                     }
@@ -562,7 +587,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         uint32_t it = 0;
         bool dead = false;
         int loaded_nt[2] = {-1, -1};               // which column tile each scale/bias buffer holds
-        for (int t = blockIdx.x; t < total_tiles && !dead; t += gridDim.x, ++it) {
+        for (int t = t_lo; t < t_hi && !dead; ++t, ++it) {
             int mt, nt;
             decode_tile(t, mt, nt);
             const int n0 = nt * BN;
@@ -689,10 +714,9 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     } else if (FUSED && warp == 2 + NUM_EPI_WARPS + NUM_XFORM_WARPS) {
         // ---------------- L2 prefetch warp ----------------
         // A transform thread can keep only two rows of loads in flight, so it cannot hide DRAM
-        // latency.  This warp runs two tiles ahead and asks the L2 for every 128-byte line of
+        // latency.  This warp runs ahead of them through the CTA's tiles and asks the L2 for every 128-byte line of
         // FP32 activations those tiles will read; it synchronises with nobody.
         const int rows = g.a_chunk_bytes >> 7;
-        const int ahead = 2 * (int)gridDim.x;
         auto prefetch_tile = [&](int t) {
             int mt, nt;
             decode_tile(t, mt, nt);
@@ -731,20 +755,13 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             }
         };
         int last_mt = -1;
-        for (int t = blockIdx.x; t < total_tiles + ahead; t += gridDim.x) {
-            // tiles t (first two iterations) and t + ahead
-            const int tp = (t < (int)blockIdx.x + ahead) ? t : -1;
-            for (int k = 0; k < 2; ++k) {
-                const int tt = k == 0 ? tp : t + ahead;
-                if (tt < 0 || tt >= total_tiles)
-                    continue;
-                int mt, nt;
-                decode_tile(tt, mt, nt);
-                if (mt == last_mt)
-                    continue;
-                last_mt = mt;
-                prefetch_tile(tt);
-            }
+        for (int t = t_lo; t < t_hi; ++t) {
+            int mt, nt;
+            decode_tile(t, mt, nt);
+            if (mt == last_mt)
+                continue;
+            last_mt = mt;
+            prefetch_tile(t);
         }
     } else if (FUSED) {
         // ---------------- activation-quantize prologue: 8 warps fill the A ring ----------------
@@ -754,9 +771,13 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         const int rows = g.a_chunk_bytes >> 7;
         uint32_t sa = 0, pa = 0;
         bool dead = false, nan = false;
-        for (int t = blockIdx.x; t < total_tiles && !dead; t += gridDim.x) {
+        int resident_mt = -1;
+        for (int t = t_lo; t < t_hi && !dead; ++t) {
             int mt, nt;
             decode_tile(t, mt, nt);
+            if (g.a_resident && mt == resident_mt)
+                continue;                          // the panel is still in the ring
+            resident_mt = mt;
             for (int cc = 0; cc < g.cchunks;) {
                 if (!mbar_wait(a_empty + 8 * sa, pa ^ 1)) { dead = true; break; }
                 const int nch = min(chunks_per_stage, g.cchunks - cc);
@@ -850,7 +871,36 @@ static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB,
     const int b_block = BN * BK;
     const int a_min_span = (g.mode == MODE_FLAT) ? g.taps : 1;
     const int64_t b_all = (int64_t)g.nblk * b_block;
-    if (b_all + 2 * g.a_chunk_bytes <= budget) {
+    g.a_resident = 0;
+    // several column tiles per row tile: try to keep the row tile's whole activation panel in the
+    // ring (read / quantized once) and stream the weights
+    bool done = false;
+    if (g.n_tiles > 1 && g.mode != MODE_TAPS) {
+        const bool conv9 = g.mode == MODE_FLAT && g.taps == 9 && g.S == 3;
+        if (conv9 || g.taps == 1) {
+            const int cps = conv9 ? 1 : (g.cchunks >= 3 ? 3 : g.cchunks);      // chunks per A stage
+            const int groups = (g.cchunks + cps - 1) / cps;
+            const int b_span = conv9 ? 3 : cps;
+            const int b_stage = b_span * b_block;
+            const int panel = groups * cps * g.a_chunk_bytes;
+            if (groups <= 8 && panel + 2 * b_stage <= budget) {
+                const int panels = (groups <= 4 && 2 * panel + 2 * b_stage <= budget) ? 2 : 1;
+                g.a_resident = 1;
+                g.m_fastest = 0;
+                g.b_resident = 0;
+                g.a_span = cps * a_min_span;
+                g.a_stage_bytes = cps * g.a_chunk_bytes;
+                g.a_stages = panels * groups;
+                g.b_span = b_span;
+                g.b_stages = (budget - g.a_stages * g.a_stage_bytes) / b_stage;
+                if (g.b_stages > 8) g.b_stages = 8;
+                done = true;
+            }
+        }
+    }
+    if (done) {
+        // configured above
+    } else if (b_all + 2 * g.a_chunk_bytes <= budget) {
         g.b_resident = 1;
         g.b_span = g.nblk;
         g.b_stages = 1;
