@@ -86,6 +86,9 @@ struct GemmArgs {
     // weight ring: a stage holds b_span consecutive blocks; resident = the whole reduction,
     // reloaded only when the column tile changes
     int b_span, b_stage_bytes, b_stages, b_resident;
+    int y_tma;                 // row-major output leaves through TMA stores
+    int vec_scale;             // w_scale / bias are 16-byte aligned
+    int stage_scales;          // x_scale * w_scale[n] and bias[n] of all N columns sit in shared memory
     int a_resident;            // a row tile's whole activation panel stays in the ring while the CTA walks its column tiles
     uint32_t a_chunk_tx, b_block_tx;   // bytes one load reports to its barrier
     const float* w_scale;
@@ -231,6 +234,7 @@ __device__ __forceinline__ void fill_chunk_rows(const GemmArgs& g, uint8_t* dst,
 template <int BN, bool FUSED>
 __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                                   const __grid_constant__ CUtensorMap tmB,
+                                                                  const __grid_constant__ CUtensorMap tmY,
                                                                   const GemmArgs g)
 {
     constexpr int NUM_EPI_WARPS = epi_warps(FUSED);
@@ -240,17 +244,25 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
 
-    // layout: [A ring][B ring][barriers + flags][scale | bias]
+    // layout: [A ring][B ring][epilogue staging for TMA stores, 4 KiB per warp][barriers + flags]
+    //         [x_scale * w_scale | bias, all N columns, when they fit]
     const uint32_t a_ring = smem_base;
     const uint32_t b_ring = a_ring + g.a_stages * g.a_stage_bytes;
     const uint32_t ctl_off = g.a_stages * g.a_stage_bytes + g.b_stages * g.b_stage_bytes;
-    const uint32_t bars = smem_base + ctl_off;
+    const uint32_t bars = smem_base + ctl_off + (g.y_tma ? NUM_EPI_WARPS * 4096 : 0);
     // barrier slots (8 bytes each): a_full[8] a_empty[8] b_full[8] b_empty[8] acc_full[2] acc_empty[2]
     const uint32_t a_full = bars, a_empty = bars + 64, b_full = bars + 128, b_empty = bars + 192;
     const uint32_t acc_full = bars + 256, acc_empty = bars + 272;
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + ctl_off + 288);
-    float* s_scale = reinterpret_cast<float*>(smem + ctl_off + 320);   // [2][BN]
-    float* s_bias = s_scale + 2 * BN;                                   // [2][BN]
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + (bars - smem_base) + 288);
+    const int n_pad = (g.N + 31) & ~31;
+    float* s_scale = reinterpret_cast<float*>(smem + (bars - smem_base) + 512);   // [n_pad], if staged
+    float* s_bias = s_scale + n_pad;
+    if (g.stage_scales) {
+        for (int i = threadIdx.x; i < n_pad; i += blockDim.x) {
+            s_scale[i] = (i < g.N) ? g.x_scale * __ldg(g.w_scale + i) : 0.f;
+            s_bias[i] = (g.bias && i < g.N) ? __ldg(g.bias + i) : 0.f;
+        }
+    }
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -274,6 +286,8 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         fence_barrier_init();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
+        if (g.y_tma)
+            tma_prefetch_desc(&tmY);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32((const void*)tmem_slot), 2 * BN);
@@ -575,34 +589,24 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         }
     } else if (warp < 2 + NUM_EPI_WARPS) {
         // ---------------- epilogue: warp w reads TMEM lane quarter w % 4 and the column
-        // slice (w - 2) / 4 of the accumulator ----------------
-        constexpr int EPI_THREADS = 32 * NUM_EPI_WARPS;
+        // slice (w - 2) / 4 of the accumulator: y = acc * (x_scale * w_scale[n]) + bias[n] ----------------
         constexpr int HALF = BN / (NUM_EPI_WARPS / 4);   // columns per warp
         constexpr int CHUNKS = HALF / 32;                // 32-column TMEM loads per warp
         constexpr int G = FUSED ? 1 : CHUNKS;            // chunks held in registers at a time
-        const int et = threadIdx.x - 64;
         const int quarter = warp & 3;
         const int half = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;       // row of the tile held by this thread
+        // row-major output: the warp's 32 x 32 block goes through a 128-byte-swizzled staging
+        // buffer and leaves as one TMA store (whole 128-byte lines; rows past M and columns
+        // past N are clipped by the tensor map)
+        uint8_t* stage = smem + ctl_off + (warp - 2) * 4096;
         uint32_t it = 0;
         bool dead = false;
-        int loaded_nt[2] = {-1, -1};               // which column tile each scale/bias buffer holds
         for (int t = t_lo; t < t_hi && !dead; ++t, ++it) {
             int mt, nt;
             decode_tile(t, mt, nt);
             const int n0 = nt * BN;
             const uint32_t buf = it & 1, aph = (it >> 1) & 1;
-            float* sc = s_scale + buf * BN;
-            float* bi = s_bias + buf * BN;
-            if (loaded_nt[buf] != nt) {            // same decision in every epilogue thread
-                for (int i = et; i < BN; i += EPI_THREADS) {
-                    const int n = n0 + i;
-                    sc[i] = (n < g.N) ? g.x_scale * __ldg(g.w_scale + n) : 0.f;
-                    bi[i] = (g.bias && n < g.N) ? __ldg(g.bias + n) : 0.f;
-                }
-                asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
-                loaded_nt[buf] = nt;
-            }
 
             // where this thread's row goes
             bool row_valid;
@@ -645,62 +649,103 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                 const uint32_t t_addr = tmem_base + buf * BN + half * HALF + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll
                 for (int c0 = 0; c0 < CHUNKS; c0 += G) {
-                if (ncol0 + c0 * 32 >= g.N)
-                    break;
-                uint32_t r[G][32];
+                    if (ncol0 + c0 * 32 >= g.N)
+                        break;
+                    uint32_t r[G][32];
 #pragma unroll
-                for (int c = 0; c < G; ++c)
-                    tmem_ld32(t_addr + (c0 + c) * 32, r[c]);
-                tmem_ld_wait();
-                if (row_valid) {
+                    for (int c = 0; c < G; ++c)
+                        tmem_ld32(t_addr + (c0 + c) * 32, r[c]);
+                    tmem_ld_wait();
 #pragma unroll
                     for (int cl = 0; cl < G; ++cl) {
-                        const int c = c0 + cl;
-                        const int nb = ncol0 + c * 32;
-                        const float* scc = sc + half * HALF + c * 32;
-                        const float* bic = bi + half * HALF + c * 32;
-                        const float4* sc4 = reinterpret_cast<const float4*>(scc);
-                        const float4* bi4 = reinterpret_cast<const float4*>(bic);
-                        if (nb + 32 <= g.N) {
-                            if (g.mode == MODE_ROWS) {
-                                if (g.N % 4 == 0) {
-                                    float4* dst = reinterpret_cast<float4*>(yrow + nb);
+                        const int nb = ncol0 + (c0 + cl) * 32;
+                        if (nb >= g.N)
+                            break;
+                        const bool full = nb + 32 <= g.N;
+                        // dequantize + bias in place
+                        if (g.stage_scales) {
+                            const float4* s4 = reinterpret_cast<const float4*>(s_scale + nb);
+                            const float4* b4 = reinterpret_cast<const float4*>(s_bias + nb);
 #pragma unroll
-                                    for (int j = 0; j < 8; ++j) {
-                                        const float4 s4 = sc4[j], b4 = bi4[j];
-                                        float4 v;
-                                        v.x = fmaf(__uint_as_float(r[cl][4 * j + 0]), s4.x, b4.x);
-                                        v.y = fmaf(__uint_as_float(r[cl][4 * j + 1]), s4.y, b4.y);
-                                        v.z = fmaf(__uint_as_float(r[cl][4 * j + 2]), s4.z, b4.z);
-                                        v.w = fmaf(__uint_as_float(r[cl][4 * j + 3]), s4.w, b4.w);
-                                        dst[j] = v;
-                                    }
-                                } else {
+                            for (int j = 0; j < 8; ++j) {
+                                const float4 sv = s4[j], bv = b4[j];
+                                r[cl][4 * j + 0] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 0]), sv.x, bv.x));
+                                r[cl][4 * j + 1] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 1]), sv.y, bv.y));
+                                r[cl][4 * j + 2] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 2]), sv.z, bv.z));
+                                r[cl][4 * j + 3] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 3]), sv.w, bv.w));
+                            }
+                        } else if (full && g.vec_scale) {
+                            const float4* s4 = reinterpret_cast<const float4*>(g.w_scale + nb);
+                            const float4* b4 = reinterpret_cast<const float4*>(g.bias + nb);
 #pragma unroll
-                                    for (int j = 0; j < 32; ++j)
-                                        yrow[nb + j] = fmaf(__uint_as_float(r[cl][j]), scc[j], bic[j]);
-                                }
-                            } else {
-                                float* dst = yrow + (int64_t)nb * nstride;
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) {
-                                    const float4 s4 = sc4[j], b4 = bi4[j];
-                                    dst[0] = fmaf(__uint_as_float(r[cl][4 * j + 0]), s4.x, b4.x);
-                                    dst[nstride] = fmaf(__uint_as_float(r[cl][4 * j + 1]), s4.y, b4.y);
-                                    dst[2 * nstride] = fmaf(__uint_as_float(r[cl][4 * j + 2]), s4.z, b4.z);
-                                    dst[3 * nstride] = fmaf(__uint_as_float(r[cl][4 * j + 3]), s4.w, b4.w);
-                                    dst += 4 * nstride;
-                                }
+                            for (int j = 0; j < 8; ++j) {
+                                const float4 sv = __ldg(s4 + j);
+                                const float4 bv = g.bias ? __ldg(b4 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                r[cl][4 * j + 0] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 0]), g.x_scale * sv.x, bv.x));
+                                r[cl][4 * j + 1] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 1]), g.x_scale * sv.y, bv.y));
+                                r[cl][4 * j + 2] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 2]), g.x_scale * sv.z, bv.z));
+                                r[cl][4 * j + 3] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 3]), g.x_scale * sv.w, bv.w));
                             }
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
-                                if (nb + j < g.N)
-                                    yrow[(int64_t)(nb + j) * nstride] = fmaf(__uint_as_float(r[cl][j]), scc[j], bic[j]);
+                                const bool in = nb + j < g.N;
+                                const float sv = in ? __ldg(g.w_scale + nb + j) : 0.f;
+                                const float bv = (in && g.bias) ? __ldg(g.bias + nb + j) : 0.f;
+                                r[cl][j] = __float_as_uint(fmaf(__uint_as_float(r[cl][j]), g.x_scale * sv, bv));
+                            }
+                        }
+                        if (g.y_tma) {
+                            // the buffer is free once the previous store has read it
+                            if (lane == 0)
+                                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                            __syncwarp();
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                *reinterpret_cast<uint4*>(stage + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                                    make_uint4(r[cl][4 * j], r[cl][4 * j + 1], r[cl][4 * j + 2], r[cl][4 * j + 3]);
+                            fence_proxy_async();
+                            __syncwarp();
+                            if (lane == 0) {
+                                asm volatile(
+                                    "cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                    ::"l"(&tmY), "r"(smem_u32(stage)), "r"(nb), "r"(mt * BM + quarter * 32)
+                                    : "memory");
+                                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                            }
+                        } else if (row_valid) {
+                            if (g.mode == MODE_ROWS) {
+                                if (full && g.N % 4 == 0) {
+                                    uint4* dst = reinterpret_cast<uint4*>(yrow + nb);
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j)
+                                        dst[j] = make_uint4(r[cl][4 * j], r[cl][4 * j + 1], r[cl][4 * j + 2], r[cl][4 * j + 3]);
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j)
+                                        if (nb + j < g.N)
+                                            yrow[nb + j] = __uint_as_float(r[cl][j]);
+                                }
+                            } else {
+                                float* dst = yrow + (int64_t)nb * nstride;
+                                if (full) {
+#pragma unroll
+                                    for (int j = 0; j < 32; j += 4) {
+                                        dst[0] = __uint_as_float(r[cl][j]);
+                                        dst[nstride] = __uint_as_float(r[cl][j + 1]);
+                                        dst[2 * nstride] = __uint_as_float(r[cl][j + 2]);
+                                        dst[3 * nstride] = __uint_as_float(r[cl][j + 3]);
+                                        dst += 4 * nstride;
+                                    }
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j)
+                                        if (nb + j < g.N)
+                                            dst[(int64_t)j * nstride] = __uint_as_float(r[cl][j]);
+                                }
                             }
                         }
                     }
-                }
                 }
             }
             // hand the accumulator back to the MMA warp
@@ -709,6 +754,8 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             if (lane == 0)
                 mbar_arrive(acc_empty + 8 * buf);
         }
+        if (g.y_tma && lane == 0)
+            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // the staging buffer must outlive its stores
         if (dead)
             atomicMin(g.status, FPQ_ERR_TIMEOUT);
     } else if (FUSED && warp == 2 + NUM_EPI_WARPS + NUM_XFORM_WARPS) {
@@ -858,7 +905,8 @@ static DeviceInfo* device_info()
 }
 
 template <int BN, bool FUSED>
-static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs& g, cudaStream_t st)
+static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY, GemmArgs& g,
+                                 cudaStream_t st)
 {
     // Split the shared-memory budget between the two rings.  A barrier handshake costs the
     // single issuing thread a few hundred cycles, so every stage is made to carry 8-36 MMAs;
@@ -866,7 +914,9 @@ static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB,
     DeviceInfo* di = device_info();
     if (!di)
         return FPQ_ERR_CUDA;
-    const int ctl = 320 + 4 * BN * 4 + 1024;
+    const int n_pad = (g.N + 31) & ~31;
+    g.stage_scales = (n_pad * 8 <= 16384) ? 1 : 0;
+    const int ctl = 512 + 1024 + (g.y_tma ? epi_warps(FUSED) * 4096 : 0) + (g.stage_scales ? n_pad * 8 : 0);
     const int budget = SMEM_BUDGET - ctl;
     const int b_block = BN * BK;
     const int a_min_span = (g.mode == MODE_FLAT) ? g.taps : 1;
@@ -964,7 +1014,7 @@ static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = g.wait_prior_grid ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, fpq_gemm_kernel<BN, FUSED>, tmA, tmB, (const GemmArgs)g) == cudaSuccess ? FPQ_OK
+    return cudaLaunchKernelEx(&cfg, fpq_gemm_kernel<BN, FUSED>, tmA, tmB, tmY, (const GemmArgs)g) == cudaSuccess ? FPQ_OK
                                                                                                       : FPQ_ERR_CUDA;
 }
 
@@ -1089,6 +1139,22 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return FPQ_ERR_CUDA;
 
+    // row-major output through TMA stores
+    CUtensorMap tmY = tmA;
+    g.y_tma = 0;
+    g.vec_scale = ((uintptr_t)p.w_scale % 16 == 0) && (p.bias == nullptr || (uintptr_t)p.bias % 16 == 0);
+    if (!p.conv && p.N % 4 == 0 && (uintptr_t)p.y % 16 == 0) {
+        cuuint64_t dimsY[2] = {(cuuint64_t)p.N, (cuuint64_t)p.M};
+        cuuint64_t stridesY[1] = {(cuuint64_t)p.N * 4};
+        cuuint32_t boxY[2] = {32, 32};
+        cuuint32_t estrY[2] = {1, 1};
+        if (enc(&tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void*)p.y, dimsY, stridesY, boxY, estrY,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return FPQ_ERR_CUDA;
+        g.y_tma = 1;
+    }
+
     const bool fused = p.x != nullptr && g.mode != MODE_TAPS;
     if (fused) {
         g.x = p.x;
@@ -1098,11 +1164,11 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
         g.W = p.W;
         g.pad = p.pad;
         g.wait_prior_grid = 0;
-        return BN == 64 ? launch_variant<64, true>(tmA, tmB, g, st) : launch_variant<128, true>(tmA, tmB, g, st);
+        return BN == 64 ? launch_variant<64, true>(tmA, tmB, tmY, g, st) : launch_variant<128, true>(tmA, tmB, tmY, g, st);
     }
     if (p.x != nullptr)
         return FPQ_ERR_UNSUPPORTED;     // the caller falls back to the two-kernel route
-    return BN == 64 ? launch_variant<64, false>(tmA, tmB, g, st) : launch_variant<128, false>(tmA, tmB, g, st);
+    return BN == 64 ? launch_variant<64, false>(tmA, tmB, tmY, g, st) : launch_variant<128, false>(tmA, tmB, tmY, g, st);
 }
 
 }  // namespace fpq
