@@ -231,7 +231,7 @@ __device__ __forceinline__ void fill_chunk_rows(const GemmArgs& g, uint8_t* dst,
 // FUSED = false: the activation operand is read as codes (TMA, written by a quantize kernel).
 // FUSED = true : 8 more warps read the FP32 activations and quantize them straight into the
 //                activation ring, so the codes never exist in global memory.
-template <int BN, bool FUSED>
+template <int BN, bool FUSED, int MODE>
 __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                                   const __grid_constant__ CUtensorMap tmB,
                                                                   const __grid_constant__ CUtensorMap tmY,
@@ -269,8 +269,11 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     const int total_tiles = g.m_tiles * g.n_tiles;
     // every CTA walks a contiguous range of the tile list, so consecutive tiles share the row tile
     // (or, in column-tile-major order, the column tile) and its resident operand
-    const int t_lo = (int)((int64_t)blockIdx.x * total_tiles / gridDim.x);
-    const int t_hi = (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x);
+    // (a_resident); otherwise the CTAs interleave, so that at any time the whole GPU works on one
+    // compact region of the activations and of the output
+    const int t_lo = g.a_resident ? (int)((int64_t)blockIdx.x * total_tiles / gridDim.x) : (int)blockIdx.x;
+    const int t_hi = g.a_resident ? (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x) : total_tiles;
+    const int t_step = g.a_resident ? 1 : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 8; ++s) {
@@ -309,18 +312,18 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     // leaves its loop, the other roles then run into their own limits and follow.
     if (warp == 0) {
         // ---------------- TMA producer (one thread; its loops never divide) ----------------
-        if (lane == 0) {
+        if (elect_one()) {
             uint32_t sa = 0, pa = 0, sb = 0, pb = 0;   // stage and phase of the next load per ring
             uint32_t na = 0, nb = 0;                   // stages issued (for the abort path)
             int resident_nt = -1, resident_mt = -1;
             bool dead = false;
             bool prior_done = !g.wait_prior_grid;
-            for (int t = t_lo; t < t_hi && !dead; ++t) {
+            for (int t = t_lo; t < t_hi && !dead; t += t_step) {
                 int mt, nt;
                 decode_tile(t, mt, nt);
                 const int n0 = nt * BN;
                 int x0 = 0, y0 = 0, b0 = 0;
-                if (g.mode == MODE_TAPS) {
+                if (MODE == MODE_TAPS) {
                     const uint32_t r1 = fdiv((uint32_t)mt, g.div_tx);
                     x0 = (mt - (int)r1 * g.tiles_x) * g.Wt * g.stride;
                     const uint32_t r2 = fdiv(r1, g.div_ty);
@@ -358,10 +361,10 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                         // activation stage: the data of the next a_span blocks
                         if (!mbar_wait(a_empty + 8 * sa, pa ^ 1)) { dead = true; break; }
                         const int nblocks = min(g.a_span, g.nblk - j);
-                        const int nloads = (g.mode == MODE_TAPS) ? nblocks : nblocks / g.taps;
+                        const int nloads = (MODE == MODE_TAPS) ? nblocks : nblocks / g.taps;
                         mbar_expect_tx(a_full + 8 * sa, (uint32_t)nloads * g.a_chunk_tx);
                         uint32_t dst = a_ring + sa * g.a_stage_bytes;
-                        if (g.mode == MODE_TAPS) {
+                        if (MODE == MODE_TAPS) {
                             int c2 = cc, t2 = tap, r2 = r, s2 = sx;
                             for (int l = 0; l < nloads; ++l, dst += g.a_chunk_bytes) {
                                 tma_load_4d(dst, &tmA, a_full + 8 * sa, c2 * BK, x0 + s2, y0 + r2, b0);
@@ -412,7 +415,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         // positions are kept as descriptor low words (16-byte units) and the two common
         // loop shapes (3x3 taps over one loaded chunk; one block per chunk) are
         // straight-line code.
-        if (lane == 0) {
+        if (elect_one()) {
             uint32_t sa = 0, pa = 0, sb = 0, pb = 0, it = 0;
             uint32_t sa0 = 0, pa0 = 0;                 // ring position of the resident activation panel
             int resident_nt = -1, resident_mt = -1;
@@ -420,7 +423,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             const uint32_t a_chunk_step = (uint32_t)g.a_chunk_bytes >> 4;
             const uint32_t b_res = smem_desc_lo(b_ring);           // resident weights start here
             const uint32_t HI = SMEM_DESC_HI_K_SW128;
-            for (int t = t_lo; t < t_hi && !dead; ++t, ++it) {
+            for (int t = t_lo; t < t_hi && !dead; t += t_step, ++it) {
                 int mt, nt;
                 decode_tile(t, mt, nt);
                 const bool new_b = !(g.b_resident && resident_nt == nt);
@@ -436,9 +439,9 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                 resident_mt = mt;
                 if (reuse_a) { sa = sa0; pa = pa0; } else { sa0 = sa; pa0 = pa; }
                 bool keep_a = false;
-                if (g.a_resident && t + 1 < t_hi) {
+                if (g.a_resident && t + t_step < t_hi) {
                     int mt2, nt2;
-                    decode_tile(t + 1, mt2, nt2);
+                    decode_tile(t + t_step, mt2, nt2);
                     keep_a = mt2 == mt;
                 }
                 const uint32_t buf = it & 1, aph = (it >> 1) & 1;
@@ -448,7 +451,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
 
-                if (g.mode == MODE_FLAT && g.taps == 9 && g.S == 3) {
+                if (MODE == MODE_FLAT && g.taps == 9 && g.S == 3) {
                     const uint32_t Wp8 = (uint32_t)g.Wp * 8u;
                     const int chunks_per_stage = g.a_span / 9;
                     for (int cc = 0; cc < g.cchunks && !dead;) {
@@ -489,7 +492,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                             mma_commit(a_empty + 8 * sa);
                         if (++sa == (uint32_t)g.a_stages) { sa = 0; pa ^= 1; }
                     }
-                } else if (g.taps == 1 && g.mode != MODE_TAPS && g.a_span <= 4 &&
+                } else if (g.taps == 1 && MODE != MODE_TAPS && g.a_span <= 4 &&
                            (g.b_resident || g.b_span == g.a_span)) {
                     // one block per 128-wide chunk; a stage carries up to 4 chunks of both operands
                     for (int cc = 0; cc < g.cchunks && !dead;) {
@@ -531,7 +534,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                     uint32_t a_chunk_lo = 0;               // FLAT/ROWS: current chunk in its stage
                     uint32_t row_off8 = 0;                 // FLAT: (r * Wp + s) * 8 of the current tap
                     const uint32_t row_wrap8 = (uint32_t)(g.Wp - g.S) * 8u;
-                    const bool flat = g.mode == MODE_FLAT, taps_mode = g.mode == MODE_TAPS;
+                    const bool flat = MODE == MODE_FLAT, taps_mode = MODE == MODE_TAPS;
                     int tap = 0, sx = 0, ja = 0, jb = 0;
                     for (int j = 0; j < g.nblk; ++j) {
                         if (ja == 0) {
@@ -602,7 +605,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         uint8_t* stage = smem + ctl_off + (warp - 2) * 4096;
         uint32_t it = 0;
         bool dead = false;
-        for (int t = t_lo; t < t_hi && !dead; ++t, ++it) {
+        for (int t = t_lo; t < t_hi && !dead; t += t_step, ++it) {
             int mt, nt;
             decode_tile(t, mt, nt);
             const int n0 = nt * BN;
@@ -612,14 +615,14 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             bool row_valid;
             float* yrow;
             int64_t nstride;
-            if (g.mode == MODE_ROWS) {
+            if (MODE == MODE_ROWS) {
                 const int64_t m = (int64_t)mt * BM + row;
                 row_valid = m < g.M;
                 nstride = 1;
                 yrow = g.y + m * g.N;
             } else {
                 int ox, oy, b;
-                if (g.mode == MODE_FLAT) {
+                if (MODE == MODE_FLAT) {
                     const uint32_t q = (uint32_t)mt * BM + row;
                     b = (int)fdiv(q, g.div_HpWp);
                     const uint32_t rem = q - (uint32_t)b * g.HpWp;
@@ -714,7 +717,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                             }
                         } else if (row_valid) {
-                            if (g.mode == MODE_ROWS) {
+                            if (MODE == MODE_ROWS) {
                                 if (full && g.N % 4 == 0) {
                                     uint4* dst = reinterpret_cast<uint4*>(yrow + nb);
 #pragma unroll
@@ -767,7 +770,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         auto prefetch_tile = [&](int t) {
             int mt, nt;
             decode_tile(t, mt, nt);
-            if (g.mode == MODE_ROWS) {
+            if (MODE == MODE_ROWS) {
                 // 128 rows of C floats: one contiguous span
                 const int64_t m0 = (int64_t)mt * BM;
                 const int64_t m1 = min(m0 + BM, g.M);
@@ -802,7 +805,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             }
         };
         int last_mt = -1;
-        for (int t = t_lo; t < t_hi; ++t) {
+        for (int t = t_lo; t < t_hi; t += t_step) {
             int mt, nt;
             decode_tile(t, mt, nt);
             if (mt == last_mt)
@@ -819,7 +822,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         uint32_t sa = 0, pa = 0;
         bool dead = false, nan = false;
         int resident_mt = -1;
-        for (int t = t_lo; t < t_hi && !dead; ++t) {
+        for (int t = t_lo; t < t_hi && !dead; t += t_step) {
             int mt, nt;
             decode_tile(t, mt, nt);
             if (g.a_resident && mt == resident_mt)
@@ -830,7 +833,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                 const int nch = min(chunks_per_stage, g.cchunks - cc);
                 uint8_t* dst = smem + sa * g.a_stage_bytes;
                 for (int l = 0; l < nch; ++l, dst += g.a_chunk_bytes) {
-                    if (g.mode == MODE_ROWS)
+                    if (MODE == MODE_ROWS)
                         fill_chunk_rows(g, dst, (int64_t)mt * BM, (cc + l) * BK, tid, nan);
                     else
                         fill_chunk_nchw(g, dst, (uint32_t)mt * BM, rows, (cc + l) * BK, tw, lane, nan);
@@ -886,7 +889,7 @@ static int pow2_at_least(int v)
 
 struct DeviceInfo {
     int sms;
-    bool smem_set[4];
+    bool smem_set[12];
 };
 
 static DeviceInfo* device_info()
@@ -904,8 +907,8 @@ static DeviceInfo* device_info()
     return &info[dev];
 }
 
-template <int BN, bool FUSED>
-static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY, GemmArgs& g,
+template <int BN, bool FUSED, int MODE>
+static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY, GemmArgs& g,
                                  cudaStream_t st)
 {
     // Split the shared-memory budget between the two rings.  A barrier handshake costs the
@@ -995,9 +998,9 @@ static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB,
         return FPQ_ERR_UNSUPPORTED;
     g.div_tiles = make_fastdiv((uint32_t)(g.m_fastest ? g.m_tiles : g.n_tiles));
     const int dyn = g.a_stages * g.a_stage_bytes + g.b_stages * g.b_stage_bytes + ctl;
-    const int slot = (BN == 64 ? 0 : 1) + (FUSED ? 2 : 0);
+    const int slot = (BN == 64 ? 0 : 1) + (FUSED ? 2 : 0) + 4 * MODE;
     if (!di->smem_set[slot]) {
-        if (cudaFuncSetAttribute(fpq_gemm_kernel<BN, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) !=
+        if (cudaFuncSetAttribute(fpq_gemm_kernel<BN, FUSED, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) !=
             cudaSuccess)
             return FPQ_ERR_CUDA;
         di->smem_set[slot] = true;
@@ -1014,8 +1017,23 @@ static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = g.wait_prior_grid ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, fpq_gemm_kernel<BN, FUSED>, tmA, tmB, tmY, (const GemmArgs)g) == cudaSuccess ? FPQ_OK
+    return cudaLaunchKernelEx(&cfg, fpq_gemm_kernel<BN, FUSED, MODE>, tmA, tmB, tmY, (const GemmArgs)g) == cudaSuccess ? FPQ_OK
                                                                                                       : FPQ_ERR_CUDA;
+}
+
+template <int BN, bool FUSED>
+static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY, GemmArgs& g,
+                                 cudaStream_t st)
+{
+    // one instantiation per addressing mode keeps every kernel's code small: the single MMA-issuing
+    // thread is sensitive to instruction fetch
+    if (g.mode == MODE_ROWS)
+        return launch_mode<BN, FUSED, MODE_ROWS>(tmA, tmB, tmY, g, st);
+    if (g.mode == MODE_FLAT)
+        return launch_mode<BN, FUSED, MODE_FLAT>(tmA, tmB, tmY, g, st);
+    if (FUSED)
+        return FPQ_ERR_UNSUPPORTED;
+    return launch_mode<BN, false, MODE_TAPS>(tmA, tmB, tmY, g, st);
 }
 
 fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
