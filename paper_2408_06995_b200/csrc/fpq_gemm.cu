@@ -89,6 +89,7 @@ struct GemmArgs {
     int y_tma;                 // row-major output leaves through TMA stores
     int vec_scale;             // w_scale / bias are 16-byte aligned
     int stage_scales;          // x_scale * w_scale[n] and bias[n] of all N columns sit in shared memory
+    int contiguous;            // tile order: 1 = every CTA walks a contiguous range, 0 = CTAs interleave
     int a_resident;            // a row tile's whole activation panel stays in the ring while the CTA walks its column tiles
     uint32_t a_chunk_tx, b_block_tx;   // bytes one load reports to its barrier
     const float* w_scale;
@@ -269,11 +270,11 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     const int total_tiles = g.m_tiles * g.n_tiles;
     // every CTA walks a contiguous range of the tile list, so consecutive tiles share the row tile
     // (or, in column-tile-major order, the column tile) and its resident operand
-    // (a_resident); otherwise the CTAs interleave, so that at any time the whole GPU works on one
+    // (a resident operand that several tiles share); otherwise the CTAs interleave, so that at any time the whole GPU works on one
     // compact region of the activations and of the output
-    const int t_lo = g.a_resident ? (int)((int64_t)blockIdx.x * total_tiles / gridDim.x) : (int)blockIdx.x;
-    const int t_hi = g.a_resident ? (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x) : total_tiles;
-    const int t_step = g.a_resident ? 1 : (int)gridDim.x;
+    const int t_lo = g.contiguous ? (int)((int64_t)blockIdx.x * total_tiles / gridDim.x) : (int)blockIdx.x;
+    const int t_hi = g.contiguous ? (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x) : total_tiles;
+    const int t_step = g.contiguous ? 1 : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 8; ++s) {
@@ -996,6 +997,7 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
     g.b_stage_bytes = g.b_span * b_block;
     if (g.a_stages < 1 || g.b_stages < 1 || (!g.b_resident && g.b_stages < 2))
         return FPQ_ERR_UNSUPPORTED;
+    g.contiguous = (g.a_resident || (g.b_resident && g.n_tiles > 1)) ? 1 : 0;
     g.div_tiles = make_fastdiv((uint32_t)(g.m_fastest ? g.m_tiles : g.n_tiles));
     const int dyn = g.a_stages * g.a_stage_bytes + g.b_stages * g.b_stage_bytes + ctl;
     const int slot = (BN == 64 ? 0 : 1) + (FUSED ? 2 : 0) + 4 * MODE;
