@@ -91,6 +91,7 @@ struct GemmArgs {
     int stage_scales;          // x_scale * w_scale[n] and bias[n] of all N columns sit in shared memory
     int contiguous;            // tile order: 1 = every CTA walks a contiguous range, 0 = CTAs interleave
     int a_resident;            // a row tile's whole activation panel stays in the ring while the CTA walks its column tiles
+    int ksplit;                // > 1: the CTAs of a cluster of this size share one output tile, each reducing a range of chunks
     uint32_t a_chunk_tx, b_block_tx;   // bytes one load reports to its barrier
     const float* w_scale;
     float x_scale;
@@ -229,6 +230,29 @@ __device__ __forceinline__ void fill_chunk_rows(const GemmArgs& g, uint8_t* dst,
     }
 }
 
+// ---- thread-block cluster: barrier over all threads of all CTAs, and reads of a peer CTA's shared memory
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+__device__ __forceinline__ float ld_peer_smem(uint32_t local_addr, uint32_t peer)
+{
+    uint32_t remote;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(peer));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
+
 // FUSED = false: the activation operand is read as codes (TMA, written by a quantize kernel).
 // FUSED = true : 8 more warps read the FP32 activations and quantize them straight into the
 //                activation ring, so the codes never exist in global memory.
@@ -272,9 +296,19 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     // (or, in column-tile-major order, the column tile) and its resident operand
     // (a resident operand that several tiles share); otherwise the CTAs interleave, so that at any time the whole GPU works on one
     // compact region of the activations and of the output
-    const int t_lo = g.contiguous ? (int)((int64_t)blockIdx.x * total_tiles / gridDim.x) : (int)blockIdx.x;
-    const int t_hi = g.contiguous ? (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x) : total_tiles;
-    const int t_step = g.contiguous ? 1 : (int)gridDim.x;
+    // Split reduction (few tiles, long reduction): a cluster of ksplit CTAs owns one tile, CTA k of the
+    // cluster reduces the chunks [c_lo, c_hi) into its own accumulator; the partial sums meet in shared
+    // memory after the role loops below.
+    const int ksplit = g.ksplit;
+    const uint32_t krank = ksplit > 1 ? cluster_rank() : 0u;
+    const int c_lo = ksplit > 1 ? (int)krank * g.cchunks / ksplit : 0;
+    const int c_hi = ksplit > 1 ? ((int)krank + 1) * g.cchunks / ksplit : g.cchunks;
+    const int nblk = (c_hi - c_lo) * g.taps;
+    const int t_lo = ksplit > 1 ? (int)blockIdx.x / ksplit
+                                : g.contiguous ? (int)((int64_t)blockIdx.x * total_tiles / gridDim.x) : (int)blockIdx.x;
+    const int t_hi = ksplit > 1 ? t_lo + 1
+                                : g.contiguous ? (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x) : total_tiles;
+    const int t_step = (ksplit > 1 || g.contiguous) ? 1 : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 8; ++s) {
@@ -309,6 +343,39 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         else             { mt = q; nt = t - q * g.n_tiles; }
     };
 
+    // row `row` of row tile mt -> its address in y (column 0), the column stride, and whether it exists
+    auto row_target = [&](int mt, int row, bool& row_valid, float*& yrow, int64_t& nstride) {
+        if (MODE == MODE_ROWS) {
+            const int64_t m = (int64_t)mt * BM + row;
+            row_valid = m < g.M;
+            nstride = 1;
+            yrow = g.y + m * g.N;
+        } else {
+            int ox, oy, b;
+            if (MODE == MODE_FLAT) {
+                const uint32_t q = (uint32_t)mt * BM + row;
+                b = (int)fdiv(q, g.div_HpWp);
+                const uint32_t rem = q - (uint32_t)b * g.HpWp;
+                oy = (int)fdiv(rem, g.div_Wp);
+                ox = (int)rem - oy * g.Wp;
+            } else {
+                const uint32_t r1 = fdiv((uint32_t)mt, g.div_tx);
+                const int x0 = (mt - (int)r1 * g.tiles_x) * g.Wt;
+                const uint32_t r2 = fdiv(r1, g.div_ty);
+                const int y0 = ((int)r1 - (int)r2 * g.tiles_y) * g.Ht;
+                const int b0 = (int)r2 * g.Bt;
+                const uint32_t q1 = fdiv((uint32_t)row, g.div_Wt);
+                ox = x0 + (row - (int)q1 * g.Wt);
+                const uint32_t q2 = fdiv(q1, g.div_Ht);
+                oy = y0 + ((int)q1 - (int)q2 * g.Ht);
+                b = b0 + (int)q2;
+            }
+            row_valid = ox < g.Wo && oy < g.Ho && b < g.B;
+            nstride = (int64_t)g.Ho * g.Wo;
+            yrow = g.y + ((int64_t)b * g.N * g.Ho + oy) * g.Wo + ox;   // + n * Ho * Wo
+        }
+    };
+
     // Every wait below is bounded; a role whose wait expires records FPQ_ERR_TIMEOUT and
     // leaves its loop, the other roles then run into their own limits and follow.
     if (warp == 0) {
@@ -335,10 +402,10 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                 resident_nt = nt;
                 const bool load_a = !(g.a_resident && resident_mt == mt);
                 resident_mt = mt;
-                int cc = 0, tap = 0, r = 0, sx = 0;    // block j = (cc, tap), tap = (r, sx)
+                int cc = c_lo, tap = 0, r = 0, sx = 0; // block j = (cc, tap), tap = (r, sx)
                 int ja = 0, jb = 0;                    // position inside the current A / B stage
                 bool early_b = false;
-                for (int j = 0; j < g.nblk; ++j) {
+                for (int j = 0; j < nblk; ++j) {
                     if (jb == 0 && load_b && !prior_done && g.b_resident) {
                         // the weights do not depend on the kernel in front: fetch them before waiting for it
                         if (!mbar_wait(b_empty + 8 * sb, pb ^ 1)) { dead = true; break; }
@@ -361,7 +428,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                     if (ja == 0 && !FUSED && load_a) {
                         // activation stage: the data of the next a_span blocks
                         if (!mbar_wait(a_empty + 8 * sa, pa ^ 1)) { dead = true; break; }
-                        const int nblocks = min(g.a_span, g.nblk - j);
+                        const int nblocks = min(g.a_span, nblk - j);
                         const int nloads = (MODE == MODE_TAPS) ? nblocks : nblocks / g.taps;
                         mbar_expect_tx(a_full + 8 * sa, (uint32_t)nloads * g.a_chunk_tx);
                         uint32_t dst = a_ring + sa * g.a_stage_bytes;
@@ -383,7 +450,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                     }
                     if (jb == 0 && load_b && !early_b) {
                         if (!mbar_wait(b_empty + 8 * sb, pb ^ 1)) { dead = true; break; }
-                        const int nblocks = min(g.b_span, g.nblk - j);
+                        const int nblocks = min(g.b_span, nblk - j);
                         mbar_expect_tx(b_full + 8 * sb, (uint32_t)nblocks * g.b_block_tx);
                         uint32_t dst = b_ring + sb * g.b_stage_bytes;
                         int c2 = cc, t2 = tap;
@@ -455,12 +522,12 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                 if (MODE == MODE_FLAT && g.taps == 9 && g.S == 3) {
                     const uint32_t Wp8 = (uint32_t)g.Wp * 8u;
                     const int chunks_per_stage = g.a_span / 9;
-                    for (int cc = 0; cc < g.cchunks && !dead;) {
+                    for (int cc = c_lo; cc < c_hi && !dead;) {
                         if (!reuse_a)
                             if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
                         tc_fence_after();
                         const uint32_t abase = smem_desc_lo(a_ring + sa * g.a_stage_bytes);
-                        const int nch = min(chunks_per_stage, g.cchunks - cc);
+                        const int nch = min(chunks_per_stage, c_hi - cc);
                         for (int c = 0; c < nch && !dead; ++c, ++cc) {
                             const uint32_t ac = abase + c * a_chunk_step;
                             const uint32_t bres = b_res + (uint32_t)cc * 9u * BSTEP;
@@ -476,7 +543,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                                 const uint32_t al = ac + (tap / 3) * Wp8 + (tap % 3) * 8u;
                                 const uint32_t bl = g.b_resident ? bres + tap * BSTEP : bst + (tap % 3) * BSTEP;
                                 // 32 reduction elements = 32 bytes inside the swizzled row: +2 units
-                                if (tap == 0 && cc == 0)
+                                if (tap == 0 && cc == c_lo)
                                     mma_f8f6f4<false>(d_tmem, al, bl, HI, g.idesc);
                                 else
                                     mma_f8f6f4<true>(d_tmem, al, bl, HI, g.idesc);
@@ -496,7 +563,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                 } else if (g.taps == 1 && MODE != MODE_TAPS && g.a_span <= 4 &&
                            (g.b_resident || g.b_span == g.a_span)) {
                     // one block per 128-wide chunk; a stage carries up to 4 chunks of both operands
-                    for (int cc = 0; cc < g.cchunks && !dead;) {
+                    for (int cc = c_lo; cc < c_hi && !dead;) {
                         if (!reuse_a)
                             if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
                         uint32_t bbase = b_res + (uint32_t)cc * BSTEP;
@@ -506,12 +573,12 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                         }
                         tc_fence_after();
                         const uint32_t abase = smem_desc_lo(a_ring + sa * g.a_stage_bytes);
-                        const int n = min(g.a_span, g.cchunks - cc);
+                        const int n = min(g.a_span, c_hi - cc);
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
                             if (c < n) {
                                 const uint32_t al = abase + c * (BM * BK / 16), bl = bbase + c * BSTEP;
-                                if (c == 0 && cc == 0)
+                                if (c == 0 && cc == c_lo)
                                     mma_f8f6f4<false>(d_tmem, al, bl, HI, g.idesc);
                                 else
                                     mma_f8f6f4<true>(d_tmem, al, bl, HI, g.idesc);
@@ -537,7 +604,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                     const uint32_t row_wrap8 = (uint32_t)(g.Wp - g.S) * 8u;
                     const bool flat = MODE == MODE_FLAT, taps_mode = MODE == MODE_TAPS;
                     int tap = 0, sx = 0, ja = 0, jb = 0;
-                    for (int j = 0; j < g.nblk; ++j) {
+                    for (int j = 0; j < nblk; ++j) {
                         if (ja == 0) {
                             if (!reuse_a)
                                 if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
@@ -558,7 +625,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                         mma_f8f6f4<true>(d_tmem, al + 2, b_lo + 2, HI, g.idesc);
                         mma_f8f6f4<true>(d_tmem, al + 4, b_lo + 4, HI, g.idesc);
                         mma_f8f6f4<true>(d_tmem, al + 6, b_lo + 6, HI, g.idesc);
-                        const bool last = (j == g.nblk - 1);
+                        const bool last = (j == nblk - 1);
                         b_lo += BSTEP;
                         if (++jb == g.b_span || last) {
                             jb = 0;
@@ -616,40 +683,31 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             bool row_valid;
             float* yrow;
             int64_t nstride;
-            if (MODE == MODE_ROWS) {
-                const int64_t m = (int64_t)mt * BM + row;
-                row_valid = m < g.M;
-                nstride = 1;
-                yrow = g.y + m * g.N;
-            } else {
-                int ox, oy, b;
-                if (MODE == MODE_FLAT) {
-                    const uint32_t q = (uint32_t)mt * BM + row;
-                    b = (int)fdiv(q, g.div_HpWp);
-                    const uint32_t rem = q - (uint32_t)b * g.HpWp;
-                    oy = (int)fdiv(rem, g.div_Wp);
-                    ox = (int)rem - oy * g.Wp;
-                } else {
-                    const uint32_t r1 = fdiv((uint32_t)mt, g.div_tx);
-                    const int x0 = (mt - (int)r1 * g.tiles_x) * g.Wt;
-                    const uint32_t r2 = fdiv(r1, g.div_ty);
-                    const int y0 = ((int)r1 - (int)r2 * g.tiles_y) * g.Ht;
-                    const int b0 = (int)r2 * g.Bt;
-                    const uint32_t q1 = fdiv((uint32_t)row, g.div_Wt);
-                    ox = x0 + (row - (int)q1 * g.Wt);
-                    const uint32_t q2 = fdiv(q1, g.div_Ht);
-                    oy = y0 + ((int)q1 - (int)q2 * g.Ht);
-                    b = b0 + (int)q2;
-                }
-                row_valid = ox < g.Wo && oy < g.Ho && b < g.B;
-                nstride = (int64_t)g.Ho * g.Wo;
-                yrow = g.y + ((int64_t)b * g.N * g.Ho + oy) * g.Wo + ox;   // + n * Ho * Wo
-            }
+            row_target(mt, row, row_valid, yrow, nstride);
 
             if (!mbar_wait(acc_full + 8 * buf, aph)) { dead = true; }
             tc_fence_after();
             const int ncol0 = n0 + half * HALF;    // first output column of this warp
-            if (!dead && ncol0 < g.N) {
+            if (ksplit > 1) {
+                // partial sums of this CTA's chunk range: column-major [BN][128] at the start of the
+                // rings, which are idle once the accumulator is complete; the cluster adds them up below
+                float* red = reinterpret_cast<float*>(smem);
+                if (!dead && ncol0 < g.N) {
+                    const uint32_t t_addr = tmem_base + buf * BN + half * HALF + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll
+                    for (int c = 0; c < CHUNKS; ++c) {
+                        if (ncol0 + c * 32 >= g.N)
+                            break;
+                        uint32_t r[32];
+                        tmem_ld32(t_addr + c * 32, r);
+                        tmem_ld_wait();
+                        float* dst = red + (half * HALF + c * 32) * BM + row;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            dst[j * BM] = __uint_as_float(r[j]);
+                    }
+                }
+            } else if (!dead && ncol0 < g.N) {
                 const uint32_t t_addr = tmem_base + buf * BN + half * HALF + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll
                 for (int c0 = 0; c0 < CHUNKS; c0 += G) {
@@ -797,7 +855,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                 if ((int)b >= g.B || y1 < y0)
                     continue;
                 const int bytes = (y1 - y0 + 1) * g.W * 4;        // contiguous per channel
-                for (int c = lane; c < g.C; c += 32) {
+                for (int c = c_lo * BK + lane; c < min(g.C, c_hi * BK); c += 32) {
                     const char* p0 = reinterpret_cast<const char*>(
                         g.x + ((int64_t)(b * (uint32_t)g.C + (uint32_t)c) * g.H + y0) * g.W);
                     for (int o = 0; o < bytes; o += 128)
@@ -829,9 +887,9 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             if (g.a_resident && mt == resident_mt)
                 continue;                          // the panel is still in the ring
             resident_mt = mt;
-            for (int cc = 0; cc < g.cchunks;) {
+            for (int cc = c_lo; cc < c_hi;) {
                 if (!mbar_wait(a_empty + 8 * sa, pa ^ 1)) { dead = true; break; }
-                const int nch = min(chunks_per_stage, g.cchunks - cc);
+                const int nch = min(chunks_per_stage, c_hi - cc);
                 uint8_t* dst = smem + sa * g.a_stage_bytes;
                 for (int l = 0; l < nch; ++l, dst += g.a_chunk_bytes) {
                     if (MODE == MODE_ROWS)
@@ -854,6 +912,46 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             atomicMin(g.status, FPQ_ERR_TIMEOUT);
     }
 
+    if (ksplit > 1) {
+        // every thread of every CTA of the cluster arrives here (all waits above are bounded)
+        __syncwarp();
+        cluster_sync_all();
+        if (warp >= 2 && warp < 2 + NUM_EPI_WARPS) {
+            // CTA k adds up the columns k, k + ksplit, ... of the tile over all CTAs of the cluster, in
+            // rank order (the same order whatever the timing), then dequantize + bias as usual
+            int mt, nt;
+            decode_tile(t_lo, mt, nt);
+            const int e = threadIdx.x - 64;
+            const int row = e & (BM - 1);
+            bool row_valid;
+            float* yrow;
+            int64_t nstride;
+            row_target(mt, row, row_valid, yrow, nstride);
+            const uint32_t red = smem_base;
+            for (int c = (int)krank + ksplit * (e >> 7); c < BN; c += ksplit * (32 * NUM_EPI_WARPS / BM)) {
+                const int n = nt * BN + c;
+                if (n >= g.N)
+                    break;
+                const uint32_t addr = red + (uint32_t)(c * BM + row) * 4u;
+                float v[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    v[k] = k < ksplit ? ld_peer_smem(addr, (uint32_t)k) : 0.f;
+                float acc = v[0];
+#pragma unroll
+                for (int k = 1; k < 8; ++k)
+                    if (k < ksplit)
+                        acc += v[k];
+                const float sv = g.stage_scales ? s_scale[n] : g.x_scale * __ldg(g.w_scale + n);
+                const float bv = g.stage_scales ? s_bias[n] : (g.bias ? __ldg(g.bias + n) : 0.f);
+                if (row_valid)
+                    yrow[(int64_t)n * nstride] = fmaf(acc, sv, bv);
+            }
+        }
+        // nobody leaves (and frees its shared memory) while a peer may still read it
+        __syncwarp();
+        cluster_sync_all();
+    }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -891,6 +989,7 @@ static int pow2_at_least(int v)
 struct DeviceInfo {
     int sms;
     bool smem_set[12];
+    int max_clusters[2][3][9];     // [BN == 128][mode][cluster size]: clusters resident at once, 0 = not asked yet, -1 = none
 };
 
 static DeviceInfo* device_info()
@@ -906,6 +1005,49 @@ static DeviceInfo* device_info()
         info[dev].sms = v;
     }
     return &info[dev];
+}
+
+template <int BN, bool FUSED, int MODE>
+static bool allow_max_smem(DeviceInfo* di)
+{
+    const int slot = (BN == 64 ? 0 : 1) + (FUSED ? 2 : 0) + 4 * MODE;
+    if (!di->smem_set[slot]) {
+        if (cudaFuncSetAttribute(fpq_gemm_kernel<BN, FUSED, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) !=
+            cudaSuccess)
+            return false;
+        di->smem_set[slot] = true;
+    }
+    return true;
+}
+
+// How many clusters of `size` CTAs of the contraction kernel the GPU holds at once.  Asked of the
+// plain kernel for both forms, so that both take the same decision (and add partial sums in the same order).
+template <int BN, int MODE>
+static int max_clusters(DeviceInfo* di, int size)
+{
+    int& slot = di->max_clusters[BN == 64 ? 0 : 1][MODE][size];
+    if (slot == 0) {
+        slot = -1;
+        if (allow_max_smem<BN, false, MODE>(di)) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)(size * di->sms));
+            cfg.blockDim = dim3(num_threads(false));
+            cfg.dynamicSmemBytes = SMEM_BUDGET;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = (unsigned)size;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, fpq_gemm_kernel<BN, false, MODE>, &cfg) == cudaSuccess && n > 0)
+                slot = n;
+            else
+                (void)cudaGetLastError();
+        }
+    }
+    return slot;
 }
 
 template <int BN, bool FUSED, int MODE>
@@ -926,10 +1068,29 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
     const int a_min_span = (g.mode == MODE_FLAT) ? g.taps : 1;
     const int64_t b_all = (int64_t)g.nblk * b_block;
     g.a_resident = 0;
+    // Few tiles and a long reduction (the low-resolution convolutions): a cluster of ksplit CTAs
+    // shares each tile.  The split takes the largest cluster that still lets all tiles run at once,
+    // then the smallest one with the same longest chunk range.
+    g.ksplit = 1;
+    const int64_t base_tiles = (int64_t)g.m_tiles * g.n_tiles;
+    if (MODE != MODE_ROWS && g.cchunks >= 2 && base_tiles * 2 <= di->sms) {
+        int s_max = (int)(di->sms / base_tiles);
+        if (s_max > 8) s_max = 8;
+        if (s_max > g.cchunks) s_max = g.cchunks;
+        while (s_max >= 2 && max_clusters<BN, MODE>(di, s_max) < base_tiles)
+            --s_max;
+        if (s_max >= 2) {
+            const int longest = (g.cchunks + s_max - 1) / s_max;
+            int sp = s_max;
+            while (sp > 2 && (g.cchunks + sp - 2) / (sp - 1) == longest)
+                --sp;
+            g.ksplit = sp;
+        }
+    }
     // several column tiles per row tile: try to keep the row tile's whole activation panel in the
     // ring (read / quantized once) and stream the weights
     bool done = false;
-    if (g.n_tiles > 1 && g.mode != MODE_TAPS) {
+    if (g.ksplit == 1 && g.n_tiles > 1 && g.mode != MODE_TAPS) {
         const bool conv9 = g.mode == MODE_FLAT && g.taps == 9 && g.S == 3;
         if (conv9 || g.taps == 1) {
             const int cps = conv9 ? 1 : (g.cchunks >= 3 ? 3 : g.cchunks);      // chunks per A stage
@@ -954,7 +1115,7 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
     }
     if (done) {
         // configured above
-    } else if (b_all + 2 * g.a_chunk_bytes <= budget) {
+    } else if (g.ksplit == 1 && b_all + 2 * g.a_chunk_bytes <= budget) {
         g.b_resident = 1;
         g.b_span = g.nblk;
         g.b_stages = 1;
@@ -999,26 +1160,35 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
         return FPQ_ERR_UNSUPPORTED;
     g.contiguous = (g.a_resident || (g.b_resident && g.n_tiles > 1)) ? 1 : 0;
     g.div_tiles = make_fastdiv((uint32_t)(g.m_fastest ? g.m_tiles : g.n_tiles));
+    // the partial sums of a split tile are staged over the rings
+    if (g.ksplit > 1 && g.a_stages * g.a_stage_bytes + g.b_stages * g.b_stage_bytes < BN * BM * 4)
+        return FPQ_ERR_UNSUPPORTED;
     const int dyn = g.a_stages * g.a_stage_bytes + g.b_stages * g.b_stage_bytes + ctl;
-    const int slot = (BN == 64 ? 0 : 1) + (FUSED ? 2 : 0) + 4 * MODE;
-    if (!di->smem_set[slot]) {
-        if (cudaFuncSetAttribute(fpq_gemm_kernel<BN, FUSED, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET) !=
-            cudaSuccess)
-            return FPQ_ERR_CUDA;
-        di->smem_set[slot] = true;
-    }
+    if (!allow_max_smem<BN, FUSED, MODE>(di))
+        return FPQ_ERR_CUDA;
     const int64_t tiles = (int64_t)g.m_tiles * g.n_tiles;
-    const int grid = (int)(tiles < di->sms ? tiles : di->sms);
+    const int grid = g.ksplit > 1 ? (int)tiles * g.ksplit : (int)(tiles < di->sms ? tiles : di->sms);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(num_threads(FUSED));
     cfg.dynamicSmemBytes = (size_t)dyn;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int nattr = 0;
+    if (g.wait_prior_grid) {
+        attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[nattr].val.programmaticStreamSerializationAllowed = 1;
+        ++nattr;
+    }
+    if (g.ksplit > 1) {
+        attr[nattr].id = cudaLaunchAttributeClusterDimension;
+        attr[nattr].val.clusterDim.x = (unsigned)g.ksplit;
+        attr[nattr].val.clusterDim.y = 1;
+        attr[nattr].val.clusterDim.z = 1;
+        ++nattr;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = g.wait_prior_grid ? 1 : 0;
+    cfg.numAttrs = (unsigned)nattr;
     return cudaLaunchKernelEx(&cfg, fpq_gemm_kernel<BN, FUSED, MODE>, tmA, tmB, tmY, (const GemmArgs)g) == cudaSuccess ? FPQ_OK
                                                                                                       : FPQ_ERR_CUDA;
 }

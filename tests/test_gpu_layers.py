@@ -110,6 +110,21 @@ def test_conv_ragged_shapes(wfmt, B, C, H, W, Co, R, pad, stride):
     _check_full(L)
 
 
+# few output tiles and a long reduction: the kernel splits the reduction over a cluster of CTAs
+@pytest.mark.parametrize("wfmt", ["e4m3", "e2m1"])
+@pytest.mark.parametrize("B,C,H,W,Co,R,pad,stride", [
+    (2, 640, 8, 8, 200, 3, 1, 1),      # 5 chunks, 2 x 2 tiles
+    (1, 1100, 8, 8, 130, 3, 1, 1),     # 9 chunks, the last one ragged; unequal ranges
+    (2, 300, 16, 16, 96, 3, 1, 2),     # stride 2, 3 chunks
+    (2, 520, 8, 8, 260, 1, 0, 1),      # 1x1, 5 chunks, three column tiles
+    (1, 256, 4, 4, 8, 3, 1, 1),        # 64-column tiles
+])
+def test_conv_split_reduction_shapes(wfmt, B, C, H, W, Co, R, pad, stride):
+    L = I.conv_layer("t", B, C, H, W, Co, R, pad=pad, stride=stride, wfmt=wfmt, rounding=True)
+    I.draw(L, 12, B + C + H + Co, "silu", 0.03, True)
+    _check_full(L)
+
+
 def test_conv_1x1_matches_linear_on_the_gpu():
     L = I.conv_layer("c", 2, 96, 8, 8, 80, 1, wfmt="e4m3")
     I.draw(L, 10, 0, "normal", 0.02, True)
