@@ -446,6 +446,21 @@ def run_own(args):
             del l4
             torch.cuda.empty_cache()
 
+    # ---- the standalone quantizers (HBM-bound): 2^26 FP32 elements, larger than L2
+    quant = None
+    if rank == 0 and not args.skip_w4:
+        nq = 1 << 26
+        xq = torch.randn(nq, device=dev, dtype=torch.float32)
+        cq = torch.empty(nq, device=dev, dtype=torch.uint8)
+        quant = {}
+        for name, fmt, by in (("act_e4m3_native", fpq.E4M3, 5.0), ("act_e5m2_general", fpq.E5M2, 5.0),
+                              ("act_e2m1_general", fpq.E2M1, 4.5)):
+            tq = per_launch_us(torch, lambda: fpq.fpq_quantize_act(xq, 0.01, fmt, cq), 10) * 1e-6
+            quant[name] = {"elements": nq, "us": tq * 1e6, "gbs": by * nq / tq / 1e9,
+                           "frac_of_hbm_peak": by * nq / tq / 1e9 / peaks["hbm_gbs"], "bytes_per_element": by}
+        del xq, cq
+        torch.cuda.empty_cache()
+
     # ---- CPU baseline: the oracle, as it stands, on the host cores (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.skip_cpu:
@@ -469,7 +484,7 @@ def run_own(args):
             "pct_dense_fp8_peak_2x_measured_bf16": 100 * value / world / (2 * peaks["bf16_tflops"]),
             "roofline": roofline, "layer_roofline": layer_roof, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
-            "weight_encode_us": enc_us, "w4a8": w4, "eager_step_us": eager_us,
+            "weight_encode_us": enc_us, "w4a8": w4, "standalone_quantizer": quant, "eager_step_us": eager_us,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -282,12 +282,6 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     const int n_pad = (g.N + 31) & ~31;
     float* s_scale = reinterpret_cast<float*>(smem + (bars - smem_base) + 512);   // [n_pad], if staged
     float* s_bias = s_scale + n_pad;
-    if (g.stage_scales) {
-        for (int i = threadIdx.x; i < n_pad; i += blockDim.x) {
-            s_scale[i] = (i < g.N) ? g.x_scale * __ldg(g.w_scale + i) : 0.f;
-            s_bias[i] = (g.bias && i < g.N) ? __ldg(g.bias + i) : 0.f;
-        }
-    }
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -667,6 +661,14 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         const int quarter = warp & 3;
         const int half = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;       // row of the tile held by this thread
+        if (g.stage_scales) {
+            // only these warps use the scales: they fetch them while the first loads and MMAs run
+            for (int i = threadIdx.x - 64; i < n_pad; i += 32 * NUM_EPI_WARPS) {
+                s_scale[i] = (i < g.N) ? g.x_scale * __ldg(g.w_scale + i) : 0.f;
+                s_bias[i] = (g.bias && i < g.N) ? __ldg(g.bias + i) : 0.f;
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * NUM_EPI_WARPS) : "memory");
+        }
         // row-major output: the warp's 32 x 32 block goes through a 128-byte-swizzled staging
         // buffer and leaves as one TMA store (whole 128-byte lines; rows past M and columns
         // past N are clipped by the tensor map)
