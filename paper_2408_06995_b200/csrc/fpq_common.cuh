@@ -75,6 +75,28 @@ __device__ __forceinline__ uint32_t quantize_bits(float t, const QFormat& f, int
     return code | (neg << f.sign_shift);
 }
 
+// Round-to-nearest-even only, any format, in a dozen instructions.  With s the step of the
+// element's binade and C = 1.5 * 2^23 * s, the FP32 sum |a| + C is rounded by the hardware to a
+// multiple of s (ties to the even multiple), and the multiple k = round(|a| / s) sits in the low
+// mantissa bits of the sum.  (exponent field - 1 of the binade) * 2^m + k is the code for normal
+// and subnormal results alike; a k of 2^(m+1) carries into the next exponent by itself.
+__device__ __forceinline__ uint32_t quantize_rne_bits(float t, const QFormat& f, bool& nan)
+{
+    const uint32_t u = __float_as_uint(t);
+    uint32_t au = u & 0x7fffffffu;
+    if (au > 0x7f800000u) {
+        nan = true;
+        return 0;
+    }
+    au = min(au, f.cmax_bits);                                   // clip (Inf included)
+    const int eb = max((int)(au >> 23), 128 - f.B);              // biased exponent of the binade whose step applies
+    const uint32_t cbits = ((uint32_t)(eb - f.m + 23) << 23) | 0x400000u;
+    const uint32_t k = __float_as_uint(__fadd_rn(__uint_as_float(au), __uint_as_float(cbits))) - cbits;
+    uint32_t code = ((uint32_t)(eb - 128 + f.B) << f.m) + k;
+    code = min(code, (uint32_t)f.code_max);
+    return code ? code | ((u >> 31) << f.sign_shift) : 0u;
+}
+
 // Four E4M3 (bias 7, saturating at 448) codes from four scaled floats with the
 // hardware convert; -0 and NaN are mapped to code 0 afterwards.
 __device__ __forceinline__ uint32_t e4m3x4_from_scaled(float t0, float t1, float t2, float t3, bool& nan)

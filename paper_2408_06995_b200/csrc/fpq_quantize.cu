@@ -30,8 +30,8 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const float* __restri
             if (FAST_E4M3) {
                 out[j] = e4m3x4_from_scaled(t0, t1, t2, t3, nan);
             } else {
-                out[j] = quantize_bits(t0, f, -1, nan) | (quantize_bits(t1, f, -1, nan) << 8) |
-                         (quantize_bits(t2, f, -1, nan) << 16) | (quantize_bits(t3, f, -1, nan) << 24);
+                out[j] = quantize_rne_bits(t0, f, nan) | (quantize_rne_bits(t1, f, nan) << 8) |
+                         (quantize_rne_bits(t2, f, nan) << 16) | (quantize_rne_bits(t3, f, nan) << 24);
             }
         }
         if (!f.four_bit) {
@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const float* __restri
     // tail (fewer than 16 elements): one thread, in order, so nibbles never race
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         for (int64_t i = nvec * 16; i < n; ++i) {
-            uint32_t c = quantize_bits(__fmul_rn(x[i], rinv), f, -1, nan);
+            uint32_t c = quantize_rne_bits(__fmul_rn(x[i], rinv), f, nan);
             if (!f.four_bit) {
                 codes[i] = (uint8_t)c;
             } else if (i & 1) {
@@ -74,9 +74,9 @@ __global__ void __launch_bounds__(256) quantize_act_scalar_kernel(const float* _
     int64_t per = f.four_bit ? 2 : 1;
     int64_t nout = (n + per - 1) / per;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < nout; o += stride) {
-        uint32_t c = quantize_bits(__fmul_rn(x[o * per], rinv), f, -1, nan);
+        uint32_t c = quantize_rne_bits(__fmul_rn(x[o * per], rinv), f, nan);
         if (f.four_bit && o * 2 + 1 < n)
-            c |= quantize_bits(__fmul_rn(x[o * 2 + 1], rinv), f, -1, nan) << 4;
+            c |= quantize_rne_bits(__fmul_rn(x[o * 2 + 1], rinv), f, nan) << 4;
         codes[o] = (uint8_t)c;
     }
     if (nan)
