@@ -80,6 +80,8 @@ def lib():
         L.fpq_o_conv2d.restype = i32
         L.fpq_o_conv2d.argtypes = [vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, vp,
                                    i64, i64, i64, i64, i64, i64, i64, i64, i64, vp, i64, vp, vp]
+        L.fpq_o_search_mse.restype = i64
+        L.fpq_o_search_mse.argtypes = [vp, i64, vp, i32, vp, i32, vp]
         _lib = L
     return _lib
 
@@ -214,3 +216,48 @@ def conv2d(x, w, w_scale, x_scale, fx: Format, fw: Format, bias=None, rounding_b
     wc = quantize_weight(w.reshape(Co, C * R * S), w_scale, fw, rounding_bits)
     xc = quantize_act(x, x_scale, fx)
     return conv2d_codes(xc, wc, w_scale, x_scale, fx, fw, bias, B, C, H, W, Co, R, S, pad, stride, idx)
+
+
+# ---- encoding and bias search (Sec. V-A, Algorithm 1) -------------------------------------
+
+FP8_ENCODINGS = (E2M5, E3M4, Format(4, 3, 8, SAT_PAPER), Format(5, 2, 16, SAT_PAPER))   # bias 2^(e-1), Sec. IV-B
+FP4_ENCODINGS = (E1M2, Format(2, 1, 2, SAT_PAPER))
+
+
+def clip_candidates(maxabs: float, count: int = 111) -> np.ndarray:
+    """Evenly spaced clipping values up to the largest magnitude of the data (Sec. V-A):
+    c_j = maxabs * j / count for j = 1..count, rounded once to FP32.  (Zero is left out: no
+    format has c = 0.)"""
+    return np.array([np.float32(float(np.float32(maxabs)) * j / count) for j in range(1, count + 1)],
+                    dtype=np.float32)
+
+
+def bias_from_clip(c: float, f: Format) -> float:
+    """The real-valued exponent bias whose clipping value is c: the clipping equation
+    c = (2 - 2^-m) 2^(2^e - b - 1) solved for b (Sec. IV-B)."""
+    return float(2 ** f.e - 1 - np.log2(float(c) / (2.0 - 2.0 ** -f.m)))
+
+
+def search_mse(x, encodings, clips) -> np.ndarray:
+    """mse[i][j] of quantizing x with encoding i clipped at clips[j] (see fpq_o_search_mse)."""
+    x = _f32(x).reshape(-1)
+    enc = np.ascontiguousarray([[f.e, f.m, f.B] for f in encodings], dtype=np.int32)
+    clips = _f32(clips)
+    mse = np.zeros((len(encodings), clips.size), dtype=np.float64)
+    lib().fpq_o_search_mse(_p(x), x.size, _p(enc), len(encodings), _p(clips), clips.size, _p(mse))
+    return mse
+
+
+def select_encoding_and_bias(mse: np.ndarray):
+    """Algorithm 1: walk the encodings (outer loop) and the bias candidates (inner loop) and keep
+    a candidate only when its error is strictly below the best so far.  The best-so-far starts
+    at +infinity: the listing's printed start value of 0 would never accept any candidate."""
+    best = (None, None)
+    prev_mse = float("inf")
+    for i in range(mse.shape[0]):
+        for j in range(mse.shape[1]):
+            curr_mse = float(mse[i, j])
+            if prev_mse > curr_mse:
+                best = (i, j)
+                prev_mse = curr_mse
+    return best

@@ -106,20 +106,20 @@ static int encode_exact(double q, ofmt f)
     return -1; /* not on the grid: a bug in the caller */
 }
 
-/* One element.  h < 0: round to nearest (ties to even); h = 0 / 1: learned
- * rounding with the hardened decision h.  Returns the code; *nan is set when
- * the scaled input is NaN. */
-int fpq_o_quantize_one(float x, float scale, int e, int m, int B, int sat, int h, int *nan)
+/* One element, value domain: the grid value q (in units of the scale) that the
+ * scaled input t = x * (1.0f / scale) is rounded to.  h < 0: round to nearest
+ * (ties to even); h = 0 / 1: learned rounding with the hardened decision h.
+ * *nan is set (and 0 returned) when the scaled input is NaN. */
+static double quantize_value(float x, float scale, ofmt f, int h, int *nan)
 {
-    ofmt f = {e, m, B, sat};
     volatile float r = 1.0f / scale;
     volatile float t = x * r;
     if (t != t) {
         if (nan)
             *nan = 1;
-        return 0;
+        return 0.0;
     }
-    double c = fpq_o_cmax(e, m, B, sat);
+    double c = fpq_o_cmax(f.e, f.m, f.B, f.sat);
     double a = (double)t;
     if (a > c)
         a = c;
@@ -136,6 +136,20 @@ int fpq_o_quantize_one(float x, float scale, int e, int m, int B, int sat, int h
         q = c;
     if (q < -c)
         q = -c;
+    return q;
+}
+
+/* One element: the code of that grid value. */
+int fpq_o_quantize_one(float x, float scale, int e, int m, int B, int sat, int h, int *nan)
+{
+    ofmt f = {e, m, B, sat};
+    int isnan = 0;
+    double q = quantize_value(x, scale, f, h, &isnan);
+    if (isnan) {
+        if (nan)
+            *nan = 1;
+        return 0;
+    }
     return encode_exact(q, f);
 }
 
@@ -318,4 +332,40 @@ int fpq_o_conv2d(const uint8_t *xc, const uint8_t *wc, const float *w_scale, flo
     free(xv);
     free(wv);
     return 0;
+}
+
+/* ---- encoding and bias search (Sec. V-A, Algorithm 1) ---------------------
+ *
+ * For every encoding candidate i (exponent bits, mantissa bits; the integer
+ * bias B_i only fixes the unit) and every clipping candidate c_j, the tensor is
+ * quantized with the format whose largest value is c_j and compared with the
+ * full-precision data:
+ *     scale_ij = (float)c_j / (float)c(F_i)      (FP32 division; this is the
+ *                real-valued bias of the clipping equation, b = B_i - log2 scale_ij)
+ *     xq       = scale_ij * q(x * (1.0f / scale_ij))   round to nearest, in double
+ *     mse_ij   = (1/n) sum (x - xq)^2                   in double, index order
+ * mse is written as [n_enc][n_clip].  The encodings use the paper's clipping
+ * value (all exponent fields finite).  Returns the number of NaN inputs. */
+int64_t fpq_o_search_mse(const float *x, int64_t n, const int32_t *enc /* [n_enc][3]: e, m, B */, int n_enc,
+                         const float *clip, int n_clip, double *mse)
+{
+    int64_t nans = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic) reduction(+ : nans)
+    for (int i = 0; i < n_enc; ++i) {
+        for (int j = 0; j < n_clip; ++j) {
+            ofmt f = {enc[3 * i], enc[3 * i + 1], enc[3 * i + 2], SAT_PAPER};
+            volatile float cf = (float)fpq_o_cmax(f.e, f.m, f.B, f.sat);
+            volatile float scale = clip[j] / cf;
+            double sum = 0.0;
+            for (int64_t k = 0; k < n; ++k) {
+                int isnan = 0;
+                double q = quantize_value(x[k], scale, f, -1, &isnan);
+                nans += isnan;
+                double err = (double)x[k] - (double)scale * q;
+                sum += err * err;
+            }
+            mse[(int64_t)i * n_clip + j] = n > 0 ? sum / (double)n : 0.0;
+        }
+    }
+    return nans;
 }
