@@ -228,6 +228,44 @@ fpq_status fpq_linear_static(const float* x, const void* w_prepared, const float
                              float* y, int64_t M, int64_t N, int64_t K, void* stream);
 
 /*
+ * Encoding and bias search of one tensor (Sec. V-A, Algorithm 1; offline, once per weight or
+ * activation tensor).  For every encoding candidate enc_host[i] (exponent and mantissa bits; the
+ * integer exp_bias only fixes the unit, sat_mode must be FPQ_SAT_PAPER) and every clipping value
+ * clip[j] > 0 the tensor is quantized, round to nearest even, with the format whose largest value
+ * is clip[j] - that is with scale = clip[j] / fpq_format_max(enc_host[i]) (FP32 division), which
+ * is the real-valued bias b = exp_bias - log2(scale) of the clipping equation (Sec. IV-B) - and
+ *   mse[i * n_clip + j] = (1/n) sum_k (x[k] - scale * q(x[k] / scale))^2.
+ * best[0], best[1] receive the encoding and clipping index that Algorithm 1 selects: candidates
+ * are visited encoding by encoding, clipping values in the inner loop, and one replaces the best
+ * so far only if its error is strictly smaller (the best so far starts at +infinity).
+ *
+ *   x          n FP32 values (n >= 0); a NaN makes every mse NaN and sets FPQ_ERR_NAN_INPUT in
+ *              the status word
+ *   enc_host   HOST array of n_enc formats, 1 <= n_enc <= 8
+ *   clip       DEVICE array of n_clip positive finite FP32 values, 1 <= n_clip <= 256,
+ *              n_enc * n_clip <= 1024 (the paper uses 4 x 111 for FP8 and 2 x 111 for FP4)
+ *   mse        DEVICE out, n_enc * n_clip doubles
+ *   best       DEVICE out, 2 int32
+ *   workspace  fpq_search_workspace_size(n_enc, n_clip) bytes, 8-byte aligned; contents need
+ *              not be kept between calls
+ * Two kernels on `stream`, no allocation, no host synchronisation.  Errors: FPQ_ERR_NULL,
+ * FPQ_ERR_SHAPE (counts out of range, n < 0), FPQ_ERR_FORMAT, FPQ_ERR_UNSUPPORTED (sat_mode),
+ * FPQ_ERR_ALIGN, FPQ_ERR_WORKSPACE, FPQ_ERR_CUDA.
+ */
+size_t fpq_search_workspace_size(int32_t n_enc, int32_t n_clip);
+fpq_status fpq_search_format(const float* x, int64_t n, const fpq_format* enc_host, int32_t n_enc, const float* clip,
+                             int32_t n_clip, double* mse, int32_t* best, void* workspace, size_t ws_bytes,
+                             void* stream);
+
+/*
+ * The clipping candidates of Sec. V-A: count evenly spaced values up to the largest magnitude
+ * of the data, clip_host[j] = maxabs * (j + 1) / count rounded once to FP32 (zero is left out:
+ * no format has a largest value of 0).  HOST output.  FPQ_ERR_SHAPE unless 1 <= count <= 256
+ * and maxabs is positive and finite.
+ */
+fpq_status fpq_search_clip_candidates(float maxabs, int32_t count, float* clip_host);
+
+/*
  * Which route fpq_linear / fpq_conv2d take (process-wide setting, not thread-safe against
  * concurrent layer calls; the results are the same bit for bit on either route):
  *   FPQ_PATH_FUSED        one kernel: the activation quantize (Sec. IV-B rounding equation) runs

@@ -68,7 +68,8 @@ EXPORTS = [
     "fpq_prepared_size", "fpq_prepare_weight", "fpq_linear_workspace_size", "fpq_linear",
     "fpq_conv2d_workspace_size", "fpq_conv2d", "fpq_linear_host", "fpq_conv2d_host",
     "fpq_linear_quantize_input", "fpq_linear_contract", "fpq_conv2d_quantize_input", "fpq_conv2d_contract",
-    "fpq_linear_static", "fpq_set_path_policy", "fpq_get_path_policy", "fpq_read_status", "fpq_status_string",
+    "fpq_linear_static", "fpq_search_workspace_size", "fpq_search_format", "fpq_search_clip_candidates",
+    "fpq_set_path_policy", "fpq_get_path_policy", "fpq_read_status", "fpq_status_string",
 ]
 
 _lib = None
@@ -120,6 +121,12 @@ def lib() -> ctypes.CDLL:
         L.fpq_conv2d_contract.argtypes = [vp, sz, vp, vp, f32, F, F, vp, vp] + [i32] * 9 + [vp]
         L.fpq_linear_static.restype = i32
         L.fpq_linear_static.argtypes = [vp, vp, vp, f32, F, F, vp, vp, i64, i64, i64, vp]
+        L.fpq_search_workspace_size.restype = sz
+        L.fpq_search_workspace_size.argtypes = [i32, i32]
+        L.fpq_search_format.restype = i32
+        L.fpq_search_format.argtypes = [vp, i64, vp, i32, vp, i32, vp, vp, vp, sz, vp]
+        L.fpq_search_clip_candidates.restype = i32
+        L.fpq_search_clip_candidates.argtypes = [f32, i32, vp]
         L.fpq_set_path_policy.restype = i32
         L.fpq_set_path_policy.argtypes = [i32]
         L.fpq_get_path_policy.restype = i32
@@ -301,6 +308,38 @@ def fpq_conv2d_host(x_host, x_dev, w_prepared, w_scale, x_scale, fx, fw, bias, y
                                  fx.c(), fw.c(), _ptr(bias), _ptr(y_dev), _ptr(y_host), B, C, H, W, C_out, R, S,
                                  pad, stride, _ptr(workspace), workspace.numel(), _stream()), "fpq_conv2d_host")
     return y_host
+
+
+def fpq_search_workspace_size(n_enc: int, n_clip: int) -> int:
+    return lib().fpq_search_workspace_size(int(n_enc), int(n_clip))
+
+
+def fpq_search_clip_candidates(maxabs: float, count: int = 111) -> torch.Tensor:
+    """The evenly spaced clipping candidates up to maxabs, as a CPU float32 tensor."""
+    out = torch.empty(count, dtype=torch.float32)
+    _check(lib().fpq_search_clip_candidates(float(maxabs), int(count), ctypes.c_void_p(out.data_ptr())),
+           "fpq_search_clip_candidates")
+    return out
+
+
+def fpq_search_format(x: torch.Tensor, encodings, clip: torch.Tensor, mse: torch.Tensor = None,
+                      best: torch.Tensor = None, workspace: torch.Tensor = None):
+    """Mean squared error of every (encoding, clipping value) candidate on x and Algorithm 1's
+    choice.  Returns (mse [n_enc][n_clip] float64, best [2] int32), both on the device."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    assert clip.is_cuda and clip.dtype == torch.float32 and clip.is_contiguous()
+    n_enc, n_clip = len(encodings), clip.numel()
+    enc = (_CFormat * n_enc)(*[f.c() for f in encodings])
+    if mse is None:
+        mse = torch.empty((n_enc, n_clip), dtype=torch.float64, device=x.device)
+    if best is None:
+        best = torch.empty(2, dtype=torch.int32, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(max(8, fpq_search_workspace_size(n_enc, n_clip)), dtype=torch.uint8, device=x.device)
+    _check(lib().fpq_search_format(_ptr(x), x.numel(), ctypes.cast(enc, ctypes.c_void_p), n_enc, _ptr(clip), n_clip,
+                                   _ptr(mse), _ptr(best), _ptr(workspace), workspace.numel(), _stream()),
+           "fpq_search_format")
+    return mse, best
 
 
 def fpq_set_path_policy(policy: int) -> None:

@@ -510,6 +510,48 @@ fpq_status fpq_conv2d_host(const float* x_host, float* x_dev, const void* w_prep
     return cudaStreamSynchronize(st) == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
 }
 
+size_t fpq_search_workspace_size(int32_t n_enc, int32_t n_clip)
+{
+    if (n_enc < 1 || n_enc > search_max_enc() || n_clip < 1 || n_clip > search_max_clip() ||
+        n_enc * n_clip > search_max_cand())
+        return 0;
+    return search_workspace_bytes(n_enc, n_clip);
+}
+
+fpq_status fpq_search_format(const float* x, int64_t n, const fpq_format* enc_host, int32_t n_enc, const float* clip,
+                             int32_t n_clip, double* mse, int32_t* best, void* workspace, size_t ws_bytes,
+                             void* stream)
+{
+    if (n < 0 || n_enc < 1 || n_enc > search_max_enc() || n_clip < 1 || n_clip > search_max_clip() ||
+        n_enc * n_clip > search_max_cand())
+        return FPQ_ERR_SHAPE;
+    if (!enc_host || !clip || !mse || !best || (n > 0 && !x))
+        return FPQ_ERR_NULL;
+    for (int i = 0; i < n_enc; ++i) {
+        QFormat q;
+        if (!resolve_format(enc_host[i], &q))
+            return FPQ_ERR_FORMAT;
+        if (enc_host[i].sat_mode != FPQ_SAT_PAPER)
+            return FPQ_ERR_UNSUPPORTED;
+    }
+    if (!aligned(x, 4) || !aligned(clip, 4) || !aligned(mse, 8) || !aligned(best, 4) || !aligned(workspace, 8))
+        return FPQ_ERR_ALIGN;
+    if (!workspace || ws_bytes < search_workspace_bytes(n_enc, n_clip))
+        return FPQ_ERR_WORKSPACE;
+    return launch_search(x, n, enc_host, n_enc, clip, n_clip, mse, best, workspace, (cudaStream_t)stream);
+}
+
+fpq_status fpq_search_clip_candidates(float maxabs, int32_t count, float* clip_host)
+{
+    if (!clip_host)
+        return FPQ_ERR_NULL;
+    if (count < 1 || count > search_max_clip() || !(maxabs > 0.f) || !isfinite(maxabs))
+        return FPQ_ERR_SHAPE;
+    for (int j = 0; j < count; ++j)
+        clip_host[j] = (float)((double)maxabs * (double)(j + 1) / (double)count);
+    return FPQ_OK;
+}
+
 fpq_status fpq_set_path_policy(int32_t policy)
 {
     if (policy != FPQ_PATH_AUTO && policy != FPQ_PATH_FUSED && policy != FPQ_PATH_TWO_KERNELS)

@@ -43,4 +43,12 @@ struct GemmProblem {
 // Returns FPQ_OK or an error; enqueues one kernel.
 fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st);
 
+// Encoding / bias search: limits, scratch size, and the two-kernel launch.
+int search_max_enc();
+int search_max_clip();
+int search_max_cand();
+size_t search_workspace_bytes(int n_enc, int n_clip);
+fpq_status launch_search(const float* x, int64_t n, const fpq_format* enc, int n_enc, const float* clip, int n_clip,
+                         double* mse, int32_t* best, void* workspace, cudaStream_t st);
+
 }  // namespace fpq

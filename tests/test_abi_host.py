@@ -72,6 +72,31 @@ def test_host_side_rejections(L):
     assert L.fpq_conv2d(big, big, big, 1.0, F, F, None, big, 1, 8, 4, 4, 8, 3, 3, 1, 1, big, 16, None) == fpq.ERR_WORKSPACE
 
 
+def test_search_host_side(L):
+    import numpy as np
+    import oracle as O
+    enc = (fpq._CFormat * 2)(fpq.Format(1, 2, 1).c(), fpq.Format(2, 1, 2).c())
+    encp = ctypes.cast(enc, ctypes.c_void_p)
+    big = ctypes.c_void_p(1024)
+    assert L.fpq_search_format(big, -1, encp, 2, big, 4, big, big, big, 1 << 30, None) == fpq.ERR_SHAPE
+    assert L.fpq_search_format(big, 8, encp, 0, big, 4, big, big, big, 1 << 30, None) == fpq.ERR_SHAPE
+    assert L.fpq_search_format(big, 8, encp, 2, big, 257, big, big, big, 1 << 30, None) == fpq.ERR_SHAPE
+    assert L.fpq_search_format(None, 8, encp, 2, big, 4, big, big, big, 1 << 30, None) == fpq.ERR_NULL
+    assert L.fpq_search_format(big, 8, encp, 2, big, 4, ctypes.c_void_p(1028), big, big, 1 << 30, None) == fpq.ERR_ALIGN
+    assert L.fpq_search_format(big, 8, encp, 2, big, 4, big, big, big, 64, None) == fpq.ERR_WORKSPACE
+    native = (fpq._CFormat * 1)(fpq.E4M3.c())
+    assert L.fpq_search_format(big, 8, ctypes.cast(native, ctypes.c_void_p), 1, big, 4, big, big, big, 1 << 30,
+                               None) == fpq.ERR_UNSUPPORTED
+    assert fpq.fpq_search_workspace_size(4, 111) == 592 * 444 * 8
+    assert fpq.fpq_search_workspace_size(8, 256) == 0            # more than 1024 candidates
+    # the clipping candidates are the oracle's, bit for bit
+    for maxabs in (3.7, 0.0123, 1e4):
+        assert np.array_equal(fpq.fpq_search_clip_candidates(maxabs, 111).numpy(), O.clip_candidates(maxabs, 111))
+    assert L.fpq_search_clip_candidates(0.0, 5, big) == fpq.ERR_SHAPE
+    assert L.fpq_search_clip_candidates(1.0, 0, big) == fpq.ERR_SHAPE
+    assert L.fpq_search_clip_candidates(float("inf"), 5, big) == fpq.ERR_SHAPE
+
+
 def test_sizes(L):
     assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E4M3, fpq.E4M3) == 100 * 320
     assert fpq.fpq_linear_workspace_size(100, 64, 321, fpq.E4M3, fpq.E2M1) == 100 * 336
