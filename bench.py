@@ -594,6 +594,57 @@ def run_suite(args):
     print(json.dumps(summary), flush=True)
 
 
+def run_search(args):
+    """The encoding / bias search (Algorithm 1) on one tensor of 2^24 FP32 values: all FP8
+    (4 x 111) and all FP4 (2 x 111) candidates.  ALU-bound: the roofline is instruction issue,
+    9 lane instructions per element and candidate against 128 lanes per SM and clock."""
+    import numpy as np
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    from paper_2408_06995_b200 import build as fpq_build
+    fpq_build.build()
+    import paper_2408_06995_b200 as fpq
+    import oracle as O
+    n = 1 << 24
+    x = torch.randn(n, device=dev, dtype=torch.float32)
+    maxabs = float(x.abs().max())
+    clips = fpq.fpq_search_clip_candidates(maxabs, 111).to(dev)
+    props = torch.cuda.get_device_properties(0)
+    sampler = ClockSampler(physical_gpu_index(0))
+    sampler.start()
+    out = {"suite": "search", "elements": n, "rows": []}
+    for name, encs_cpu in (("fp8_4x111", O.FP8_ENCODINGS), ("fp4_2x111", O.FP4_ENCODINGS)):
+        encs = [fpq.Format(f.e, f.m, f.B, fpq.SAT_PAPER) for f in encs_cpu]
+        ncand = len(encs) * 111
+        mse = torch.empty((len(encs), 111), dtype=torch.float64, device=dev)
+        best = torch.empty(2, dtype=torch.int32, device=dev)
+        wk = torch.empty(fpq.fpq_search_workspace_size(len(encs), 111), dtype=torch.uint8, device=dev)
+        t = per_launch_us(torch, lambda: fpq.fpq_search_format(x, encs, clips, mse, best, wk), 5) * 1e-6
+        b = best.cpu().numpy()
+        row = {"name": name, "candidates": ncand, "us": t * 1e6, "element_candidates_per_s": n * ncand / t,
+               "lane_instructions_per_s": 9.0 * n * ncand / t, "hbm_gbs": 4.0 * n / t / 1e9,
+               "selected": {"encoding": f"E{encs_cpu[b[0]].e}M{encs_cpu[b[0]].m}", "clip_index": int(b[1])}}
+        out["rows"].append(row)
+    clocks = sampler.stop()
+    peak = props.multi_processor_count * 128 * (clocks["sm_mhz"] or 1965.0) * 1e6
+    for row in out["rows"]:
+        row["roofline"] = {"bound": "alu", "achieved": row["lane_instructions_per_s"] / 1e12, "peak": peak / 1e12,
+                           "unit": "T lane-instructions/s", "frac": row["lane_instructions_per_s"] / peak,
+                           "peak_source": "SM count x 128 lanes x sampled SM clock"}
+    out["clocks"] = clocks
+    if not args.skip_cpu:
+        xs = x[: 1 << 16].cpu().numpy()
+        t0 = time.perf_counter()
+        O.search_mse(xs, O.FP8_ENCODINGS, clips.cpu().numpy())
+        dt = time.perf_counter() - t0
+        out["cpu_baseline"] = {"value": xs.size * 444 / dt, "unit": "element-candidates/s", "cores": os.cpu_count(),
+                               "kind": "oracle", "sample": "the first 2^16 elements, 4 x 111 candidates"}
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -602,11 +653,13 @@ def main():
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline leg")
     ap.add_argument("--skip-w4", action="store_true", help="leave out the W4A8 side measurement")
-    ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd", "sd_trace"],
+    ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd", "sd_trace", "search"],
                     help="print a per-shape table of a whole workload instead of the headline line")
     args = ap.parse_args()
     if args.suite == "sd_trace":
         run_trace(args)
+    elif args.suite == "search":
+        run_search(args)
     elif args.suite:
         run_suite(args)
     elif args.impl == "reference":
