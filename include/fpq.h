@@ -228,6 +228,19 @@ fpq_status fpq_linear_static(const float* x, const void* w_prepared, const float
                              float* y, int64_t M, int64_t N, int64_t K, void* stream);
 
 /*
+ * Zero census of a quantized tensor (the sparsity measurement of the paper's evaluation, Sec.
+ * "Sparsity": the fraction of weights that are zero after quantization).  Counts the values of
+ * `codes` whose code is 0; the quantizers never produce a negative zero, so this is every zero.
+ *   codes   n codes as written by fpq_quantize_weight / fpq_quantize_act: one per byte, or for
+ *           formats of at most 4 bits two per byte, even index in the low nibble (a high nibble
+ *           of padding after an odd n is not counted)
+ *   count   DEVICE out, one uint64 (8-byte aligned), overwritten
+ * One memset and one kernel on `stream`.  Errors: FPQ_ERR_FORMAT, FPQ_ERR_SHAPE (n < 0),
+ * FPQ_ERR_NULL, FPQ_ERR_ALIGN, FPQ_ERR_CUDA.
+ */
+fpq_status fpq_zero_census(const uint8_t* codes, int64_t n, fpq_format fmt, uint64_t* count, void* stream);
+
+/*
  * Encoding and bias search of one tensor (Sec. V-A, Algorithm 1; offline, once per weight or
  * activation tensor).  For every encoding candidate enc_host[i] (exponent and mantissa bits; the
  * integer exp_bias only fixes the unit, sat_mode must be FPQ_SAT_PAPER) and every clipping value

@@ -261,3 +261,17 @@ def select_encoding_and_bias(mse: np.ndarray):
                 best = (i, j)
                 prev_mse = curr_mse
     return best
+
+
+# ---- sparsity of a quantized tensor (the paper's sparsity study) --------------------------
+
+def zero_count(codes, n: int, f: Format) -> int:
+    """How many of the n quantized values are zero (code 0: the quantizer has no negative zero).
+    `codes` is laid out as quantize_weight / quantize_act write it."""
+    flat = np.ascontiguousarray(codes, dtype=np.uint8).reshape(-1)
+    if f.bits == 8:
+        return int(np.count_nonzero(flat[:n] == 0))
+    values = np.empty(flat.size * 2, dtype=np.uint8)
+    values[0::2] = flat & 0xF
+    values[1::2] = flat >> 4
+    return int(np.count_nonzero(values[:n] == 0))

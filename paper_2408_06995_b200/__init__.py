@@ -69,7 +69,7 @@ EXPORTS = [
     "fpq_conv2d_workspace_size", "fpq_conv2d", "fpq_linear_host", "fpq_conv2d_host",
     "fpq_linear_quantize_input", "fpq_linear_contract", "fpq_conv2d_quantize_input", "fpq_conv2d_contract",
     "fpq_linear_static", "fpq_search_workspace_size", "fpq_search_format", "fpq_search_clip_candidates",
-    "fpq_set_path_policy", "fpq_get_path_policy", "fpq_read_status", "fpq_status_string",
+    "fpq_zero_census", "fpq_set_path_policy", "fpq_get_path_policy", "fpq_read_status", "fpq_status_string",
 ]
 
 _lib = None
@@ -121,6 +121,8 @@ def lib() -> ctypes.CDLL:
         L.fpq_conv2d_contract.argtypes = [vp, sz, vp, vp, f32, F, F, vp, vp] + [i32] * 9 + [vp]
         L.fpq_linear_static.restype = i32
         L.fpq_linear_static.argtypes = [vp, vp, vp, f32, F, F, vp, vp, i64, i64, i64, vp]
+        L.fpq_zero_census.restype = i32
+        L.fpq_zero_census.argtypes = [vp, i64, F, vp, vp]
         L.fpq_search_workspace_size.restype = sz
         L.fpq_search_workspace_size.argtypes = [i32, i32]
         L.fpq_search_format.restype = i32
@@ -308,6 +310,15 @@ def fpq_conv2d_host(x_host, x_dev, w_prepared, w_scale, x_scale, fx, fw, bias, y
                                  fx.c(), fw.c(), _ptr(bias), _ptr(y_dev), _ptr(y_host), B, C, H, W, C_out, R, S,
                                  pad, stride, _ptr(workspace), workspace.numel(), _stream()), "fpq_conv2d_host")
     return y_host
+
+
+def fpq_zero_census(codes: torch.Tensor, n: int, fmt: Format, count: torch.Tensor = None) -> torch.Tensor:
+    """Number of zero codes among the n values of `codes` (device int64 tensor with one entry)."""
+    assert codes.is_cuda and codes.dtype == torch.uint8 and codes.is_contiguous()
+    if count is None:
+        count = torch.empty(1, dtype=torch.int64, device=codes.device)
+    _check(lib().fpq_zero_census(_ptr(codes), int(n), fmt.c(), _ptr(count), _stream()), "fpq_zero_census")
+    return count
 
 
 def fpq_search_workspace_size(n_enc: int, n_clip: int) -> int:

@@ -510,6 +510,22 @@ fpq_status fpq_conv2d_host(const float* x_host, float* x_dev, const void* w_prep
     return cudaStreamSynchronize(st) == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
 }
 
+fpq_status fpq_zero_census(const uint8_t* codes, int64_t n, fpq_format fmt, uint64_t* count, void* stream)
+{
+    QFormat q;
+    if (!resolve_format(fmt, &q))
+        return FPQ_ERR_FORMAT;
+    if (n < 0)
+        return FPQ_ERR_SHAPE;
+    if (!count || (n > 0 && !codes))
+        return FPQ_ERR_NULL;
+    if (!aligned(count, 8))
+        return FPQ_ERR_ALIGN;
+    return launch_zero_census(codes, n, q.four_bit, (unsigned long long*)count, (cudaStream_t)stream) == cudaSuccess
+               ? FPQ_OK
+               : FPQ_ERR_CUDA;
+}
+
 size_t fpq_search_workspace_size(int32_t n_enc, int32_t n_clip)
 {
     if (n_enc < 1 || n_enc > search_max_enc() || n_clip < 1 || n_clip > search_max_clip() ||

@@ -269,12 +269,12 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
 
-    // layout: [A ring][B ring][epilogue staging for TMA stores, 4 KiB per warp][barriers + flags]
+    // layout: [A ring][B ring][epilogue staging for TMA stores, 2 x 4 KiB per warp][barriers + flags]
     //         [x_scale * w_scale | bias, all N columns, when they fit]
     const uint32_t a_ring = smem_base;
     const uint32_t b_ring = a_ring + g.a_stages * g.a_stage_bytes;
     const uint32_t ctl_off = g.a_stages * g.a_stage_bytes + g.b_stages * g.b_stage_bytes;
-    const uint32_t bars = smem_base + ctl_off + (g.y_tma ? NUM_EPI_WARPS * 4096 : 0);
+    const uint32_t bars = smem_base + ctl_off + (g.y_tma ? NUM_EPI_WARPS * 8192 : 0);
     // barrier slots (8 bytes each): a_full[8] a_empty[8] b_full[8] b_empty[8] acc_full[2] acc_empty[2]
     const uint32_t a_full = bars, a_empty = bars + 64, b_full = bars + 128, b_empty = bars + 192;
     const uint32_t acc_full = bars + 256, acc_empty = bars + 272;
@@ -672,7 +672,8 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         // row-major output: the warp's 32 x 32 block goes through a 128-byte-swizzled staging
         // buffer and leaves as one TMA store (whole 128-byte lines; rows past M and columns
         // past N are clipped by the tensor map)
-        uint8_t* stage = smem + ctl_off + (warp - 2) * 4096;
+        uint8_t* stage0 = smem + ctl_off + (warp - 2) * 8192;     // two 4 KiB buffers, used in turn
+        uint32_t nstore = 0;
         uint32_t it = 0;
         bool dead = false;
         for (int t = t_lo; t < t_hi && !dead; t += t_step, ++it) {
@@ -760,9 +761,11 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                             }
                         }
                         if (g.y_tma) {
-                            // the buffer is free once the previous store has read it
+                            // the buffer is free once the store before the previous one has read it
+                            uint8_t* stage = stage0 + (nstore & 1u) * 4096;
+                            ++nstore;
                             if (lane == 0)
-                                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                                asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                             __syncwarp();
 #pragma unroll
                             for (int j = 0; j < 8; ++j)
@@ -1064,7 +1067,7 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
         return FPQ_ERR_CUDA;
     const int n_pad = (g.N + 31) & ~31;
     g.stage_scales = (n_pad * 8 <= 16384) ? 1 : 0;
-    const int ctl = 512 + 1024 + (g.y_tma ? epi_warps(FUSED) * 4096 : 0) + (g.stage_scales ? n_pad * 8 : 0);
+    const int ctl = 512 + 1024 + (g.y_tma ? epi_warps(FUSED) * 8192 : 0) + (g.stage_scales ? n_pad * 8 : 0);
     const int budget = SMEM_BUDGET - ctl;
     const int b_block = BN * BK;
     const int a_min_span = (g.mode == MODE_FLAT) ? g.taps : 1;

@@ -16,6 +16,7 @@ cudaError_t launch_quantize_rows_e4m3(const float* x, int64_t M, int64_t K, int6
                                       cudaStream_t st);
 cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int H, int W, int pad, int Cp, float scale,
                                               uint8_t* codes, cudaStream_t st);
+cudaError_t launch_zero_census(const uint8_t* codes, int64_t n, int four_bit, unsigned long long* count, cudaStream_t st);
 cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, uint8_t* prepared,
                                   cudaStream_t st);
 

@@ -337,6 +337,70 @@ cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int 
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------
+// Zero census of a code tensor (the sparsity measurement): how many of the n values are the
+// code 0.  16 bytes per thread and step, one atomic per block.  *count must be 0 at the start.
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) zero_census_kernel(const uint8_t* __restrict__ codes, int64_t n, int four_bit,
+                                                          unsigned long long* __restrict__ count)
+{
+    const int64_t nbytes = four_bit ? n / 2 : n;              // whole bytes; an odd 4-bit tail is handled below
+    const int64_t head = min(nbytes, (int64_t)((16 - ((uintptr_t)codes & 15)) & 15));
+    const int64_t nvec = (nbytes - head) / 16;
+    const uint4* v4 = reinterpret_cast<const uint4*>(codes + head);
+    unsigned zeros = 0;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t v = tid; v < nvec; v += stride) {
+        const uint4 q = __ldg(v4 + v);
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (four_bit) {
+                // a nibble is zero iff none of its four bits is set
+                uint32_t t = w[k] | (w[k] >> 1);
+                t |= t >> 2;
+                zeros += 8 - __popc(t & 0x11111111u);
+            } else {
+                uint32_t t = w[k] | (w[k] >> 4);
+                t |= t >> 2;
+                t |= t >> 1;
+                zeros += 4 - __popc(t & 0x01010101u);
+            }
+        }
+    }
+    // bytes before the first and after the last aligned 16-byte group
+    for (int64_t i = tid; i < nbytes - nvec * 16; i += stride) {
+        const uint8_t c = codes[i < head ? i : i + nvec * 16];
+        zeros += four_bit ? ((c & 0xf) == 0) + ((c >> 4) == 0) : (c == 0);
+    }
+    if (four_bit && (n & 1) && tid == 0)
+        zeros += (codes[nbytes] & 0xf) == 0;                   // last value sits alone in a low nibble
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+        zeros += __shfl_xor_sync(0xffffffffu, zeros, o);
+    __shared__ unsigned s_z[8];
+    if ((threadIdx.x & 31) == 0)
+        s_z[threadIdx.x >> 5] = zeros;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long t = 0;
+        for (int w = 0; w < 8; ++w)
+            t += s_z[w];
+        if (t)
+            atomicAdd(count, t);
+    }
+}
+
+cudaError_t launch_zero_census(const uint8_t* codes, int64_t n, int four_bit, unsigned long long* count, cudaStream_t st)
+{
+    cudaError_t e = cudaMemsetAsync(count, 0, sizeof(unsigned long long), st);
+    if (e != cudaSuccess || n == 0)
+        return e;
+    const int64_t nbytes = four_bit ? (n + 1) / 2 : n;
+    zero_census_kernel<<<grid_for(nbytes / 16 + 1, 256), 256, 0, st>>>(codes, n, four_bit, count);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, uint8_t* prepared,
                                   cudaStream_t st)
 {

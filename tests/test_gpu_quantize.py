@@ -132,3 +132,20 @@ def test_full_size_activation_tensor_sampled():
     got = fpq.fpq_quantize_act(torch.from_numpy(x).cuda(), float(scale), fpq.E4M3).cpu().numpy()
     want = O.quantize_act(x, scale, O.E4M3)
     assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("fname", ["E4M3", "E2M1", "E3M4", "E1M2"])
+@pytest.mark.parametrize("n", [0, 1, 15, 16, 33, 4097, 1 << 20, (1 << 20) + 3])
+def test_zero_census_matches_the_oracle(fname, n):
+    fo, fg = getattr(O, fname), getattr(fpq, fname)
+    rng = np.random.default_rng(n + 17)
+    x = (rng.standard_normal(n) * 0.3).astype(np.float32)
+    x[rng.random(n) < 0.1] = 0.0
+    scale = 0.4 if fo.bits == 8 else 0.2
+    codes = O.quantize_act(x, scale, fo).reshape(-1)
+    # one byte of offset: the kernel must cope with a start that is not 16-byte aligned
+    buf = torch.zeros(codes.size + 1, dtype=torch.uint8, device="cuda")
+    buf[1:] = torch.from_numpy(codes).cuda()
+    for view in (buf[1:], buf[1:].clone()):
+        got = int(fpq.fpq_zero_census(view, n, fg).cpu()[0])
+        assert got == O.zero_count(codes, n, fo)

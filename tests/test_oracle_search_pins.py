@@ -124,3 +124,18 @@ def test_narrow_data_takes_the_most_mantissa_bits_and_heavy_tails_take_fewer():
     i, _ = O.select_encoding_and_bias(O.search_mse(heavy, O.FP8_ENCODINGS,
                                                    O.clip_candidates(np.abs(heavy).max(), 16)))
     assert O.FP8_ENCODINGS[i].m < 5
+
+
+def test_zero_count_is_the_number_of_values_that_decode_to_zero():
+    rng = np.random.default_rng(11)
+    for f in (O.E4M3, O.E2M1, O.E1M2, O.E3M4):
+        for n in (1, 2, 7, 1000, 1001):
+            x = (rng.standard_normal(n) * 0.3).astype(np.float32)
+            x[rng.random(n) < 0.2] = 0.0
+            codes = O.quantize_act(x, 0.5, f)
+            table = O.decode_table(f)
+            decoded = np.array([table[O.quantize_one(v, 0.5, f)] for v in x])
+            assert O.zero_count(codes, n, f) == int(np.count_nonzero(decoded == 0.0))
+    assert O.zero_count(np.array([0x10, 0x00, 0x0F], dtype=np.uint8), 5, O.E2M1) == 3   # 0,1 | 0,0 | f,(pad)
+    assert O.zero_count(np.array([0x10, 0x00, 0x0F], dtype=np.uint8), 6, O.E2M1) == 4
+    assert O.zero_count(np.array([0, 0x80, 3, 0], dtype=np.uint8), 4, O.E4M3) == 2      # 0x80 would be -0: not produced, not counted
