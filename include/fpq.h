@@ -228,6 +228,31 @@ fpq_status fpq_linear_static(const float* x, const void* w_prepared, const float
                              float* y, int64_t M, int64_t N, int64_t K, void* stream);
 
 /*
+ * Convolution whose input is the channel concatenation of two tensors that are quantized
+ * separately, each with its own scale (Sec. VI-A: the skip connection and the previous layer's
+ * output of a decoder block have different value distributions and are quantized apart before
+ * they are concatenated):
+ *   y[b][n][oy][ox] = w_scale[n] * ( x1_scale * sum over the C1 channels of x1
+ *                                  + x2_scale * sum over the C2 channels of x2 ) + bias[n]
+ * with the sums as in fpq_conv2d.  x1 is NCHW [B][C1][H][W], x2 is [B][C2][H][W]; the
+ * concatenated FP32 tensor is never formed.  The weights are [C_out][C1 + C2][R][S] codes from
+ * fpq_quantize_weight (x1's channels first), passed through fpq_prepare_weight_split (buffer of
+ * fpq_prepared_size_split bytes, 128-byte aligned): that copy starts x2's channels at a multiple
+ * of 128 so that no 128-wide chunk of the reduction mixes the two scales.
+ * workspace: fpq_conv2d_split_workspace_size bytes, 128-byte aligned, scratch.
+ * Formats, alignment, errors and stream behaviour as fpq_conv2d (three kernels).
+ */
+size_t fpq_prepared_size_split(fpq_format fmt, int32_t N, int32_t C1, int32_t C2, int32_t R, int32_t S);
+fpq_status fpq_prepare_weight_split(const uint8_t* codes, fpq_format fmt, int32_t N, int32_t C1, int32_t C2,
+                                    int32_t R, int32_t S, void* prepared, void* stream);
+size_t fpq_conv2d_split_workspace_size(int B, int C1, int C2, int H, int W, int C_out, int R, int S, int pad,
+                                       int stride, fpq_format fx, fpq_format fw);
+fpq_status fpq_conv2d_split(const float* x1, int C1, float x1_scale, const float* x2, int C2, float x2_scale,
+                            const void* w_prepared, const float* w_scale, fpq_format fx, fpq_format fw,
+                            const float* bias, float* y, int B, int H, int W, int C_out, int R, int S, int pad,
+                            int stride, void* workspace, size_t ws_bytes, void* stream);
+
+/*
  * Zero census of a quantized tensor (the sparsity measurement of the paper's evaluation, Sec.
  * "Sparsity": the fraction of weights that are zero after quantization).  Counts the values of
  * `codes` whose code is 0; the quantizers never produce a negative zero, so this is every zero.

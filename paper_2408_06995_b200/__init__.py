@@ -69,7 +69,8 @@ EXPORTS = [
     "fpq_conv2d_workspace_size", "fpq_conv2d", "fpq_linear_host", "fpq_conv2d_host",
     "fpq_linear_quantize_input", "fpq_linear_contract", "fpq_conv2d_quantize_input", "fpq_conv2d_contract",
     "fpq_linear_static", "fpq_search_workspace_size", "fpq_search_format", "fpq_search_clip_candidates",
-    "fpq_zero_census", "fpq_set_path_policy", "fpq_get_path_policy", "fpq_read_status", "fpq_status_string",
+    "fpq_zero_census", "fpq_prepared_size_split", "fpq_prepare_weight_split", "fpq_conv2d_split_workspace_size",
+    "fpq_conv2d_split", "fpq_set_path_policy", "fpq_get_path_policy", "fpq_read_status", "fpq_status_string",
 ]
 
 _lib = None
@@ -121,6 +122,14 @@ def lib() -> ctypes.CDLL:
         L.fpq_conv2d_contract.argtypes = [vp, sz, vp, vp, f32, F, F, vp, vp] + [i32] * 9 + [vp]
         L.fpq_linear_static.restype = i32
         L.fpq_linear_static.argtypes = [vp, vp, vp, f32, F, F, vp, vp, i64, i64, i64, vp]
+        L.fpq_prepared_size_split.restype = sz
+        L.fpq_prepared_size_split.argtypes = [F, i32, i32, i32, i32, i32]
+        L.fpq_prepare_weight_split.restype = i32
+        L.fpq_prepare_weight_split.argtypes = [vp, F, i32, i32, i32, i32, i32, vp, vp]
+        L.fpq_conv2d_split_workspace_size.restype = sz
+        L.fpq_conv2d_split_workspace_size.argtypes = [i32] * 10 + [F, F]
+        L.fpq_conv2d_split.restype = i32
+        L.fpq_conv2d_split.argtypes = [vp, i32, f32, vp, i32, f32, vp, vp, F, F, vp, vp] + [i32] * 8 + [vp, sz, vp]
         L.fpq_zero_census.restype = i32
         L.fpq_zero_census.argtypes = [vp, i64, F, vp, vp]
         L.fpq_search_workspace_size.restype = sz
@@ -310,6 +319,32 @@ def fpq_conv2d_host(x_host, x_dev, w_prepared, w_scale, x_scale, fx, fw, bias, y
                                  fx.c(), fw.c(), _ptr(bias), _ptr(y_dev), _ptr(y_host), B, C, H, W, C_out, R, S,
                                  pad, stride, _ptr(workspace), workspace.numel(), _stream()), "fpq_conv2d_host")
     return y_host
+
+
+def fpq_prepare_weight_split(codes: torch.Tensor, fmt: Format, N: int, C1: int, C2: int, R: int, S: int) -> torch.Tensor:
+    """Contraction-ready weights of a convolution over two concatenated input tensors."""
+    size = lib().fpq_prepared_size_split(fmt.c(), N, C1, C2, R, S)
+    assert size > 0, "invalid split layer"
+    prepared = torch.empty(size, dtype=torch.uint8, device=codes.device)
+    _check(lib().fpq_prepare_weight_split(_ptr(codes), fmt.c(), N, C1, C2, R, S, _ptr(prepared), _stream()),
+           "fpq_prepare_weight_split")
+    return prepared
+
+
+def fpq_conv2d_split_workspace_size(B, C1, C2, H, W, C_out, R, S, pad, stride, fx: Format, fw: Format) -> int:
+    return lib().fpq_conv2d_split_workspace_size(B, C1, C2, H, W, C_out, R, S, pad, stride, fx.c(), fw.c())
+
+
+def fpq_conv2d_split(x1, x1_scale, x2, x2_scale, w_prepared, w_scale, fx: Format, fw: Format, bias, y, R, S, pad,
+                     stride, workspace):
+    """Convolution over the channel concatenation of x1 and x2, quantized with their own scales."""
+    B, C1, H, W = x1.shape
+    C2 = x2.shape[1]
+    C_out = y.shape[1]
+    _check(lib().fpq_conv2d_split(_ptr(x1), C1, float(x1_scale), _ptr(x2), C2, float(x2_scale), _ptr(w_prepared),
+                                  _ptr(w_scale), fx.c(), fw.c(), _ptr(bias), _ptr(y), B, H, W, C_out, R, S, pad, stride,
+                                  _ptr(workspace), workspace.numel(), _stream()), "fpq_conv2d_split")
+    return y
 
 
 def fpq_zero_census(codes: torch.Tensor, n: int, fmt: Format, count: torch.Tensor = None) -> torch.Tensor:

@@ -187,8 +187,8 @@ fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_la
         return FPQ_ERR_NULL;
     if (!aligned(prepared, 128))
         return FPQ_ERR_ALIGN;
-    return launch_prepare_weight(codes, d->N, d->C, d->R * d->S, (int)padded_c(d->C), q.four_bit, (uint8_t*)prepared,
-                                 (cudaStream_t)stream) == cudaSuccess
+    return launch_prepare_weight(codes, d->N, d->C, d->R * d->S, (int)padded_c(d->C), q.four_bit, 0, 0,
+                                 (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
                ? FPQ_OK
                : FPQ_ERR_CUDA;
 }
@@ -375,8 +375,8 @@ fpq_status fpq_conv2d_quantize_input(const float* x, float x_scale, fpq_format f
         return FPQ_ERR_ALIGN;
     if (!status_word())
         return FPQ_ERR_CUDA;
-    return launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H, W, pad, (int)round_up(C, 16), x_scale, (uint8_t*)workspace,
-                                             (cudaStream_t)stream) == cudaSuccess
+    return launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H, W, pad, (int)round_up(C, 16), (int)round_up(C, 16), 0, x_scale,
+                                             (uint8_t*)workspace, (cudaStream_t)stream) == cudaSuccess
                ? FPQ_OK
                : FPQ_ERR_CUDA;
 }
@@ -462,6 +462,126 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
         return s;
     return conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out,
                                 R, S, pad, stride, stream, 1, nullptr);
+}
+
+// ---- convolution over two concatenated input tensors, each with its own scale ----------------
+
+static fpq_status split_shape(int C1, int C2)
+{
+    if (C1 < 1 || C2 < 1 || (int64_t)C1 + C2 > (1 << 20))
+        return FPQ_ERR_SHAPE;
+    return FPQ_OK;
+}
+
+size_t fpq_prepared_size_split(fpq_format fmt, int32_t N, int32_t C1, int32_t C2, int32_t R, int32_t S)
+{
+    QFormat q;
+    fpq_layer_desc d = {FPQ_CONV2D, N, C1 + C2, R, S};
+    if (!resolve_format(fmt, &q) || split_shape(C1, C2) != FPQ_OK || check_desc(&d) != FPQ_OK)
+        return 0;
+    size_t elems = (size_t)N * R * S * (size_t)(padded_c(C1) + padded_c(C2));
+    return q.four_bit ? elems / 2 : elems;
+}
+
+fpq_status fpq_prepare_weight_split(const uint8_t* codes, fpq_format fmt, int32_t N, int32_t C1, int32_t C2,
+                                    int32_t R, int32_t S, void* prepared, void* stream)
+{
+    QFormat q;
+    if (!resolve_format(fmt, &q))
+        return FPQ_ERR_FORMAT;
+    fpq_status s = split_shape(C1, C2);
+    if (s != FPQ_OK)
+        return s;
+    fpq_layer_desc d = {FPQ_CONV2D, N, C1 + C2, R, S};
+    s = check_desc(&d);
+    if (s != FPQ_OK)
+        return s;
+    if (!codes || !prepared)
+        return FPQ_ERR_NULL;
+    if (!aligned(prepared, 128))
+        return FPQ_ERR_ALIGN;
+    return launch_prepare_weight(codes, N, C1 + C2, R * S, (int)(padded_c(C1) + padded_c(C2)), q.four_bit, C1,
+                                 (int)padded_c(C1), (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
+               ? FPQ_OK
+               : FPQ_ERR_CUDA;
+}
+
+static size_t split_row_bytes(int C1, int C2) { return (size_t)(padded_c(C1) + round_up(C2, 16)); }
+
+size_t fpq_conv2d_split_workspace_size(int B, int C1, int C2, int H, int W, int C_out, int R, int S, int pad,
+                                       int stride, fpq_format fx, fpq_format fw)
+{
+    int Ho, Wo;
+    if (check_pair(fx, fw) != FPQ_OK || split_shape(C1, C2) != FPQ_OK ||
+        conv_shape(B, C1 + C2, H, W, C_out, R, S, pad, stride, &Ho, &Wo) != FPQ_OK)
+        return 0;
+    return (size_t)B * (H + 2 * pad) * (W + 2 * pad) * split_row_bytes(C1, C2);
+}
+
+fpq_status fpq_conv2d_split(const float* x1, int C1, float x1_scale, const float* x2, int C2, float x2_scale,
+                            const void* w_prepared, const float* w_scale, fpq_format fx, fpq_format fw,
+                            const float* bias, float* y, int B, int H, int W, int C_out, int R, int S, int pad,
+                            int stride, void* workspace, size_t ws_bytes, void* stream)
+{
+    fpq_status s = check_pair(fx, fw);
+    if (s != FPQ_OK)
+        return s;
+    s = split_shape(C1, C2);
+    if (s != FPQ_OK)
+        return s;
+    int Ho, Wo;
+    s = conv_shape(B, C1 + C2, H, W, C_out, R, S, pad, stride, &Ho, &Wo);
+    if (s != FPQ_OK)
+        return s;
+    if (B == 0 || C_out == 0)
+        return FPQ_OK;
+    if (B > 65535)
+        return FPQ_ERR_SHAPE;
+    const size_t row = split_row_bytes(C1, C2);
+    if (!workspace || ws_bytes < (size_t)B * (H + 2 * pad) * (W + 2 * pad) * row)
+        return FPQ_ERR_WORKSPACE;
+    if (!x1 || !x2 || !w_prepared || !w_scale || !y)
+        return FPQ_ERR_NULL;
+    if (!aligned(workspace, 128) || !aligned(x1, 4) || !aligned(x2, 4) || !aligned(y, 4) || !aligned(w_prepared, 128) ||
+        !aligned(w_scale, 4) || (bias && !aligned(bias, 4)))
+        return FPQ_ERR_ALIGN;
+    if (!status_word())
+        return FPQ_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int C1p = (int)padded_c(C1);
+    // each tensor is quantized with its own scale into its own channel range of the framed
+    // channels-last codes; the concatenated FP32 tensor is never formed
+    if (launch_quantize_nchw_to_nhwc_e4m3(x1, B, C1, H, W, pad, C1p, (int)row, 0, x1_scale, (uint8_t*)workspace, st) !=
+            cudaSuccess ||
+        launch_quantize_nchw_to_nhwc_e4m3(x2, B, C2, H, W, pad, (int)round_up(C2, 16), (int)row, C1p, x2_scale,
+                                          (uint8_t*)workspace, st) != cudaSuccess)
+        return FPQ_ERR_CUDA;
+    GemmProblem p{};
+    p.conv = 1;
+    p.after_stage1 = 1;
+    p.w4 = is_e2m1(fw) ? 1 : 0;
+    p.M = (int64_t)B * Ho * Wo;
+    p.N = C_out;
+    p.Cp = C1p + (int)padded_c(C2);
+    p.Ca = (int)row;
+    p.B = B;
+    p.H = H;
+    p.W = W;
+    p.Ho = Ho;
+    p.Wo = Wo;
+    p.R = R;
+    p.S = S;
+    p.pad = pad;
+    p.stride = stride;
+    p.a_codes = (const uint8_t*)workspace;
+    p.w_prepared = w_prepared;
+    p.w_scale = w_scale;
+    p.x_scale = x1_scale;
+    p.x_scale2 = x2_scale;
+    p.c_seg = C1p / 128;
+    p.bias = bias;
+    p.y = y;
+    return launch_gemm(p, st);
 }
 
 fpq_status fpq_linear_host(const float* x_host, float* x_dev, const void* w_prepared, const float* w_scale,

@@ -92,6 +92,10 @@ struct GemmArgs {
     int contiguous;            // tile order: 1 = every CTA walks a contiguous range, 0 = CTAs interleave
     int a_resident;            // a row tile's whole activation panel stays in the ring while the CTA walks its column tiles
     int ksplit;                // > 1: the CTAs of a cluster of this size share one output tile, each reducing a range of chunks
+    // input of two concatenated tensors: chunks [0, seg_chunk) carry x_scale and are shared out over the
+    // cluster's first seg_ranks CTAs, the others carry x_scale2 and go to the remaining CTAs; 0 = one tensor
+    int seg_chunk, seg_ranks;
+    float x_scale2;
     uint32_t a_chunk_tx, b_block_tx;   // bytes one load reports to its barrier
     const float* w_scale;
     float x_scale;
@@ -295,8 +299,19 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     // memory after the role loops below.
     const int ksplit = g.ksplit;
     const uint32_t krank = ksplit > 1 ? cluster_rank() : 0u;
-    const int c_lo = ksplit > 1 ? (int)krank * g.cchunks / ksplit : 0;
-    const int c_hi = ksplit > 1 ? ((int)krank + 1) * g.cchunks / ksplit : g.cchunks;
+    int c_lo = 0, c_hi = g.cchunks;
+    if (ksplit > 1 && !g.seg_chunk) {
+        c_lo = (int)krank * g.cchunks / ksplit;
+        c_hi = ((int)krank + 1) * g.cchunks / ksplit;
+    } else if (ksplit > 1) {
+        // a CTA's range never crosses from one input tensor into the other: their scales differ
+        const int first = (int)krank < g.seg_ranks;
+        const int k = first ? (int)krank : (int)krank - g.seg_ranks;
+        const int ranks = first ? g.seg_ranks : ksplit - g.seg_ranks;
+        const int base = first ? 0 : g.seg_chunk, len = first ? g.seg_chunk : g.cchunks - g.seg_chunk;
+        c_lo = base + k * len / ranks;
+        c_hi = base + (k + 1) * len / ranks;
+    }
     const int nblk = (c_hi - c_lo) * g.taps;
     const int t_lo = ksplit > 1 ? (int)blockIdx.x / ksplit
                                 : g.contiguous ? (int)((int64_t)blockIdx.x * total_tiles / gridDim.x) : (int)blockIdx.x;
@@ -942,15 +957,21 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
                     v[k] = k < ksplit ? ld_peer_smem(addr, (uint32_t)k) : 0.f;
-                float acc = v[0];
+                const int first_ranks = g.seg_chunk ? g.seg_ranks : ksplit;
+                float acc = v[0], acc2 = 0.f;              // sums over the first / second input tensor
 #pragma unroll
                 for (int k = 1; k < 8; ++k)
-                    if (k < ksplit)
-                        acc += v[k];
+                    if (k < ksplit) {
+                        if (k < first_ranks) acc += v[k];
+                        else                 acc2 += v[k];
+                    }
                 const float sv = g.stage_scales ? s_scale[n] : g.x_scale * __ldg(g.w_scale + n);
                 const float bv = g.stage_scales ? s_bias[n] : (g.bias ? __ldg(g.bias + n) : 0.f);
+                float out = fmaf(acc, sv, bv);
+                if (g.seg_chunk)
+                    out = fmaf(acc2, g.x_scale2 * __ldg(g.w_scale + n), out);
                 if (row_valid)
-                    yrow[(int64_t)n * nstride] = fmaf(acc, sv, bv);
+                    yrow[(int64_t)n * nstride] = out;
             }
         }
         // nobody leaves (and frees its shared memory) while a peer may still read it
@@ -1078,7 +1099,28 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
     // then the smallest one with the same longest chunk range.
     g.ksplit = 1;
     const int64_t base_tiles = (int64_t)g.m_tiles * g.n_tiles;
-    if (MODE != MODE_ROWS && g.cchunks >= 2 && base_tiles * 2 <= di->sms) {
+    if (g.seg_chunk) {
+        // two input tensors: always a cluster, at least one CTA per tensor; as many CTAs as keep
+        // every tile resident at once when the tiles are few, a pair per tile otherwise
+        if (MODE == MODE_ROWS || FUSED || g.seg_chunk >= g.cchunks)
+            return FPQ_ERR_UNSUPPORTED;
+        int sp = 2;
+        if (base_tiles * 2 <= di->sms) {
+            sp = (int)(di->sms / base_tiles);
+            if (sp > 8) sp = 8;
+            if (sp > g.cchunks) sp = g.cchunks;
+            while (sp > 2 && max_clusters<BN, MODE>(di, sp) < base_tiles)
+                --sp;
+        }
+        int r1 = (sp * g.seg_chunk + g.cchunks / 2) / g.cchunks;
+        if (r1 < 1) r1 = 1;
+        if (r1 > sp - 1) r1 = sp - 1;
+        if (r1 > g.seg_chunk) r1 = g.seg_chunk;
+        int r2 = sp - r1;
+        if (r2 > g.cchunks - g.seg_chunk) r2 = g.cchunks - g.seg_chunk;
+        g.seg_ranks = r1;
+        g.ksplit = r1 + r2;
+    } else if (MODE != MODE_ROWS && g.cchunks >= 2 && base_tiles * 2 <= di->sms) {
         int s_max = (int)(di->sms / base_tiles);
         if (s_max > 8) s_max = 8;
         if (s_max > g.cchunks) s_max = g.cchunks;
@@ -1172,6 +1214,8 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
     if (!allow_max_smem<BN, FUSED, MODE>(di))
         return FPQ_ERR_CUDA;
     const int64_t tiles = (int64_t)g.m_tiles * g.n_tiles;
+    if (g.ksplit > 1 && tiles * g.ksplit > 0x7fffff00ll)
+        return FPQ_ERR_SHAPE;
     const int grid = g.ksplit > 1 ? (int)tiles * g.ksplit : (int)(tiles < di->sms ? tiles : di->sms);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
@@ -1231,6 +1275,8 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
     g.B = p.B;
     g.w_scale = p.w_scale;
     g.x_scale = p.x_scale;
+    g.seg_chunk = p.c_seg;
+    g.x_scale2 = p.x_scale2;
     g.bias = p.bias;
     g.y = p.y;
     g.status = status_word();

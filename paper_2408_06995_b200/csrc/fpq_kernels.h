@@ -14,11 +14,11 @@ cudaError_t launch_quantize_weight(const float* w, int64_t N, int64_t K, const f
                                    const uint8_t* rbits, uint8_t* codes, cudaStream_t st);
 cudaError_t launch_quantize_rows_e4m3(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, uint8_t* codes,
                                       cudaStream_t st);
-cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int H, int W, int pad, int Cp, float scale,
-                                              uint8_t* codes, cudaStream_t st);
+cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int H, int W, int pad, int Cp, int row,
+                                              int c_off, float scale, uint8_t* codes, cudaStream_t st);
 cudaError_t launch_zero_census(const uint8_t* codes, int64_t n, int four_bit, unsigned long long* count, cudaStream_t st);
-cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, uint8_t* prepared,
-                                  cudaStream_t st);
+cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, int C1, int C1p,
+                                  uint8_t* prepared, cudaStream_t st);
 
 // Geometry of one contraction launch (linear: taps = 1, rows of Ca codes).
 struct GemmProblem {
@@ -39,6 +39,10 @@ struct GemmProblem {
     float x_scale;
     const float* bias;
     float* y;
+    // input made of two concatenated tensors with their own scales: the first c_seg 128-wide chunks
+    // of the reduction belong to the first tensor (x_scale), the rest to the second (x_scale2); 0 = one tensor
+    int c_seg;
+    float x_scale2;
 };
 
 // Returns FPQ_OK or an error; enqueues one kernel.

@@ -166,15 +166,17 @@ __global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const float* __
 }
 
 // ---------------------------------------------------------------------------------
-// NCHW FP32 -> channels-last codes with a zero frame: [B][H+2p][W+2p][Cp] (Cp = C
-// rounded up to 16, channel padding and frame = code 0), the A operand of the
-// implicit-GEMM convolution.  A block transposes 128 channels x 32 pixels through
+// NCHW FP32 -> channels-last codes with a zero frame: [B][H+2p][W+2p][row] (channel padding
+// and frame = code 0), the A operand of the implicit-GEMM convolution.  The kernel fills the
+// channels [c_off, c_off + Cp) of every pixel row (Cp = C rounded up to 16, or further for the
+// first of two concatenated tensors); row = Cp and c_off = 0 for a single input tensor.  A block transposes 128 channels x 32 pixels through
 // shared memory: loads are coalesced along pixels (16 in flight per thread), stores
 // are whole 128-byte channel rows.  The blocks also share out the frame pixels.
 // ---------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const float* __restrict__ x, int C, int H,
-                                                                         int W, int pad, int Cp, float rinv,
-                                                                         uint8_t* __restrict__ codes, int* status)
+                                                                         int W, int pad, int Cp, int row, int c_off,
+                                                                         float rinv, uint8_t* __restrict__ codes,
+                                                                         int* status)
 {
     __shared__ __align__(16) uint8_t tile[32][128 + 16];
     // the contraction queued behind this kernel may start its set-up (it waits for this grid
@@ -187,7 +189,7 @@ __global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const f
     const int p0 = blockIdx.x * 32;
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 pixels x 8 channel groups of 16
     const float* xb = x + (int64_t)b * C * HW;
-    uint8_t* ob = codes + (int64_t)b * Hp * Wp * Cp;
+    uint8_t* ob = codes + (int64_t)b * Hp * Wp * row + c_off;
     const int p = p0 + tx;
     {
         const int cl = ty * 16;
@@ -217,7 +219,7 @@ __global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const f
         if (pp < HW && c < Cp) {
             const int yy = pp / W, xx = pp - yy * W;
             const uint4 v = *reinterpret_cast<const uint4*>(&tile[pl][ch]);
-            *reinterpret_cast<uint4*>(ob + ((int64_t)(yy + pad) * Wp + (xx + pad)) * Cp + c) = v;
+            *reinterpret_cast<uint4*>(ob + ((int64_t)(yy + pad) * Wp + (xx + pad)) * row + c) = v;
         }
     }
     // frame pixels of this image, shared out over the blocks of the image's pixel axis
@@ -240,7 +242,7 @@ __global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const f
                 const int e = k % (2 * pad);
                 xp = (e < pad) ? e : W + e;
             }
-            *reinterpret_cast<uint4*>(ob + ((int64_t)yp * Wp + xp) * Cp + c0 + ch) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4*>(ob + ((int64_t)yp * Wp + xp) * row + c0 + ch) = make_uint4(0, 0, 0, 0);
         }
     }
     if (nan)
@@ -249,10 +251,13 @@ __global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const f
 
 // ---------------------------------------------------------------------------------
 // Contraction-ready weight copy: [N][C][R][S] codes -> [N][R*S][Cp] codes, zero padded.
-// One thread per output byte.
+// One thread per output byte.  For an input made of two concatenated tensors (C1 > 0) the
+// channels from C1 on start at position C1p (C1 rounded up to 128), so that each tensor's
+// channels fill whole 128-wide chunks of the reduction.
 // ---------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) prepare_weight_kernel(const uint8_t* __restrict__ codes, int N, int C, int RS,
-                                                             int Cp, int four_bit, uint8_t* __restrict__ prepared)
+                                                             int Cp, int four_bit, int C1, int C1p,
+                                                             uint8_t* __restrict__ prepared)
 {
     int64_t row_out = four_bit ? (int64_t)RS * Cp / 2 : (int64_t)RS * Cp;
     int64_t total = (int64_t)N * row_out;
@@ -267,7 +272,13 @@ __global__ void __launch_bounds__(256) prepare_weight_kernel(const uint8_t* __re
             int64_t e = within * per + q;       // element index in [RS][Cp]
             int tap = (int)(e / Cp), c = (int)(e % Cp);
             uint32_t code = 0;
-            if (c < C) {
+            bool real = c < C;
+            if (C1 > 0) {
+                real = c < C1 || (c >= C1p && c - C1p + C1 < C);
+                if (c >= C1p)
+                    c = c - C1p + C1;
+            }
+            if (real) {
                 int64_t k = (int64_t)c * RS + tap;   // source order [C][R][S]
                 if (four_bit) {
                     uint8_t bsrc = __ldg(codes + n * row_in + (k >> 1));
@@ -329,11 +340,12 @@ cudaError_t launch_quantize_rows_e4m3(const float* x, int64_t M, int64_t K, int6
     return cudaGetLastError();
 }
 
-cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int H, int W, int pad, int Cp, float scale,
-                                              uint8_t* codes, cudaStream_t st)
+cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int H, int W, int pad, int Cp, int row,
+                                              int c_off, float scale, uint8_t* codes, cudaStream_t st)
 {
     dim3 grid((H * W + 31) / 32, (Cp + 127) / 128, B);
-    quantize_nchw_to_nhwc_e4m3_kernel<<<grid, 256, 0, st>>>(x, C, H, W, pad, Cp, 1.0f / scale, codes, status_word());
+    quantize_nchw_to_nhwc_e4m3_kernel<<<grid, 256, 0, st>>>(x, C, H, W, pad, Cp, row, c_off, 1.0f / scale, codes,
+                                                            status_word());
     return cudaGetLastError();
 }
 
@@ -401,11 +413,11 @@ cudaError_t launch_zero_census(const uint8_t* codes, int64_t n, int four_bit, un
     return cudaGetLastError();
 }
 
-cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, uint8_t* prepared,
-                                  cudaStream_t st)
+cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, int C1, int C1p,
+                                  uint8_t* prepared, cudaStream_t st)
 {
     int64_t total = (int64_t)N * RS * Cp / (four_bit ? 2 : 1);
-    prepare_weight_kernel<<<grid_for(total, 256), 256, 0, st>>>(codes, N, C, RS, Cp, four_bit, prepared);
+    prepare_weight_kernel<<<grid_for(total, 256), 256, 0, st>>>(codes, N, C, RS, Cp, four_bit, C1, C1p, prepared);
     return cudaGetLastError();
 }
 
