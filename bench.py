@@ -645,6 +645,67 @@ def run_search(args):
     print(json.dumps(out), flush=True)
 
 
+def run_split(args):
+    """The decoder convolutions of the SD-v1-style U-Net whose input is a concatenation (previous
+    layer's output + skip connection), W4A8, batch 2: the two-scale call against the ordinary call
+    on the already concatenated tensor."""
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    from paper_2408_06995_b200 import build as fpq_build
+    fpq_build.build()
+    import paper_2408_06995_b200 as fpq
+    peaks = load_peaks()
+    shapes = [("up3.res.conv1", 1280, 1280, 8, 1280, 3), ("up2.res0.conv1", 1280, 1280, 16, 1280, 3),
+              ("up2.res2.conv1", 1280, 640, 16, 1280, 3), ("up1.res0.conv1", 1280, 640, 32, 640, 3),
+              ("up1.res1.conv1", 640, 640, 32, 640, 3), ("up1.res2.conv1", 640, 320, 32, 640, 3),
+              ("up0.res0.conv1", 640, 320, 64, 320, 3), ("up0.res1.conv1", 320, 320, 64, 320, 3),
+              ("up0.res1.skip", 320, 320, 64, 320, 1)]
+    B, fw = 2, fpq.E2M1
+    rows = []
+    for name, C1, C2, HW, Co, R in shapes:
+        pad = R // 2
+        nsets = max(2, int(3 * (128 << 20) / (B * (C1 + C2 + Co) * HW * HW * 4)) + 1)
+        nsets = min(nsets, 64)
+        x1 = [torch.randn(B, C1, HW, HW, device=dev) for _ in range(nsets)]
+        x2 = [torch.randn(B, C2, HW, HW, device=dev) * 3 for _ in range(nsets)]
+        xc = [torch.cat([a, b], dim=1).contiguous() for a, b in zip(x1, x2)]
+        ys = [torch.empty(B, Co, HW, HW, device=dev) for _ in range(nsets)]
+        w = torch.randn(Co, (C1 + C2) * R * R, device=dev) * 0.02
+        ws = (w.abs().amax(dim=1) / 6.0).contiguous()
+        codes = fpq.fpq_quantize_weight(w, ws, fw, None)
+        prep_s = fpq.fpq_prepare_weight_split(codes, fw, Co, C1, C2, R, R)
+        prep_c = fpq.fpq_prepare_weight(codes, fw, fpq.CONV2D, Co, C1 + C2, R, R)
+        bias = torch.zeros(Co, device=dev)
+        wk = torch.empty(fpq.fpq_conv2d_split_workspace_size(B, C1, C2, HW, HW, Co, R, R, pad, 1, fpq.E4M3, fw),
+                         dtype=torch.uint8, device=dev)
+        s1, s2, sc = float(x1[0].abs().max()) / 448, float(x2[0].abs().max()) / 448, float(xc[0].abs().max()) / 448
+        k = [0]
+
+        def split_call():
+            i = k[0] = (k[0] + 1) % nsets
+            fpq.fpq_conv2d_split(x1[i], s1, x2[i], s2, prep_s, ws, fpq.E4M3, fw, bias, ys[i], R, R, pad, 1, wk)
+
+        def plain_call():
+            i = k[0] = (k[0] + 1) % nsets
+            fpq.fpq_conv2d(xc[i], prep_c, ws, sc, fpq.E4M3, fw, bias, Co, R, R, pad, 1, ys[i], wk)
+
+        t_s = per_launch_us(torch, split_call, 4 * nsets)
+        t_p = per_launch_us(torch, plain_call, 4 * nsets)
+        flops = 2.0 * B * HW * HW * Co * (C1 + C2) * R * R
+        by = 4.0 * B * (C1 + C2 + Co) * HW * HW + Co * (C1 + C2) * R * R / 2 + 8 * Co
+        rows.append({"name": name, "C1": C1, "C2": C2, "HW": HW, "C_out": Co, "R": R, "us_split": t_s, "us_plain": t_p,
+                     "tflops_split": flops / t_s / 1e6, "t_hbm_us": by / peaks["hbm_gbs"] / 1e3,
+                     "t_tensor_us": flops / NOMINAL_FP8_TFLOPS / 1e6})
+        del x1, x2, xc, ys
+        torch.cuda.empty_cache()
+    print(json.dumps({"suite": "sd_split", "batch": B, "rows": rows,
+                      "sum_us": {"split": sum(r["us_split"] for r in rows), "plain": sum(r["us_plain"] for r in rows)}}),
+          flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -653,13 +714,15 @@ def main():
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline leg")
     ap.add_argument("--skip-w4", action="store_true", help="leave out the W4A8 side measurement")
-    ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd", "sd_trace", "search"],
+    ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd", "sd_trace", "search", "sd_split"],
                     help="print a per-shape table of a whole workload instead of the headline line")
     args = ap.parse_args()
     if args.suite == "sd_trace":
         run_trace(args)
     elif args.suite == "search":
         run_search(args)
+    elif args.suite == "sd_split":
+        run_split(args)
     elif args.suite:
         run_suite(args)
     elif args.impl == "reference":

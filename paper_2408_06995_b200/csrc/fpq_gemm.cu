@@ -96,6 +96,7 @@ struct GemmArgs {
     // cluster's first seg_ranks CTAs, the others carry x_scale2 and go to the remaining CTAs; 0 = one tensor
     int seg_chunk, seg_ranks;
     float x_scale2;
+    int seg_acc;               // two tensors without a cluster: each has its own accumulator, the epilogue joins them
     uint32_t a_chunk_tx, b_block_tx;   // bytes one load reports to its barrier
     const float* w_scale;
     float x_scale;
@@ -337,7 +338,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             tma_prefetch_desc(&tmY);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32((const void*)tmem_slot), 2 * BN);
+        tmem_alloc(smem_u32((const void*)tmem_slot), g.seg_acc ? 4 * BN : 2 * BN);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -527,6 +528,8 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                     if (!mbar_wait(b_full + 8 * sb, pb)) { dead = true; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
+                // chunks from seg_from on (the second input tensor) add up in the accumulator 2 * BN columns further
+                const int seg_from = (!FUSED && g.seg_acc) ? g.seg_chunk : 0x7fffffff;
 
                 if (MODE == MODE_FLAT && g.taps == 9 && g.S == 3) {
                     const uint32_t Wp8 = (uint32_t)g.Wp * 8u;
@@ -540,6 +543,8 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                         for (int c = 0; c < nch && !dead; ++c, ++cc) {
                             const uint32_t ac = abase + c * a_chunk_step;
                             const uint32_t bres = b_res + (uint32_t)cc * 9u * BSTEP;
+                            const uint32_t d = cc >= seg_from ? d_tmem + 2 * BN : d_tmem;
+                            const bool fresh = cc == c_lo || cc == seg_from;
                             uint32_t bst = 0;
 #pragma unroll
                             for (int tap = 0; tap < 9; ++tap) {
@@ -552,13 +557,13 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                                 const uint32_t al = ac + (tap / 3) * Wp8 + (tap % 3) * 8u;
                                 const uint32_t bl = g.b_resident ? bres + tap * BSTEP : bst + (tap % 3) * BSTEP;
                                 // 32 reduction elements = 32 bytes inside the swizzled row: +2 units
-                                if (tap == 0 && cc == c_lo)
-                                    mma_f8f6f4<false>(d_tmem, al, bl, HI, g.idesc);
+                                if (tap == 0 && fresh)
+                                    mma_f8f6f4<false>(d, al, bl, HI, g.idesc);
                                 else
-                                    mma_f8f6f4<true>(d_tmem, al, bl, HI, g.idesc);
-                                mma_f8f6f4<true>(d_tmem, al + 2, bl + 2, HI, g.idesc);
-                                mma_f8f6f4<true>(d_tmem, al + 4, bl + 4, HI, g.idesc);
-                                mma_f8f6f4<true>(d_tmem, al + 6, bl + 6, HI, g.idesc);
+                                    mma_f8f6f4<true>(d, al, bl, HI, g.idesc);
+                                mma_f8f6f4<true>(d, al + 2, bl + 2, HI, g.idesc);
+                                mma_f8f6f4<true>(d, al + 4, bl + 4, HI, g.idesc);
+                                mma_f8f6f4<true>(d, al + 6, bl + 6, HI, g.idesc);
                                 if (!g.b_resident && tap % 3 == 2) {
                                     mma_commit(b_empty + 8 * sb);
                                     if (++sb == (uint32_t)g.b_stages) { sb = 0; pb ^= 1; }
@@ -587,13 +592,14 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                         for (int c = 0; c < 4; ++c) {
                             if (c < n) {
                                 const uint32_t al = abase + c * (BM * BK / 16), bl = bbase + c * BSTEP;
-                                if (c == 0 && cc == c_lo)
-                                    mma_f8f6f4<false>(d_tmem, al, bl, HI, g.idesc);
+                                const uint32_t d = cc + c >= seg_from ? d_tmem + 2 * BN : d_tmem;
+                                if (cc + c == c_lo || cc + c == seg_from)
+                                    mma_f8f6f4<false>(d, al, bl, HI, g.idesc);
                                 else
-                                    mma_f8f6f4<true>(d_tmem, al, bl, HI, g.idesc);
-                                mma_f8f6f4<true>(d_tmem, al + 2, bl + 2, HI, g.idesc);
-                                mma_f8f6f4<true>(d_tmem, al + 4, bl + 4, HI, g.idesc);
-                                mma_f8f6f4<true>(d_tmem, al + 6, bl + 6, HI, g.idesc);
+                                    mma_f8f6f4<true>(d, al, bl, HI, g.idesc);
+                                mma_f8f6f4<true>(d, al + 2, bl + 2, HI, g.idesc);
+                                mma_f8f6f4<true>(d, al + 4, bl + 4, HI, g.idesc);
+                                mma_f8f6f4<true>(d, al + 6, bl + 6, HI, g.idesc);
                             }
                         }
                         if (!g.b_resident) {
@@ -613,6 +619,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                     const uint32_t row_wrap8 = (uint32_t)(g.Wp - g.S) * 8u;
                     const bool flat = MODE == MODE_FLAT, taps_mode = MODE == MODE_TAPS;
                     int tap = 0, sx = 0, ja = 0, jb = 0;
+                    int ccg = c_lo;                        // chunk of the current block
                     for (int j = 0; j < nblk; ++j) {
                         if (ja == 0) {
                             if (!reuse_a)
@@ -627,13 +634,14 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                             b_lo = smem_desc_lo(b_ring + sb * g.b_stage_bytes);
                         }
                         const uint32_t al = flat ? a_chunk_lo + row_off8 : a_lo;
-                        if (j == 0)
-                            mma_f8f6f4<false>(d_tmem, al, b_lo, HI, g.idesc);
+                        const uint32_t d = ccg >= seg_from ? d_tmem + 2 * BN : d_tmem;
+                        if (j == 0 || (tap == 0 && ccg == seg_from))
+                            mma_f8f6f4<false>(d, al, b_lo, HI, g.idesc);
                         else
-                            mma_f8f6f4<true>(d_tmem, al, b_lo, HI, g.idesc);
-                        mma_f8f6f4<true>(d_tmem, al + 2, b_lo + 2, HI, g.idesc);
-                        mma_f8f6f4<true>(d_tmem, al + 4, b_lo + 4, HI, g.idesc);
-                        mma_f8f6f4<true>(d_tmem, al + 6, b_lo + 6, HI, g.idesc);
+                            mma_f8f6f4<true>(d, al, b_lo, HI, g.idesc);
+                        mma_f8f6f4<true>(d, al + 2, b_lo + 2, HI, g.idesc);
+                        mma_f8f6f4<true>(d, al + 4, b_lo + 4, HI, g.idesc);
+                        mma_f8f6f4<true>(d, al + 6, b_lo + 6, HI, g.idesc);
                         const bool last = (j == nblk - 1);
                         b_lo += BSTEP;
                         if (++jb == g.b_span || last) {
@@ -649,6 +657,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                         if (taps_mode) a_lo += a_chunk_step;
                         if (++tap == g.taps) {
                             tap = 0; sx = 0; row_off8 = 0;
+                            ++ccg;
                             a_chunk_lo += a_chunk_step;
                             if (!taps_mode) a_lo = a_chunk_lo;
                         }
@@ -773,6 +782,17 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                                 const float sv = in ? __ldg(g.w_scale + nb + j) : 0.f;
                                 const float bv = (in && g.bias) ? __ldg(g.bias + nb + j) : 0.f;
                                 r[cl][j] = __float_as_uint(fmaf(__uint_as_float(r[cl][j]), g.x_scale * sv, bv));
+                            }
+                        }
+                        if (!FUSED && g.seg_acc) {
+                            // the second input tensor's sums, with its own scale
+                            uint32_t r2[32];
+                            tmem_ld32(t_addr + 2 * BN + (c0 + cl) * 32, r2);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const float sv = nb + j < g.N ? g.x_scale2 * __ldg(g.w_scale + nb + j) : 0.f;
+                                r[cl][j] = __float_as_uint(fmaf(__uint_as_float(r2[j]), sv, __uint_as_float(r[cl][j])));
                             }
                         }
                         if (g.y_tma) {
@@ -982,7 +1002,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 2 * BN);
+        tmem_dealloc(tmem_base, g.seg_acc ? 4 * BN : 2 * BN);
     }
 }
 
@@ -1100,26 +1120,33 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
     g.ksplit = 1;
     const int64_t base_tiles = (int64_t)g.m_tiles * g.n_tiles;
     if (g.seg_chunk) {
-        // two input tensors: always a cluster, at least one CTA per tensor; as many CTAs as keep
-        // every tile resident at once when the tiles are few, a pair per tile otherwise
+        // two input tensors: with few tiles a cluster per tile, at least one CTA per tensor and as
+        // many CTAs as keep every tile resident at once; with many tiles no cluster
         if (MODE == MODE_ROWS || FUSED || g.seg_chunk >= g.cchunks)
             return FPQ_ERR_UNSUPPORTED;
         int sp = 2;
-        if (base_tiles * 2 <= di->sms) {
+        g.seg_acc = 0;
+        if (base_tiles * 2 > di->sms) {
+            // plenty of tiles: the usual persistent walk, one accumulator per tensor
+            sp = 1;
+            g.seg_acc = 1;
+        } else {
             sp = (int)(di->sms / base_tiles);
             if (sp > 8) sp = 8;
             if (sp > g.cchunks) sp = g.cchunks;
             while (sp > 2 && max_clusters<BN, MODE>(di, sp) < base_tiles)
                 --sp;
         }
-        int r1 = (sp * g.seg_chunk + g.cchunks / 2) / g.cchunks;
-        if (r1 < 1) r1 = 1;
-        if (r1 > sp - 1) r1 = sp - 1;
-        if (r1 > g.seg_chunk) r1 = g.seg_chunk;
-        int r2 = sp - r1;
-        if (r2 > g.cchunks - g.seg_chunk) r2 = g.cchunks - g.seg_chunk;
-        g.seg_ranks = r1;
-        g.ksplit = r1 + r2;
+        if (!g.seg_acc) {
+            int r1 = (sp * g.seg_chunk + g.cchunks / 2) / g.cchunks;
+            if (r1 < 1) r1 = 1;
+            if (r1 > sp - 1) r1 = sp - 1;
+            if (r1 > g.seg_chunk) r1 = g.seg_chunk;
+            int r2 = sp - r1;
+            if (r2 > g.cchunks - g.seg_chunk) r2 = g.cchunks - g.seg_chunk;
+            g.seg_ranks = r1;
+            g.ksplit = r1 + r2;
+        }
     } else if (MODE != MODE_ROWS && g.cchunks >= 2 && base_tiles * 2 <= di->sms) {
         int s_max = (int)(di->sms / base_tiles);
         if (s_max > 8) s_max = 8;
