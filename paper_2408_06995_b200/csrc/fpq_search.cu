@@ -16,7 +16,7 @@ constexpr int SEARCH_PER_THREAD = 16;
 constexpr int SEARCH_MAX_ENC = 8;
 constexpr int SEARCH_MAX_CLIP = 256;
 constexpr int SEARCH_MAX_CAND = 1024;
-constexpr int SEARCH_MAX_BLOCKS = 592;
+constexpr int SEARCH_MAX_BLOCKS = 1184;
 
 struct SearchEnc {
     uint32_t cmax_bits;      // FP32 bit pattern of the format's own clipping value
@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(SEARCH_THREADS) search_mse_kernel(const Search
         atomicMin(a.status, FPQ_ERR_NAN_INPUT);
 }
 
-// Block partial sums -> mse (added in block order, so the result does not depend on timing), then
+// Block partial sums -> mse (added in a fixed order, so the result does not depend on timing), then
 // Algorithm 1: encodings in the outer loop, clipping candidates in the inner one, a candidate is
 // kept only when its error is strictly below the best so far, which starts at +infinity.
 __global__ void __launch_bounds__(1024) search_finish_kernel(const double* __restrict__ partial, int blocks, int n_enc,
@@ -126,11 +126,17 @@ __global__ void __launch_bounds__(1024) search_finish_kernel(const double* __res
                                                              int32_t* __restrict__ best)
 {
     const int ncand = n_enc * n_clip;
-    for (int c = threadIdx.x; c < ncand; c += blockDim.x) {
+    // one warp per candidate: lane l adds the blocks l, l + 32, ... in order, then a fixed shuffle tree
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int c = warp; c < ncand; c += (int)(blockDim.x >> 5)) {
         double s = 0.0;
-        for (int b = 0; b < blocks; ++b)
+        for (int b = lane; b < blocks; b += 32)
             s += partial[(int64_t)b * ncand + c];
-        mse[c] = n > 0 ? s / (double)n : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+            s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0)
+            mse[c] = n > 0 ? s / (double)n : 0.0;
     }
     __syncthreads();
     if (threadIdx.x == 0) {

@@ -87,7 +87,7 @@ def test_search_host_side(L):
     native = (fpq._CFormat * 1)(fpq.E4M3.c())
     assert L.fpq_search_format(big, 8, ctypes.cast(native, ctypes.c_void_p), 1, big, 4, big, big, big, 1 << 30,
                                None) == fpq.ERR_UNSUPPORTED
-    assert fpq.fpq_search_workspace_size(4, 111) == 592 * 444 * 8
+    assert fpq.fpq_search_workspace_size(4, 111) == 1184 * 444 * 8
     assert fpq.fpq_search_workspace_size(8, 256) == 0            # more than 1024 candidates
     # the clipping candidates are the oracle's, bit for bit
     for maxabs in (3.7, 0.0123, 1e4):
