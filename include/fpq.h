@@ -286,7 +286,7 @@ fpq_status fpq_zero_census(const uint8_t* codes, int64_t n, fpq_format fmt, uint
  *   best       DEVICE out, 2 int32
  *   workspace  fpq_search_workspace_size(n_enc, n_clip) bytes, 8-byte aligned; contents need
  *              not be kept between calls
- * Two kernels on `stream`, no allocation, no host synchronisation.  Errors: FPQ_ERR_NULL,
+ * Three kernels on `stream`, no allocation, no host synchronisation.  Errors: FPQ_ERR_NULL,
  * FPQ_ERR_SHAPE (counts out of range, n < 0), FPQ_ERR_FORMAT, FPQ_ERR_UNSUPPORTED (sat_mode),
  * FPQ_ERR_ALIGN, FPQ_ERR_WORKSPACE, FPQ_ERR_CUDA.
  */

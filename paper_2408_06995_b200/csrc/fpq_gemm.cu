@@ -977,14 +977,22 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
                     v[k] = k < ksplit ? ld_peer_smem(addr, (uint32_t)k) : 0.f;
-                const int first_ranks = g.seg_chunk ? g.seg_ranks : ksplit;
                 float acc = v[0], acc2 = 0.f;              // sums over the first / second input tensor
+                if (!g.seg_chunk) {
 #pragma unroll
-                for (int k = 1; k < 8; ++k)
-                    if (k < ksplit) {
-                        if (k < first_ranks) acc += v[k];
-                        else                 acc2 += v[k];
+                    for (int k = 1; k < 8; ++k)
+                        if (k < ksplit)
+                            acc += v[k];
+                } else {
+                    // selects, not branches (v[k] is 0 beyond the cluster): branching per rank here
+                    // was measured to cost microseconds
+                    acc = 0.f;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        acc += k < g.seg_ranks ? v[k] : 0.f;
+                        acc2 += k < g.seg_ranks ? 0.f : v[k];
                     }
+                }
                 const float sv = g.stage_scales ? s_scale[n] : g.x_scale * __ldg(g.w_scale + n);
                 const float bv = g.stage_scales ? s_bias[n] : (g.bias ? __ldg(g.bias + n) : 0.f);
                 float out = fmaf(acc, sv, bv);
@@ -1147,7 +1155,10 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
             g.seg_ranks = r1;
             g.ksplit = r1 + r2;
         }
-    } else if (MODE != MODE_ROWS && g.cchunks >= 2 && base_tiles * 2 <= di->sms) {
+    } else if (g.cchunks >= 2 && base_tiles * 2 <= di->sms &&
+               (MODE != MODE_ROWS || (g.m_tiles == 1 && g.cchunks >= 32))) {
+        // (row-major outputs leave the cluster's reduction column by column, which only pays for a single
+        // row tile with a very long reduction: measured on the SD-v1 linears)
         int s_max = (int)(di->sms / base_tiles);
         if (s_max > 8) s_max = 8;
         if (s_max > g.cchunks) s_max = g.cchunks;

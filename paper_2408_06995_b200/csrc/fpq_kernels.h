@@ -48,7 +48,7 @@ struct GemmProblem {
 // Returns FPQ_OK or an error; enqueues one kernel.
 fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st);
 
-// Encoding / bias search: limits, scratch size, and the two-kernel launch.
+// Encoding / bias search: limits, scratch size, and the launch (three kernels).
 int search_max_enc();
 int search_max_clip();
 int search_max_cand();

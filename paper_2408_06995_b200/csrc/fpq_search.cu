@@ -118,41 +118,60 @@ __global__ void __launch_bounds__(SEARCH_THREADS) search_mse_kernel(const Search
         atomicMin(a.status, FPQ_ERR_NAN_INPUT);
 }
 
-// Block partial sums -> mse (added in a fixed order, so the result does not depend on timing), then
-// Algorithm 1: encodings in the outer loop, clipping candidates in the inner one, a candidate is
-// kept only when its error is strictly below the best so far, which starts at +infinity.
-__global__ void __launch_bounds__(1024) search_finish_kernel(const double* __restrict__ partial, int blocks, int n_enc,
-                                                             int n_clip, int64_t n, double* __restrict__ mse,
-                                                             int32_t* __restrict__ best)
+// Block partial sums -> mse.  A block of 32 x 32 threads owns 32 candidates: thread (slice, ci) adds
+// the blocks slice, slice + 32, ... of candidate c0 + ci (coalesced along ci), then the 32 slices are
+// added in order: the same order whatever the timing.
+__global__ void __launch_bounds__(1024) search_reduce_kernel(const double* __restrict__ partial, int blocks, int ncand,
+                                                             int64_t n, double* __restrict__ mse)
 {
-    const int ncand = n_enc * n_clip;
-    // one warp per candidate: lane l adds the blocks l, l + 32, ... in order, then a fixed shuffle tree
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int c = warp; c < ncand; c += (int)(blockDim.x >> 5)) {
-        double s = 0.0;
-        for (int b = lane; b < blocks; b += 32)
+    __shared__ double s_part[32][33];
+    const int ci = threadIdx.x & 31, slice = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + ci;
+    double s = 0.0;
+    if (c < ncand)
+        for (int b = slice; b < blocks; b += 32)
             s += partial[(int64_t)b * ncand + c];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1)
-            s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (lane == 0)
-            mse[c] = n > 0 ? s / (double)n : 0.0;
-    }
+    s_part[slice][ci] = s;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        double prev_mse = INFINITY;
-        int bi = -1, bj = -1;
-        for (int i = 0; i < n_enc; ++i)
-            for (int j = 0; j < n_clip; ++j) {
-                const double curr_mse = mse[i * n_clip + j];
-                if (prev_mse > curr_mse) {
-                    bi = i;
-                    bj = j;
-                    prev_mse = curr_mse;
-                }
-            }
-        best[0] = bi;
-        best[1] = bj;
+    if (slice == 0 && c < ncand) {
+        double t = 0.0;
+#pragma unroll
+        for (int k = 0; k < 32; ++k)
+            t += s_part[k][ci];
+        mse[c] = n > 0 ? t / (double)n : 0.0;
+    }
+}
+
+// Algorithm 1: encodings in the outer loop, clipping candidates in the inner one, a candidate is
+// kept only when its error is strictly below the best so far, which starts at +infinity.  One warp:
+// lane l scans its contiguous stretch of that order, then the lanes are combined in lane order
+// with the same strict comparison, which gives what the sequential scan gives.
+__global__ void __launch_bounds__(32) search_select_kernel(const double* __restrict__ mse, int n_enc, int n_clip,
+                                                           int32_t* __restrict__ best)
+{
+    const int ncand = n_enc * n_clip, lane = threadIdx.x;
+    const int per = (ncand + 31) / 32;
+    double prev_mse = INFINITY;
+    int arg = -1;
+    for (int c = lane * per; c < min(ncand, (lane + 1) * per); ++c) {
+        const double curr_mse = mse[c];
+        if (prev_mse > curr_mse) {
+            arg = c;
+            prev_mse = curr_mse;
+        }
+    }
+    // lane 0 walks the 32 results in order
+    for (int l = 1; l < 32; ++l) {
+        const double other = __shfl_sync(0xffffffffu, prev_mse, l);
+        const int other_arg = __shfl_sync(0xffffffffu, arg, l);
+        if (lane == 0 && prev_mse > other) {
+            prev_mse = other;
+            arg = other_arg;
+        }
+    }
+    if (lane == 0) {
+        best[0] = arg < 0 ? -1 : arg / n_clip;
+        best[1] = arg < 0 ? -1 : arg % n_clip;
     }
 }
 
@@ -203,7 +222,8 @@ fpq_status launch_search(const float* x, int64_t n, const fpq_format* enc, int n
     search_mse_kernel<<<(unsigned)blocks, SEARCH_THREADS, smem, st>>>(a);
     if (cudaGetLastError() != cudaSuccess)
         return FPQ_ERR_CUDA;
-    search_finish_kernel<<<1, 1024, 0, st>>>((const double*)workspace, (int)blocks, n_enc, n_clip, n, mse, best);
+    search_reduce_kernel<<<(ncand + 31) / 32, 1024, 0, st>>>((const double*)workspace, (int)blocks, ncand, n, mse);
+    search_select_kernel<<<1, 32, 0, st>>>(mse, n_enc, n_clip, best);
     return cudaGetLastError() == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
 }
 
