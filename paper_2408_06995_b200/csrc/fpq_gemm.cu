@@ -249,12 +249,18 @@ __device__ __forceinline__ uint32_t cluster_rank()
     return r;
 }
 
-__device__ __forceinline__ float ld_peer_smem(uint32_t local_addr, uint32_t peer)
+// address of this CTA's shared-memory location `local_addr` in CTA `peer` of the cluster
+__device__ __forceinline__ uint32_t peer_smem_addr(uint32_t local_addr, uint32_t peer)
 {
     uint32_t remote;
-    float v;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(peer));
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return remote;
+}
+
+__device__ __forceinline__ float ld_cluster_smem(uint32_t cluster_addr)
+{
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
     return v;
 }
 
@@ -967,39 +973,55 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             float* yrow;
             int64_t nstride;
             row_target(mt, row, row_valid, yrow, nstride);
-            const uint32_t red = smem_base;
-            for (int c = (int)krank + ksplit * (e >> 7); c < BN; c += ksplit * (32 * NUM_EPI_WARPS / BM)) {
-                const int n = nt * BN + c;
-                if (n >= g.N)
+            // this CTA's staging area as seen in every CTA of the cluster
+            uint32_t peer[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                peer[k] = k < ksplit ? peer_smem_addr(smem_base, (uint32_t)k) : 0u;
+            // four columns per round: their 4 x ksplit loads are in flight together (one round is one
+            // trip through the cluster's shared-memory network)
+            const int cstep = ksplit * (32 * NUM_EPI_WARPS / BM);
+            for (int c = (int)krank + ksplit * (e >> 7); c < BN; c += 4 * cstep) {
+                if (nt * BN + c >= g.N)
                     break;
-                const uint32_t addr = red + (uint32_t)(c * BM + row) * 4u;
-                float v[8];
+                float v[4][8];
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    v[k] = k < ksplit ? ld_peer_smem(addr, (uint32_t)k) : 0.f;
-                float acc = v[0], acc2 = 0.f;              // sums over the first / second input tensor
-                if (!g.seg_chunk) {
+                for (int u = 0; u < 4; ++u) {
+                    const int cu = c + u * cstep;
+                    const uint32_t off = (uint32_t)(cu * BM + row) * 4u;
 #pragma unroll
-                    for (int k = 1; k < 8; ++k)
-                        if (k < ksplit)
-                            acc += v[k];
-                } else {
-                    // selects, not branches (v[k] is 0 beyond the cluster): branching per rank here
-                    // was measured to cost microseconds
-                    acc = 0.f;
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        acc += k < g.seg_ranks ? v[k] : 0.f;
-                        acc2 += k < g.seg_ranks ? 0.f : v[k];
-                    }
+                    for (int k = 0; k < 8; ++k)
+                        v[u][k] = (k < ksplit && cu < BN) ? ld_cluster_smem(peer[k] + off) : 0.f;
                 }
-                const float sv = g.stage_scales ? s_scale[n] : g.x_scale * __ldg(g.w_scale + n);
-                const float bv = g.stage_scales ? s_bias[n] : (g.bias ? __ldg(g.bias + n) : 0.f);
-                float out = fmaf(acc, sv, bv);
-                if (g.seg_chunk)
-                    out = fmaf(acc2, g.x_scale2 * __ldg(g.w_scale + n), out);
-                if (row_valid)
-                    yrow[(int64_t)n * nstride] = out;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int cu = c + u * cstep;
+                    const int n = nt * BN + cu;
+                    if (cu >= BN || n >= g.N)
+                        break;
+                    float acc = v[u][0], acc2 = 0.f;       // sums over the first / second input tensor
+                    if (!g.seg_chunk) {
+#pragma unroll
+                        for (int k = 1; k < 8; ++k)
+                            if (k < ksplit)
+                                acc += v[u][k];
+                    } else {
+                        // selects, not branches (v is 0 beyond the cluster)
+                        acc = 0.f;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            acc += k < g.seg_ranks ? v[u][k] : 0.f;
+                            acc2 += k < g.seg_ranks ? 0.f : v[u][k];
+                        }
+                    }
+                    const float sv = g.stage_scales ? s_scale[n] : g.x_scale * __ldg(g.w_scale + n);
+                    const float bv = g.stage_scales ? s_bias[n] : (g.bias ? __ldg(g.bias + n) : 0.f);
+                    float out = fmaf(acc, sv, bv);
+                    if (g.seg_chunk)
+                        out = fmaf(acc2, g.x_scale2 * __ldg(g.w_scale + n), out);
+                    if (row_valid)
+                        yrow[(int64_t)n * nstride] = out;
+                }
             }
         }
         // nobody leaves (and frees its shared memory) while a peer may still read it
