@@ -257,10 +257,13 @@ __device__ __forceinline__ uint32_t peer_smem_addr(uint32_t local_addr, uint32_t
     return remote;
 }
 
-__device__ __forceinline__ float ld_cluster_smem(uint32_t cluster_addr)
+__device__ __forceinline__ float4 ld_cluster_smem4(uint32_t cluster_addr)
 {
-    float v;
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(cluster_addr)
+                 : "memory");
     return v;
 }
 
@@ -967,60 +970,74 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             // rank order (the same order whatever the timing), then dequantize + bias as usual
             int mt, nt;
             decode_tile(t_lo, mt, nt);
+            // a thread owns four consecutive rows (one 16-byte load per peer and column) and every
+            // NUM_EPI_WARPS-th of this CTA's columns
             const int e = threadIdx.x - 64;
-            const int row = e & (BM - 1);
-            bool row_valid;
-            float* yrow;
-            int64_t nstride;
-            row_target(mt, row, row_valid, yrow, nstride);
+            const int rg = e & 31, cs = e >> 5;
+            bool row_valid[4];
+            float* yrow[4];
+            int64_t nstride = 1;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                row_target(mt, 4 * rg + q, row_valid[q], yrow[q], nstride);
             // this CTA's staging area as seen in every CTA of the cluster
             uint32_t peer[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k)
                 peer[k] = k < ksplit ? peer_smem_addr(smem_base, (uint32_t)k) : 0u;
-            // four columns per round: their 4 x ksplit loads are in flight together (one round is one
-            // trip through the cluster's shared-memory network)
-            const int cstep = ksplit * (32 * NUM_EPI_WARPS / BM);
-            for (int c = (int)krank + ksplit * (e >> 7); c < BN; c += 4 * cstep) {
+            // two columns per round: their 2 x ksplit loads are in flight together
+            const int cstep = ksplit * NUM_EPI_WARPS;
+            for (int c = (int)krank + ksplit * cs; c < BN; c += 2 * cstep) {
                 if (nt * BN + c >= g.N)
                     break;
-                float v[4][8];
+                float4 v[2][8];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < 2; ++u) {
                     const int cu = c + u * cstep;
-                    const uint32_t off = (uint32_t)(cu * BM + row) * 4u;
+                    const uint32_t off = (uint32_t)(cu * BM + 4 * rg) * 4u;
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        v[u][k] = (k < ksplit && cu < BN) ? ld_cluster_smem(peer[k] + off) : 0.f;
+                        v[u][k] = (k < ksplit && cu < BN) ? ld_cluster_smem4(peer[k] + off) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < 2; ++u) {
                     const int cu = c + u * cstep;
                     const int n = nt * BN + cu;
                     if (cu >= BN || n >= g.N)
                         break;
-                    float acc = v[u][0], acc2 = 0.f;       // sums over the first / second input tensor
+                    float4 acc = v[u][0], acc2 = make_float4(0.f, 0.f, 0.f, 0.f);   // first / second input tensor
                     if (!g.seg_chunk) {
 #pragma unroll
                         for (int k = 1; k < 8; ++k)
-                            if (k < ksplit)
-                                acc += v[u][k];
+                            if (k < ksplit) {
+                                acc.x += v[u][k].x; acc.y += v[u][k].y; acc.z += v[u][k].z; acc.w += v[u][k].w;
+                            }
                     } else {
                         // selects, not branches (v is 0 beyond the cluster)
-                        acc = 0.f;
+                        acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                         for (int k = 0; k < 8; ++k) {
-                            acc += k < g.seg_ranks ? v[u][k] : 0.f;
-                            acc2 += k < g.seg_ranks ? 0.f : v[u][k];
+                            const bool one = k < g.seg_ranks;
+                            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+                            const float4 a1 = one ? v[u][k] : z, a2 = one ? z : v[u][k];
+                            acc.x += a1.x; acc.y += a1.y; acc.z += a1.z; acc.w += a1.w;
+                            acc2.x += a2.x; acc2.y += a2.y; acc2.z += a2.z; acc2.w += a2.w;
                         }
                     }
                     const float sv = g.stage_scales ? s_scale[n] : g.x_scale * __ldg(g.w_scale + n);
                     const float bv = g.stage_scales ? s_bias[n] : (g.bias ? __ldg(g.bias + n) : 0.f);
-                    float out = fmaf(acc, sv, bv);
-                    if (g.seg_chunk)
-                        out = fmaf(acc2, g.x_scale2 * __ldg(g.w_scale + n), out);
-                    if (row_valid)
-                        yrow[(int64_t)n * nstride] = out;
+                    float out[4] = {fmaf(acc.x, sv, bv), fmaf(acc.y, sv, bv), fmaf(acc.z, sv, bv), fmaf(acc.w, sv, bv)};
+                    if (g.seg_chunk) {
+                        const float sv2 = g.x_scale2 * __ldg(g.w_scale + n);
+                        out[0] = fmaf(acc2.x, sv2, out[0]);
+                        out[1] = fmaf(acc2.y, sv2, out[1]);
+                        out[2] = fmaf(acc2.z, sv2, out[2]);
+                        out[3] = fmaf(acc2.w, sv2, out[3]);
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (row_valid[q])
+                            yrow[q][(int64_t)n * nstride] = out[q];
                 }
             }
         }
