@@ -1195,9 +1195,9 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
             g.ksplit = r1 + r2;
         }
     } else if (g.cchunks >= 2 && base_tiles * 2 <= di->sms &&
-               (MODE != MODE_ROWS || (g.m_tiles == 1 && g.cchunks >= 32))) {
+               (MODE != MODE_ROWS || (g.m_tiles == 1 && (g.cchunks >= 32 || (g.M <= 8 && g.cchunks >= 8))))) {
         // (row-major outputs leave the cluster's reduction column by column, which only pays for a single
-        // row tile with a very long reduction: measured on the SD-v1 linears)
+        // row tile with a very long reduction or a handful of rows: measured on the SD-v1 linears)
         int s_max = (int)(di->sms / base_tiles);
         if (s_max > 8) s_max = 8;
         if (s_max > g.cchunks) s_max = g.cchunks;
