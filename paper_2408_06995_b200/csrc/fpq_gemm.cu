@@ -18,7 +18,13 @@
 //         moved by whole 128-byte rows;
 //   TAPS  any stride: one 4-D box (channels, x, y, image) per block.
 // A ring stage carries the data of several blocks (one barrier handshake per stage);
-// weights whose whole reduction fits in shared memory stay resident across row tiles.
+// weights whose whole reduction fits in shared memory stay resident across row tiles, or a
+// row tile's activation panel stays resident across its column tiles.
+//
+// Layers with few tiles and a long reduction run as thread-block clusters: the CTAs of a
+// cluster reduce disjoint chunk ranges of one tile and add their partial sums through
+// distributed shared memory.  A layer whose input is two concatenated tensors with their own
+// scales keeps one accumulator per tensor (or gives each tensor its own CTAs of the cluster).
 #include <cuda.h>
 
 #include "fpq_common.cuh"
@@ -268,7 +274,7 @@ __device__ __forceinline__ float4 ld_cluster_smem4(uint32_t cluster_addr)
 }
 
 // FUSED = false: the activation operand is read as codes (TMA, written by a quantize kernel).
-// FUSED = true : 8 more warps read the FP32 activations and quantize them straight into the
+// FUSED = true : 16 more warps read the FP32 activations and quantize them straight into the
 //                activation ring, so the codes never exist in global memory.
 template <int BN, bool FUSED, int MODE>
 __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
@@ -922,7 +928,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             prefetch_tile(t);
         }
     } else if (FUSED) {
-        // ---------------- activation-quantize prologue: 8 warps fill the A ring ----------------
+        // ---------------- activation-quantize prologue: the transform warps fill the A ring ----------------
         const int tw = warp - (2 + NUM_EPI_WARPS);      // channel group tw % 8, row phase tw / 8
         const int tid = threadIdx.x - 32 * (2 + NUM_EPI_WARPS);
         const int chunks_per_stage = g.a_span / g.taps;
