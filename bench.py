@@ -38,7 +38,7 @@ NOMINAL_FP4_TFLOPS = 9000.0
 # launch with flushed caches and stops counting when the kernel ends, so output that is still in L2
 # at that point (all of it, for these sizes) is missing from the write side.
 TRAFFIC = {
-    "fpq_gemm_kernel (contraction + epilogue)": 9712128 + 4096,
+    "fpq_gemm_kernel (contraction + epilogue)": 9712896 + 6912,
     "quantize_nchw_to_nhwc_e4m3_kernel (activation quantize)": 33567232 + 0,
 }
 
@@ -562,6 +562,10 @@ def run_suite(args):
         raise SystemExit("unknown suite")
     rows = []
     tot = {"auto": 0.0, "fused": 0.0, "two_kernels": 0.0, "best": 0.0, "flops": 0.0, "bytes": 0.0, "bound": 0.0}
+    if args.only:
+        layers = [L for L in layers if args.only in L.name]
+        if not layers:
+            raise SystemExit(f"no layer of suite {args.suite} has {args.only!r} in its name")
     for L in layers:
         lay = LayerOnGpu(L, fpq, torch, dev, l2_bytes=(128 << 20) if args.suite != "sd" else (48 << 20))
         n = max(4, min(40, 3 * lay.nsets))
@@ -718,6 +722,7 @@ def main():
     ap.add_argument("--skip-w4", action="store_true", help="leave out the W4A8 side measurement")
     ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd", "sd_trace", "search", "sd_split"],
                     help="print a per-shape table of a whole workload instead of the headline line")
+    ap.add_argument("--only", default=None, help="with --suite ldm|transformer|sd: only the layers whose name contains this")
     args = ap.parse_args()
     if args.suite == "sd_trace":
         run_trace(args)
