@@ -186,6 +186,24 @@ def test_config4_full_size_sampled():
         _check_sampled(L, 1 << 12, 10 + j)
 
 
+def _sd_shapes():
+    out = []
+    for item in I.distinct_shapes(I.sd_v1_unet_layers()):
+        out.append(item[0] if isinstance(item, tuple) else item)
+    return out
+
+
+@pytest.mark.parametrize("j", range(58))
+def test_config5_every_sd_unet_shape_sampled(j):
+    # all distinct conv / linear shapes of one SD-v1-style U-Net step (W4A8 with rounding decisions),
+    # at the sizes and in the launch configuration the bench times; the oracle checks a sample
+    shapes = _sd_shapes()
+    assert len(shapes) == 58
+    L = shapes[j]
+    I.draw(L, 5, 10 * j, "normal", 0.02, True)
+    _check_sampled(L, 600, 100 + j)
+
+
 # ---- the two-kernel route (activation codes in a workspace, then the contraction) ---------------
 
 def _staged(L, ws, xs):
