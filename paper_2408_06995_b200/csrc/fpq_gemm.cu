@@ -46,7 +46,9 @@ __host__ __device__ constexpr int num_threads(bool fused)
 }
 constexpr int SMEM_BUDGET = 227 * 1024;   // the most dynamic shared memory a CTA can have on sm_100
 
-enum { MODE_ROWS = 0, MODE_FLAT = 1, MODE_TAPS = 2 };
+// MODE_FLAT2 is FLAT with two row tiles per unit; it has its own instantiation because the kernels are
+// sensitive to code size (the extra path cost the plain FLAT kernel 7 us when it was a run-time branch)
+enum { MODE_ROWS = 0, MODE_FLAT = 1, MODE_TAPS = 2, MODE_FLAT2 = 3 };
 
 // Division of a 31-bit unsigned number by a constant known on the host:
 // n / d = (umulhi(n, mul) + n) >> shift.
@@ -103,6 +105,8 @@ struct GemmArgs {
     int seg_chunk, seg_ranks;
     float x_scale2;
     int seg_acc;               // two tensors without a cluster: each has its own accumulator, the epilogue joins them
+    int pair;                  // a tile unit is two consecutive row tiles (256 rows) that share every weight stage;
+                               // m_tiles then counts pairs
     uint32_t a_chunk_tx, b_block_tx;   // bytes one load reports to its barrier
     const float* w_scale;
     float x_scale;
@@ -313,6 +317,10 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     // Split reduction (few tiles, long reduction): a cluster of ksplit CTAs owns one tile, CTA k of the
     // cluster reduces the chunks [c_lo, c_hi) into its own accumulator; the partial sums meet in shared
     // memory after the role loops below.
+    // two row tiles per unit: only the plain form of the stride-1 convolution uses it
+    constexpr bool pair = MODE == MODE_FLAT2;
+    constexpr bool FLATM = MODE == MODE_FLAT || MODE == MODE_FLAT2;
+    const int tile_rows = pair ? 2 * BM : BM;
     const int ksplit = g.ksplit;
     const uint32_t krank = ksplit > 1 ? cluster_rank() : 0u;
     int c_lo = 0, c_hi = g.cchunks;
@@ -353,7 +361,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             tma_prefetch_desc(&tmY);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32((const void*)tmem_slot), g.seg_acc ? 4 * BN : 2 * BN);
+        tmem_alloc(smem_u32((const void*)tmem_slot), (g.seg_acc || pair) ? 4 * BN : 2 * BN);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -377,7 +385,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             yrow = g.y + m * g.N;
         } else {
             int ox, oy, b;
-            if (MODE == MODE_FLAT) {
+            if (FLATM) {
                 const uint32_t q = (uint32_t)mt * BM + row;
                 b = (int)fdiv(q, g.div_HpWp);
                 const uint32_t rem = q - (uint32_t)b * g.HpWp;
@@ -468,7 +476,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                             for (int l = 0; l < nloads; ++l, dst += g.a_chunk_bytes)
                                 for (int bx = 0; bx < g.a_boxes; ++bx)
                                     tma_load_4d(dst + bx * g.a_box_rows * 128, &tmA, a_full + 8 * sa, (cc + l) * BK,
-                                                mt * BM + bx * g.a_box_rows, 0, 0);
+                                                mt * tile_rows + bx * g.a_box_rows, 0, 0);
                         }
                         ++na;
                         if (++sa == (uint32_t)g.a_stages) { sa = 0; pa ^= 1; }
@@ -546,7 +554,45 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                 // chunks from seg_from on (the second input tensor) add up in the accumulator 2 * BN columns further
                 const int seg_from = (!FUSED && g.seg_acc) ? g.seg_chunk : 0x7fffffff;
 
-                if (MODE == MODE_FLAT && g.taps == 9 && g.S == 3) {
+                if (pair) {
+                    // 3 x 3 taps over a 256-row chunk, weights streamed one tap per stage: every
+                    // weight block feeds the MMAs of both row tiles (accumulators d0, d1), which halves
+                    // the weight bytes that have to reach shared memory per MMA
+                    const uint32_t Wp8 = (uint32_t)g.Wp * 8u;
+                    const uint32_t d0 = tmem_base + buf * 2 * BN, d1 = d0 + BN;
+                    for (int cc = c_lo; cc < c_hi && !dead; ++cc) {
+                        if (!mbar_wait(a_full + 8 * sa, pa)) { dead = true; break; }
+                        tc_fence_after();
+                        const uint32_t ac = smem_desc_lo(a_ring + sa * g.a_stage_bytes);
+                        uint32_t bst = 0;
+#pragma unroll
+                        for (int tap = 0; tap < 9; ++tap) {
+                            if (!mbar_wait(b_full + 8 * sb, pb)) { dead = true; break; }
+                            tc_fence_after();
+                            bst = smem_desc_lo(b_ring + sb * g.b_stage_bytes);
+                            const uint32_t al = ac + (tap / 3) * Wp8 + (tap % 3) * 8u;
+                            const uint32_t al1 = al + BM * 8u;           // 128 rows of 128 bytes further down
+                            const uint32_t bl = bst;
+                            if (tap == 0 && cc == c_lo) {
+                                mma_f8f6f4<false>(d0, al, bl, HI, g.idesc);
+                                mma_f8f6f4<false>(d1, al1, bl, HI, g.idesc);
+                            } else {
+                                mma_f8f6f4<true>(d0, al, bl, HI, g.idesc);
+                                mma_f8f6f4<true>(d1, al1, bl, HI, g.idesc);
+                            }
+                            mma_f8f6f4<true>(d0, al + 2, bl + 2, HI, g.idesc);
+                            mma_f8f6f4<true>(d1, al1 + 2, bl + 2, HI, g.idesc);
+                            mma_f8f6f4<true>(d0, al + 4, bl + 4, HI, g.idesc);
+                            mma_f8f6f4<true>(d1, al1 + 4, bl + 4, HI, g.idesc);
+                            mma_f8f6f4<true>(d0, al + 6, bl + 6, HI, g.idesc);
+                            mma_f8f6f4<true>(d1, al1 + 6, bl + 6, HI, g.idesc);
+                            mma_commit(b_empty + 8 * sb);
+                            if (++sb == (uint32_t)g.b_stages) { sb = 0; pb ^= 1; }
+                        }
+                        mma_commit(a_empty + 8 * sa);
+                        if (++sa == (uint32_t)g.a_stages) { sa = 0; pa ^= 1; }
+                    }
+                } else if (FLATM && g.taps == 9 && g.S == 3) {
                     const uint32_t Wp8 = (uint32_t)g.Wp * 8u;
                     const int chunks_per_stage = g.a_span / 9;
                     for (int cc = c_lo; cc < c_hi && !dead;) {
@@ -632,7 +678,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                     uint32_t a_chunk_lo = 0;               // FLAT/ROWS: current chunk in its stage
                     uint32_t row_off8 = 0;                 // FLAT: (r * Wp + s) * 8 of the current tap
                     const uint32_t row_wrap8 = (uint32_t)(g.Wp - g.S) * 8u;
-                    const bool flat = MODE == MODE_FLAT, taps_mode = MODE == MODE_TAPS;
+                    const bool flat = FLATM, taps_mode = MODE == MODE_TAPS;
                     int tap = 0, sx = 0, ja = 0, jb = 0;
                     int ccg = c_lo;                        // chunk of the current block
                     for (int j = 0; j < nblk; ++j) {
@@ -725,7 +771,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             bool row_valid;
             float* yrow;
             int64_t nstride;
-            row_target(mt, row, row_valid, yrow, nstride);
+            row_target(pair ? 2 * mt : mt, row, row_valid, yrow, nstride);
 
             if (!mbar_wait(acc_full + 8 * buf, aph)) { dead = true; }
             tc_fence_after();
@@ -750,115 +796,121 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                     }
                 }
             } else if (!dead && ncol0 < g.N) {
-                const uint32_t t_addr = tmem_base + buf * BN + half * HALF + ((uint32_t)(quarter * 32) << 16);
+                // (two accumulators when the unit is a pair of row tiles)
+                for (int h = 0; h < (pair ? 2 : 1); ++h) {
+                    if (h)
+                        row_target(2 * mt + 1, row, row_valid, yrow, nstride);
+                    const uint32_t t_addr = tmem_base + (pair ? buf * 2 + h : buf) * BN + half * HALF +
+                                            ((uint32_t)(quarter * 32) << 16);
 #pragma unroll
-                for (int c0 = 0; c0 < CHUNKS; c0 += G) {
-                    if (ncol0 + c0 * 32 >= g.N)
-                        break;
-                    uint32_t r[G][32];
-#pragma unroll
-                    for (int c = 0; c < G; ++c)
-                        tmem_ld32(t_addr + (c0 + c) * 32, r[c]);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int cl = 0; cl < G; ++cl) {
-                        const int nb = ncol0 + (c0 + cl) * 32;
-                        if (nb >= g.N)
+                    for (int c0 = 0; c0 < CHUNKS; c0 += G) {
+                        if (ncol0 + c0 * 32 >= g.N)
                             break;
-                        const bool full = nb + 32 <= g.N;
-                        // dequantize + bias in place
-                        if (g.stage_scales) {
-                            const float4* s4 = reinterpret_cast<const float4*>(s_scale + nb);
-                            const float4* b4 = reinterpret_cast<const float4*>(s_bias + nb);
+                        uint32_t r[G][32];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const float4 sv = s4[j], bv = b4[j];
-                                r[cl][4 * j + 0] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 0]), sv.x, bv.x));
-                                r[cl][4 * j + 1] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 1]), sv.y, bv.y));
-                                r[cl][4 * j + 2] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 2]), sv.z, bv.z));
-                                r[cl][4 * j + 3] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 3]), sv.w, bv.w));
-                            }
-                        } else if (full && g.vec_scale) {
-                            const float4* s4 = reinterpret_cast<const float4*>(g.w_scale + nb);
-                            const float4* b4 = reinterpret_cast<const float4*>(g.bias + nb);
+                        for (int c = 0; c < G; ++c)
+                            tmem_ld32(t_addr + (c0 + c) * 32, r[c]);
+                        tmem_ld_wait();
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const float4 sv = __ldg(s4 + j);
-                                const float4 bv = g.bias ? __ldg(b4 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-                                r[cl][4 * j + 0] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 0]), g.x_scale * sv.x, bv.x));
-                                r[cl][4 * j + 1] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 1]), g.x_scale * sv.y, bv.y));
-                                r[cl][4 * j + 2] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 2]), g.x_scale * sv.z, bv.z));
-                                r[cl][4 * j + 3] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 3]), g.x_scale * sv.w, bv.w));
-                            }
-                        } else {
+                        for (int cl = 0; cl < G; ++cl) {
+                            const int nb = ncol0 + (c0 + cl) * 32;
+                            if (nb >= g.N)
+                                break;
+                            const bool full = nb + 32 <= g.N;
+                            // dequantize + bias in place
+                            if (g.stage_scales) {
+                                const float4* s4 = reinterpret_cast<const float4*>(s_scale + nb);
+                                const float4* b4 = reinterpret_cast<const float4*>(s_bias + nb);
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const bool in = nb + j < g.N;
-                                const float sv = in ? __ldg(g.w_scale + nb + j) : 0.f;
-                                const float bv = (in && g.bias) ? __ldg(g.bias + nb + j) : 0.f;
-                                r[cl][j] = __float_as_uint(fmaf(__uint_as_float(r[cl][j]), g.x_scale * sv, bv));
-                            }
-                        }
-                        if (!FUSED && g.seg_acc) {
-                            // the second input tensor's sums, with its own scale
-                            uint32_t r2[32];
-                            tmem_ld32(t_addr + 2 * BN + (c0 + cl) * 32, r2);
-                            tmem_ld_wait();
+                                for (int j = 0; j < 8; ++j) {
+                                    const float4 sv = s4[j], bv = b4[j];
+                                    r[cl][4 * j + 0] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 0]), sv.x, bv.x));
+                                    r[cl][4 * j + 1] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 1]), sv.y, bv.y));
+                                    r[cl][4 * j + 2] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 2]), sv.z, bv.z));
+                                    r[cl][4 * j + 3] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 3]), sv.w, bv.w));
+                                }
+                            } else if (full && g.vec_scale) {
+                                const float4* s4 = reinterpret_cast<const float4*>(g.w_scale + nb);
+                                const float4* b4 = reinterpret_cast<const float4*>(g.bias + nb);
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const float sv = nb + j < g.N ? g.x_scale2 * __ldg(g.w_scale + nb + j) : 0.f;
-                                r[cl][j] = __float_as_uint(fmaf(__uint_as_float(r2[j]), sv, __uint_as_float(r[cl][j])));
-                            }
-                        }
-                        if (g.y_tma) {
-                            // the buffer is free once the store before the previous one has read it
-                            uint8_t* stage = stage0 + (nstore & 1u) * 4096;
-                            ++nstore;
-                            if (lane == 0)
-                                asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                            __syncwarp();
-#pragma unroll
-                            for (int j = 0; j < 8; ++j)
-                                *reinterpret_cast<uint4*>(stage + lane * 128 + ((j ^ (lane & 7)) << 4)) =
-                                    make_uint4(r[cl][4 * j], r[cl][4 * j + 1], r[cl][4 * j + 2], r[cl][4 * j + 3]);
-                            fence_proxy_async();
-                            __syncwarp();
-                            if (lane == 0) {
-                                asm volatile(
-                                    "cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                                    ::"l"(&tmY), "r"(smem_u32(stage)), "r"(nb), "r"(mt * BM + quarter * 32)
-                                    : "memory");
-                                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                            }
-                        } else if (row_valid) {
-                            if (MODE == MODE_ROWS) {
-                                if (full && g.N % 4 == 0) {
-                                    uint4* dst = reinterpret_cast<uint4*>(yrow + nb);
-#pragma unroll
-                                    for (int j = 0; j < 8; ++j)
-                                        dst[j] = make_uint4(r[cl][4 * j], r[cl][4 * j + 1], r[cl][4 * j + 2], r[cl][4 * j + 3]);
-                                } else {
-#pragma unroll
-                                    for (int j = 0; j < 32; ++j)
-                                        if (nb + j < g.N)
-                                            yrow[nb + j] = __uint_as_float(r[cl][j]);
+                                for (int j = 0; j < 8; ++j) {
+                                    const float4 sv = __ldg(s4 + j);
+                                    const float4 bv = g.bias ? __ldg(b4 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                    r[cl][4 * j + 0] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 0]), g.x_scale * sv.x, bv.x));
+                                    r[cl][4 * j + 1] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 1]), g.x_scale * sv.y, bv.y));
+                                    r[cl][4 * j + 2] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 2]), g.x_scale * sv.z, bv.z));
+                                    r[cl][4 * j + 3] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 3]), g.x_scale * sv.w, bv.w));
                                 }
                             } else {
-                                float* dst = yrow + (int64_t)nb * nstride;
-                                if (full) {
 #pragma unroll
-                                    for (int j = 0; j < 32; j += 4) {
-                                        dst[0] = __uint_as_float(r[cl][j]);
-                                        dst[nstride] = __uint_as_float(r[cl][j + 1]);
-                                        dst[2 * nstride] = __uint_as_float(r[cl][j + 2]);
-                                        dst[3 * nstride] = __uint_as_float(r[cl][j + 3]);
-                                        dst += 4 * nstride;
+                                for (int j = 0; j < 32; ++j) {
+                                    const bool in = nb + j < g.N;
+                                    const float sv = in ? __ldg(g.w_scale + nb + j) : 0.f;
+                                    const float bv = (in && g.bias) ? __ldg(g.bias + nb + j) : 0.f;
+                                    r[cl][j] = __float_as_uint(fmaf(__uint_as_float(r[cl][j]), g.x_scale * sv, bv));
+                                }
+                            }
+                            if (!FUSED && g.seg_acc) {
+                                // the second input tensor's sums, with its own scale
+                                uint32_t r2[32];
+                                tmem_ld32(t_addr + 2 * BN + (c0 + cl) * 32, r2);
+                                tmem_ld_wait();
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) {
+                                    const float sv = nb + j < g.N ? g.x_scale2 * __ldg(g.w_scale + nb + j) : 0.f;
+                                    r[cl][j] = __float_as_uint(fmaf(__uint_as_float(r2[j]), sv, __uint_as_float(r[cl][j])));
+                                }
+                            }
+                            if (g.y_tma) {
+                                // the buffer is free once the store before the previous one has read it
+                                uint8_t* stage = stage0 + (nstore & 1u) * 4096;
+                                ++nstore;
+                                if (lane == 0)
+                                    asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                                __syncwarp();
+#pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    *reinterpret_cast<uint4*>(stage + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                                        make_uint4(r[cl][4 * j], r[cl][4 * j + 1], r[cl][4 * j + 2], r[cl][4 * j + 3]);
+                                fence_proxy_async();
+                                __syncwarp();
+                                if (lane == 0) {
+                                    asm volatile(
+                                        "cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                        ::"l"(&tmY), "r"(smem_u32(stage)), "r"(nb), "r"(mt * BM + quarter * 32)
+                                        : "memory");
+                                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                                }
+                            } else if (row_valid) {
+                                if (MODE == MODE_ROWS) {
+                                    if (full && g.N % 4 == 0) {
+                                        uint4* dst = reinterpret_cast<uint4*>(yrow + nb);
+#pragma unroll
+                                        for (int j = 0; j < 8; ++j)
+                                            dst[j] = make_uint4(r[cl][4 * j], r[cl][4 * j + 1], r[cl][4 * j + 2], r[cl][4 * j + 3]);
+                                    } else {
+#pragma unroll
+                                        for (int j = 0; j < 32; ++j)
+                                            if (nb + j < g.N)
+                                                yrow[nb + j] = __uint_as_float(r[cl][j]);
                                     }
                                 } else {
+                                    float* dst = yrow + (int64_t)nb * nstride;
+                                    if (full) {
 #pragma unroll
-                                    for (int j = 0; j < 32; ++j)
-                                        if (nb + j < g.N)
-                                            dst[(int64_t)j * nstride] = __uint_as_float(r[cl][j]);
+                                        for (int j = 0; j < 32; j += 4) {
+                                            dst[0] = __uint_as_float(r[cl][j]);
+                                            dst[nstride] = __uint_as_float(r[cl][j + 1]);
+                                            dst[2 * nstride] = __uint_as_float(r[cl][j + 2]);
+                                            dst[3 * nstride] = __uint_as_float(r[cl][j + 3]);
+                                            dst += 4 * nstride;
+                                        }
+                                    } else {
+#pragma unroll
+                                        for (int j = 0; j < 32; ++j)
+                                            if (nb + j < g.N)
+                                                dst[(int64_t)j * nstride] = __uint_as_float(r[cl][j]);
+                                    }
                                 }
                             }
                         }
@@ -1055,7 +1107,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, g.seg_acc ? 4 * BN : 2 * BN);
+        tmem_dealloc(tmem_base, (g.seg_acc || pair) ? 4 * BN : 2 * BN);
     }
 }
 
@@ -1087,8 +1139,8 @@ static int pow2_at_least(int v)
 
 struct DeviceInfo {
     int sms;
-    bool smem_set[12];
-    int max_clusters[2][3][9];     // [BN == 128][mode][cluster size]: clusters resident at once, 0 = not asked yet, -1 = none
+    bool smem_set[16];
+    int max_clusters[2][4][9];     // [BN == 128][mode][cluster size]: clusters resident at once, 0 = not asked yet, -1 = none
 };
 
 static DeviceInfo* device_info()
@@ -1172,7 +1224,9 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
     // then the smallest one with the same longest chunk range.
     g.ksplit = 1;
     const int64_t base_tiles = (int64_t)g.m_tiles * g.n_tiles;
-    if (g.seg_chunk) {
+    if (g.pair) {
+        // paired row tiles: plain streaming of both operands, no cluster
+    } else if (g.seg_chunk) {
         // two input tensors: with few tiles a cluster per tile, at least one CTA per tensor and as
         // many CTAs as keep every tile resident at once; with many tiles no cluster
         if (MODE == MODE_ROWS || FUSED || g.seg_chunk >= g.cchunks)
@@ -1220,7 +1274,7 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
     // several column tiles per row tile: try to keep the row tile's whole activation panel in the
     // ring (read / quantized once) and stream the weights
     bool done = false;
-    if (g.ksplit == 1 && g.n_tiles > 1 && g.mode != MODE_TAPS) {
+    if (g.ksplit == 1 && !g.pair && g.n_tiles > 1 && g.mode != MODE_TAPS) {
         const bool conv9 = g.mode == MODE_FLAT && g.taps == 9 && g.S == 3;
         if (conv9 || g.taps == 1) {
             const int cps = conv9 ? 1 : (g.cchunks >= 3 ? 3 : g.cchunks);      // chunks per A stage
@@ -1245,7 +1299,7 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
     }
     if (done) {
         // configured above
-    } else if (g.ksplit == 1 && b_all + 2 * g.a_chunk_bytes <= budget) {
+    } else if (g.ksplit == 1 && !g.pair && b_all + 2 * g.a_chunk_bytes <= budget) {
         g.b_resident = 1;
         g.b_span = g.nblk;
         g.b_stages = 1;
@@ -1266,7 +1320,7 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
         g.m_fastest = 0;
         int chunks;
         if (g.mode == MODE_FLAT && g.taps > 1) {
-            g.b_span = (g.taps == 9 && g.S == 3) ? 3 : 1;
+            g.b_span = (g.taps == 9 && g.S == 3 && !g.pair) ? 3 : 1;
             g.a_span = g.taps;                                // one chunk per stage serves all taps
             chunks = 1;
             g.a_stages = 2;
@@ -1333,6 +1387,11 @@ static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB,
     // thread is sensitive to instruction fetch
     if (g.mode == MODE_ROWS)
         return launch_mode<BN, FUSED, MODE_ROWS>(tmA, tmB, tmY, g, st);
+    if (g.mode == MODE_FLAT && g.pair) {
+        if (FUSED)
+            return FPQ_ERR_UNSUPPORTED;
+        return launch_mode<BN, false, MODE_FLAT2>(tmA, tmB, tmY, g, st);
+    }
     if (g.mode == MODE_FLAT)
         return launch_mode<BN, FUSED, MODE_FLAT>(tmA, tmB, tmY, g, st);
     if (FUSED)
@@ -1401,8 +1460,26 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
             g.Wp = Wp;
             g.HpWp = Hp * Wp;
             mtiles = flat_tiles;
-            g.a_boxes = halo_rows > 256 ? 2 : 1;
-            g.a_box_rows = (int)round_up((halo_rows + g.a_boxes - 1) / g.a_boxes, 8);
+            int rows = halo_rows;
+            // Streamed 3 x 3 weights fill shared memory at about half the rate the MMAs of one row tile
+            // consume them (measured: ~32 bytes per clock and SM arrive, 64 + 11 are needed).  Two row
+            // tiles per unit share every weight block; taken when that beats the loss of parallelism.
+            // (measured time per unit in MMA-bound tile times: 2.04 alone, 2 x 1.62 as a pair)
+            DeviceInfo* di = device_info();
+            const int64_t b_all = (int64_t)g.nblk * BN * BK;
+            if (di && p.R == 3 && p.S == 3 && p.x == nullptr && p.c_seg == 0 && b_all > 160 * 1024 &&
+                halo_rows + BM <= 2 * 256 - 16) {
+                const int64_t alone = flat_tiles * g.n_tiles, pairs = (flat_tiles + 1) / 2 * g.n_tiles;
+                const double t_alone = (double)((alone + di->sms - 1) / di->sms) * 2.04;
+                const double t_pair = (double)((pairs + di->sms - 1) / di->sms) * 2.0 * 1.62;
+                if (alone * 2 > di->sms && t_pair < t_alone) {
+                    g.pair = 1;
+                    mtiles = (flat_tiles + 1) / 2;
+                    rows = halo_rows + BM;
+                }
+            }
+            g.a_boxes = rows > 256 ? 2 : 1;
+            g.a_box_rows = (int)round_up((rows + g.a_boxes - 1) / g.a_boxes, 8);
             dimsA[0] = (cuuint64_t)p.Ca; dimsA[1] = (cuuint64_t)framed; dimsA[2] = 1; dimsA[3] = 1;
             stridesA[0] = (cuuint64_t)p.Ca; stridesA[1] = stridesA[2] = (cuuint64_t)p.Ca * framed;
             boxA[0] = BK; boxA[1] = (cuuint32_t)g.a_box_rows; boxA[2] = 1; boxA[3] = 1;
