@@ -125,6 +125,14 @@ def test_conv_split_reduction_shapes(wfmt, B, C, H, W, Co, R, pad, stride):
     _check_full(L)
 
 
+def test_conv_paired_row_tiles_every_element():
+    # more 3x3 tiles than SMs with streamed weights: the kernel walks pairs of row tiles that share
+    # each weight stage (154 tiles, the last pair is half empty)
+    L = I.conv_layer("t", 17, 256, 32, 32, 128, 3, wfmt="e2m1", rounding=True)
+    I.draw(L, 14, 0, "silu", 0.03, True)
+    _check_full(L)
+
+
 def test_conv_1x1_matches_linear_on_the_gpu():
     L = I.conv_layer("c", 2, 96, 8, 8, 80, 1, wfmt="e4m3")
     I.draw(L, 10, 0, "normal", 0.02, True)
