@@ -1472,7 +1472,11 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
                 const int64_t alone = flat_tiles * g.n_tiles, pairs = (flat_tiles + 1) / 2 * g.n_tiles;
                 const double t_alone = (double)((alone + di->sms - 1) / di->sms) * 2.04;
                 const double t_pair = (double)((pairs + di->sms - 1) / di->sms) * 2.0 * 1.62;
-                if (alone * 2 > di->sms && t_pair < t_alone) {
+                // (a row tile's whole activation panel resident across its column tiles measured a
+                // little faster than pairing where it fits)
+                const int64_t panel = (int64_t)g.cchunks * round_up(halo_rows, 8) * 128;
+                const bool panel_fits = g.n_tiles > 1 && g.cchunks <= 8 && panel + 6 * BN * BK <= SMEM_BUDGET - 12 * 1024;
+                if (alone * 2 > di->sms && t_pair < t_alone && !panel_fits) {
                     g.pair = 1;
                     mtiles = (flat_tiles + 1) / 2;
                     rows = halo_rows + BM;
