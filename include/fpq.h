@@ -14,6 +14,10 @@
  *     (fpq_read_status).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *     stream).  Calls only enqueue work; they do not synchronise unless stated.
+ *   - Calls may come from several host threads (each with its own stream and
+ *     buffers); the library takes turns inside where it keeps per-device tables.
+ *     fpq_set_path_policy and fpq_linear_static are the exceptions stated at their
+ *     declarations.
  *   - Errors are return codes (negative).  Whatever the host can check (null or
  *     misaligned pointers, impossible formats, shapes, workspace size) is
  *     rejected before anything is launched.

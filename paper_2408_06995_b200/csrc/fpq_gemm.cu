@@ -27,6 +27,8 @@
 // scales keeps one accumulator per tensor (or gives each tensor its own CTAs of the cluster).
 #include <cuda.h>
 
+#include <mutex>
+
 #include "fpq_common.cuh"
 #include "fpq_kernels.h"
 
@@ -1401,6 +1403,10 @@ static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB,
 
 fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
 {
+    // the per-device tables behind the plan (SM count, kernel attributes, cluster occupancy) are filled
+    // on first use: host threads take turns here
+    static std::mutex plan_mutex;
+    std::lock_guard<std::mutex> lock(plan_mutex);
     EncodeTiledFn enc = encode_fn();
     if (!enc)
         return FPQ_ERR_CUDA;

@@ -6,6 +6,8 @@
 // quantized and compared a few hundred times.  A thread keeps 16 elements in registers
 // and walks the candidate list; per candidate and element the quantize-dequantize-error
 // chain is nine instructions (see search_mse_kernel).
+#include <mutex>
+
 #include "fpq_common.cuh"
 #include "fpq_kernels.h"
 
@@ -208,6 +210,8 @@ fpq_status launch_search(const float* x, int64_t n, const fpq_format* enc, int n
     if (blocks < 1)
         blocks = 1;
     const size_t smem = (size_t)(SEARCH_THREADS / 32) * ncand * sizeof(double) + (size_t)ncand * 2 * sizeof(float);
+    static std::mutex attr_mutex;
+    std::lock_guard<std::mutex> lock(attr_mutex);
     static bool smem_set[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
