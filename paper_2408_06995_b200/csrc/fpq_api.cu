@@ -300,6 +300,14 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
     if (!aligned(x, 16) || !aligned(y, 16) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
         (bias && !aligned(bias, 4)))
         return FPQ_ERR_ALIGN;
+    // a handful of rows (time-embedding projections): one pass over the weights on the CUDA cores,
+    // whatever the route policy says; the workspace is not touched
+    if (small_m_linear_applies(M, K) && N <= 0x7fffffff) {
+        if (!status_word())
+            return FPQ_ERR_CUDA;
+        return launch_small_m_linear(x, (int)M, (int)K, w_prepared, is_e2m1(fw) ? 1 : 0, (int)N, w_scale, x_scale, bias, y,
+                                     (cudaStream_t)stream);
+    }
     // one kernel: the activations are quantized inside the contraction's operand staging
     // (AUTO takes the two-kernel route: measured faster on B200 so far)
     if (g_path_policy == FPQ_PATH_FUSED) {

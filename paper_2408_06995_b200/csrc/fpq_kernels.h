@@ -48,6 +48,11 @@ struct GemmProblem {
 // Returns FPQ_OK or an error; enqueues one kernel.
 fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st);
 
+// Linear layer with at most 8 rows on the CUDA cores (one pass over the weights).
+bool small_m_linear_applies(int64_t M, int64_t K);
+fpq_status launch_small_m_linear(const float* x, int M, int K, const void* w_prepared, int w4, int N, const float* w_scale,
+                                 float x_scale, const float* bias, float* y, cudaStream_t st);
+
 // Encoding / bias search: limits, scratch size, and the launch (three kernels).
 int search_max_enc();
 int search_max_clip();

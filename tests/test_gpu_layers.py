@@ -54,6 +54,16 @@ def test_linear_ragged_shapes(wfmt, M, K, N):
     _check_full(L, use_bias=False)
 
 
+# at most 8 rows: one pass over the weights on the CUDA cores instead of the tensor-core kernel
+@pytest.mark.parametrize("wfmt", ["e4m3", "e2m1"])
+@pytest.mark.parametrize("M,K,N", [(1, 128, 8), (2, 320, 1280), (3, 1000, 77), (8, 1280, 320), (8, 3072, 40), (5, 130, 1),
+                                   (8, 3200, 16), (4, 5120, 130)])   # K = 130 is not a multiple of 4: tensor-core path
+def test_linear_few_rows(wfmt, M, K, N):
+    L = I.linear_layer("t", M, K, N, wfmt, rounding=(wfmt == "e2m1"))
+    I.draw(L, 15, M + K + N, "normal", 0.02, True, 0.01, (0.01, 20.0))
+    _check_full(L)
+
+
 @pytest.mark.parametrize("wfmt", ["e4m3", "e2m1"])
 def test_linear_small_integers_are_exact(wfmt):
     rng = np.random.default_rng(3)
