@@ -132,7 +132,9 @@ fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_la
  * x FP32 [M][K] row-major, y FP32 [M][N] row-major, both 16-byte aligned; bias
  * [N] or NULL.  The activations are quantized with (fx, x_scale) exactly as
  * fpq_quantize_act does; products are exact and accumulated in FP32 on the
- * tensor cores.  Supported operand pairs: fx = E4M3 bias 7 FPQ_SAT_NATIVE with
+ * tensor cores (layers of at most 8 rows with K a multiple of 4 run on the CUDA
+ * cores instead: the same exact products, another order of the FP32 additions;
+ * the workspace is then left untouched).  Supported operand pairs: fx = E4M3 bias 7 FPQ_SAT_NATIVE with
  * fw = the same, or fw = E2M1 bias 1.  Anything else: FPQ_ERR_UNSUPPORTED.
  * workspace: fpq_linear_workspace_size bytes, 128-byte aligned; contents are
  * scratch.
