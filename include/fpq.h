@@ -188,7 +188,14 @@ fpq_status fpq_conv2d_contract(const void* workspace, size_t ws_bytes, const voi
  * Host-buffer forms of the two layers: x_host / y_host are host pointers
  * (pinned memory for asynchronous copies), x_dev / y_dev are device staging
  * buffers of the same sizes owned by the caller.  The call copies x in, runs the
- * layer, copies y out and waits for the stream.
+ * layer, copies y out and returns when y_host is complete.  Large batches are
+ * pipelined in up to 8 slices (rows / images) so that the copy-in of one slice,
+ * the layer on the previous one and the copy-out of the one before overlap; the
+ * result is the same bit for bit.  For this the library keeps two streams and a
+ * few events per device, created at the first host-form call (the one exception
+ * to "allocates nothing"); host-form calls on one device must not run concurrently.
+ * A linear layer is sliced only if K and N are multiples of 4 (slices of x and y
+ * must keep fpq_linear's 16-byte alignment).
  */
 fpq_status fpq_linear_host(const float* x_host, float* x_dev, const void* w_prepared,
                            const float* w_scale, float x_scale, fpq_format fx, fpq_format fw,

@@ -2,6 +2,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "fpq_common.cuh"
 #include "fpq_kernels.h"
 
@@ -592,6 +594,100 @@ fpq_status fpq_conv2d_split(const float* x1, int C1, float x1_scale, const float
     return launch_gemm(p, st);
 }
 
+}  // extern "C"
+
+// ---- host-buffer forms: copy in, layer, copy out, pipelined over slices of the batch --------------
+//
+// The two copies of one slice cannot overlap, but the copy-in of slice i + 1, the layer on slice i
+// and the copy-out of slice i - 1 can (PCIe carries both directions at once).  The pipeline needs a
+// stream per direction and an event per hand-over: they are created once per device at the first
+// host-form call and kept.
+
+namespace fpq {
+
+constexpr int HOST_SLICES = 8;
+
+struct HostPipe {
+    bool ready;
+    cudaStream_t in, out;
+    cudaEvent_t start, end, copied[HOST_SLICES], computed[HOST_SLICES];
+};
+
+static HostPipe* host_pipe()
+{
+    static std::mutex m;
+    static HostPipe pipes[64] = {};
+    std::lock_guard<std::mutex> lock(m);
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
+        return nullptr;
+    HostPipe& p = pipes[dev];
+    if (!p.ready) {
+        bool ok = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&p.end, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < HOST_SLICES; ++i)
+            ok = cudaEventCreateWithFlags(&p.copied[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&p.computed[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok)
+            return nullptr;
+        p.ready = true;
+    }
+    return &p;
+}
+
+// units = rows (linear) or images (conv); in_stride / out_stride = floats per unit; layer(u0, n) enqueues
+// the layer on units [u0, u0 + n) of the device buffers on `st`.
+template <typename Layer>
+static fpq_status host_pipeline(const float* x_host, float* x_dev, float* y_dev, float* y_host, int64_t units,
+                                int64_t in_stride, int64_t out_stride, cudaStream_t st, Layer layer)
+{
+    if (units == 0)
+        return FPQ_OK;
+    HostPipe* hp = host_pipe();
+    if (!hp)
+        return FPQ_ERR_CUDA;
+    // slices only when the copies are long enough to be worth overlapping
+    const int64_t bytes = 4 * units * (in_stride + out_stride);
+    int64_t slices = bytes >= (8ll << 20) ? HOST_SLICES : 1;
+    if (slices > units)
+        slices = units;
+    bool ok = cudaEventRecord(hp->start, st) == cudaSuccess && cudaStreamWaitEvent(hp->in, hp->start, 0) == cudaSuccess &&
+              cudaStreamWaitEvent(hp->out, hp->start, 0) == cudaSuccess;
+    for (int64_t i = 0; ok && i < slices; ++i) {
+        const int64_t u0 = units * i / slices, n = units * (i + 1) / slices - u0;
+        ok = cudaMemcpyAsync(x_dev + u0 * in_stride, x_host + u0 * in_stride, sizeof(float) * (size_t)(n * in_stride),
+                             cudaMemcpyHostToDevice, hp->in) == cudaSuccess &&
+             cudaEventRecord(hp->copied[i], hp->in) == cudaSuccess;
+    }
+    fpq_status s = ok ? FPQ_OK : FPQ_ERR_CUDA;
+    for (int64_t i = 0; s == FPQ_OK && i < slices; ++i) {
+        const int64_t u0 = units * i / slices, n = units * (i + 1) / slices - u0;
+        if (cudaStreamWaitEvent(st, hp->copied[i], 0) != cudaSuccess) {
+            s = FPQ_ERR_CUDA;
+            break;
+        }
+        s = layer(u0, n);
+        if (s != FPQ_OK)
+            break;
+        if (cudaEventRecord(hp->computed[i], st) != cudaSuccess || cudaStreamWaitEvent(hp->out, hp->computed[i], 0) != cudaSuccess ||
+            cudaMemcpyAsync(y_host + u0 * out_stride, y_dev + u0 * out_stride, sizeof(float) * (size_t)(n * out_stride),
+                            cudaMemcpyDeviceToHost, hp->out) != cudaSuccess)
+            s = FPQ_ERR_CUDA;
+    }
+    // whatever happened, nothing of this call may still be in flight on the side streams afterwards
+    const bool drained = cudaStreamSynchronize(hp->in) == cudaSuccess && cudaStreamSynchronize(hp->out) == cudaSuccess &&
+                         cudaStreamSynchronize(st) == cudaSuccess;
+    if (s != FPQ_OK)
+        return s;
+    return drained ? FPQ_OK : FPQ_ERR_CUDA;
+}
+
+}  // namespace fpq
+
+extern "C" {
+
 fpq_status fpq_linear_host(const float* x_host, float* x_dev, const void* w_prepared, const float* w_scale,
                            float x_scale, fpq_format fx, fpq_format fw, const float* bias, float* y_dev,
                            float* y_host, int64_t M, int64_t N, int64_t K, void* workspace, size_t ws_bytes,
@@ -601,16 +697,24 @@ fpq_status fpq_linear_host(const float* x_host, float* x_dev, const void* w_prep
         return FPQ_ERR_NULL;
     if (M < 0 || N < 0 || K < 0)
         return FPQ_ERR_SHAPE;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (cudaMemcpyAsync(x_dev, x_host, sizeof(float) * (size_t)M * K, cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return FPQ_ERR_CUDA;
-    fpq_status s = fpq_linear(x_dev, w_prepared, w_scale, x_scale, fx, fw, bias, y_dev, M, N, K, workspace, ws_bytes,
-                              stream);
-    if (s != FPQ_OK)
-        return s;
-    if (cudaMemcpyAsync(y_host, y_dev, sizeof(float) * (size_t)M * N, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return FPQ_ERR_CUDA;
-    return cudaStreamSynchronize(st) == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
+    // (row slices stay 16-byte aligned only if whole rows are: otherwise one slice)
+    const bool sliceable = (K % 4 == 0) && (N % 4 == 0);
+    auto layer = [&](int64_t m0, int64_t m) {
+        return fpq_linear(x_dev + m0 * K, w_prepared, w_scale, x_scale, fx, fw, bias, y_dev + m0 * N, m, N, K, workspace,
+                          ws_bytes, stream);
+    };
+    if (!sliceable) {
+        cudaStream_t st = (cudaStream_t)stream;
+        if (cudaMemcpyAsync(x_dev, x_host, sizeof(float) * (size_t)M * K, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return FPQ_ERR_CUDA;
+        fpq_status s = layer(0, M);
+        if (s != FPQ_OK)
+            return s;
+        if (cudaMemcpyAsync(y_host, y_dev, sizeof(float) * (size_t)M * N, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return FPQ_ERR_CUDA;
+        return cudaStreamSynchronize(st) == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
+    }
+    return host_pipeline(x_host, x_dev, y_dev, y_host, M, K, N, (cudaStream_t)stream, layer);
 }
 
 fpq_status fpq_conv2d_host(const float* x_host, float* x_dev, const void* w_prepared, const float* w_scale,
@@ -624,18 +728,12 @@ fpq_status fpq_conv2d_host(const float* x_host, float* x_dev, const void* w_prep
     fpq_status s = conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo);
     if (s != FPQ_OK)
         return s;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (cudaMemcpyAsync(x_dev, x_host, sizeof(float) * (size_t)B * C * H * W, cudaMemcpyHostToDevice, st) !=
-        cudaSuccess)
-        return FPQ_ERR_CUDA;
-    s = fpq_conv2d(x_dev, w_prepared, w_scale, x_scale, fx, fw, bias, y_dev, B, C, H, W, C_out, R, S, pad, stride,
-                   workspace, ws_bytes, stream);
-    if (s != FPQ_OK)
-        return s;
-    if (cudaMemcpyAsync(y_host, y_dev, sizeof(float) * (size_t)B * C_out * Ho * Wo, cudaMemcpyDeviceToHost, st) !=
-        cudaSuccess)
-        return FPQ_ERR_CUDA;
-    return cudaStreamSynchronize(st) == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
+    const int64_t in_stride = (int64_t)C * H * W, out_stride = (int64_t)C_out * Ho * Wo;
+    auto layer = [&](int64_t b0, int64_t b) {
+        return fpq_conv2d(x_dev + b0 * in_stride, w_prepared, w_scale, x_scale, fx, fw, bias, y_dev + b0 * out_stride, (int)b,
+                          C, H, W, C_out, R, S, pad, stride, workspace, ws_bytes, stream);
+    };
+    return host_pipeline(x_host, x_dev, y_dev, y_host, B, in_stride, out_stride, (cudaStream_t)stream, layer);
 }
 
 fpq_status fpq_zero_census(const uint8_t* codes, int64_t n, fpq_format fmt, uint64_t* count, void* stream)

@@ -273,3 +273,47 @@ def test_two_kernel_route_matches_the_oracle_and_the_fused_call(wfmt):
             inner = got[:, L.pad:L.pad + L.H, L.pad:L.pad + L.W, : L.C]
             assert np.array_equal(inner, want.transpose(0, 2, 3, 1))
             assert got.sum() == inner.sum()                    # frame and channel padding are code 0
+
+
+# ---- host-buffer forms (copy in, layer, copy out; pipelined in slices when the batch is large) ----------
+
+@pytest.mark.parametrize("kind,shape", [
+    ("conv", (16, 64, 32, 32, 64, 3)),        # 8 MiB of copies: eight slices of two images
+    ("conv", (3, 20, 9, 7, 37, 3)),           # small: one slice
+    ("conv", (5, 130, 32, 32, 140, 1)),       # 5 images in 5 slices
+    ("linear", (4096, 320, 320)),             # sliced by rows
+    ("linear", (3000, 640, 200)),             # 3000 rows in 8 unequal slices
+    ("linear", (4096, 130, 322)),             # rows are not 16-byte multiples: one slice
+])
+def test_host_forms_equal_the_device_forms(kind, shape):
+    if kind == "conv":
+        B, C, H, W, Co, R = shape
+        L = I.conv_layer("h", B, C, H, W, Co, R, wfmt="e4m3", rounding=True)
+    else:
+        M, K, N = shape
+        L = I.linear_layer("h", M, K, N, "e2m1", rounding=True)
+    I.draw(L, 16, sum(shape), "normal", 0.02, True)
+    ws, xs = layer_scales(L)
+    gfw, _ = FMT[L.wfmt]
+    _, prep = gpu_prepare(L, ws)
+    want = gpu_layer(L, ws, xs)
+    xh = torch.from_numpy(L.x).pin_memory()
+    xd = torch.empty_like(xh, device="cuda")
+    wsd = torch.from_numpy(ws).cuda()
+    bias = torch.from_numpy(L.bias).cuda()
+    if kind == "conv":
+        yd = torch.empty((L.B, L.N, L.Ho, L.Wo), dtype=torch.float32, device="cuda")
+        wk = torch.empty(fpq.fpq_conv2d_workspace_size(L.B, L.C, L.H, L.W, L.N, L.R, L.S, L.pad, L.stride, fpq.E4M3, gfw),
+                         dtype=torch.uint8, device="cuda")
+    else:
+        yd = torch.empty((L.M, L.N), dtype=torch.float32, device="cuda")
+        wk = torch.empty(max(1, fpq.fpq_linear_workspace_size(L.M, L.N, L.K, fpq.E4M3, gfw)), dtype=torch.uint8, device="cuda")
+    yh = torch.empty(yd.shape, dtype=torch.float32).pin_memory()
+    for _ in range(2):                                    # twice: the pipeline's streams and events are reused
+        yh.fill_(float("nan"))
+        if kind == "conv":
+            fpq.fpq_conv2d_host(xh, xd, prep, wsd, xs, fpq.E4M3, gfw, bias, yd, yh, L.R, L.S, L.pad, L.stride, wk)
+        else:
+            fpq.fpq_linear_host(xh, xd, prep, wsd, xs, fpq.E4M3, gfw, bias, yd, yh, wk)
+        assert fpq.fpq_read_status() == fpq.OK
+        assert np.array_equal(yh.numpy(), want)
