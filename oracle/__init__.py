@@ -2,8 +2,9 @@
 
 Thin numpy/ctypes front end of ``fpq_oracle.c``: the plain definition of the
 paper's floating-point quantizer (Sec. IV-B), its learned-rounding variant with
-hardened decisions (Sec. V-B) and the quantized linear / conv layer (Sec. V-B,
-Sec. VI-A), summed in double.  Nothing in the product path may import this
+hardened decisions (Sec. V-B), the quantized linear / conv layer (Sec. V-B,
+Sec. VI-A), summed in double, the encoding / bias search (Sec. V-A) and one
+evaluation of the rounding-learning objective and its gradient (Sec. V-B).  Nothing in the product path may import this
 package: it exists so that tests, the smoke check and the benchmark's
 CPU-baseline leg have something independent to compare the CUDA library with.
 """
@@ -82,6 +83,8 @@ def lib():
                                    i64, i64, i64, i64, i64, i64, i64, i64, i64, vp, i64, vp, vp]
         L.fpq_o_search_mse.restype = i64
         L.fpq_o_search_mse.argtypes = [vp, i64, vp, i32, vp, i32, vp]
+        L.fpq_o_soft_weight.restype = i64
+        L.fpq_o_soft_weight.argtypes = [vp, i64, i64, vp, i32, i32, i32, i32, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -275,3 +278,64 @@ def zero_count(codes, n: int, f: Format) -> int:
     values[0::2] = flat & 0xF
     values[1::2] = flat >> 4
     return int(np.count_nonzero(values[:n] == 0))
+
+
+# ---- rounding learning (Sec. V-B) -----------------------------------------------------------
+
+
+def soft_weight(w, scale, f: Format, alpha):
+    """Soft-rounded weights W^q(alpha) of the learned-rounding equation (Sec. V-B) and their
+    derivative with respect to alpha, both [N][K] float64."""
+    w = _f32(w)
+    alpha = _f32(alpha)
+    scale = _f32(scale)
+    N, K = w.shape
+    assert alpha.shape == (N, K) and scale.shape == (N,)
+    wq = np.zeros((N, K), dtype=np.float64)
+    dwq = np.zeros((N, K), dtype=np.float64)
+    lib().fpq_o_soft_weight(_p(w), N, K, _p(scale), f.e, f.m, f.B, f.sat, _p(alpha), _p(wq), _p(dwq))
+    return wq, dwq
+
+
+def rounding_regularizer(alpha):
+    """lambda(alpha) = 1 - (2 |sigma(alpha) - 0.5|)^20 per element (Sec. V-B) and its derivative."""
+    al = np.asarray(alpha, dtype=np.float64)
+    sig = 1.0 / (1.0 + np.exp(-al))
+    u = 2.0 * np.abs(sig - 0.5)
+    lam = 1.0 - u ** 20
+    dlam = -20.0 * u ** 19 * 2.0 * np.sign(sig - 0.5) * sig * (1.0 - sig)
+    return lam, dlam
+
+
+def round_learn_loss(w, scale, f: Format, alpha, a, reg: float):
+    """The rounding-learning objective of Sec. V-B for a bias-free linear layer with calibration
+    activations a [M][K]:  mean((A W^q(alpha)^T - A W^T)^2) + reg * sum_i lambda(alpha_i).
+    Returns (mse, sum of lambda)."""
+    w64 = np.asarray(_f32(w), dtype=np.float64)
+    a64 = np.asarray(_f32(a), dtype=np.float64)
+    wq, _ = soft_weight(w, scale, f, alpha)
+    y = a64 @ w64.T
+    yq = a64 @ wq.T
+    lam, _ = rounding_regularizer(_f32(alpha))
+    return float(np.mean((yq - y) ** 2)), float(lam.sum())
+
+
+def round_learn_step(w, scale, f: Format, alpha, a, reg: float):
+    """One evaluation of the objective and of its gradient with respect to alpha.
+    Chain rule on the definition: d mse / d W^q = (2 / (M N)) (Y^q - Y)^T A, times the element's
+    own d W^q / d alpha, plus reg * d lambda / d alpha.  Also returns the per-element sum of
+    absolute terms of the gradient's contraction (for the parity tolerance)."""
+    w64 = np.asarray(_f32(w), dtype=np.float64)
+    a64 = np.asarray(_f32(a), dtype=np.float64)
+    M = a64.shape[0]
+    N = w64.shape[0]
+    wq, dwq = soft_weight(w, scale, f, alpha)
+    y = a64 @ w64.T
+    yq = a64 @ wq.T
+    d = yq - y
+    mse = float(np.mean(d ** 2))
+    lam, dlam = rounding_regularizer(_f32(alpha))
+    g = (2.0 / (M * N)) * (d.T @ a64)
+    grad = g * dwq + reg * dlam
+    absum = (2.0 / (M * N)) * (np.abs(d).T @ np.abs(a64)) * np.abs(dwq)
+    return {"mse": mse, "reg": float(lam.sum()), "grad": grad, "absum": absum, "wq": wq, "d": d}

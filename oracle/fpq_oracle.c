@@ -14,7 +14,8 @@
  *   - round to nearest        Sec. IV-B, X_fp = clamp(s_i round(X'/s_i); -c, c)
  *   - per-element step s_i    Sec. IV-B, the two-case equation for s_i
  *   - learned rounding        Sec. V-B, W_q = clamp(s (floor(W/s) + sigma(alpha)); -c, c)
- *                             with sigma(alpha) hardened to 0 or 1 at inference
+ *                             with sigma(alpha) hardened to 0 or 1 at inference;
+ *                             the soft form and its derivative for the learning step
  *   - the quantized layer     Sec. V-B (Y = W A), Sec. VI-A (conv and linear
  *                             weights and activations are quantized, everything
  *                             else stays FP32)
@@ -365,6 +366,54 @@ int64_t fpq_o_search_mse(const float *x, int64_t n, const int32_t *enc /* [n_enc
                 sum += err * err;
             }
             mse[(int64_t)i * n_clip + j] = n > 0 ? sum / (double)n : 0.0;
+        }
+    }
+    return nans;
+}
+
+/* ---- rounding learning (Sec. V-B) ------------------------------------------ */
+
+/* Soft-rounded weights of Sec. V-B, the learned-rounding equation before hardening:
+ *     a      = clamp(w * (1.0f / scale); -c, c)           (FP32 scaling as everywhere above)
+ *     pre    = s(a) * (floor(a / s(a)) + sigma(alpha))    sigma(alpha) = 1 / (1 + exp(-alpha))
+ *     wq     = scale * clamp(pre; -c, c)                  back in the weight's own units
+ * and its derivative with respect to alpha,
+ *     dwq    = scale * s(a) * sigma (1 - sigma)           where pre lies in [-c, c], else 0
+ * (floor is piecewise constant; a clamp passes the gradient inside its range and
+ * blocks it outside).  Everything after the FP32 scaling is double.  A NaN weight
+ * gives wq = dwq = 0.  wq, dwq: [N][K] doubles. */
+int64_t fpq_o_soft_weight(const float *w, int64_t N, int64_t K, const float *scale, int e, int m, int B,
+                          int sat, const float *alpha, double *wq, double *dwq)
+{
+    ofmt f = {e, m, B, sat};
+    double c = fpq_o_cmax(e, m, B, sat);
+    int64_t nans = 0;
+    for (int64_t n = 0; n < N; ++n) {
+        for (int64_t k = 0; k < K; ++k) {
+            int64_t i = n * K + k;
+            volatile float r = 1.0f / scale[n];
+            volatile float t = w[i] * r;
+            if (t != t) {
+                wq[i] = 0.0;
+                dwq[i] = 0.0;
+                ++nans;
+                continue;
+            }
+            double a = (double)t;
+            if (a > c)
+                a = c;
+            if (a < -c)
+                a = -c;
+            double s = step_of(a, f);
+            double sig = 1.0 / (1.0 + exp(-(double)alpha[i]));
+            double pre = s * (floor(a / s) + sig);
+            double q = pre;
+            if (q > c)
+                q = c;
+            if (q < -c)
+                q = -c;
+            wq[i] = (double)scale[n] * q;
+            dwq[i] = (pre >= -c && pre <= c) ? (double)scale[n] * s * sig * (1.0 - sig) : 0.0;
         }
     }
     return nans;
