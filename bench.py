@@ -651,6 +651,67 @@ def run_search(args):
     print(json.dumps(out), flush=True)
 
 
+def run_round_learn(args):
+    """One rounding-learning step (Sec. V-B objective + gradient + descent update) on the linear layers of
+    the SD-v1-style transformer blocks, FP4 E2M1 weights, calibration rows = the tokens of one latent at
+    that level.  Two FP32 contractions of 2 M N K flop each on the CUDA cores: the roofline is the FP32
+    multiply-add rate, SMs x 128 lanes x 2 flop x sampled SM clock."""
+    import numpy as np
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    from paper_2408_06995_b200 import build as fpq_build
+    fpq_build.build()
+    import paper_2408_06995_b200 as fpq
+    import oracle as O
+    shapes = [("qkv_320_960", 4096, 960, 320), ("attn_out_320_320", 4096, 320, 320),
+              ("geglu_320_2560", 4096, 2560, 320), ("ffn_out_1280_320", 4096, 320, 1280),
+              ("geglu_640_5120", 1024, 5120, 640), ("ffn_out_5120_1280", 256, 1280, 5120)]
+    if args.only:
+        shapes = [sh for sh in shapes if args.only in sh[0]]
+        if not shapes:
+            raise SystemExit(f"no shape of suite round_learn has {args.only!r} in its name")
+    props = torch.cuda.get_device_properties(0)
+    sampler = ClockSampler(physical_gpu_index(0))
+    sampler.start()
+    out = {"suite": "round_learn", "dtype": "f32", "rows": []}
+    for name, M, N, K in shapes:
+        w = torch.randn((N, K), device=dev) * 0.02
+        scale = (w.abs().amax(dim=1) / 6.0).contiguous()
+        a = torch.randn((M, K), device=dev)
+        alpha = torch.randn((N, K), device=dev) * 2.0
+        grad = torch.empty_like(alpha)
+        loss = torch.empty(2, dtype=torch.float64, device=dev)
+        wk = torch.empty(fpq.fpq_round_learn_workspace_size(M, N, K), dtype=torch.uint8, device=dev)
+        fn = lambda: fpq.fpq_round_learn_step(w, scale, fpq.E2M1, alpha, a, 0.01, 1.0, grad, loss, wk)
+        t = per_launch_us(torch, fn, 10) * 1e-6
+        flop = 4.0 * M * N * K
+        out["rows"].append({"name": name, "M": M, "N": N, "K": K, "us": t * 1e6, "tflops": flop / t / 1e12,
+                            "steps_per_s": 1.0 / t})
+    clocks = sampler.stop()
+    peak = props.multi_processor_count * 128 * 2 * (clocks["sm_mhz"] or 1965.0) * 1e6
+    for row in out["rows"]:
+        row["roofline"] = {"bound": "alu", "achieved": row["tflops"], "peak": peak / 1e12, "unit": "TFLOP/s",
+                           "frac": row["tflops"] * 1e12 / peak,
+                           "peak_source": "SM count x 128 FP32 lanes x 2 flop x sampled SM clock"}
+    out["clocks"] = clocks
+    if not args.skip_cpu:
+        name, M, N, K = min(shapes, key=lambda sh: sh[1] * sh[2] * sh[3])
+        rng = np.random.default_rng(0)
+        w = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+        sc = (np.abs(w).max(axis=1) / 6.0).astype(np.float32)
+        al = (rng.standard_normal((N, K)) * 2).astype(np.float32)
+        a = rng.standard_normal((M, K)).astype(np.float32)
+        t0 = time.perf_counter()
+        O.round_learn_step(w, sc, O.E2M1, al, a, 0.01)
+        dt = time.perf_counter() - t0
+        out["cpu_baseline"] = {"value": 1.0 / dt, "unit": "steps/s", "cores": os.cpu_count(), "kind": "oracle",
+                               "sample": f"one step of {name} (M={M})"}
+    print(json.dumps(out), flush=True)
+
+
 def run_split(args):
     """The decoder convolutions of the SD-v1-style U-Net whose input is a concatenation (previous
     layer's output + skip connection), W4A8, batch 2: the two-scale call against the ordinary call
@@ -720,9 +781,9 @@ def main():
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline leg")
     ap.add_argument("--skip-w4", action="store_true", help="leave out the W4A8 side measurement")
-    ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd", "sd_trace", "search", "sd_split"],
+    ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd", "sd_trace", "search", "sd_split", "round_learn"],
                     help="print a per-shape table of a whole workload instead of the headline line")
-    ap.add_argument("--only", default=None, help="with --suite ldm|transformer|sd: only the layers whose name contains this")
+    ap.add_argument("--only", default=None, help="with --suite ldm|transformer|sd|round_learn: only the layers whose name contains this")
     args = ap.parse_args()
     if args.suite == "sd_trace":
         run_trace(args)
@@ -730,6 +791,8 @@ def main():
         run_search(args)
     elif args.suite == "sd_split":
         run_split(args)
+    elif args.suite == "round_learn":
+        run_round_learn(args)
     elif args.suite:
         run_suite(args)
     elif args.impl == "reference":

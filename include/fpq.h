@@ -317,6 +317,50 @@ fpq_status fpq_search_format(const float* x, int64_t n, const fpq_format* enc_ho
 fpq_status fpq_search_clip_candidates(float maxabs, int32_t count, float* clip_host);
 
 /*
+ * Rounding learning (Sec. V-B): one evaluation of the objective and of its gradient for the weights
+ * of a bias-free linear layer (the paper's own example; a convolution is the same call on its
+ * unfolded input rows).  With sigma(t) = 1 / (1 + exp(-t)), gamma = scale[n] and, per weight,
+ * a = clamp(w * (1.0f / gamma); -c, c), s = the grid step of a's binade (Sec. IV-B step equation):
+ *     Wq(alpha)  = gamma * clamp(s * (floor(a / s) + sigma(alpha)); -c, c)      learned-rounding equation
+ *     mse        = mean over [M][N] of (A Wq^T - A W^T)^2                        layer-output error
+ *     lambda     = 1 - (2 |sigma(alpha) - 0.5|)^20                               regulariser, per weight
+ *     objective  = mse + reg * sum of lambda over all weights
+ *     grad       = d objective / d alpha  (floor has zero derivative; a clamp passes the derivative
+ *                  inside [-c, c] and blocks it outside)
+ * The paper prints "+ lambda(alpha)" without saying how the per-weight terms combine or how they
+ * are weighted: they are summed and the caller gives the weight `reg`.  The activations are used as
+ * given (FP32, the same on both sides of the difference, as in the paper's equations).
+ * Everything is computed in FP32, the precision the method is stated in: the two contractions are
+ * FP32 multiply-adds (A (Wq - W)^T, which is A Wq^T - A W^T by linearity, and its transpose product
+ * with A), the sums of squares and of lambda are accumulated in double.
+ *   w       [N][K] FP32 weights, scale [N] (as fpq_quantize_weight)
+ *   fmt     weight format (any valid format; the paper learns rounding for FP4 only)
+ *   alpha   [N][K] FP32, read; overwritten by alpha - lr * grad when lr != 0 (plain gradient descent)
+ *   a       [M][K] FP32 calibration activations, row-major
+ *   reg,lr  finite
+ *   grad    out, [N][K] FP32
+ *   loss    out, 2 doubles (8-byte aligned): {mse, sum of lambda}
+ *   workspace  fpq_round_learn_workspace_size(M, N, K) bytes, 256-byte aligned, contents not kept
+ * One memset and four kernels on `stream`; no allocation, no host synchronisation.  A NaN weight
+ * contributes nothing and sets FPQ_ERR_NAN_INPUT in the device status.  Limits: 1 <= M < 2^31 - 128,
+ * 1 <= N, K <= 65535 * 128, N * K < 2^40.  Errors: FPQ_ERR_FORMAT, FPQ_ERR_SHAPE, FPQ_ERR_NULL,
+ * FPQ_ERR_ALIGN, FPQ_ERR_WORKSPACE, FPQ_ERR_CUDA.  The workspace size is 0 for shapes out of range.
+ */
+size_t fpq_round_learn_workspace_size(int64_t M, int64_t N, int64_t K);
+fpq_status fpq_round_learn_step(const float* w, const float* scale, fpq_format fmt, float* alpha, const float* a,
+                                int64_t M, int64_t N, int64_t K, float reg, float lr, float* grad, double* loss,
+                                void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * The inference rule of Sec. V-B: sigma(alpha) < 0.5 rounds down, sigma(alpha) >= 0.5 rounds up, i.e.
+ * decision bit = (alpha >= 0).  Writes the bits in the layout fpq_quantize_weight reads (1 bit per
+ * weight, LSB first along K, every row padded to a whole byte; padding bits are 0).
+ *   alpha [N][K] FP32; rounding_bits out, N * ceil(K / 8) bytes.  One kernel on `stream`.
+ * Errors: FPQ_ERR_SHAPE, FPQ_ERR_NULL, FPQ_ERR_ALIGN, FPQ_ERR_CUDA.
+ */
+fpq_status fpq_round_learn_harden(const float* alpha, int64_t N, int64_t K, uint8_t* rounding_bits, void* stream);
+
+/*
  * Which route fpq_linear / fpq_conv2d take (process-wide setting, not thread-safe against
  * concurrent layer calls; the results are the same bit for bit on either route):
  *   FPQ_PATH_FUSED        one kernel: the activation quantize (Sec. IV-B rounding equation) runs

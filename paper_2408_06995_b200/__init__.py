@@ -69,6 +69,7 @@ EXPORTS = [
     "fpq_conv2d_workspace_size", "fpq_conv2d", "fpq_linear_host", "fpq_conv2d_host",
     "fpq_linear_quantize_input", "fpq_linear_contract", "fpq_conv2d_quantize_input", "fpq_conv2d_contract",
     "fpq_linear_static", "fpq_search_workspace_size", "fpq_search_format", "fpq_search_clip_candidates",
+    "fpq_round_learn_workspace_size", "fpq_round_learn_step", "fpq_round_learn_harden",
     "fpq_zero_census", "fpq_prepared_size_split", "fpq_prepare_weight_split", "fpq_conv2d_split_workspace_size",
     "fpq_conv2d_split", "fpq_set_path_policy", "fpq_get_path_policy", "fpq_read_status", "fpq_status_string",
 ]
@@ -88,6 +89,12 @@ def lib() -> ctypes.CDLL:
         i32, i64, f32 = ctypes.c_int32, ctypes.c_int64, ctypes.c_float
         vp, sz = ctypes.c_void_p, ctypes.c_size_t
         F, D = _CFormat, ctypes.POINTER(_CLayerDesc)
+        L.fpq_round_learn_workspace_size.restype = sz
+        L.fpq_round_learn_workspace_size.argtypes = [i64, i64, i64]
+        L.fpq_round_learn_step.restype = i32
+        L.fpq_round_learn_step.argtypes = [vp, vp, F, vp, vp, i64, i64, i64, f32, f32, vp, vp, vp, sz, vp]
+        L.fpq_round_learn_harden.restype = i32
+        L.fpq_round_learn_harden.argtypes = [vp, i64, i64, vp, vp]
         L.fpq_scale_from_max.restype = f32
         L.fpq_scale_from_max.argtypes = [f32, F]
         L.fpq_format_max.restype = f32
@@ -386,6 +393,42 @@ def fpq_search_format(x: torch.Tensor, encodings, clip: torch.Tensor, mse: torch
                                    _ptr(mse), _ptr(best), _ptr(workspace), workspace.numel(), _stream()),
            "fpq_search_format")
     return mse, best
+
+
+def fpq_round_learn_workspace_size(M: int, N: int, K: int) -> int:
+    return lib().fpq_round_learn_workspace_size(int(M), int(N), int(K))
+
+
+def fpq_round_learn_step(w: torch.Tensor, scale: torch.Tensor, fmt: Format, alpha: torch.Tensor, a: torch.Tensor,
+                         reg: float, lr: float = 0.0, grad: torch.Tensor = None, loss: torch.Tensor = None,
+                         workspace: torch.Tensor = None):
+    """One evaluation of the rounding-learning objective and its gradient (Sec. V-B); alpha is updated in
+    place when lr != 0.  Returns (grad [N][K] float32, loss [2] float64 = {mse, sum of lambda}), on the device."""
+    for t_ in (w, scale, alpha, a):
+        assert t_.is_cuda and t_.dtype == torch.float32 and t_.is_contiguous()
+    N, K = w.shape
+    M = a.shape[0]
+    assert a.shape == (M, K) and alpha.shape == (N, K) and scale.shape == (N,)
+    if grad is None:
+        grad = torch.empty((N, K), dtype=torch.float32, device=w.device)
+    if loss is None:
+        loss = torch.empty(2, dtype=torch.float64, device=w.device)
+    if workspace is None:
+        workspace = torch.empty(max(256, fpq_round_learn_workspace_size(M, N, K)), dtype=torch.uint8, device=w.device)
+    _check(lib().fpq_round_learn_step(_ptr(w), _ptr(scale), fmt.c(), _ptr(alpha), _ptr(a), M, N, K, float(reg),
+                                      float(lr), _ptr(grad), _ptr(loss), _ptr(workspace), workspace.numel(),
+                                      _stream()), "fpq_round_learn_step")
+    return grad, loss
+
+
+def fpq_round_learn_harden(alpha: torch.Tensor, bits: torch.Tensor = None) -> torch.Tensor:
+    """Decision bits (alpha >= 0) packed as fpq_quantize_weight reads them: [N][ceil(K/8)] bytes."""
+    assert alpha.is_cuda and alpha.dtype == torch.float32 and alpha.is_contiguous() and alpha.dim() == 2
+    N, K = alpha.shape
+    if bits is None:
+        bits = torch.empty((N, (K + 7) // 8), dtype=torch.uint8, device=alpha.device)
+    _check(lib().fpq_round_learn_harden(_ptr(alpha), N, K, _ptr(bits), _stream()), "fpq_round_learn_harden")
+    return bits
 
 
 def fpq_set_path_policy(policy: int) -> None:

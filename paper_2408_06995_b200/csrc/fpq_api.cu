@@ -794,6 +794,50 @@ fpq_status fpq_search_clip_candidates(float maxabs, int32_t count, float* clip_h
     return FPQ_OK;
 }
 
+static bool round_learn_shape_ok(int64_t M, int64_t N, int64_t K)
+{
+    const int64_t lim = (int64_t)1 << 31;
+    return M >= 1 && N >= 1 && K >= 1 && M < lim - 128 && N <= 65535 * 128 && K <= 65535 * 128 &&
+           N * K < ((int64_t)1 << 40) && M * round_up(N, 4) < ((int64_t)1 << 40);
+}
+
+size_t fpq_round_learn_workspace_size(int64_t M, int64_t N, int64_t K)
+{
+    if (!round_learn_shape_ok(M, N, K))
+        return 0;
+    return round_learn_workspace_bytes(M, N, K);
+}
+
+fpq_status fpq_round_learn_step(const float* w, const float* scale, fpq_format fmt, float* alpha, const float* a,
+                                int64_t M, int64_t N, int64_t K, float reg, float lr, float* grad, double* loss,
+                                void* workspace, size_t ws_bytes, void* stream)
+{
+    QFormat q;
+    if (!resolve_format(fmt, &q))
+        return FPQ_ERR_FORMAT;
+    if (!round_learn_shape_ok(M, N, K) || !isfinite(reg) || !isfinite(lr))
+        return FPQ_ERR_SHAPE;
+    if (!w || !scale || !alpha || !a || !grad || !loss)
+        return FPQ_ERR_NULL;
+    if (!aligned(w, 4) || !aligned(scale, 4) || !aligned(alpha, 4) || !aligned(a, 4) || !aligned(grad, 4) ||
+        !aligned(loss, 8) || !aligned(workspace, 256))
+        return FPQ_ERR_ALIGN;
+    if (!workspace || ws_bytes < round_learn_workspace_bytes(M, N, K))
+        return FPQ_ERR_WORKSPACE;
+    return launch_round_learn(w, scale, q, alpha, a, M, N, K, reg, lr, grad, loss, workspace, (cudaStream_t)stream);
+}
+
+fpq_status fpq_round_learn_harden(const float* alpha, int64_t N, int64_t K, uint8_t* rounding_bits, void* stream)
+{
+    if (N < 0 || K < 0 || (K > 0 && N > (((int64_t)1 << 40) / K)))
+        return FPQ_ERR_SHAPE;
+    if (N * K > 0 && (!alpha || !rounding_bits))
+        return FPQ_ERR_NULL;
+    if (!aligned(alpha, 4))
+        return FPQ_ERR_ALIGN;
+    return launch_round_harden(alpha, N, K, rounding_bits, (cudaStream_t)stream);
+}
+
 fpq_status fpq_set_path_policy(int32_t policy)
 {
     if (policy != FPQ_PATH_AUTO && policy != FPQ_PATH_FUSED && policy != FPQ_PATH_TWO_KERNELS)

@@ -61,4 +61,12 @@ size_t search_workspace_bytes(int n_enc, int n_clip);
 fpq_status launch_search(const float* x, int64_t n, const fpq_format* enc, int n_enc, const float* clip, int n_clip,
                          double* mse, int32_t* best, void* workspace, cudaStream_t st);
 
+// Rounding learning (Sec. V-B): scratch size, one objective + gradient evaluation (a memset and four kernels),
+// and the hardening of alpha into decision bits.
+size_t round_learn_workspace_bytes(int64_t M, int64_t N, int64_t K);
+fpq_status launch_round_learn(const float* w, const float* scale, const QFormat& f, float* alpha, const float* a,
+                              int64_t M, int64_t N, int64_t K, float reg, float lr, float* grad, double* loss,
+                              void* workspace, cudaStream_t st);
+fpq_status launch_round_harden(const float* alpha, int64_t N, int64_t K, uint8_t* bits, cudaStream_t st);
+
 }  // namespace fpq

@@ -106,3 +106,15 @@ def test_sizes(L):
     assert fpq.fpq_prepared_size(fpq.E2M1, fpq.CONV2D, 10, 320, 3, 3) == 10 * 9 * 384 // 2
     assert fpq.fpq_prepared_size(fpq.E2M1, fpq.LINEAR, 10, 320, 3, 3) == 0
     assert fpq.status_string(fpq.ERR_TIMEOUT) == "device-side wait timed out"
+
+
+def test_round_learn_rejections(L):
+    p = ctypes.c_void_p(256)   # never dereferenced: rejected first
+    F = fpq.E2M1.c()
+    assert L.fpq_round_learn_step(p, p, fpq.Format(6, 3, 7).c(), p, p, 4, 4, 4, 0.0, 0.0, p, p, p, 1 << 30, None) == fpq.ERR_FORMAT
+    assert L.fpq_round_learn_step(p, p, F, p, p, 0, 4, 4, 0.0, 0.0, p, p, p, 1 << 30, None) == fpq.ERR_SHAPE
+    assert L.fpq_round_learn_step(p, p, F, None, p, 4, 4, 4, 0.0, 0.0, p, p, p, 1 << 30, None) == fpq.ERR_NULL
+    assert L.fpq_round_learn_step(p, p, F, p, p, 4, 4, 4, 0.0, 0.0, p, ctypes.c_void_p(260), p, 1 << 30, None) == fpq.ERR_ALIGN
+    assert L.fpq_round_learn_step(p, p, F, p, p, 4, 4, 4, 0.0, 0.0, p, p, p, 16, None) == fpq.ERR_WORKSPACE
+    assert L.fpq_round_learn_step(p, p, F, p, p, 4, 4, 4, float("nan"), 0.0, p, p, p, 1 << 30, None) == fpq.ERR_SHAPE
+    assert L.fpq_round_learn_workspace_size(0, 4, 4) == 0
