@@ -121,6 +121,12 @@ fpq_status fpq_quantize_act(const float* x, int64_t n, float scale, fpq_format f
  * fpq_prepared_size(fmt, d) bytes and be 128-byte aligned.  The layout is
  * internal: rows of C padded with zero codes to a multiple of 128, taps
  * outermost within a row ([N][R*S][C_pad]).  May be saved and reloaded as bytes.
+ * E4M3 (bias 7, FPQ_SAT_NATIVE) and E2M1 (bias 1) codes are kept as they are (E2M1 two per
+ * byte).  Any other format whose every value is also a finite E4M3 value - E1M2 with bias 1,
+ * E2M1 with bias 2, small formats such as E3M2 bias 3 or E2M3 bias 1 - is re-encoded here,
+ * exactly, into one E4M3 byte per weight, so that the layer calls can run it; formats that do
+ * not fit (more than 3 mantissa bits, a wider exponent range, the paper's E4M3 code for 480)
+ * are copied unchanged and the layer calls refuse them.
  */
 size_t fpq_prepared_size(fpq_format fmt, const fpq_layer_desc* d);
 fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_layer_desc* d,
@@ -135,7 +141,9 @@ fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_la
  * tensor cores (layers of at most 8 rows with K a multiple of 4 run on the CUDA
  * cores instead: the same exact products, another order of the FP32 additions;
  * the workspace is then left untouched).  Supported operand pairs: fx = E4M3 bias 7 FPQ_SAT_NATIVE with
- * fw = the same, or fw = E2M1 bias 1.  Anything else: FPQ_ERR_UNSUPPORTED.
+ * fw = the same, fw = E2M1 bias 1, or any fw that fpq_prepare_weight re-encodes exactly into E4M3 (see
+ * there; the weights then occupy one byte each and run at the E4M3 rate).  Anything else:
+ * FPQ_ERR_UNSUPPORTED.
  * workspace: fpq_linear_workspace_size bytes, 128-byte aligned; contents are
  * scratch.
  */

@@ -73,6 +73,52 @@ static bool is_e2m1(fpq_format f)
     return f.exp_bits == 2 && f.man_bits == 1 && f.exp_bias == 1;
 }
 
+// Value of one code of format f (format equation of Sec. IV-B), sign included.
+static double code_value(int code, fpq_format f)
+{
+    int em = f.exp_bits + f.man_bits;
+    int p = (code >> f.man_bits) & ((1 << f.exp_bits) - 1);
+    int d = code & ((1 << f.man_bits) - 1);
+    double v = p == 0 ? ldexp((double)d, 1 - f.exp_bias - f.man_bits)
+                      : ldexp(1.0 + ldexp((double)d, -f.man_bits), p - f.exp_bias);
+    return ((code >> em) & 1) ? -v : v;
+}
+
+// Exact re-encode of a weight format into the contraction's E4M3 operand type: true when every value of
+// f (that its quantizer can produce) is also a finite value of E4M3 with bias 7; table[code of f] = the
+// E4M3 code of the same value (a zero of either sign maps to +0; codes f never produces map to 0).
+static bool embeds_in_e4m3(fpq_format f, CodeTable* tab)
+{
+    QFormat q;
+    if (!resolve_format(f, &q))
+        return false;
+    const fpq_format e4m3 = {4, 3, 7, FPQ_SAT_NATIVE};
+    int ncodes = 1 << (1 + f.exp_bits + f.man_bits);
+    int mag_mask = (1 << (f.exp_bits + f.man_bits)) - 1;
+    for (int c = 0; c < 256; ++c) {
+        uint8_t out = 0;
+        if (c < ncodes && (c & mag_mask) <= q.code_max) {
+            double v = code_value(c, f);
+            if (v != 0.0) {
+                int found = -1;
+                for (int k = 1; k <= 0x7E && found < 0; ++k)
+                    if (code_value(k, e4m3) == fabs(v))
+                        found = k;
+                if (found < 0)
+                    return false;
+                out = (uint8_t)(found | (v < 0.0 ? 0x80 : 0));
+            }
+        }
+        if (tab)
+            tab->t[c] = out;
+    }
+    return true;
+}
+
+// Weight formats the contraction reads as they are, and formats re-encoded when the weights are prepared.
+static bool weight_native(fpq_format f) { return is_e4m3_native(f) || is_e2m1(f); }
+static bool weight_reencoded(fpq_format f) { return !weight_native(f) && embeds_in_e4m3(f, nullptr); }
+
 static int g_path_policy = FPQ_PATH_AUTO;
 
 static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
@@ -86,7 +132,7 @@ static fpq_status check_pair(fpq_format fx, fpq_format fw)
         return FPQ_ERR_FORMAT;
     if (!is_e4m3_native(fx))
         return FPQ_ERR_UNSUPPORTED;
-    if (!is_e4m3_native(fw) && !is_e2m1(fw))
+    if (!weight_native(fw) && !weight_reencoded(fw))
         return FPQ_ERR_UNSUPPORTED;
     return FPQ_OK;
 }
@@ -173,7 +219,7 @@ size_t fpq_prepared_size(fpq_format fmt, const fpq_layer_desc* d)
     if (!resolve_format(fmt, &q) || check_desc(d) != FPQ_OK)
         return 0;
     size_t elems = (size_t)d->N * d->R * d->S * (size_t)padded_c(d->C);
-    return q.four_bit ? elems / 2 : elems;
+    return (q.four_bit && !weight_reencoded(fmt)) ? elems / 2 : elems;
 }
 
 fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_layer_desc* d, void* prepared,
@@ -189,8 +235,10 @@ fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_la
         return FPQ_ERR_NULL;
     if (!aligned(prepared, 128))
         return FPQ_ERR_ALIGN;
+    CodeTable tab;
+    const bool re = weight_reencoded(fmt) && embeds_in_e4m3(fmt, &tab);
     return launch_prepare_weight(codes, d->N, d->C, d->R * d->S, (int)padded_c(d->C), q.four_bit, 0, 0,
-                                 (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
+                                 re ? &tab : nullptr, (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
                ? FPQ_OK
                : FPQ_ERR_CUDA;
 }
@@ -490,7 +538,7 @@ size_t fpq_prepared_size_split(fpq_format fmt, int32_t N, int32_t C1, int32_t C2
     if (!resolve_format(fmt, &q) || split_shape(C1, C2) != FPQ_OK || check_desc(&d) != FPQ_OK)
         return 0;
     size_t elems = (size_t)N * R * S * (size_t)(padded_c(C1) + padded_c(C2));
-    return q.four_bit ? elems / 2 : elems;
+    return (q.four_bit && !weight_reencoded(fmt)) ? elems / 2 : elems;
 }
 
 fpq_status fpq_prepare_weight_split(const uint8_t* codes, fpq_format fmt, int32_t N, int32_t C1, int32_t C2,
@@ -510,8 +558,11 @@ fpq_status fpq_prepare_weight_split(const uint8_t* codes, fpq_format fmt, int32_
         return FPQ_ERR_NULL;
     if (!aligned(prepared, 128))
         return FPQ_ERR_ALIGN;
+    CodeTable tab;
+    const bool re = weight_reencoded(fmt) && embeds_in_e4m3(fmt, &tab);
     return launch_prepare_weight(codes, N, C1 + C2, R * S, (int)(padded_c(C1) + padded_c(C2)), q.four_bit, C1,
-                                 (int)padded_c(C1), (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
+                                 (int)padded_c(C1), re ? &tab : nullptr, (uint8_t*)prepared,
+                                 (cudaStream_t)stream) == cudaSuccess
                ? FPQ_OK
                : FPQ_ERR_CUDA;
 }

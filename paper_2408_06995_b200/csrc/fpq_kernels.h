@@ -17,8 +17,13 @@ cudaError_t launch_quantize_rows_e4m3(const float* x, int64_t M, int64_t K, int6
 cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int H, int W, int pad, int Cp, int row,
                                               int c_off, float scale, uint8_t* codes, cudaStream_t st);
 cudaError_t launch_zero_census(const uint8_t* codes, int64_t n, int four_bit, unsigned long long* count, cudaStream_t st);
+// Code-to-code table of an exact re-encode (weight format -> E4M3), passed to the kernel by value.
+struct CodeTable {
+    uint8_t t[256];
+};
+// table != NULL: every code is looked up and the prepared copy holds one byte per weight.
 cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, int C1, int C1p,
-                                  uint8_t* prepared, cudaStream_t st);
+                                  const CodeTable* table, uint8_t* prepared, cudaStream_t st);
 
 // Geometry of one contraction launch (linear: taps = 1, rows of Ca codes).
 struct GemmProblem {

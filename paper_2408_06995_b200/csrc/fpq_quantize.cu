@@ -256,13 +256,17 @@ __global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const f
 // channels fill whole 128-wide chunks of the reduction.
 // ---------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) prepare_weight_kernel(const uint8_t* __restrict__ codes, int N, int C, int RS,
-                                                             int Cp, int four_bit, int C1, int C1p,
-                                                             uint8_t* __restrict__ prepared)
+                                                             int Cp, int in_four_bit, int use_table, CodeTable table,
+                                                             int C1, int C1p, uint8_t* __restrict__ prepared)
 {
+    __shared__ uint8_t s_tab[256];
+    s_tab[threadIdx.x] = table.t[threadIdx.x];
+    __syncthreads();
+    const int four_bit = in_four_bit && !use_table;      // layout of the prepared copy
     int64_t row_out = four_bit ? (int64_t)RS * Cp / 2 : (int64_t)RS * Cp;
     int64_t total = (int64_t)N * row_out;
     int64_t K = (int64_t)C * RS;
-    int64_t row_in = four_bit ? (K + 1) / 2 : K;
+    int64_t row_in = in_four_bit ? (K + 1) / 2 : K;
     int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += stride) {
         int64_t n = o / row_out, within = o % row_out;
@@ -280,12 +284,14 @@ __global__ void __launch_bounds__(256) prepare_weight_kernel(const uint8_t* __re
             }
             if (real) {
                 int64_t k = (int64_t)c * RS + tap;   // source order [C][R][S]
-                if (four_bit) {
+                if (in_four_bit) {
                     uint8_t bsrc = __ldg(codes + n * row_in + (k >> 1));
                     code = (k & 1) ? (bsrc >> 4) : (bsrc & 0xf);
                 } else {
                     code = __ldg(codes + n * row_in + k);
                 }
+                if (use_table)
+                    code = s_tab[code];
             }
             outb |= code << (4 * q * four_bit);
         }
@@ -414,10 +420,14 @@ cudaError_t launch_zero_census(const uint8_t* codes, int64_t n, int four_bit, un
 }
 
 cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, int C1, int C1p,
-                                  uint8_t* prepared, cudaStream_t st)
+                                  const CodeTable* table, uint8_t* prepared, cudaStream_t st)
 {
-    int64_t total = (int64_t)N * RS * Cp / (four_bit ? 2 : 1);
-    prepare_weight_kernel<<<grid_for(total, 256), 256, 0, st>>>(codes, N, C, RS, Cp, four_bit, C1, C1p, prepared);
+    int64_t total = (int64_t)N * RS * Cp / ((four_bit && !table) ? 2 : 1);
+    CodeTable tab = {};
+    if (table)
+        tab = *table;
+    prepare_weight_kernel<<<grid_for(total, 256), 256, 0, st>>>(codes, N, C, RS, Cp, four_bit, table ? 1 : 0, tab, C1, C1p,
+                                                                prepared);
     return cudaGetLastError();
 }
 

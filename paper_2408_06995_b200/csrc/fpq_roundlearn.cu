@@ -335,10 +335,11 @@ struct Plan {
     size_t off_E, off_DQ, off_D, off_DP, off_GP, bytes;
 };
 
-// Enough slices of a reduction of length R for about two resident blocks per SM, each at least 256 long.
+// As many slices of a reduction of length R as still fit into one wave of two resident blocks per SM (one more
+// would add a second, nearly empty wave), each at least 256 long.
 void slice(int64_t tiles, int64_t R, int* splits, int64_t* per)
 {
-    int64_t want = (2 * 148 + tiles - 1) / tiles;
+    int64_t want = (2 * 148) / tiles;
     int64_t cap = (R + 255) / 256;
     int64_t s = want < cap ? want : cap;
     s = s < 1 ? 1 : (s > 64 ? 64 : s);

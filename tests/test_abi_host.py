@@ -118,3 +118,24 @@ def test_round_learn_rejections(L):
     assert L.fpq_round_learn_step(p, p, F, p, p, 4, 4, 4, 0.0, 0.0, p, p, p, 16, None) == fpq.ERR_WORKSPACE
     assert L.fpq_round_learn_step(p, p, F, p, p, 4, 4, 4, float("nan"), 0.0, p, p, p, 1 << 30, None) == fpq.ERR_SHAPE
     assert L.fpq_round_learn_workspace_size(0, 4, 4) == 0
+
+
+def test_weight_formats_the_layer_accepts(L):
+    F = fpq.E4M3.c()
+    big = ctypes.c_void_p(1024)
+
+    def accepted(fw):
+        # a NULL activation pointer is rejected after the operand pair has been checked
+        return L.fpq_linear(None, big, big, 1.0, F, fw.c(), None, big, 8, 8, 8, big, 1 << 20, None) != fpq.ERR_UNSUPPORTED
+
+    # read by the tensor cores as they are
+    assert accepted(fpq.E4M3) and accepted(fpq.E2M1)
+    # every value is also an E4M3 value: re-encoded when the weights are prepared
+    assert accepted(fpq.E1M2) and accepted(fpq.Format(2, 1, 2)) and accepted(fpq.Format(3, 2, 3))
+    # more mantissa bits or a wider exponent range than E4M3 holds, or the code 480 of the paper's E4M3
+    assert not accepted(fpq.E3M4) and not accepted(fpq.E2M5) and not accepted(fpq.E5M2)
+    assert not accepted(fpq.Format(4, 3, 7, fpq.SAT_PAPER)) and not accepted(fpq.Format(4, 3, 8, fpq.SAT_NATIVE))
+    d = fpq._CLayerDesc(fpq.LINEAR, 8, 200, 1, 1)
+    assert L.fpq_prepared_size(fpq.E2M1.c(), ctypes.byref(d)) == 8 * 256 // 2
+    assert L.fpq_prepared_size(fpq.E1M2.c(), ctypes.byref(d)) == 8 * 256      # one E4M3 byte per weight
+    assert L.fpq_prepared_size(fpq.E4M3.c(), ctypes.byref(d)) == 8 * 256
