@@ -40,6 +40,23 @@ __device__ __forceinline__ SoftTerms soft_terms(float al)
     return o;
 }
 
+// Two FP32 values in one 64-bit register, and the packed multiply-add on such pairs (each half an IEEE fused
+// multiply-add, round to nearest): half the issue slots of two scalar instructions.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void fma2(unsigned long long& d, unsigned long long a, unsigned long long b)
+{
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b));
+}
+
 __device__ __forceinline__ double warp_sum(double v)
 {
 #pragma unroll
@@ -186,12 +203,12 @@ __global__ void __launch_bounds__(256, 2) sgemm128(const float* __restrict__ P, 
         }
     };
 
-    float acc[8][8];
+    unsigned long long acc2[8][4];   // acc2[a][b] = outputs (a, 2 b) and (a, 2 b + 1) of the thread's 8 x 8
 #pragma unroll
     for (int a = 0; a < 8; ++a)
 #pragma unroll
-        for (int b = 0; b < 8; ++b)
-            acc[a][b] = 0.f;
+        for (int b = 0; b < 4; ++b)
+            acc2[a][b] = 0ull;
 
     const int ty = t >> 4, tx = t & 15;
     int buf = 0;
@@ -215,12 +232,14 @@ __global__ void __launch_bounds__(256, 2) sgemm128(const float* __restrict__ P, 
             float4 q0 = *reinterpret_cast<const float4*>(&Qs[buf][r][tx * 4]);
             float4 q1 = *reinterpret_cast<const float4*>(&Qs[buf][r][64 + tx * 4]);
             float pv[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
-            float qv[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+            unsigned long long qq[4] = {pack2(q0.x, q0.y), pack2(q0.z, q0.w), pack2(q1.x, q1.y), pack2(q1.z, q1.w)};
 #pragma unroll
-            for (int a = 0; a < 8; ++a)
+            for (int a = 0; a < 8; ++a) {
+                unsigned long long pp = pack2(pv[a], pv[a]);
 #pragma unroll
-                for (int b = 0; b < 8; ++b)
-                    acc[a][b] = fmaf(pv[a], qv[b], acc[a][b]);
+                for (int b = 0; b < 4; ++b)
+                    fma2(acc2[a][b], pp, qq[b]);
+            }
         }
         if (more) {
             stash(Ps[buf ^ 1], pf);
@@ -229,6 +248,13 @@ __global__ void __launch_bounds__(256, 2) sgemm128(const float* __restrict__ P, 
         __syncthreads();
         buf ^= 1;
     }
+
+    float acc[8][8];
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+            unpack2(acc2[a][b], acc[a][2 * b], acc[a][2 * b + 1]);
 
     float sq = 0.f;
     const bool vec_c = (ldc % 4 == 0) && (((uintptr_t)C) % 16 == 0);
