@@ -360,6 +360,20 @@ fpq_status fpq_round_learn_step(const float* w, const float* scale, fpq_format f
                                 void* workspace, size_t ws_bytes, void* stream);
 
 /*
+ * Rounding learning for a convolution (Sec. V-B: the method also applies to convolutional layers): writes
+ * the convolution's input rows out, so that fpq_round_learn_step on `rows` and the weights flattened to
+ * [C_out][C*R*S] (the layout fpq_quantize_weight takes) is the step for the convolution.
+ *   x     FP32 NCHW [B][C][H][W]
+ *   rows  out, FP32 [B*H_out*W_out][C*R*S]: row (b, oy, ox), column (c, r, s) =
+ *         x[b][c][oy*stride - pad + r][ox*stride - pad + s], 0 in the padding;
+ *         H_out = (H + 2 pad - R) / stride + 1, likewise W_out
+ * One kernel on `stream`.  Errors: FPQ_ERR_SHAPE (sizes out of range, window larger than the padded
+ * input, R or S above 64), FPQ_ERR_NULL, FPQ_ERR_ALIGN, FPQ_ERR_CUDA.
+ */
+fpq_status fpq_round_learn_unfold(const float* x, int32_t B, int32_t C, int32_t H, int32_t W, int32_t R, int32_t S,
+                                  int32_t pad, int32_t stride, float* rows, void* stream);
+
+/*
  * The inference rule of Sec. V-B: sigma(alpha) < 0.5 rounds down, sigma(alpha) >= 0.5 rounds up, i.e.
  * decision bit = (alpha >= 0).  Writes the bits in the layout fpq_quantize_weight reads (1 bit per
  * weight, LSB first along K, every row padded to a whole byte; padding bits are 0).

@@ -339,3 +339,21 @@ def round_learn_step(w, scale, f: Format, alpha, a, reg: float):
     grad = g * dwq + reg * dlam
     absum = (2.0 / (M * N)) * (np.abs(d).T @ np.abs(a64)) * np.abs(dwq)
     return {"mse": mse, "reg": float(lam.sum()), "grad": grad, "absum": absum, "wq": wq, "d": d}
+
+
+def unfold(x, R: int, S: int, pad: int, stride: int) -> np.ndarray:
+    """Input rows of a convolution (Sec. V-B applies the learning step to convolutions as well): row
+    (b, oy, ox), column (c, r, s) = x[b][c][oy*stride - pad + r][ox*stride - pad + s], zero in the padding.
+    Plain loops over the window."""
+    x = _f32(x)
+    B, C, H, W = x.shape
+    Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
+    xp = np.zeros((B, C, H + 2 * pad, W + 2 * pad), dtype=np.float32)
+    xp[:, :, pad:pad + H, pad:pad + W] = x
+    rows = np.zeros((B, Ho, Wo, C, R, S), dtype=np.float32)
+    for oy in range(Ho):
+        for ox in range(Wo):
+            for r in range(R):
+                for s in range(S):
+                    rows[:, oy, ox, :, r, s] = xp[:, :, oy * stride + r, ox * stride + s]
+    return rows.reshape(B * Ho * Wo, C * R * S)

@@ -69,7 +69,7 @@ EXPORTS = [
     "fpq_conv2d_workspace_size", "fpq_conv2d", "fpq_linear_host", "fpq_conv2d_host",
     "fpq_linear_quantize_input", "fpq_linear_contract", "fpq_conv2d_quantize_input", "fpq_conv2d_contract",
     "fpq_linear_static", "fpq_search_workspace_size", "fpq_search_format", "fpq_search_clip_candidates",
-    "fpq_round_learn_workspace_size", "fpq_round_learn_step", "fpq_round_learn_harden",
+    "fpq_round_learn_workspace_size", "fpq_round_learn_step", "fpq_round_learn_harden", "fpq_round_learn_unfold",
     "fpq_zero_census", "fpq_prepared_size_split", "fpq_prepare_weight_split", "fpq_conv2d_split_workspace_size",
     "fpq_conv2d_split", "fpq_set_path_policy", "fpq_get_path_policy", "fpq_read_status", "fpq_status_string",
 ]
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
         L.fpq_round_learn_workspace_size.argtypes = [i64, i64, i64]
         L.fpq_round_learn_step.restype = i32
         L.fpq_round_learn_step.argtypes = [vp, vp, F, vp, vp, i64, i64, i64, f32, f32, vp, vp, vp, sz, vp]
+        L.fpq_round_learn_unfold.restype = i32
+        L.fpq_round_learn_unfold.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, i32, vp, vp]
         L.fpq_round_learn_harden.restype = i32
         L.fpq_round_learn_harden.argtypes = [vp, i64, i64, vp, vp]
         L.fpq_scale_from_max.restype = f32
@@ -419,6 +421,18 @@ def fpq_round_learn_step(w: torch.Tensor, scale: torch.Tensor, fmt: Format, alph
                                       float(lr), _ptr(grad), _ptr(loss), _ptr(workspace), workspace.numel(),
                                       _stream()), "fpq_round_learn_step")
     return grad, loss
+
+
+def fpq_round_learn_unfold(x: torch.Tensor, R: int, S: int, pad: int, stride: int, rows: torch.Tensor = None) -> torch.Tensor:
+    """Input rows [B*H_out*W_out][C*R*S] of a convolution over x (NCHW), columns in [C][R][S] order."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous() and x.dim() == 4
+    B, C, H, W = x.shape
+    Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
+    if rows is None:
+        rows = torch.empty((B * Ho * Wo, C * R * S), dtype=torch.float32, device=x.device)
+    _check(lib().fpq_round_learn_unfold(_ptr(x), B, C, H, W, R, S, pad, stride, _ptr(rows), _stream()),
+           "fpq_round_learn_unfold")
+    return rows
 
 
 def fpq_round_learn_harden(alpha: torch.Tensor, bits: torch.Tensor = None) -> torch.Tensor:

@@ -878,6 +878,26 @@ fpq_status fpq_round_learn_step(const float* w, const float* scale, fpq_format f
     return launch_round_learn(w, scale, q, alpha, a, M, N, K, reg, lr, grad, loss, workspace, (cudaStream_t)stream);
 }
 
+fpq_status fpq_round_learn_unfold(const float* x, int32_t B, int32_t C, int32_t H, int32_t W, int32_t R, int32_t S,
+                                  int32_t pad, int32_t stride, float* rows, void* stream)
+{
+    if (B < 0 || C < 1 || H < 1 || W < 1 || R < 1 || S < 1 || pad < 0 || stride < 1 || R > 64 || S > 64)
+        return FPQ_ERR_SHAPE;
+    if (H + 2 * (int64_t)pad < R || W + 2 * (int64_t)pad < S)
+        return FPQ_ERR_SHAPE;
+    int Ho = (H + 2 * pad - R) / stride + 1, Wo = (W + 2 * pad - S) / stride + 1;
+    int64_t K = (int64_t)C * R * S;
+    if (K > ((int64_t)1 << 30) || (int64_t)B * Ho * Wo > ((int64_t)1 << 40) / K || (int64_t)B * C * H * W > ((int64_t)1 << 40))
+        return FPQ_ERR_SHAPE;
+    if (B == 0)
+        return FPQ_OK;
+    if (!x || !rows)
+        return FPQ_ERR_NULL;
+    if (!aligned(x, 4) || !aligned(rows, 4))
+        return FPQ_ERR_ALIGN;
+    return launch_unfold(x, B, C, H, W, R, S, pad, stride, Ho, Wo, rows, (cudaStream_t)stream);
+}
+
 fpq_status fpq_round_learn_harden(const float* alpha, int64_t N, int64_t K, uint8_t* rounding_bits, void* stream)
 {
     if (N < 0 || K < 0 || (K > 0 && N > (((int64_t)1 << 40) / K)))

@@ -72,6 +72,8 @@ size_t round_learn_workspace_bytes(int64_t M, int64_t N, int64_t K);
 fpq_status launch_round_learn(const float* w, const float* scale, const QFormat& f, float* alpha, const float* a,
                               int64_t M, int64_t N, int64_t K, float reg, float lr, float* grad, double* loss,
                               void* workspace, cudaStream_t st);
+fpq_status launch_unfold(const float* x, int B, int C, int H, int W, int R, int S, int pad, int stride, int Ho, int Wo,
+                         float* rows, cudaStream_t st);
 fpq_status launch_round_harden(const float* alpha, int64_t N, int64_t K, uint8_t* bits, cudaStream_t st);
 
 }  // namespace fpq

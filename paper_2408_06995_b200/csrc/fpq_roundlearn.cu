@@ -11,6 +11,7 @@
 //   sgemm128<false>         partial sums of D^T A over slices of the M rows
 //   grad_finalize_kernel    slices added in a fixed order, chain rule, optional descent update
 //   harden_kernel           the inference rule: decision bit = (sigma(alpha) >= 0.5)
+//   unfold_kernel           a convolution's input rows, so that the same step serves convolution weights
 #include <math.h>
 
 #include "fpq_kernels.h"
@@ -346,6 +347,27 @@ __global__ void __launch_bounds__(256) harden_kernel(const float* __restrict__ a
     }
 }
 
+// Input rows of a convolution written out: row (b, oy, ox), column (c, r, s) in the weight's own [C][R][S]
+// order, zero where the tap falls into the padding.  One thread per output element (writes coalesced).
+__global__ void __launch_bounds__(256) unfold_kernel(const float* __restrict__ x, int C, int H, int W, int R, int S,
+                                                     int pad, int stride, int Ho, int Wo, int64_t total,
+                                                     float* __restrict__ rows)
+{
+    const int64_t K = (int64_t)C * R * S;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t m = i / K;
+        int k = (int)(i - m * K);
+        int s = k % S, r = (k / S) % R, c = k / (S * R);
+        int ox = (int)(m % Wo), oy = (int)((m / Wo) % Ho);
+        int64_t b = m / ((int64_t)Wo * Ho);
+        int iy = oy * stride - pad + r, ix = ox * stride - pad + s;
+        float v = 0.f;
+        if (iy >= 0 && iy < H && ix >= 0 && ix < W)
+            v = __ldg(x + ((b * C + c) * H + iy) * W + ix);
+        rows[i] = v;
+    }
+}
+
 int grid_for(int64_t total)
 {
     int64_t blocks = (total + 255) / 256;
@@ -441,6 +463,16 @@ fpq_status launch_round_harden(const float* alpha, int64_t N, int64_t K, uint8_t
     if (N * row_bytes == 0)
         return FPQ_OK;
     harden_kernel<<<grid_for(N * row_bytes), 256, 0, st>>>(alpha, N, K, row_bytes, bits);
+    return cudaGetLastError() == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
+}
+
+fpq_status launch_unfold(const float* x, int B, int C, int H, int W, int R, int S, int pad, int stride, int Ho, int Wo,
+                         float* rows, cudaStream_t st)
+{
+    int64_t total = (int64_t)B * Ho * Wo * C * R * S;
+    if (total == 0)
+        return FPQ_OK;
+    unfold_kernel<<<grid_for(total), 256, 0, st>>>(x, C, H, W, R, S, pad, stride, Ho, Wo, total, rows);
     return cudaGetLastError() == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
 }
 

@@ -122,3 +122,32 @@ def test_learned_bits_feed_the_weight_encoder():
     codes = fpq.fpq_quantize_weight(wd, sd, fpq.E2M1, bits)
     want = O.quantize_weight(w, scale, O.E2M1, bits.cpu().numpy())
     assert np.array_equal(codes.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("shape", [(2, 3, 7, 6, 3, 3, 1, 1), (1, 4, 8, 8, 3, 3, 1, 2), (3, 130, 9, 11, 1, 1, 0, 1),
+                                   (2, 40, 16, 16, 3, 3, 1, 1), (1, 2, 6, 6, 3, 2, 0, 1)])
+def test_unfold_matches_the_oracle_bit_for_bit(shape):
+    B, C, H, W, R, S, pad, stride = shape
+    rng = np.random.default_rng(sum(shape))
+    x = rng.standard_normal((B, C, H, W)).astype(np.float32)
+    rows = fpq.fpq_round_learn_unfold(torch.from_numpy(x).cuda(), R, S, pad, stride)
+    assert np.array_equal(rows.cpu().numpy(), O.unfold(x, R, S, pad, stride))
+
+
+def test_round_learn_step_for_a_convolution():
+    # 3 x 3 convolution weights [Co][C][3][3] learned against the layer's own input: unfold, then the same step
+    rng = np.random.default_rng(17)
+    B, C, H, W, Co = 2, 24, 12, 12, 40
+    x = rng.standard_normal((B, C, H, W)).astype(np.float32)
+    w = (rng.standard_normal((Co, C * 9)) * 0.03).astype(np.float32)
+    scale = np.array([O.scale_from_max(v, O.E2M1) for v in np.abs(w).max(axis=1)], dtype=np.float32)
+    alpha = (rng.standard_normal(w.shape) * 2).astype(np.float32)
+    d = "cuda"
+    rows = fpq.fpq_round_learn_unfold(torch.from_numpy(x).to(d), 3, 3, 1, 1)
+    grad, loss = fpq.fpq_round_learn_step(torch.from_numpy(w).to(d), torch.from_numpy(scale).to(d), fpq.E2M1,
+                                          torch.from_numpy(alpha).to(d), rows, 0.01)
+    r = O.round_learn_step(w, scale, O.E2M1, alpha, O.unfold(x, 3, 3, 1, 1), 0.01)
+    assert float(loss[0]) == pytest.approx(r["mse"], rel=LOSS_RTOL)
+    tol = 2.0 * GRAD_RTOL_ABSUM * r["absum"] + 1e-5 * 0.01 * np.abs(O.rounding_regularizer(alpha)[1]) + 1e-16 \
+        + 4.0 * np.spacing(np.abs(r["grad"]).astype(np.float32)).astype(np.float64)
+    assert np.all(np.abs(grad.cpu().numpy() - r["grad"]) <= tol)

@@ -143,3 +143,18 @@ def test_gradient_matches_autograd_through_a_grid_neighbour_search():
     assert r["mse"] + reg * r["reg"] == pytest.approx(float(loss.detach()), rel=1e-12)
     np.testing.assert_allclose(r["grad"], al.grad.numpy(), rtol=1e-10, atol=1e-16)
     np.testing.assert_allclose(r["wq"], wq.detach().numpy(), rtol=1e-14, atol=0)
+
+
+@pytest.mark.parametrize("shape", [(2, 3, 7, 6, 3, 3, 1, 1), (1, 4, 8, 8, 3, 3, 1, 2), (2, 5, 5, 9, 1, 1, 0, 1), (1, 2, 6, 6, 3, 2, 0, 1)])
+def test_unfold_is_the_library_unfold_and_turns_the_convolution_into_a_product(shape):
+    B, C, H, W, R, S, pad, stride = shape
+    rng = np.random.default_rng(sum(shape))
+    x = rng.standard_normal((B, C, H, W)).astype(np.float32)
+    rows = O.unfold(x, R, S, pad, stride)
+    lib = torch.nn.functional.unfold(torch.from_numpy(x), (R, S), padding=pad, stride=stride)   # [B][C*R*S][L]
+    assert np.array_equal(rows, lib.permute(0, 2, 1).reshape(rows.shape).numpy())
+    # rows times flattened weights = the convolution
+    w = rng.standard_normal((4, C, R, S)).astype(np.float32)
+    y = torch.nn.functional.conv2d(torch.from_numpy(x).double(), torch.from_numpy(w).double(), padding=pad, stride=stride)
+    got = rows.astype(np.float64) @ w.reshape(4, -1).astype(np.float64).T
+    np.testing.assert_allclose(got, y.permute(0, 2, 3, 1).reshape(got.shape).numpy(), rtol=1e-12, atol=1e-12)
