@@ -384,11 +384,11 @@ struct Plan {
 };
 
 // As many slices of a reduction of length R as still fit into one wave of two resident blocks per SM (one more
-// would add a second, nearly empty wave), each at least 256 long.
+// would add a second, nearly empty wave), each at least 128 long.
 void slice(int64_t tiles, int64_t R, int* splits, int64_t* per)
 {
     int64_t want = (2 * 148) / tiles;
-    int64_t cap = (R + 255) / 256;
+    int64_t cap = (R + 127) / 128;
     int64_t s = want < cap ? want : cap;
     s = s < 1 ? 1 : (s > 64 ? 64 : s);
     *per = round_up((R + s - 1) / s, BK);
