@@ -712,6 +712,52 @@ def run_round_learn(args):
     print(json.dumps(out), flush=True)
 
 
+def run_formats(args):
+    """The weight encodings the search can select, as the same linear layers (SD-v1-style transformer block,
+    M = 8192): read by the tensor cores as they are (E4M3, E2M1), re-encoded exactly into E4M3 when the
+    weights are prepared (E1M2), or run on the CUDA cores with FP32 multiply-adds (E3M4, E2M5, E5M2)."""
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    from paper_2408_06995_b200 import build as fpq_build
+    fpq_build.build()
+    import paper_2408_06995_b200 as fpq
+    shapes = [("qkv_320_960", 8192, 960, 320), ("ffn_out_1280_320", 8192, 320, 1280)]
+    formats = [("e4m3", fpq.E4M3, "tensor cores"), ("e2m1", fpq.E2M1, "tensor cores"),
+               ("e1m2", fpq.E1M2, "tensor cores, weights re-encoded into E4M3"),
+               ("e3m4", fpq.E3M4, "CUDA cores (FP32 multiply-adds)"),
+               ("e2m5", fpq.E2M5, "CUDA cores (FP32 multiply-adds)"),
+               ("e5m2_bias16", fpq.Format(5, 2, 16, fpq.SAT_PAPER), "CUDA cores (FP32 multiply-adds)")]
+    props = torch.cuda.get_device_properties(0)
+    sampler = ClockSampler(physical_gpu_index(0))
+    sampler.start()
+    rows = []
+    for name, M, N, K in shapes:
+        x = torch.randn((M, K), device=dev)
+        xs = float(x.abs().max()) / 448.0
+        w = torch.randn((N, K), device=dev) * 0.02
+        bias = torch.randn(N, device=dev) * 0.01
+        y = torch.empty((M, N), device=dev)
+        for fname, f, route in formats:
+            ws = (w.abs().amax(dim=1) / fpq.fpq_format_max(f)).contiguous()
+            codes = fpq.fpq_quantize_weight(w, ws, f, None)
+            prep = fpq.fpq_prepare_weight(codes, f, fpq.LINEAR, N, K)
+            wk = torch.empty(max(256, fpq.fpq_linear_workspace_size(M, N, K, fpq.E4M3, f)), dtype=torch.uint8, device=dev)
+            t = per_launch_us(torch, lambda: fpq.fpq_linear(x, prep, ws, xs, fpq.E4M3, f, bias, N, y, wk), 10) * 1e-6
+            rows.append({"name": name, "weights": fname, "route": route, "M": M, "N": N, "K": K, "us": t * 1e6,
+                         "tflops": 2.0 * M * N * K / t / 1e12, "weight_bytes": prep.numel()})
+    clocks = sampler.stop()
+    fp32_peak = props.multi_processor_count * 128 * 2 * (clocks["sm_mhz"] or 1965.0) * 1e6
+    for r in rows:
+        if r["route"].startswith("CUDA"):
+            r["roofline"] = {"bound": "alu", "achieved": r["tflops"], "peak": fp32_peak / 1e12, "unit": "TFLOP/s",
+                             "frac": r["tflops"] * 1e12 / fp32_peak,
+                             "peak_source": "SM count x 128 FP32 lanes x 2 flop x sampled SM clock"}
+    print(json.dumps({"suite": "formats", "rows": rows, "clocks": clocks}), flush=True)
+
+
 def run_split(args):
     """The decoder convolutions of the SD-v1-style U-Net whose input is a concatenation (previous
     layer's output + skip connection), W4A8, batch 2: the two-scale call against the ordinary call
@@ -781,7 +827,7 @@ def main():
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline leg")
     ap.add_argument("--skip-w4", action="store_true", help="leave out the W4A8 side measurement")
-    ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd", "sd_trace", "search", "sd_split", "round_learn"],
+    ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd", "sd_trace", "search", "sd_split", "round_learn", "formats"],
                     help="print a per-shape table of a whole workload instead of the headline line")
     ap.add_argument("--only", default=None, help="with --suite ldm|transformer|sd|round_learn: only the layers whose name contains this")
     args = ap.parse_args()
@@ -793,6 +839,8 @@ def main():
         run_split(args)
     elif args.suite == "round_learn":
         run_round_learn(args)
+    elif args.suite == "formats":
+        run_formats(args)
     elif args.suite:
         run_suite(args)
     elif args.impl == "reference":

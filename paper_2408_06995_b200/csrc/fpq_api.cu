@@ -119,6 +119,25 @@ static bool embeds_in_e4m3(fpq_format f, CodeTable* tab)
 static bool weight_native(fpq_format f) { return is_e4m3_native(f) || is_e2m1(f); }
 static bool weight_reencoded(fpq_format f) { return !weight_native(f) && embeds_in_e4m3(f, nullptr); }
 
+// Operand pairs the tensor-core contraction has no type for run on the CUDA cores (fpq_linear and fpq_conv2d
+// only; the staged, host-buffer, two-tensor and built-in-scratch forms keep to the tensor-core pairs).
+static bool general_pair(fpq_format fx, fpq_format fw)
+{
+    QFormat q;
+    if (!resolve_format(fx, &q) || !resolve_format(fw, &q))
+        return false;
+    return !(is_e4m3_native(fx) && (weight_native(fw) || weight_reencoded(fw)));
+}
+
+// Format of the codes in the prepared copy: re-encoded weights are E4M3 there.
+static QFormat prepared_format(fpq_format fw)
+{
+    const fpq_format e4m3 = {4, 3, 7, FPQ_SAT_NATIVE};
+    QFormat q;
+    resolve_format(weight_reencoded(fw) ? e4m3 : fw, &q);
+    return q;
+}
+
 static int g_path_policy = FPQ_PATH_AUTO;
 
 static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
@@ -245,6 +264,13 @@ fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_la
 
 size_t fpq_linear_workspace_size(int64_t M, int64_t N, int64_t K, fpq_format fx, fpq_format fw)
 {
+    if (general_pair(fx, fw)) {
+        if (M < 0 || N < 0 || K < 1 || M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff)
+            return 0;
+        GeneralLayer g = {};
+        g.M = M, g.N = N, g.K = K;
+        return general_layer_workspace_bytes(g);
+    }
     (void)N;
     if (check_pair(fx, fw) != FPQ_OK || M < 0 || K < 0)
         return 0;
@@ -340,6 +366,27 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
                       fpq_format fw, const float* bias, float* y, int64_t M, int64_t N, int64_t K, void* workspace,
                       size_t ws_bytes, void* stream)
 {
+    if (general_pair(fx, fw)) {
+        if (M < 0 || N < 0 || K < 0 || M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff)
+            return FPQ_ERR_SHAPE;
+        if (M == 0 || N == 0)
+            return FPQ_OK;
+        if (K == 0)
+            return FPQ_ERR_SHAPE;
+        GeneralLayer g = {};
+        g.M = M, g.N = N, g.K = K, g.C = (int)K, g.R = 1, g.S = 1, g.Cp = (int)padded_c(K);
+        resolve_format(fx, &g.fx);
+        g.fw = prepared_format(fw);
+        g.x = x, g.w_prepared = w_prepared, g.w_scale = w_scale, g.x_scale = x_scale, g.bias = bias, g.y = y;
+        if (!x || !w_prepared || !w_scale || !y)
+            return FPQ_ERR_NULL;
+        if (!aligned(x, 16) || !aligned(y, 16) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
+            (bias && !aligned(bias, 4)) || !aligned(workspace, 256))
+            return FPQ_ERR_ALIGN;
+        if (!workspace || ws_bytes < general_layer_workspace_bytes(g))
+            return FPQ_ERR_WORKSPACE;
+        return launch_general_layer(g, workspace, (cudaStream_t)stream);
+    }
     bool empty = false;
     fpq_status s = linear_checks(fx, fw, M, N, K, workspace, ws_bytes, &empty);
     if (s != FPQ_OK || empty)
@@ -387,10 +434,35 @@ static fpq_status conv_shape(int B, int C, int H, int W, int C_out, int R, int S
     return FPQ_OK;
 }
 
+// Geometry of a convolution on the CUDA-core route; false if the shape is out of range.
+static bool general_conv(GeneralLayer* g, fpq_format fx, fpq_format fw, int B, int C, int H, int W, int C_out, int R,
+                         int S, int pad, int stride)
+{
+    int Ho, Wo;
+    if (conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo) != FPQ_OK)
+        return false;
+    int64_t K = (int64_t)C * R * S, M = (int64_t)B * Ho * Wo;
+    if (K > 0x7fffffff || M > 0x7fffffff || (K > 0 && M > ((int64_t)1 << 38) / K))
+        return false;
+    g->conv = 1;
+    g->M = M, g->N = C_out, g->K = K;
+    g->B = B, g->C = C, g->H = H, g->W = W, g->R = R, g->S = S, g->pad = pad, g->stride = stride, g->Ho = Ho, g->Wo = Wo;
+    g->Cp = (int)padded_c(C);
+    resolve_format(fx, &g->fx);
+    g->fw = prepared_format(fw);
+    return true;
+}
+
 size_t fpq_conv2d_workspace_size(int B, int C, int H, int W, int C_out, int R, int S, int pad, int stride,
                                  fpq_format fx, fpq_format fw)
 {
     int Ho, Wo;
+    if (general_pair(fx, fw)) {
+        GeneralLayer g = {};
+        if (!general_conv(&g, fx, fw, B, C, H, W, C_out, R, S, pad, stride))
+            return 0;
+        return general_layer_workspace_bytes(g);
+    }
     if (check_pair(fx, fw) != FPQ_OK || conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo) != FPQ_OK)
         return 0;
     return (size_t)B * (H + 2 * pad) * (W + 2 * pad) * (size_t)round_up(C, 16);
@@ -496,6 +568,22 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
                       fpq_format fw, const float* bias, float* y, int B, int C, int H, int W, int C_out, int R, int S,
                       int pad, int stride, void* workspace, size_t ws_bytes, void* stream)
 {
+    if (general_pair(fx, fw)) {
+        GeneralLayer g = {};
+        if (!general_conv(&g, fx, fw, B, C, H, W, C_out, R, S, pad, stride))
+            return FPQ_ERR_SHAPE;
+        if (B == 0 || C_out == 0)
+            return FPQ_OK;
+        g.x = x, g.w_prepared = w_prepared, g.w_scale = w_scale, g.x_scale = x_scale, g.bias = bias, g.y = y;
+        if (!x || !w_prepared || !w_scale || !y)
+            return FPQ_ERR_NULL;
+        if (!aligned(x, 4) || !aligned(y, 4) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
+            (bias && !aligned(bias, 4)) || !aligned(workspace, 256))
+            return FPQ_ERR_ALIGN;
+        if (!workspace || ws_bytes < general_layer_workspace_bytes(g))
+            return FPQ_ERR_WORKSPACE;
+        return launch_general_layer(g, workspace, (cudaStream_t)stream);
+    }
     int Ho, Wo;
     bool empty = false;
     fpq_status s = conv_checks(fx, fw, B, C, H, W, C_out, R, S, pad, stride, workspace, ws_bytes, &Ho, &Wo, &empty);

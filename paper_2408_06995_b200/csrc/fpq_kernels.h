@@ -74,6 +74,27 @@ fpq_status launch_round_learn(const float* w, const float* scale, const QFormat&
                               void* workspace, cudaStream_t st);
 fpq_status launch_unfold(const float* x, int B, int C, int H, int W, int R, int S, int pad, int stride, int Ho, int Wo,
                          float* rows, cudaStream_t st);
+fpq_status launch_sgemm_nt(const float* P, int64_t ldp, const float* Q, int64_t ldq, float* C, int64_t ldc, int64_t I,
+                           int64_t J, int64_t R, cudaStream_t st);
 fpq_status launch_round_harden(const float* alpha, int64_t N, int64_t K, uint8_t* bits, cudaStream_t st);
+
+// Layer on the CUDA cores for operand formats the tensor-core contraction has no type for (any valid pair):
+// activations quantized to their grid values in FP32, weight codes decoded to FP32, FP32 multiply-add
+// contraction (exact products, FP32 sums, as on the tensor cores), dequantize + bias.
+struct GeneralLayer {
+    int conv;                 // 0 linear ([M][K] rows), 1 convolution (NCHW)
+    int64_t M, N, K;          // K = C * R * S for a convolution
+    int B, C, H, W, R, S, pad, stride, Ho, Wo;
+    QFormat fx, fw;           // fw: the format of the codes in the prepared copy
+    int Cp;                   // padded channels of the prepared copy ([N][R*S][Cp])
+    const float* x;
+    const void* w_prepared;
+    const float* w_scale;
+    float x_scale;
+    const float* bias;
+    float* y;
+};
+size_t general_layer_workspace_bytes(const GeneralLayer& g);
+fpq_status launch_general_layer(const GeneralLayer& g, void* workspace, cudaStream_t st);
 
 }  // namespace fpq

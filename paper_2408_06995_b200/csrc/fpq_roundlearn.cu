@@ -466,6 +466,17 @@ fpq_status launch_round_harden(const float* alpha, int64_t N, int64_t K, uint8_t
     return cudaGetLastError() == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
 }
 
+// C[i][j] = sum_r P[i][r] Q[j][r] (both operands with the reduction index contiguous), FP32 multiply-adds.
+fpq_status launch_sgemm_nt(const float* P, int64_t ldp, const float* Q, int64_t ldq, float* C, int64_t ldc, int64_t I,
+                           int64_t J, int64_t R, cudaStream_t st)
+{
+    if (I == 0 || J == 0)
+        return FPQ_OK;
+    dim3 g((unsigned)((I + TILE - 1) / TILE), (unsigned)((J + TILE - 1) / TILE), 1);
+    sgemm128<true><<<g, 256, 0, st>>>(P, ldp, Q, ldq, C, ldc, (int)I, (int)J, R, R, nullptr);
+    return cudaGetLastError() == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
+}
+
 fpq_status launch_unfold(const float* x, int B, int C, int H, int W, int R, int S, int pad, int stride, int Ho, int Wo,
                          float* rows, cudaStream_t st)
 {

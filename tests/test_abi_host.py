@@ -57,10 +57,18 @@ def test_host_side_rejections(L):
     # contraction: operand pairs
     e2m1, e3m4 = fpq.E2M1.c(), fpq.E3M4.c()
     big = ctypes.c_void_p(1024)
-    assert L.fpq_linear(big, big, big, 1.0, e3m4, F, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_UNSUPPORTED
-    assert L.fpq_linear(big, big, big, 1.0, F, e3m4, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_UNSUPPORTED
+    # the staged forms keep to the pairs the tensor cores read
+    assert L.fpq_linear_quantize_input(big, 1.0, e3m4, F, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_UNSUPPORTED
+    assert L.fpq_linear_quantize_input(big, 1.0, F, e3m4, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_UNSUPPORTED
     paper_sat = fpq.Format(4, 3, 7, fpq.SAT_PAPER).c()
-    assert L.fpq_linear(big, big, big, 1.0, paper_sat, F, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_UNSUPPORTED
+    assert L.fpq_linear_quantize_input(big, 1.0, paper_sat, F, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_UNSUPPORTED
+    # fpq_linear / fpq_conv2d take every valid pair (the others on the CUDA cores) and check it like any other
+    assert L.fpq_linear(None, big, big, 1.0, e3m4, F, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_NULL
+    assert L.fpq_linear(big, big, big, 1.0, F, e3m4, None, big, 8, 8, 8, big, 8, None) == fpq.ERR_WORKSPACE
+    assert L.fpq_linear(big, big, big, 1.0, F, e3m4, None, big, 8, 8, 8, ctypes.c_void_p(1152), 1 << 20, None) == fpq.ERR_ALIGN
+    assert L.fpq_linear(big, big, big, 1.0, fpq.Format(6, 3, 7).c(), F, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_FORMAT
+    assert L.fpq_conv2d(big, big, big, 1.0, F, e3m4, None, big, 1, 8, 2, 2, 8, 3, 3, 0, 1, big, 1 << 20, None) == fpq.ERR_SHAPE
+    assert L.fpq_conv2d(big, big, big, 1.0, F, e3m4, None, big, 1, 8, 4, 4, 8, 3, 3, 1, 1, big, 16, None) == fpq.ERR_WORKSPACE
     assert L.fpq_linear(big, big, big, 1.0, F, e2m1, None, big, -1, 8, 8, big, 1 << 20, None) == fpq.ERR_SHAPE
     assert L.fpq_linear(None, big, big, 1.0, F, F, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_NULL
     assert L.fpq_linear(ctypes.c_void_p(1028), big, big, 1.0, F, F, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_ALIGN
@@ -100,7 +108,8 @@ def test_search_host_side(L):
 def test_sizes(L):
     assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E4M3, fpq.E4M3) == 100 * 320
     assert fpq.fpq_linear_workspace_size(100, 64, 321, fpq.E4M3, fpq.E2M1) == 100 * 336
-    assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E3M4, fpq.E4M3) == 0
+    assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E3M4, fpq.E4M3) > 100 * 320     # CUDA-core route: FP32 scratch
+    assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.Format(6, 3, 7), fpq.E4M3) == 0
     assert fpq.fpq_conv2d_workspace_size(2, 4, 8, 8, 16, 3, 3, 1, 1, fpq.E4M3, fpq.E2M1) == 2 * 100 * 16
     assert fpq.fpq_prepared_size(fpq.E4M3, fpq.LINEAR, 10, 320) == 10 * 384
     assert fpq.fpq_prepared_size(fpq.E2M1, fpq.CONV2D, 10, 320, 3, 3) == 10 * 9 * 384 // 2
@@ -125,8 +134,8 @@ def test_weight_formats_the_layer_accepts(L):
     big = ctypes.c_void_p(1024)
 
     def accepted(fw):
-        # a NULL activation pointer is rejected after the operand pair has been checked
-        return L.fpq_linear(None, big, big, 1.0, F, fw.c(), None, big, 8, 8, 8, big, 1 << 20, None) != fpq.ERR_UNSUPPORTED
+        # (by the tensor-core forms) a NULL activation pointer is rejected after the operand pair has been checked
+        return L.fpq_linear_quantize_input(None, 1.0, F, fw.c(), 8, 8, 8, big, 1 << 20, None) != fpq.ERR_UNSUPPORTED
 
     # read by the tensor cores as they are
     assert accepted(fpq.E4M3) and accepted(fpq.E2M1)

@@ -1,0 +1,79 @@
+"""Layers whose operand formats the tensor cores have no type for (E3M4, E2M5, E5M2, the paper's E4M3 with
+all exponent fields finite - what the FP8 encoding search of Sec. V-A may select - or activations in a format
+other than native E4M3): fpq_linear / fpq_conv2d run them on the CUDA cores with the same arithmetic model
+(exact products of grid values, FP32 sums), so the bar is the one of the tensor-core path."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2408_06995_b200 as fpq
+from paper_2408_06995_b200 import inputs as I
+from _helpers import assert_close, to_oracle
+
+pytestmark = pytest.mark.gpu
+
+E4M3_PAPER = fpq.Format(4, 3, 7, fpq.SAT_PAPER)
+E4M3_B8 = fpq.Format(4, 3, 8, fpq.SAT_PAPER)        # the paper's default bias 2^(e-1)
+E5M2_B16 = fpq.Format(5, 2, 16, fpq.SAT_PAPER)
+E2M1_TINY = fpq.Format(2, 1, 12, fpq.SAT_PAPER)      # a 4-bit format whose values E4M3 cannot hold
+
+PAIRS = [(fpq.E4M3, fpq.E3M4), (fpq.E4M3, fpq.E2M5), (fpq.E4M3, fpq.E5M2), (fpq.E4M3, E5M2_B16), (fpq.E4M3, E4M3_PAPER),
+         (fpq.E4M3, E4M3_B8), (fpq.E4M3, E2M1_TINY),
+         (fpq.E5M2, fpq.E4M3), (fpq.E3M4, fpq.E2M1), (E4M3_PAPER, fpq.E1M2), (fpq.E2M5, fpq.E3M4)]
+
+
+def _run(L, gfx, gfw, use_bias=True):
+    ofx, ofw = to_oracle(gfx), to_oracle(gfw)
+    d = "cuda"
+    w2 = L.w.reshape(L.N, -1)
+    ws = np.array([fpq.fpq_scale_from_max(float(v), gfw) for v in np.abs(w2).max(axis=1)], dtype=np.float32)
+    assert np.array_equal(ws, np.array([O.scale_from_max(v, ofw) for v in np.abs(w2).max(axis=1)], dtype=np.float32))
+    xs = fpq.fpq_scale_from_max(float(np.abs(L.x).max()), gfx)
+    assert np.float32(xs) == O.scale_from_max(float(np.abs(L.x).max()), ofx)
+    rb = O.pack_bits(L.bits) if L.bits is not None else None
+    codes = fpq.fpq_quantize_weight(torch.from_numpy(w2).to(d), torch.from_numpy(ws).to(d), gfw,
+                                    None if rb is None else torch.from_numpy(rb).to(d))
+    assert np.array_equal(codes.cpu().numpy(), O.quantize_weight(w2, ws, ofw, rb))
+    x = torch.from_numpy(L.x).to(d)
+    bias = torch.from_numpy(L.bias).to(d) if use_bias else None
+    wsd = torch.from_numpy(ws).to(d)
+    if L.kind == "linear":
+        prep = fpq.fpq_prepare_weight(codes, gfw, fpq.LINEAR, L.N, L.K)
+        y = fpq.fpq_linear(x, prep, wsd, xs, gfx, gfw, bias, L.N)
+        yr, ab = O.linear(L.x, L.w, ws, xs, ofx, ofw, L.bias if use_bias else None, rb)
+    else:
+        prep = fpq.fpq_prepare_weight(codes, gfw, fpq.CONV2D, L.N, L.C, L.R, L.S)
+        y = fpq.fpq_conv2d(x, prep, wsd, xs, gfx, gfw, bias, L.N, L.R, L.S, L.pad, L.stride)
+        yr, ab = O.conv2d(L.x, L.w, ws, xs, ofx, ofw, L.bias if use_bias else None, rb, L.pad, L.stride)
+    assert fpq.fpq_read_status() == fpq.OK
+    y = y.cpu().numpy()
+    assert y.shape == yr.shape
+    return assert_close(y, yr, ab)
+
+
+@pytest.mark.parametrize("gfx,gfw", PAIRS)
+@pytest.mark.parametrize("M,K,N", [(130, 200, 72), (300, 320, 260), (2, 129, 5)])
+def test_linear(gfx, gfw, M, K, N):
+    L = I.linear_layer("t", M, K, N, rounding=(M == 130))
+    I.draw(L, 31, M + K + N, "normal", 0.02, True, 0.01, (0.001, 20.0))
+    _run(L, gfx, gfw)
+    _run(L, gfx, gfw, use_bias=False)
+
+
+@pytest.mark.parametrize("gfx,gfw", [(fpq.E4M3, fpq.E3M4), (fpq.E4M3, E5M2_B16), (fpq.E4M3, E4M3_B8), (fpq.E5M2, fpq.E2M1),
+                                     (fpq.E3M4, fpq.E1M2)])
+@pytest.mark.parametrize("shape", [(2, 40, 12, 12, 72, 3, 1), (1, 130, 9, 11, 33, 3, 2), (3, 64, 8, 8, 130, 1, 1)])
+def test_conv(gfx, gfw, shape):
+    B, C, H, W, Co, R, stride = shape
+    L = I.conv_layer("t", B, C, H, W, Co, R, stride=stride, rounding=(stride == 2))
+    I.draw(L, 32, B + C + Co, "silu", 0.03, True, 0.01)
+    _run(L, gfx, gfw)
+
+
+def test_every_fp8_search_candidate_runs_as_a_layer():
+    # the four FP8 encodings of Algorithm 1 with the paper's default bias, as weight formats of one layer
+    L = I.linear_layer("t", 96, 256, 64)
+    I.draw(L, 33, 0, "normal", 0.02, True, 0.01)
+    for enc in O.FP8_ENCODINGS:
+        _run(L, fpq.E4M3, fpq.Format(enc.e, enc.m, enc.B, fpq.SAT_PAPER))
