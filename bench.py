@@ -715,7 +715,8 @@ def run_round_learn(args):
 def run_formats(args):
     """The weight encodings the search can select, as the same linear layers (SD-v1-style transformer block,
     M = 8192): read by the tensor cores as they are (E4M3, E2M1), re-encoded exactly into E4M3 when the
-    weights are prepared (E1M2), or run on the CUDA cores with FP32 multiply-adds (E3M4, E2M5, E5M2)."""
+    weights are prepared (E1M2), prepared as the sum of two E4M3 terms and contracted over twice the
+    reduction length (E3M4, E2M5), or run on the CUDA cores with FP32 multiply-adds (E5M2)."""
     import torch
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device")
@@ -727,8 +728,9 @@ def run_formats(args):
     shapes = [("qkv_320_960", 8192, 960, 320), ("ffn_out_1280_320", 8192, 320, 1280)]
     formats = [("e4m3", fpq.E4M3, "tensor cores"), ("e2m1", fpq.E2M1, "tensor cores"),
                ("e1m2", fpq.E1M2, "tensor cores, weights re-encoded into E4M3"),
-               ("e3m4", fpq.E3M4, "CUDA cores (FP32 multiply-adds)"),
-               ("e2m5", fpq.E2M5, "CUDA cores (FP32 multiply-adds)"),
+               ("e3m4", fpq.E3M4, "tensor cores, weights prepared as two E4M3 terms"),
+               ("e2m5", fpq.E2M5, "tensor cores, weights prepared as two E4M3 terms"),
+               ("e4m3_all_finite", fpq.Format(4, 3, 7, fpq.SAT_PAPER), "tensor cores, weights prepared as two E4M3 terms"),
                ("e5m2_bias16", fpq.Format(5, 2, 16, fpq.SAT_PAPER), "CUDA cores (FP32 multiply-adds)")]
     props = torch.cuda.get_device_properties(0)
     sampler = ClockSampler(physical_gpu_index(0))

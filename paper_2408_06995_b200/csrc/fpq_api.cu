@@ -115,9 +115,55 @@ static bool embeds_in_e4m3(fpq_format f, CodeTable* tab)
     return true;
 }
 
-// Weight formats the contraction reads as they are, and formats re-encoded when the weights are prepared.
+// Exact split of a weight format into two E4M3 terms: true when every value v of f is first + second with
+// first = the largest E4M3 magnitude not above |v| (sign of v) and second = v - first also a finite E4M3
+// value (formats with up to 7 significant bits inside E4M3's exponent range: E3M4, E2M5, the paper's E4M3
+// with its code for 480 = 448 + 32).  Tables: code of f -> E4M3 code of each term.
+static bool splits_in_two_e4m3(fpq_format f, CodeTable* first, CodeTable* second)
+{
+    QFormat q;
+    if (!resolve_format(f, &q))
+        return false;
+    const fpq_format e4m3 = {4, 3, 7, FPQ_SAT_NATIVE};
+    int ncodes = 1 << (1 + f.exp_bits + f.man_bits);
+    int mag_mask = (1 << (f.exp_bits + f.man_bits)) - 1;
+    for (int c = 0; c < 256; ++c) {
+        uint8_t o1 = 0, o2 = 0;
+        if (c < ncodes && (c & mag_mask) <= q.code_max) {
+            double v = code_value(c, f), a = fabs(v);
+            if (a != 0.0) {
+                int k1 = 0;                               // E4M3 magnitudes increase with the code
+                for (int k = 1; k <= 0x7E; ++k)
+                    if (code_value(k, e4m3) <= a)
+                        k1 = k;
+                double rest = a - code_value(k1, e4m3);
+                int k2 = rest == 0.0 ? 0 : -1;
+                for (int k = 1; k <= 0x7E && k2 < 0; ++k)
+                    if (code_value(k, e4m3) == rest)
+                        k2 = k;
+                if (k2 < 0)
+                    return false;
+                uint8_t sign = v < 0.0 ? 0x80 : 0;
+                o1 = (uint8_t)(k1 ? (k1 | sign) : 0);
+                o2 = (uint8_t)(k2 ? (k2 | sign) : 0);
+            }
+        }
+        if (first)
+            first->t[c] = o1;
+        if (second)
+            second->t[c] = o2;
+    }
+    return true;
+}
+
+// Weight formats the contraction reads as they are, formats re-encoded when the weights are prepared, and
+// formats prepared as two E4M3 terms (twice the reduction length on the tensor cores).
 static bool weight_native(fpq_format f) { return is_e4m3_native(f) || is_e2m1(f); }
 static bool weight_reencoded(fpq_format f) { return !weight_native(f) && embeds_in_e4m3(f, nullptr); }
+static bool weight_two_term(fpq_format f)
+{
+    return !weight_native(f) && !embeds_in_e4m3(f, nullptr) && splits_in_two_e4m3(f, nullptr, nullptr);
+}
 
 // Operand pairs the tensor-core contraction has no type for run on the CUDA cores (fpq_linear and fpq_conv2d
 // only; the staged, host-buffer, two-tensor and built-in-scratch forms keep to the tensor-core pairs).
@@ -126,7 +172,13 @@ static bool general_pair(fpq_format fx, fpq_format fw)
     QFormat q;
     if (!resolve_format(fx, &q) || !resolve_format(fw, &q))
         return false;
-    return !(is_e4m3_native(fx) && (weight_native(fw) || weight_reencoded(fw)));
+    return !(is_e4m3_native(fx) && (weight_native(fw) || weight_reencoded(fw) || weight_two_term(fw)));
+}
+
+static bool two_term_pair(fpq_format fx, fpq_format fw)
+{
+    QFormat q;
+    return resolve_format(fx, &q) && resolve_format(fw, &q) && is_e4m3_native(fx) && weight_two_term(fw);
 }
 
 // Format of the codes in the prepared copy: re-encoded weights are E4M3 there.
@@ -134,9 +186,11 @@ static QFormat prepared_format(fpq_format fw)
 {
     const fpq_format e4m3 = {4, 3, 7, FPQ_SAT_NATIVE};
     QFormat q;
-    resolve_format(weight_reencoded(fw) ? e4m3 : fw, &q);
+    resolve_format((weight_reencoded(fw) || weight_two_term(fw)) ? e4m3 : fw, &q);
     return q;
 }
+
+static const fpq_format kE4M3Native = {4, 3, 7, FPQ_SAT_NATIVE};
 
 static int g_path_policy = FPQ_PATH_AUTO;
 
@@ -238,6 +292,8 @@ size_t fpq_prepared_size(fpq_format fmt, const fpq_layer_desc* d)
     if (!resolve_format(fmt, &q) || check_desc(d) != FPQ_OK)
         return 0;
     size_t elems = (size_t)d->N * d->R * d->S * (size_t)padded_c(d->C);
+    if (weight_two_term(fmt))
+        return 2 * elems;
     return (q.four_bit && !weight_reencoded(fmt)) ? elems / 2 : elems;
 }
 
@@ -254,10 +310,15 @@ fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_la
         return FPQ_ERR_NULL;
     if (!aligned(prepared, 128))
         return FPQ_ERR_ALIGN;
-    CodeTable tab;
+    CodeTable tab, tab2;
+    if (weight_two_term(fmt) && splits_in_two_e4m3(fmt, &tab, &tab2))
+        return launch_prepare_weight(codes, d->N, d->C, d->R * d->S, 2 * (int)padded_c(d->C), q.four_bit, 0, 0, &tab,
+                                     &tab2, (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
+                   ? FPQ_OK
+                   : FPQ_ERR_CUDA;
     const bool re = weight_reencoded(fmt) && embeds_in_e4m3(fmt, &tab);
     return launch_prepare_weight(codes, d->N, d->C, d->R * d->S, (int)padded_c(d->C), q.four_bit, 0, 0,
-                                 re ? &tab : nullptr, (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
+                                 re ? &tab : nullptr, nullptr, (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
                ? FPQ_OK
                : FPQ_ERR_CUDA;
 }
@@ -271,6 +332,8 @@ size_t fpq_linear_workspace_size(int64_t M, int64_t N, int64_t K, fpq_format fx,
         g.M = M, g.N = N, g.K = K;
         return general_layer_workspace_bytes(g);
     }
+    if (two_term_pair(fx, fw))
+        return (M < 0 || K < 0 || K > 0x3fffffff) ? 0 : (size_t)(M * 2 * padded_c(K));
     (void)N;
     if (check_pair(fx, fw) != FPQ_OK || M < 0 || K < 0)
         return 0;
@@ -377,6 +440,7 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
         g.M = M, g.N = N, g.K = K, g.C = (int)K, g.R = 1, g.S = 1, g.Cp = (int)padded_c(K);
         resolve_format(fx, &g.fx);
         g.fw = prepared_format(fw);
+        g.w_two_term = weight_two_term(fw) ? 1 : 0;
         g.x = x, g.w_prepared = w_prepared, g.w_scale = w_scale, g.x_scale = x_scale, g.bias = bias, g.y = y;
         if (!x || !w_prepared || !w_scale || !y)
             return FPQ_ERR_NULL;
@@ -386,6 +450,31 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
         if (!workspace || ws_bytes < general_layer_workspace_bytes(g))
             return FPQ_ERR_WORKSPACE;
         return launch_general_layer(g, workspace, (cudaStream_t)stream);
+    }
+    if (two_term_pair(fx, fw)) {
+        // weights prepared as two E4M3 terms: activation codes written twice per row, then the ordinary
+        // contraction over twice the (padded) reduction length
+        if (K < 0 || K > 0x3fffffff)
+            return FPQ_ERR_SHAPE;
+        const int64_t K2 = 2 * padded_c(K);
+        bool empty = false;
+        fpq_status s = linear_checks(fx, kE4M3Native, M, N, K2, workspace, ws_bytes, &empty);
+        if (s != FPQ_OK || empty)
+            return s;
+        if (K == 0)
+            return FPQ_ERR_SHAPE;
+        if (!x || !w_prepared || !w_scale || !y)
+            return FPQ_ERR_NULL;
+        if (!aligned(x, 16) || !aligned(y, 16) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
+            (bias && !aligned(bias, 4)))
+            return FPQ_ERR_ALIGN;
+        if (!status_word())
+            return FPQ_ERR_CUDA;
+        if (launch_quantize_rows_e4m3_twice(x, M, K, K2 / 2, x_scale, (uint8_t*)workspace, (cudaStream_t)stream) !=
+            cudaSuccess)
+            return FPQ_ERR_CUDA;
+        return linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, kE4M3Native, bias, y, M, N, K2,
+                                    stream, 1, nullptr);
     }
     bool empty = false;
     fpq_status s = linear_checks(fx, fw, M, N, K, workspace, ws_bytes, &empty);
@@ -450,6 +539,7 @@ static bool general_conv(GeneralLayer* g, fpq_format fx, fpq_format fw, int B, i
     g->Cp = (int)padded_c(C);
     resolve_format(fx, &g->fx);
     g->fw = prepared_format(fw);
+    g->w_two_term = weight_two_term(fw) ? 1 : 0;
     return true;
 }
 
@@ -462,6 +552,11 @@ size_t fpq_conv2d_workspace_size(int B, int C, int H, int W, int C_out, int R, i
         if (!general_conv(&g, fx, fw, B, C, H, W, C_out, R, S, pad, stride))
             return 0;
         return general_layer_workspace_bytes(g);
+    }
+    if (two_term_pair(fx, fw)) {
+        if (conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo) != FPQ_OK)
+            return 0;
+        return (size_t)B * (H + 2 * pad) * (W + 2 * pad) * (size_t)(2 * padded_c(C));
     }
     if (check_pair(fx, fw) != FPQ_OK || conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo) != FPQ_OK)
         return 0;
@@ -584,6 +679,34 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
             return FPQ_ERR_WORKSPACE;
         return launch_general_layer(g, workspace, (cudaStream_t)stream);
     }
+    if (two_term_pair(fx, fw)) {
+        // weights prepared as two E4M3 terms per tap: the activation codes fill two channel ranges of the
+        // framed channels-last scratch, then the ordinary convolution over 2 * (padded C) channels
+        if (C < 1 || C > 0x3fffffff / 2)
+            return FPQ_ERR_SHAPE;
+        const int Cp = (int)padded_c(C), C2 = 2 * Cp;
+        int Ho2, Wo2;
+        bool empty2 = false;
+        fpq_status s2 = conv_checks(fx, kE4M3Native, B, C2, H, W, C_out, R, S, pad, stride, workspace, ws_bytes, &Ho2, &Wo2,
+                                    &empty2);
+        if (s2 != FPQ_OK || empty2)
+            return s2;
+        if (!x || !w_prepared || !w_scale || !y)
+            return FPQ_ERR_NULL;
+        if (!aligned(x, 4) || !aligned(y, 4) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
+            (bias && !aligned(bias, 4)))
+            return FPQ_ERR_ALIGN;
+        if (!status_word())
+            return FPQ_ERR_CUDA;
+        cudaStream_t st = (cudaStream_t)stream;
+        if (launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H, W, pad, Cp, C2, 0, x_scale, (uint8_t*)workspace, st) !=
+                cudaSuccess ||
+            launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H, W, pad, Cp, C2, Cp, x_scale, (uint8_t*)workspace, st) !=
+                cudaSuccess)
+            return FPQ_ERR_CUDA;
+        return conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, kE4M3Native, bias, y, B, C2, H, W,
+                                    C_out, R, S, pad, stride, stream, 1, nullptr);
+    }
     int Ho, Wo;
     bool empty = false;
     fpq_status s = conv_checks(fx, fw, B, C, H, W, C_out, R, S, pad, stride, workspace, ws_bytes, &Ho, &Wo, &empty);
@@ -649,7 +772,7 @@ fpq_status fpq_prepare_weight_split(const uint8_t* codes, fpq_format fmt, int32_
     CodeTable tab;
     const bool re = weight_reencoded(fmt) && embeds_in_e4m3(fmt, &tab);
     return launch_prepare_weight(codes, N, C1 + C2, R * S, (int)(padded_c(C1) + padded_c(C2)), q.four_bit, C1,
-                                 (int)padded_c(C1), re ? &tab : nullptr, (uint8_t*)prepared,
+                                 (int)padded_c(C1), re ? &tab : nullptr, nullptr, (uint8_t*)prepared,
                                  (cudaStream_t)stream) == cudaSuccess
                ? FPQ_OK
                : FPQ_ERR_CUDA;

@@ -40,14 +40,21 @@ __global__ void __launch_bounds__(256) quantize_values_kernel(const float* __res
 
 // prepared [N][RS][Cp] (one byte per code, or two codes per byte, even index in the low nibble) ->
 // values [N][C*RS] with column c * RS + tap, the order of the boundary's [C][R][S] weights.
+// two_term: a prepared row holds [first terms | second terms], Cp bytes each, and a weight is their sum (exact).
 __global__ void __launch_bounds__(256) decode_prepared_kernel(const uint8_t* __restrict__ prepared, int64_t N, int C,
-                                                              int RS, int Cp, QFormat f, float* __restrict__ wv)
+                                                              int RS, int Cp, QFormat f, int two_term,
+                                                              float* __restrict__ wv)
 {
     const int64_t K = (int64_t)C * RS, total = N * K;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         int64_t n = i / K;
         int k = (int)(i - n * K);
         int c = k / RS, tap = k - c * RS;
+        if (two_term) {
+            int64_t e1 = (n * RS + tap) * (2 * (int64_t)Cp) + c;
+            wv[i] = decode_code(__ldg(prepared + e1), f) + decode_code(__ldg(prepared + e1 + Cp), f);
+            continue;
+        }
         int64_t e = (n * RS + tap) * Cp + c;
         uint32_t code;
         if (f.four_bit) {
@@ -128,7 +135,7 @@ fpq_status launch_general_layer(const GeneralLayer& g, void* workspace, cudaStre
         return FPQ_ERR_CUDA;
     quantize_values_kernel<<<grid_for(p.n_x), 256, 0, st>>>(g.x, p.n_x, g.x_scale, g.fx, xv, status);
     decode_prepared_kernel<<<grid_for(g.N * g.K), 256, 0, st>>>((const uint8_t*)g.w_prepared, g.N, g.C, g.R * g.S, g.Cp,
-                                                               g.fw, wv);
+                                                               g.fw, g.w_two_term, wv);
     const float* a = xv;
     if (g.conv) {
         fpq_status s = launch_unfold(xv, g.B, g.C, g.H, g.W, g.R, g.S, g.pad, g.stride, g.Ho, g.Wo, rows, st);

@@ -21,9 +21,12 @@ cudaError_t launch_zero_census(const uint8_t* codes, int64_t n, int four_bit, un
 struct CodeTable {
     uint8_t t[256];
 };
-// table != NULL: every code is looked up and the prepared copy holds one byte per weight.
+// table != NULL: every code is looked up and the prepared copy holds one byte per weight.  table2 != NULL as
+// well: Cp counts two halves per row, the first filled through table, the second through table2.
 cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, int C1, int C1p,
-                                  const CodeTable* table, uint8_t* prepared, cudaStream_t st);
+                                  const CodeTable* table, const CodeTable* table2, uint8_t* prepared, cudaStream_t st);
+cudaError_t launch_quantize_rows_e4m3_twice(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, uint8_t* codes,
+                                            cudaStream_t st);
 
 // Geometry of one contraction launch (linear: taps = 1, rows of Ca codes).
 struct GemmProblem {
@@ -87,6 +90,7 @@ struct GeneralLayer {
     int B, C, H, W, R, S, pad, stride, Ho, Wo;
     QFormat fx, fw;           // fw: the format of the codes in the prepared copy
     int Cp;                   // padded channels of the prepared copy ([N][R*S][Cp])
+    int w_two_term;           // the prepared copy holds two E4M3 terms per weight ([N][R*S][2 Cp])
     const float* x;
     const void* w_prepared;
     const float* w_scale;

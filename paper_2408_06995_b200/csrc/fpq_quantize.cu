@@ -129,6 +129,9 @@ __global__ void __launch_bounds__(256) quantize_weight_kernel(const float* __res
 // Row-major activations [M][K] FP32 -> codes [M][Kp] (Kp = K rounded up to 16, pad = 0),
 // the A operand of the linear contraction.  16 elements per thread.
 // ---------------------------------------------------------------------------------
+// TWICE: every row is written two times side by side, [M][2 Kp] (Kp a multiple of 128), for weights that
+// are the sum of two E4M3 terms: the reduction then runs over (x | x) against (first terms | second terms).
+template <bool TWICE>
 __global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const float* __restrict__ x, int64_t M, int64_t K,
                                                                  int64_t Kp, float rinv, uint8_t* __restrict__ codes,
                                                                  int* status)
@@ -159,7 +162,13 @@ __global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const float* __
             out[j] = e4m3x4_from_scaled(__fmul_rn(a0, rinv), __fmul_rn(a1, rinv), __fmul_rn(a2, rinv),
                                         __fmul_rn(a3, rinv), nan);
         }
-        reinterpret_cast<uint4*>(codes)[v] = make_uint4(out[0], out[1], out[2], out[3]);
+        if (TWICE) {
+            int64_t o = row * 2 * vec_per_row + v % vec_per_row;
+            reinterpret_cast<uint4*>(codes)[o] = make_uint4(out[0], out[1], out[2], out[3]);
+            reinterpret_cast<uint4*>(codes)[o + vec_per_row] = make_uint4(out[0], out[1], out[2], out[3]);
+        } else {
+            reinterpret_cast<uint4*>(codes)[v] = make_uint4(out[0], out[1], out[2], out[3]);
+        }
     }
     if (nan)
         atomicMin(status, FPQ_ERR_NAN_INPUT);
@@ -257,10 +266,13 @@ __global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const f
 // ---------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) prepare_weight_kernel(const uint8_t* __restrict__ codes, int N, int C, int RS,
                                                              int Cp, int in_four_bit, int use_table, CodeTable table,
-                                                             int C1, int C1p, uint8_t* __restrict__ prepared)
+                                                             int two_term, CodeTable table2, int C1, int C1p,
+                                                             uint8_t* __restrict__ prepared)
 {
-    __shared__ uint8_t s_tab[256];
+    // two_term: a row holds the channels twice, [first terms | second terms], Cp / 2 positions each
+    __shared__ uint8_t s_tab[256], s_tab2[256];
     s_tab[threadIdx.x] = table.t[threadIdx.x];
+    s_tab2[threadIdx.x] = table2.t[threadIdx.x];
     __syncthreads();
     const int four_bit = in_four_bit && !use_table;      // layout of the prepared copy
     int64_t row_out = four_bit ? (int64_t)RS * Cp / 2 : (int64_t)RS * Cp;
@@ -276,6 +288,11 @@ __global__ void __launch_bounds__(256) prepare_weight_kernel(const uint8_t* __re
             int64_t e = within * per + q;       // element index in [RS][Cp]
             int tap = (int)(e / Cp), c = (int)(e % Cp);
             uint32_t code = 0;
+            bool second = false;
+            if (two_term && c >= Cp / 2) {
+                second = true;
+                c -= Cp / 2;
+            }
             bool real = c < C;
             if (C1 > 0) {
                 real = c < C1 || (c >= C1p && c - C1p + C1 < C);
@@ -291,7 +308,7 @@ __global__ void __launch_bounds__(256) prepare_weight_kernel(const uint8_t* __re
                     code = __ldg(codes + n * row_in + k);
                 }
                 if (use_table)
-                    code = s_tab[code];
+                    code = second ? s_tab2[code] : s_tab[code];
             }
             outb |= code << (4 * q * four_bit);
         }
@@ -342,7 +359,17 @@ cudaError_t launch_quantize_rows_e4m3(const float* x, int64_t M, int64_t K, int6
                                       cudaStream_t st)
 {
     int64_t total = M * (Kp / 16);
-    quantize_rows_e4m3_kernel<<<grid_for(total, 256), 256, 0, st>>>(x, M, K, Kp, 1.0f / scale, codes, status_word());
+    quantize_rows_e4m3_kernel<false><<<grid_for(total, 256), 256, 0, st>>>(x, M, K, Kp, 1.0f / scale, codes,
+                                                                          status_word());
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_rows_e4m3_twice(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, uint8_t* codes,
+                                            cudaStream_t st)
+{
+    int64_t total = M * (Kp / 16);
+    quantize_rows_e4m3_kernel<true><<<grid_for(total, 256), 256, 0, st>>>(x, M, K, Kp, 1.0f / scale, codes,
+                                                                         status_word());
     return cudaGetLastError();
 }
 
@@ -420,14 +447,16 @@ cudaError_t launch_zero_census(const uint8_t* codes, int64_t n, int four_bit, un
 }
 
 cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, int C1, int C1p,
-                                  const CodeTable* table, uint8_t* prepared, cudaStream_t st)
+                                  const CodeTable* table, const CodeTable* table2, uint8_t* prepared, cudaStream_t st)
 {
     int64_t total = (int64_t)N * RS * Cp / ((four_bit && !table) ? 2 : 1);
-    CodeTable tab = {};
+    CodeTable tab = {}, tab2 = {};
     if (table)
         tab = *table;
-    prepare_weight_kernel<<<grid_for(total, 256), 256, 0, st>>>(codes, N, C, RS, Cp, four_bit, table ? 1 : 0, tab, C1, C1p,
-                                                                prepared);
+    if (table2)
+        tab2 = *table2;
+    prepare_weight_kernel<<<grid_for(total, 256), 256, 0, st>>>(codes, N, C, RS, Cp, four_bit, table ? 1 : 0, tab,
+                                                                table2 ? 1 : 0, tab2, C1, C1p, prepared);
     return cudaGetLastError();
 }
 

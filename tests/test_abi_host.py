@@ -65,7 +65,8 @@ def test_host_side_rejections(L):
     # fpq_linear / fpq_conv2d take every valid pair (the others on the CUDA cores) and check it like any other
     assert L.fpq_linear(None, big, big, 1.0, e3m4, F, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_NULL
     assert L.fpq_linear(big, big, big, 1.0, F, e3m4, None, big, 8, 8, 8, big, 8, None) == fpq.ERR_WORKSPACE
-    assert L.fpq_linear(big, big, big, 1.0, F, e3m4, None, big, 8, 8, 8, ctypes.c_void_p(1152), 1 << 20, None) == fpq.ERR_ALIGN
+    assert L.fpq_linear(big, big, big, 1.0, F, e3m4, None, big, 8, 8, 8, ctypes.c_void_p(1032), 1 << 20, None) == fpq.ERR_ALIGN
+    assert L.fpq_linear(big, big, big, 1.0, e3m4, F, None, big, 8, 8, 8, ctypes.c_void_p(1152), 1 << 20, None) == fpq.ERR_ALIGN
     assert L.fpq_linear(big, big, big, 1.0, fpq.Format(6, 3, 7).c(), F, None, big, 8, 8, 8, big, 1 << 20, None) == fpq.ERR_FORMAT
     assert L.fpq_conv2d(big, big, big, 1.0, F, e3m4, None, big, 1, 8, 2, 2, 8, 3, 3, 0, 1, big, 1 << 20, None) == fpq.ERR_SHAPE
     assert L.fpq_conv2d(big, big, big, 1.0, F, e3m4, None, big, 1, 8, 4, 4, 8, 3, 3, 1, 1, big, 16, None) == fpq.ERR_WORKSPACE
@@ -144,7 +145,11 @@ def test_weight_formats_the_layer_accepts(L):
     # more mantissa bits or a wider exponent range than E4M3 holds, or the code 480 of the paper's E4M3
     assert not accepted(fpq.E3M4) and not accepted(fpq.E2M5) and not accepted(fpq.E5M2)
     assert not accepted(fpq.Format(4, 3, 7, fpq.SAT_PAPER)) and not accepted(fpq.Format(4, 3, 8, fpq.SAT_NATIVE))
+    # E3M4 / E2M5 weights are prepared as two E4M3 terms: twice the bytes, twice the activation codes
     d = fpq._CLayerDesc(fpq.LINEAR, 8, 200, 1, 1)
+    assert L.fpq_prepared_size(fpq.E3M4.c(), ctypes.byref(d)) == 2 * 8 * 256
+    assert L.fpq_prepared_size(fpq.E5M2.c(), ctypes.byref(d)) == 8 * 256       # CUDA-core route: codes as they are
+    assert fpq.fpq_linear_workspace_size(100, 64, 200, fpq.E4M3, fpq.E2M5) == 100 * 512
     assert L.fpq_prepared_size(fpq.E2M1.c(), ctypes.byref(d)) == 8 * 256 // 2
     assert L.fpq_prepared_size(fpq.E1M2.c(), ctypes.byref(d)) == 8 * 256      # one E4M3 byte per weight
     assert L.fpq_prepared_size(fpq.E4M3.c(), ctypes.byref(d)) == 8 * 256
