@@ -730,7 +730,7 @@ def run_formats(args):
                ("e1m2", fpq.E1M2, "tensor cores, weights re-encoded into E4M3"),
                ("e3m4", fpq.E3M4, "tensor cores, weights prepared as two E4M3 terms"),
                ("e2m5", fpq.E2M5, "tensor cores, weights prepared as two E4M3 terms"),
-               ("e4m3_all_finite", fpq.Format(4, 3, 7, fpq.SAT_PAPER), "tensor cores, weights prepared as two E4M3 terms"),
+               ("e4m3_bias8", fpq.Format(4, 3, 8, fpq.SAT_PAPER), "tensor cores, weights prepared as two E4M3 terms"),
                ("e5m2_bias16", fpq.Format(5, 2, 16, fpq.SAT_PAPER), "CUDA cores (FP32 multiply-adds)")]
     props = torch.cuda.get_device_properties(0)
     sampler = ClockSampler(physical_gpu_index(0))

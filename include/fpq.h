@@ -126,11 +126,12 @@ fpq_status fpq_quantize_act(const float* x, int64_t n, float scale, fpq_format f
  * E2M1 with bias 2, small formats such as E3M2 bias 3 or E2M3 bias 1 - is re-encoded here,
  * exactly, into one E4M3 byte per weight.  A format whose every value is the sum of two finite
  * E4M3 values (the largest E4M3 magnitude not above it, and the rest: E3M4 bias 4, E2M5 bias 2,
- * E4M3 bias 7 with all exponent fields finite, where 480 = 448 + 32) is prepared as those two
- * terms, two bytes per weight ([N][R*S][2 C_pad]); fpq_linear / fpq_conv2d then contract over
- * twice the reduction length on the tensor cores - exact products, FP32 sums, as for one term.
- * Every other format (E5M2, whose exponent range E4M3 cannot hold; E4M3 with bias 8, whose
- * smallest subnormals it cannot hold) is copied unchanged and runs on the CUDA cores.
+ * E4M3 bias 7 with all exponent fields finite, where 480 = 448 + 32; and, after a factor 2^k that
+ * the layer's dequantization takes back exactly, formats such as the paper's default E4M3 with
+ * bias 8) is prepared as those two terms, two bytes per weight ([N][R*S][2 C_pad]); fpq_linear /
+ * fpq_conv2d then contract over twice the reduction length on the tensor cores - exact products,
+ * FP32 sums, as for one term.  Every other format (E5M2, whose exponent range is twice that of
+ * E4M3) is copied unchanged and runs on the CUDA cores.
  */
 size_t fpq_prepared_size(fpq_format fmt, const fpq_layer_desc* d);
 fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_layer_desc* d,

@@ -119,7 +119,7 @@ static bool embeds_in_e4m3(fpq_format f, CodeTable* tab)
 // first = the largest E4M3 magnitude not above |v| (sign of v) and second = v - first also a finite E4M3
 // value (formats with up to 7 significant bits inside E4M3's exponent range: E3M4, E2M5, the paper's E4M3
 // with its code for 480 = 448 + 32).  Tables: code of f -> E4M3 code of each term.
-static bool splits_in_two_e4m3(fpq_format f, CodeTable* first, CodeTable* second)
+static bool splits_in_two_e4m3_at(fpq_format f, int shift, CodeTable* first, CodeTable* second)
 {
     QFormat q;
     if (!resolve_format(f, &q))
@@ -130,7 +130,7 @@ static bool splits_in_two_e4m3(fpq_format f, CodeTable* first, CodeTable* second
     for (int c = 0; c < 256; ++c) {
         uint8_t o1 = 0, o2 = 0;
         if (c < ncodes && (c & mag_mask) <= q.code_max) {
-            double v = code_value(c, f), a = fabs(v);
+            double v = ldexp(code_value(c, f), shift), a = fabs(v);
             if (a != 0.0) {
                 int k1 = 0;                               // E4M3 magnitudes increase with the code
                 for (int k = 1; k <= 0x7E; ++k)
@@ -156,13 +156,28 @@ static bool splits_in_two_e4m3(fpq_format f, CodeTable* first, CodeTable* second
     return true;
 }
 
+// The terms are those of 2^shift * v for the smallest |shift| <= 16 that works (0 first): a format whose bias
+// puts it outside E4M3's range (the paper's default E4M3 with bias 8: shift 1) still splits, and the layer
+// multiplies the dequantization scale by 2^-shift, which is exact.
+static bool splits_in_two_e4m3(fpq_format f, CodeTable* first, CodeTable* second, int* shift)
+{
+    for (int m = 0; m <= 16; ++m)
+        for (int sgn = 1; sgn >= (m ? -1 : 1); sgn -= 2)
+            if (splits_in_two_e4m3_at(f, sgn * m, first, second)) {
+                if (shift)
+                    *shift = sgn * m;
+                return true;
+            }
+    return false;
+}
+
 // Weight formats the contraction reads as they are, formats re-encoded when the weights are prepared, and
 // formats prepared as two E4M3 terms (twice the reduction length on the tensor cores).
 static bool weight_native(fpq_format f) { return is_e4m3_native(f) || is_e2m1(f); }
 static bool weight_reencoded(fpq_format f) { return !weight_native(f) && embeds_in_e4m3(f, nullptr); }
 static bool weight_two_term(fpq_format f)
 {
-    return !weight_native(f) && !embeds_in_e4m3(f, nullptr) && splits_in_two_e4m3(f, nullptr, nullptr);
+    return !weight_native(f) && !embeds_in_e4m3(f, nullptr) && splits_in_two_e4m3(f, nullptr, nullptr, nullptr);
 }
 
 // Operand pairs the tensor-core contraction has no type for run on the CUDA cores (fpq_linear and fpq_conv2d
@@ -191,6 +206,14 @@ static QFormat prepared_format(fpq_format fw)
 }
 
 static const fpq_format kE4M3Native = {4, 3, 7, FPQ_SAT_NATIVE};
+
+// 2^-shift of a two-term weight format: what the prepared terms have to be multiplied by.
+static float two_term_unshift(fpq_format fw)
+{
+    int shift = 0;
+    splits_in_two_e4m3(fw, nullptr, nullptr, &shift);
+    return ldexpf(1.0f, -shift);
+}
 
 static int g_path_policy = FPQ_PATH_AUTO;
 
@@ -311,7 +334,7 @@ fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_la
     if (!aligned(prepared, 128))
         return FPQ_ERR_ALIGN;
     CodeTable tab, tab2;
-    if (weight_two_term(fmt) && splits_in_two_e4m3(fmt, &tab, &tab2))
+    if (weight_two_term(fmt) && splits_in_two_e4m3(fmt, &tab, &tab2, nullptr))
         return launch_prepare_weight(codes, d->N, d->C, d->R * d->S, 2 * (int)padded_c(d->C), q.four_bit, 0, 0, &tab,
                                      &tab2, (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
                    ? FPQ_OK
@@ -441,6 +464,7 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
         resolve_format(fx, &g.fx);
         g.fw = prepared_format(fw);
         g.w_two_term = weight_two_term(fw) ? 1 : 0;
+        g.w_mul = g.w_two_term ? two_term_unshift(fw) : 1.0f;
         g.x = x, g.w_prepared = w_prepared, g.w_scale = w_scale, g.x_scale = x_scale, g.bias = bias, g.y = y;
         if (!x || !w_prepared || !w_scale || !y)
             return FPQ_ERR_NULL;
@@ -473,8 +497,9 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
         if (launch_quantize_rows_e4m3_twice(x, M, K, K2 / 2, x_scale, (uint8_t*)workspace, (cudaStream_t)stream) !=
             cudaSuccess)
             return FPQ_ERR_CUDA;
-        return linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, kE4M3Native, bias, y, M, N, K2,
-                                    stream, 1, nullptr);
+        // (the contraction uses the activation scale only to dequantize: the weights' power of two goes there)
+        return linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale * two_term_unshift(fw), fx,
+                                    kE4M3Native, bias, y, M, N, K2, stream, 1, nullptr);
     }
     bool empty = false;
     fpq_status s = linear_checks(fx, fw, M, N, K, workspace, ws_bytes, &empty);
@@ -540,6 +565,7 @@ static bool general_conv(GeneralLayer* g, fpq_format fx, fpq_format fw, int B, i
     resolve_format(fx, &g->fx);
     g->fw = prepared_format(fw);
     g->w_two_term = weight_two_term(fw) ? 1 : 0;
+    g->w_mul = g->w_two_term ? two_term_unshift(fw) : 1.0f;
     return true;
 }
 
@@ -704,8 +730,8 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
             launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H, W, pad, Cp, C2, Cp, x_scale, (uint8_t*)workspace, st) !=
                 cudaSuccess)
             return FPQ_ERR_CUDA;
-        return conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, kE4M3Native, bias, y, B, C2, H, W,
-                                    C_out, R, S, pad, stride, stream, 1, nullptr);
+        return conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale * two_term_unshift(fw), fx,
+                                    kE4M3Native, bias, y, B, C2, H, W, C_out, R, S, pad, stride, stream, 1, nullptr);
     }
     int Ho, Wo;
     bool empty = false;

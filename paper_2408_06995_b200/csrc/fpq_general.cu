@@ -42,7 +42,7 @@ __global__ void __launch_bounds__(256) quantize_values_kernel(const float* __res
 // values [N][C*RS] with column c * RS + tap, the order of the boundary's [C][R][S] weights.
 // two_term: a prepared row holds [first terms | second terms], Cp bytes each, and a weight is their sum (exact).
 __global__ void __launch_bounds__(256) decode_prepared_kernel(const uint8_t* __restrict__ prepared, int64_t N, int C,
-                                                              int RS, int Cp, QFormat f, int two_term,
+                                                              int RS, int Cp, QFormat f, int two_term, float w_mul,
                                                               float* __restrict__ wv)
 {
     const int64_t K = (int64_t)C * RS, total = N * K;
@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(256) decode_prepared_kernel(const uint8_t* __r
         int c = k / RS, tap = k - c * RS;
         if (two_term) {
             int64_t e1 = (n * RS + tap) * (2 * (int64_t)Cp) + c;
-            wv[i] = decode_code(__ldg(prepared + e1), f) + decode_code(__ldg(prepared + e1 + Cp), f);
+            wv[i] = (decode_code(__ldg(prepared + e1), f) + decode_code(__ldg(prepared + e1 + Cp), f)) * w_mul;
             continue;
         }
         int64_t e = (n * RS + tap) * Cp + c;
@@ -135,7 +135,7 @@ fpq_status launch_general_layer(const GeneralLayer& g, void* workspace, cudaStre
         return FPQ_ERR_CUDA;
     quantize_values_kernel<<<grid_for(p.n_x), 256, 0, st>>>(g.x, p.n_x, g.x_scale, g.fx, xv, status);
     decode_prepared_kernel<<<grid_for(g.N * g.K), 256, 0, st>>>((const uint8_t*)g.w_prepared, g.N, g.C, g.R * g.S, g.Cp,
-                                                               g.fw, g.w_two_term, wv);
+                                                               g.fw, g.w_two_term, g.w_mul, wv);
     const float* a = xv;
     if (g.conv) {
         fpq_status s = launch_unfold(xv, g.B, g.C, g.H, g.W, g.R, g.S, g.pad, g.stride, g.Ho, g.Wo, rows, st);

@@ -91,6 +91,7 @@ struct GeneralLayer {
     QFormat fx, fw;           // fw: the format of the codes in the prepared copy
     int Cp;                   // padded channels of the prepared copy ([N][R*S][Cp])
     int w_two_term;           // the prepared copy holds two E4M3 terms per weight ([N][R*S][2 Cp])
+    float w_mul;              // power of two the sum of the two terms is multiplied by (1 unless w_two_term)
     const float* x;
     const void* w_prepared;
     const float* w_scale;

@@ -149,6 +149,9 @@ def test_weight_formats_the_layer_accepts(L):
     d = fpq._CLayerDesc(fpq.LINEAR, 8, 200, 1, 1)
     assert L.fpq_prepared_size(fpq.E3M4.c(), ctypes.byref(d)) == 2 * 8 * 256
     assert L.fpq_prepared_size(fpq.E5M2.c(), ctypes.byref(d)) == 8 * 256       # CUDA-core route: codes as they are
+    # the paper's default E4M3 (bias 8): two terms after a factor of two that the dequantization scale takes back
+    assert L.fpq_prepared_size(fpq.Format(4, 3, 8, fpq.SAT_PAPER).c(), ctypes.byref(d)) == 2 * 8 * 256
+    assert L.fpq_prepared_size(fpq.Format(5, 2, 16, fpq.SAT_PAPER).c(), ctypes.byref(d)) == 8 * 256
     assert fpq.fpq_linear_workspace_size(100, 64, 200, fpq.E4M3, fpq.E2M5) == 100 * 512
     assert L.fpq_prepared_size(fpq.E2M1.c(), ctypes.byref(d)) == 8 * 256 // 2
     assert L.fpq_prepared_size(fpq.E1M2.c(), ctypes.byref(d)) == 8 * 256      # one E4M3 byte per weight
