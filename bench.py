@@ -732,6 +732,10 @@ def run_formats(args):
                ("e2m5", fpq.E2M5, "tensor cores, weights prepared as two E4M3 terms"),
                ("e4m3_bias8", fpq.Format(4, 3, 8, fpq.SAT_PAPER), "tensor cores, weights prepared as two E4M3 terms"),
                ("e5m2_bias16", fpq.Format(5, 2, 16, fpq.SAT_PAPER), "CUDA cores (FP32 multiply-adds)")]
+    if args.only:
+        formats = [f for f in formats if args.only in f[0]]
+        if not formats:
+            raise SystemExit(f"no weight format of suite formats has {args.only!r} in its name")
     props = torch.cuda.get_device_properties(0)
     sampler = ClockSampler(physical_gpu_index(0))
     sampler.start()
@@ -831,7 +835,8 @@ def main():
     ap.add_argument("--skip-w4", action="store_true", help="leave out the W4A8 side measurement")
     ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd", "sd_trace", "search", "sd_split", "round_learn", "formats"],
                     help="print a per-shape table of a whole workload instead of the headline line")
-    ap.add_argument("--only", default=None, help="with --suite ldm|transformer|sd|round_learn: only the layers whose name contains this")
+    ap.add_argument("--only", default=None, help="with --suite ldm|transformer|sd|round_learn: only the layers whose name contains this; "
+                    "with --suite formats: only the weight formats whose name contains this")
     args = ap.parse_args()
     if args.suite == "sd_trace":
         run_trace(args)
