@@ -9,9 +9,10 @@
  *
  * Conventions
  *   - Every pointer is a DEVICE pointer unless its name ends in _host.
- *   - The caller owns every buffer.  The library allocates nothing in these
- *     calls and keeps no state except one sticky device status word
- *     (fpq_read_status).
+ *   - The caller owns every buffer.  The library allocates no device memory in
+ *     these calls and keeps no state except one sticky device status word
+ *     (fpq_read_status) and host-side tables of things worked out once (launch
+ *     plans per device, how each weight format is run).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *     stream).  Calls only enqueue work; they do not synchronise unless stated.
  *   - Calls may come from several host threads (each with its own stream and

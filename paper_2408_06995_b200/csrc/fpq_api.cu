@@ -2,6 +2,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <map>
 #include <mutex>
 
 #include "fpq_common.cuh"
@@ -171,14 +172,48 @@ static bool splits_in_two_e4m3(fpq_format f, CodeTable* first, CodeTable* second
     return false;
 }
 
-// Weight formats the contraction reads as they are, formats re-encoded when the weights are prepared, and
-// formats prepared as two E4M3 terms (twice the reduction length on the tensor cores).
-static bool weight_native(fpq_format f) { return is_e4m3_native(f) || is_e2m1(f); }
-static bool weight_reencoded(fpq_format f) { return !weight_native(f) && embeds_in_e4m3(f, nullptr); }
-static bool weight_two_term(fpq_format f)
+// How the layer calls run a weight format: read by the tensor cores as it is, re-encoded into one E4M3
+// term when the weights are prepared, prepared as two E4M3 terms (twice the reduction length), or on the
+// CUDA cores.  Working this out walks all codes of the format, so the answer (a pure function of the four
+// format fields) is kept per format; host threads take turns at the table.
+enum { W_INVALID = 0, W_NATIVE, W_ONE_TERM, W_TWO_TERM, W_OTHER };
+struct WeightClass {
+    int kind;
+    int shift;             // W_TWO_TERM: the terms are those of 2^shift * value
+    CodeTable t1, t2;      // W_ONE_TERM: t1; W_TWO_TERM: t1 (first terms), t2 (second terms)
+};
+
+static const WeightClass& classify_weight(fpq_format f)
 {
-    return !weight_native(f) && !embeds_in_e4m3(f, nullptr) && splits_in_two_e4m3(f, nullptr, nullptr, nullptr);
+    static std::mutex mu;
+    static std::map<uint64_t, WeightClass> known;
+    static const WeightClass invalid = {};
+    if (f.exp_bits < 1 || f.exp_bits > 8 || f.man_bits < 1 || f.man_bits > 8 || f.sat_mode < 0 || f.sat_mode > 1)
+        return invalid;
+    const uint64_t key = ((uint64_t)(uint8_t)f.exp_bits << 56) | ((uint64_t)(uint8_t)f.man_bits << 48) |
+                         ((uint64_t)(uint8_t)f.sat_mode << 40) | (uint64_t)(uint32_t)f.exp_bias;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = known.find(key);
+    if (it != known.end())
+        return it->second;
+    WeightClass c = {};
+    QFormat q;
+    if (!resolve_format(f, &q))
+        c.kind = W_INVALID;
+    else if (is_e4m3_native(f) || is_e2m1(f))
+        c.kind = W_NATIVE;
+    else if (embeds_in_e4m3(f, &c.t1))
+        c.kind = W_ONE_TERM;
+    else if (splits_in_two_e4m3(f, &c.t1, &c.t2, &c.shift))
+        c.kind = W_TWO_TERM;
+    else
+        c.kind = W_OTHER;
+    return known.emplace(key, c).first->second;
 }
+
+static bool weight_native(fpq_format f) { return classify_weight(f).kind == W_NATIVE; }
+static bool weight_reencoded(fpq_format f) { return classify_weight(f).kind == W_ONE_TERM; }
+static bool weight_two_term(fpq_format f) { return classify_weight(f).kind == W_TWO_TERM; }
 
 // Operand pairs the tensor-core contraction has no type for run on the CUDA cores (fpq_linear and fpq_conv2d
 // only; the staged, host-buffer, two-tensor and built-in-scratch forms keep to the tensor-core pairs).
@@ -208,12 +243,7 @@ static QFormat prepared_format(fpq_format fw)
 static const fpq_format kE4M3Native = {4, 3, 7, FPQ_SAT_NATIVE};
 
 // 2^-shift of a two-term weight format: what the prepared terms have to be multiplied by.
-static float two_term_unshift(fpq_format fw)
-{
-    int shift = 0;
-    splits_in_two_e4m3(fw, nullptr, nullptr, &shift);
-    return ldexpf(1.0f, -shift);
-}
+static float two_term_unshift(fpq_format fw) { return ldexpf(1.0f, -classify_weight(fw).shift); }
 
 static int g_path_policy = FPQ_PATH_AUTO;
 
@@ -333,15 +363,15 @@ fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_la
         return FPQ_ERR_NULL;
     if (!aligned(prepared, 128))
         return FPQ_ERR_ALIGN;
-    CodeTable tab, tab2;
-    if (weight_two_term(fmt) && splits_in_two_e4m3(fmt, &tab, &tab2, nullptr))
-        return launch_prepare_weight(codes, d->N, d->C, d->R * d->S, 2 * (int)padded_c(d->C), q.four_bit, 0, 0, &tab,
-                                     &tab2, (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
+    const WeightClass& wc = classify_weight(fmt);
+    if (wc.kind == W_TWO_TERM)
+        return launch_prepare_weight(codes, d->N, d->C, d->R * d->S, 2 * (int)padded_c(d->C), q.four_bit, 0, 0, &wc.t1,
+                                     &wc.t2, (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
                    ? FPQ_OK
                    : FPQ_ERR_CUDA;
-    const bool re = weight_reencoded(fmt) && embeds_in_e4m3(fmt, &tab);
+    const bool re = wc.kind == W_ONE_TERM;
     return launch_prepare_weight(codes, d->N, d->C, d->R * d->S, (int)padded_c(d->C), q.four_bit, 0, 0,
-                                 re ? &tab : nullptr, nullptr, (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
+                                 re ? &wc.t1 : nullptr, nullptr, (uint8_t*)prepared, (cudaStream_t)stream) == cudaSuccess
                ? FPQ_OK
                : FPQ_ERR_CUDA;
 }
@@ -795,10 +825,10 @@ fpq_status fpq_prepare_weight_split(const uint8_t* codes, fpq_format fmt, int32_
         return FPQ_ERR_NULL;
     if (!aligned(prepared, 128))
         return FPQ_ERR_ALIGN;
-    CodeTable tab;
-    const bool re = weight_reencoded(fmt) && embeds_in_e4m3(fmt, &tab);
+    const WeightClass& wc = classify_weight(fmt);
+    const bool re = wc.kind == W_ONE_TERM;
     return launch_prepare_weight(codes, N, C1 + C2, R * S, (int)(padded_c(C1) + padded_c(C2)), q.four_bit, C1,
-                                 (int)padded_c(C1), re ? &tab : nullptr, nullptr, (uint8_t*)prepared,
+                                 (int)padded_c(C1), re ? &wc.t1 : nullptr, nullptr, (uint8_t*)prepared,
                                  (cudaStream_t)stream) == cudaSuccess
                ? FPQ_OK
                : FPQ_ERR_CUDA;
