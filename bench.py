@@ -461,6 +461,36 @@ def run_own(args):
         del xq, cq
         torch.cuda.empty_cache()
 
+    # ---- side measurements of the rows built around the layer (details: --suite round_learn / formats)
+    side = None
+    if rank == 0 and not args.skip_w4:
+        side = {}
+        M, N, K = 4096, 960, 320
+        w = torch.randn((N, K), device=dev) * 0.02
+        a = torch.randn((M, K), device=dev)
+        alpha = torch.randn((N, K), device=dev) * 2.0
+        sc = (w.abs().amax(dim=1) / 6.0).contiguous()
+        grad, loss = torch.empty_like(alpha), torch.empty(2, dtype=torch.float64, device=dev)
+        wk = torch.empty(fpq.fpq_round_learn_workspace_size(M, N, K), dtype=torch.uint8, device=dev)
+        t = per_launch_us(torch, lambda: fpq.fpq_round_learn_step(w, sc, fpq.E2M1, alpha, a, 0.01, 1.0, grad, loss, wk),
+                          10) * 1e-6
+        fp32_peak = torch.cuda.get_device_properties(dev).multi_processor_count * 128 * 2 * \
+            (clocks.get("sm_mhz") or 1965.0) * 1e6
+        side["round_learn_step_qkv_320_960_m4096"] = {"us": t * 1e6, "tflops_fp32": 4.0 * M * N * K / t / 1e12,
+                                                      "frac_of_fp32_fma_peak": 4.0 * M * N * K / t / fp32_peak}
+        M = 8192
+        x = torch.randn((M, K), device=dev)
+        y = torch.empty((M, N), device=dev)
+        for fname, f in (("e4m3", fpq.E4M3), ("e1m2_reencoded", fpq.E1M2), ("e3m4_two_terms", fpq.E3M4),
+                         ("e5m2_bias16_cuda_cores", fpq.Format(5, 2, 16, fpq.SAT_PAPER))):
+            ws = (w.abs().amax(dim=1) / fpq.fpq_format_max(f)).contiguous()
+            prep = fpq.fpq_prepare_weight(fpq.fpq_quantize_weight(w, ws, f, None), f, fpq.LINEAR, N, K)
+            wk = torch.empty(max(256, fpq.fpq_linear_workspace_size(M, N, K, fpq.E4M3, f)), dtype=torch.uint8, device=dev)
+            t = per_launch_us(torch, lambda: fpq.fpq_linear(x, prep, ws, 0.01, fpq.E4M3, f, None, N, y, wk), 10) * 1e-6
+            side["linear_qkv_320_960_m8192_weights_" + fname] = {"us": t * 1e6, "tflops": 2.0 * M * N * K / t / 1e12}
+        del w, a, alpha, x, y, wk
+        torch.cuda.empty_cache()
+
     # ---- CPU baseline: the oracle, as it stands, on the host cores (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.skip_cpu:
@@ -487,6 +517,7 @@ def run_own(args):
             "roofline": roofline, "layer_roofline": layer_roof, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
             "weight_encode_us": enc_us, "w4a8": w4, "standalone_quantizer": quant, "eager_step_us": eager_us,
+            "side_measurements": side,
         }
         print(json.dumps(line), flush=True)
     if world > 1:
