@@ -77,3 +77,25 @@ def test_every_fp8_search_candidate_runs_as_a_layer():
     I.draw(L, 33, 0, "normal", 0.02, True, 0.01)
     for enc in O.FP8_ENCODINGS:
         _run(L, fpq.E4M3, fpq.Format(enc.e, enc.m, enc.B, fpq.SAT_PAPER))
+
+
+@pytest.mark.parametrize("gfw", [fpq.E3M4, E5M2_B16])
+def test_empty_and_nan_inputs(gfw):
+    d = "cuda"
+    N, K = 8, 32
+    w = torch.randn((N, K), device=d) * 0.02
+    ws = (w.abs().amax(dim=1) / fpq.fpq_format_max(gfw)).contiguous()
+    prep = fpq.fpq_prepare_weight(fpq.fpq_quantize_weight(w, ws, gfw, None), gfw, fpq.LINEAR, N, K)
+    # no rows: nothing to do, no error
+    y0 = fpq.fpq_linear(torch.empty((0, K), device=d), prep, ws, 0.01, fpq.E4M3, gfw, None, N)
+    assert y0.shape == (0, N) and fpq.fpq_read_status() == fpq.OK
+    # a NaN activation is quantized to zero and reported through the status word
+    x = torch.randn((16, K), device=d)
+    x[3, 5] = float("nan")
+    y = fpq.fpq_linear(x, prep, ws, 0.01, fpq.E4M3, gfw, None, N)
+    assert fpq.fpq_read_status() == fpq.ERR_NAN_INPUT
+    assert torch.isfinite(y).all()
+    x[3, 5] = 0.0
+    y2 = fpq.fpq_linear(x, prep, ws, 0.01, fpq.E4M3, gfw, None, N)
+    assert fpq.fpq_read_status() == fpq.OK
+    assert torch.equal(y, y2)

@@ -151,3 +151,20 @@ def test_round_learn_step_for_a_convolution():
     tol = 2.0 * GRAD_RTOL_ABSUM * r["absum"] + 1e-5 * 0.01 * np.abs(O.rounding_regularizer(alpha)[1]) + 1e-16 \
         + 4.0 * np.spacing(np.abs(r["grad"]).astype(np.float32)).astype(np.float64)
     assert np.all(np.abs(grad.cpu().numpy() - r["grad"]) <= tol)
+
+
+def test_nan_weight_is_reported_and_contributes_nothing():
+    w, scale, alpha, a = _case(64, 20, 24, O.E2M1, 3)
+    d = "cuda"
+    args = [torch.from_numpy(v).to(d) for v in (w, scale, alpha, a)]
+    g0, l0 = fpq.fpq_round_learn_step(args[0], args[1], fpq.E2M1, args[2], args[3], 0.0)
+    assert fpq.fpq_read_status() == fpq.OK
+    wn = args[0].clone()
+    wn[2, 7] = float("nan")
+    g1, l1 = fpq.fpq_round_learn_step(wn, args[1], fpq.E2M1, args[2], args[3], 0.0)
+    assert fpq.fpq_read_status() == fpq.ERR_NAN_INPUT
+    assert torch.isfinite(g1).all() and torch.isfinite(l1).all()
+    assert float(g1[2, 7]) == 0.0
+    # rows of other output channels do not see the NaN weight at all
+    keep = [n for n in range(20) if n != 2]
+    assert torch.equal(g0[keep], g1[keep])
