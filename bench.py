@@ -482,7 +482,8 @@ def run_own(args):
         x = torch.randn((M, K), device=dev)
         y = torch.empty((M, N), device=dev)
         for fname, f in (("e4m3", fpq.E4M3), ("e1m2_reencoded", fpq.E1M2), ("e3m4_two_terms", fpq.E3M4),
-                         ("e5m2_bias16_cuda_cores", fpq.Format(5, 2, 16, fpq.SAT_PAPER))):
+                         ("e5m2_bias16_two_terms", fpq.Format(5, 2, 16, fpq.SAT_PAPER)),
+                         ("e6m1_cuda_cores", fpq.Format(6, 1, 31, fpq.SAT_PAPER))):
             ws = (w.abs().amax(dim=1) / fpq.fpq_format_max(f)).contiguous()
             prep = fpq.fpq_prepare_weight(fpq.fpq_quantize_weight(w, ws, f, None), f, fpq.LINEAR, N, K)
             wk = torch.empty(max(256, fpq.fpq_linear_workspace_size(M, N, K, fpq.E4M3, f)), dtype=torch.uint8, device=dev)
@@ -746,8 +747,9 @@ def run_round_learn(args):
 def run_formats(args):
     """The weight encodings the search can select, as the same linear layers (SD-v1-style transformer block,
     M = 8192): read by the tensor cores as they are (E4M3, E2M1), re-encoded exactly into E4M3 when the
-    weights are prepared (E1M2), prepared as the sum of two E4M3 terms and contracted over twice the
-    reduction length (E3M4, E2M5), or run on the CUDA cores with FP32 multiply-adds (E5M2)."""
+    weights are prepared (E1M2), prepared as the sum of two E4M3 (E3M4, E2M5, E4M3 bias 8) or E5M2 (E5M2 bias 16)
+    terms and contracted over twice the reduction length, or run on the CUDA cores with FP32 multiply-adds
+    (E6M1, whose 64 binades no two tensor-core terms span: a stand-in for whatever the tensor cores cannot hold)."""
     import torch
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device")
@@ -758,11 +760,13 @@ def run_formats(args):
     import paper_2408_06995_b200 as fpq
     shapes = [("qkv_320_960", 8192, 960, 320), ("ffn_out_1280_320", 8192, 320, 1280)]
     formats = [("e4m3", fpq.E4M3, "tensor cores"), ("e2m1", fpq.E2M1, "tensor cores"),
+               ("e5m2_ocp", fpq.E5M2, "tensor cores"),
                ("e1m2", fpq.E1M2, "tensor cores, weights re-encoded into E4M3"),
                ("e3m4", fpq.E3M4, "tensor cores, weights prepared as two E4M3 terms"),
                ("e2m5", fpq.E2M5, "tensor cores, weights prepared as two E4M3 terms"),
                ("e4m3_bias8", fpq.Format(4, 3, 8, fpq.SAT_PAPER), "tensor cores, weights prepared as two E4M3 terms"),
-               ("e5m2_bias16", fpq.Format(5, 2, 16, fpq.SAT_PAPER), "CUDA cores (FP32 multiply-adds)")]
+               ("e5m2_bias16", fpq.Format(5, 2, 16, fpq.SAT_PAPER), "tensor cores, weights prepared as two E5M2 terms"),
+               ("e6m1", fpq.Format(6, 1, 31, fpq.SAT_PAPER), "CUDA cores (FP32 multiply-adds)")]
     if args.only:
         formats = [f for f in formats if args.only in f[0]]
         if not formats:

@@ -122,8 +122,8 @@ fpq_status fpq_quantize_act(const float* x, int64_t n, float scale, fpq_format f
  * fpq_prepared_size(fmt, d) bytes and be 128-byte aligned.  The layout is
  * internal: rows of C padded with zero codes to a multiple of 128, taps
  * outermost within a row ([N][R*S][C_pad]).  May be saved and reloaded as bytes.
- * E4M3 (bias 7, FPQ_SAT_NATIVE) and E2M1 (bias 1) codes are kept as they are (E2M1 two per
- * byte).  Any other format whose every value is also a finite E4M3 value - E1M2 with bias 1,
+ * E4M3 (bias 7, FPQ_SAT_NATIVE), E5M2 (bias 15, FPQ_SAT_NATIVE) and E2M1 (bias 1) codes are
+ * kept as they are (E2M1 two per byte).  Any other format whose every value is also a finite E4M3 value - E1M2 with bias 1,
  * E2M1 with bias 2, small formats such as E3M2 bias 3 or E2M3 bias 1 - is re-encoded here,
  * exactly, into one E4M3 byte per weight.  A format whose every value is the sum of two finite
  * E4M3 values (the largest E4M3 magnitude not above it, and the rest: E3M4 bias 4, E2M5 bias 2,
@@ -131,8 +131,9 @@ fpq_status fpq_quantize_act(const float* x, int64_t n, float scale, fpq_format f
  * the layer's dequantization takes back exactly, formats such as the paper's default E4M3 with
  * bias 8) is prepared as those two terms, two bytes per weight ([N][R*S][2 C_pad]); fpq_linear /
  * fpq_conv2d then contract over twice the reduction length on the tensor cores - exact products,
- * FP32 sums, as for one term.  Every other format (E5M2, whose exponent range is twice that of
- * E4M3) is copied unchanged and runs on the CUDA cores.
+ * FP32 sums, as for one term.  The paper's E5M2 (bias 16, all exponent fields finite) is prepared
+ * the same way as two terms of the tensor cores' own E5M2.  Every other format (beyond two such
+ * terms, e.g. 6 exponent bits) is copied unchanged and runs on the CUDA cores.
  */
 size_t fpq_prepared_size(fpq_format fmt, const fpq_layer_desc* d);
 fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_layer_desc* d,
@@ -147,14 +148,15 @@ fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_la
  * tensor cores (layers of at most 8 rows with K a multiple of 4 run on the CUDA
  * cores instead: the same exact products, another order of the FP32 additions;
  * the workspace is then left untouched).  Supported operand pairs: fx = E4M3 bias 7 FPQ_SAT_NATIVE with
- * fw = the same, fw = E2M1 bias 1, or any fw that fpq_prepare_weight re-encodes exactly into one or two
- * E4M3 terms (see there) run on the tensor cores.  Every other valid pair (any fx, any fw) runs on the CUDA
+ * fw = the same, fw = E5M2 bias 15 FPQ_SAT_NATIVE, fw = E2M1 bias 1, or any fw that fpq_prepare_weight
+ * re-encodes exactly into one or two terms of those types (see there) run on the tensor cores.  Every other valid pair (any fx, any fw) runs on the CUDA
  * cores: activations quantized to their grid values in FP32, weights decoded to FP32, an FP32 multiply-add
  * contraction - the same arithmetic model (exact products, FP32 sums) at roughly a tenth of the speed; the
  * workspace is then FP32 scratch (fpq_linear_workspace_size says how much) and must be 256-byte aligned.
- * This holds for fpq_linear and fpq_conv2d and their host-buffer forms; the staged (quantize_input /
- * contract), two-tensor and built-in-scratch forms take only the pairs the tensor cores read directly or
- * after the one-term re-encode, and return FPQ_ERR_UNSUPPORTED otherwise.
+ * This holds for fpq_linear and fpq_conv2d and their host-buffer forms (and for fpq_linear_static as far as
+ * its fixed scratch reaches: FPQ_ERR_WORKSPACE beyond); the staged (quantize_input / contract) and two-tensor
+ * forms take only the pairs the tensor cores read directly or after the one-term re-encode, and return
+ * FPQ_ERR_UNSUPPORTED otherwise.
  * workspace: fpq_linear_workspace_size bytes, 128-byte aligned; contents are
  * scratch.
  */

@@ -69,6 +69,11 @@ static bool is_e4m3_native(fpq_format f)
     return f.exp_bits == 4 && f.man_bits == 3 && f.exp_bias == 7 && f.sat_mode == FPQ_SAT_NATIVE;
 }
 
+static bool is_e5m2_native(fpq_format f)
+{
+    return f.exp_bits == 5 && f.man_bits == 2 && f.exp_bias == 15 && f.sat_mode == FPQ_SAT_NATIVE;
+}
+
 static bool is_e2m1(fpq_format f)
 {
     return f.exp_bits == 2 && f.man_bits == 1 && f.exp_bias == 1;
@@ -120,12 +125,12 @@ static bool embeds_in_e4m3(fpq_format f, CodeTable* tab)
 // first = the largest E4M3 magnitude not above |v| (sign of v) and second = v - first also a finite E4M3
 // value (formats with up to 7 significant bits inside E4M3's exponent range: E3M4, E2M5, the paper's E4M3
 // with its code for 480 = 448 + 32).  Tables: code of f -> E4M3 code of each term.
-static bool splits_in_two_e4m3_at(fpq_format f, int shift, CodeTable* first, CodeTable* second)
+static bool splits_in_two_at(fpq_format f, fpq_format e4m3 /* the container type */, int top_code, int shift,
+                             CodeTable* first, CodeTable* second)
 {
     QFormat q;
     if (!resolve_format(f, &q))
         return false;
-    const fpq_format e4m3 = {4, 3, 7, FPQ_SAT_NATIVE};
     int ncodes = 1 << (1 + f.exp_bits + f.man_bits);
     int mag_mask = (1 << (f.exp_bits + f.man_bits)) - 1;
     for (int c = 0; c < 256; ++c) {
@@ -133,13 +138,13 @@ static bool splits_in_two_e4m3_at(fpq_format f, int shift, CodeTable* first, Cod
         if (c < ncodes && (c & mag_mask) <= q.code_max) {
             double v = ldexp(code_value(c, f), shift), a = fabs(v);
             if (a != 0.0) {
-                int k1 = 0;                               // E4M3 magnitudes increase with the code
-                for (int k = 1; k <= 0x7E; ++k)
+                int k1 = 0;                               // magnitudes increase with the code
+                for (int k = 1; k <= top_code; ++k)
                     if (code_value(k, e4m3) <= a)
                         k1 = k;
                 double rest = a - code_value(k1, e4m3);
                 int k2 = rest == 0.0 ? 0 : -1;
-                for (int k = 1; k <= 0x7E && k2 < 0; ++k)
+                for (int k = 1; k <= top_code && k2 < 0; ++k)
                     if (code_value(k, e4m3) == rest)
                         k2 = k;
                 if (k2 < 0)
@@ -160,17 +165,21 @@ static bool splits_in_two_e4m3_at(fpq_format f, int shift, CodeTable* first, Cod
 // The terms are those of 2^shift * v for the smallest |shift| <= 16 that works (0 first): a format whose bias
 // puts it outside E4M3's range (the paper's default E4M3 with bias 8: shift 1) still splits, and the layer
 // multiplies the dequantization scale by 2^-shift, which is exact.
-static bool splits_in_two_e4m3(fpq_format f, CodeTable* first, CodeTable* second, int* shift)
+static bool splits_in_two(fpq_format f, fpq_format container, int top_code, CodeTable* first, CodeTable* second,
+                          int* shift)
 {
     for (int m = 0; m <= 16; ++m)
         for (int sgn = 1; sgn >= (m ? -1 : 1); sgn -= 2)
-            if (splits_in_two_e4m3_at(f, sgn * m, first, second)) {
+            if (splits_in_two_at(f, container, top_code, sgn * m, first, second)) {
                 if (shift)
                     *shift = sgn * m;
                 return true;
             }
     return false;
 }
+
+static const fpq_format kE4M3Native = {4, 3, 7, FPQ_SAT_NATIVE};
+static const fpq_format kE5M2Native = {5, 2, 15, FPQ_SAT_NATIVE};
 
 // How the layer calls run a weight format: read by the tensor cores as it is, re-encoded into one E4M3
 // term when the weights are prepared, prepared as two E4M3 terms (twice the reduction length), or on the
@@ -180,6 +189,7 @@ enum { W_INVALID = 0, W_NATIVE, W_ONE_TERM, W_TWO_TERM, W_OTHER };
 struct WeightClass {
     int kind;
     int shift;             // W_TWO_TERM: the terms are those of 2^shift * value
+    int e5m2;              // W_TWO_TERM: the terms are E5M2 (bias 15) codes instead of E4M3 codes
     CodeTable t1, t2;      // W_ONE_TERM: t1; W_TWO_TERM: t1 (first terms), t2 (second terms)
 };
 
@@ -200,12 +210,14 @@ static const WeightClass& classify_weight(fpq_format f)
     QFormat q;
     if (!resolve_format(f, &q))
         c.kind = W_INVALID;
-    else if (is_e4m3_native(f) || is_e2m1(f))
+    else if (is_e4m3_native(f) || is_e2m1(f) || is_e5m2_native(f))
         c.kind = W_NATIVE;
     else if (embeds_in_e4m3(f, &c.t1))
         c.kind = W_ONE_TERM;
-    else if (splits_in_two_e4m3(f, &c.t1, &c.t2, &c.shift))
+    else if (splits_in_two(f, kE4M3Native, 0x7E, &c.t1, &c.t2, &c.shift))
         c.kind = W_TWO_TERM;
+    else if (splits_in_two(f, kE5M2Native, 0x7B, &c.t1, &c.t2, &c.shift))
+        c.kind = W_TWO_TERM, c.e5m2 = 1;                  // the paper's E5M2 with all 32 exponent fields finite
     else
         c.kind = W_OTHER;
     return known.emplace(key, c).first->second;
@@ -236,11 +248,10 @@ static QFormat prepared_format(fpq_format fw)
 {
     const fpq_format e4m3 = {4, 3, 7, FPQ_SAT_NATIVE};
     QFormat q;
-    resolve_format((weight_reencoded(fw) || weight_two_term(fw)) ? e4m3 : fw, &q);
+    const WeightClass& wc = classify_weight(fw);
+    resolve_format(wc.kind == W_TWO_TERM ? (wc.e5m2 ? kE5M2Native : kE4M3Native) : (wc.kind == W_ONE_TERM ? e4m3 : fw), &q);
     return q;
 }
-
-static const fpq_format kE4M3Native = {4, 3, 7, FPQ_SAT_NATIVE};
 
 // 2^-shift of a two-term weight format: what the prepared terms have to be multiplied by.
 static float two_term_unshift(fpq_format fw) { return ldexpf(1.0f, -classify_weight(fw).shift); }
@@ -453,6 +464,7 @@ static fpq_status linear_contract_impl(const void* workspace, size_t ws_bytes, c
     p.C = (int)K;
     p.after_stage1 = after_stage1;
     p.w4 = is_e2m1(fw) ? 1 : 0;
+    p.w_e5m2 = is_e5m2_native(fw) ? 1 : 0;
     p.M = M;
     p.N = (int)N;
     p.Cp = (int)padded_c(K);
@@ -512,7 +524,8 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
             return FPQ_ERR_SHAPE;
         const int64_t K2 = 2 * padded_c(K);
         bool empty = false;
-        fpq_status s = linear_checks(fx, kE4M3Native, M, N, K2, workspace, ws_bytes, &empty);
+        const fpq_format term = classify_weight(fw).e5m2 ? kE5M2Native : kE4M3Native;
+        fpq_status s = linear_checks(fx, term, M, N, K2, workspace, ws_bytes, &empty);
         if (s != FPQ_OK || empty)
             return s;
         if (K == 0)
@@ -528,8 +541,8 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
             cudaSuccess)
             return FPQ_ERR_CUDA;
         // (the contraction uses the activation scale only to dequantize: the weights' power of two goes there)
-        return linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale * two_term_unshift(fw), fx,
-                                    kE4M3Native, bias, y, M, N, K2, stream, 1, nullptr);
+        return linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale * two_term_unshift(fw), fx, term, bias,
+                                    y, M, N, K2, stream, 1, nullptr);
     }
     bool empty = false;
     fpq_status s = linear_checks(fx, fw, M, N, K, workspace, ws_bytes, &empty);
@@ -543,7 +556,7 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
         return FPQ_ERR_ALIGN;
     // a handful of rows (time-embedding projections): one pass over the weights on the CUDA cores,
     // whatever the route policy says; the workspace is not touched
-    if (small_m_linear_applies(M, K) && N <= 0x7fffffff) {
+    if (small_m_linear_applies(M, K) && N <= 0x7fffffff && !is_e5m2_native(fw)) {
         if (!status_word())
             return FPQ_ERR_CUDA;
         return launch_small_m_linear(x, (int)M, (int)K, w_prepared, is_e2m1(fw) ? 1 : 0, (int)N, w_scale, x_scale, bias, y,
@@ -685,6 +698,7 @@ static fpq_status conv2d_contract_impl(const void* workspace, size_t ws_bytes, c
     p.C = C;
     p.after_stage1 = after_stage1;
     p.w4 = is_e2m1(fw) ? 1 : 0;
+    p.w_e5m2 = is_e5m2_native(fw) ? 1 : 0;
     p.M = (int64_t)B * Ho * Wo;
     p.N = C_out;
     p.Cp = (int)padded_c(C);
@@ -743,8 +757,8 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
         const int Cp = (int)padded_c(C), C2 = 2 * Cp;
         int Ho2, Wo2;
         bool empty2 = false;
-        fpq_status s2 = conv_checks(fx, kE4M3Native, B, C2, H, W, C_out, R, S, pad, stride, workspace, ws_bytes, &Ho2, &Wo2,
-                                    &empty2);
+        const fpq_format term = classify_weight(fw).e5m2 ? kE5M2Native : kE4M3Native;
+        fpq_status s2 = conv_checks(fx, term, B, C2, H, W, C_out, R, S, pad, stride, workspace, ws_bytes, &Ho2, &Wo2, &empty2);
         if (s2 != FPQ_OK || empty2)
             return s2;
         if (!x || !w_prepared || !w_scale || !y)
@@ -760,8 +774,8 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
             launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H, W, pad, Cp, C2, Cp, x_scale, (uint8_t*)workspace, st) !=
                 cudaSuccess)
             return FPQ_ERR_CUDA;
-        return conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale * two_term_unshift(fw), fx,
-                                    kE4M3Native, bias, y, B, C2, H, W, C_out, R, S, pad, stride, stream, 1, nullptr);
+        return conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale * two_term_unshift(fw), fx, term, bias,
+                                    y, B, C2, H, W, C_out, R, S, pad, stride, stream, 1, nullptr);
     }
     int Ho, Wo;
     bool empty = false;
@@ -888,6 +902,7 @@ fpq_status fpq_conv2d_split(const float* x1, int C1, float x1_scale, const float
     p.conv = 1;
     p.after_stage1 = 1;
     p.w4 = is_e2m1(fw) ? 1 : 0;
+    p.w_e5m2 = is_e5m2_native(fw) ? 1 : 0;
     p.M = (int64_t)B * Ho * Wo;
     p.N = C_out;
     p.Cp = C1p + (int)padded_c(C2);

@@ -305,7 +305,7 @@ __device__ __forceinline__ uint32_t smem_desc_lo(uint32_t addr)
 }
 constexpr uint32_t SMEM_DESC_HI_K_SW128 = 64u | (1u << 14) | (2u << 29);
 
-// Instruction descriptor: FP32 accumulator, operand formats (0 = E4M3, 5 = E2M1),
+// Instruction descriptor: FP32 accumulator, operand formats (0 = E4M3, 1 = E5M2, 5 = E2M1),
 // both operands K-major, M = 128, N = n.
 __host__ __device__ inline uint32_t idesc_f8f6f4(uint32_t a_fmt, uint32_t b_fmt, uint32_t n)
 {

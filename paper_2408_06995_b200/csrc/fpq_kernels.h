@@ -33,6 +33,7 @@ struct GemmProblem {
     int conv;            // 0 linear, 1 conv
     int after_stage1;    // launched right behind this library's own activation-quantize kernel
     int w4;              // weights are E2M1
+    int w_e5m2;          // weights are E5M2 (bias 15, native saturation): the tensor cores' second 8-bit type
     int64_t M;           // linear rows
     int N;               // outputs / out channels
     int Cp;              // padded reduction length per tap in the weight copy (multiple of 128)

@@ -9,7 +9,7 @@ from paper_2408_06995_b200 import build as fpq_build
 
 fpq_build.build()
 
-FMT = {"e4m3": (fpq.E4M3, O.E4M3), "e2m1": (fpq.E2M1, O.E2M1),
+FMT = {"e4m3": (fpq.E4M3, O.E4M3), "e2m1": (fpq.E2M1, O.E2M1), "e5m2": (fpq.E5M2, O.E5M2),
        # weight formats that the layer re-encodes exactly into E4M3 when the weights are prepared
        "e1m2": (fpq.E1M2, O.E1M2),
        "e2m1b2": (fpq.Format(2, 1, 2, fpq.SAT_PAPER), O.Format(2, 1, 2, O.SAT_PAPER)),

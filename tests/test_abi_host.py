@@ -138,20 +138,25 @@ def test_weight_formats_the_layer_accepts(L):
         # (by the tensor-core forms) a NULL activation pointer is rejected after the operand pair has been checked
         return L.fpq_linear_quantize_input(None, 1.0, F, fw.c(), 8, 8, 8, big, 1 << 20, None) != fpq.ERR_UNSUPPORTED
 
-    # read by the tensor cores as they are
-    assert accepted(fpq.E4M3) and accepted(fpq.E2M1)
+    # read by the tensor cores as they are (E4M3, E2M1 and the OCP E5M2)
+    assert accepted(fpq.E4M3) and accepted(fpq.E2M1) and accepted(fpq.E5M2)
     # every value is also an E4M3 value: re-encoded when the weights are prepared
     assert accepted(fpq.E1M2) and accepted(fpq.Format(2, 1, 2)) and accepted(fpq.Format(3, 2, 3))
     # more mantissa bits or a wider exponent range than E4M3 holds, or the code 480 of the paper's E4M3
-    assert not accepted(fpq.E3M4) and not accepted(fpq.E2M5) and not accepted(fpq.E5M2)
+    assert not accepted(fpq.E3M4) and not accepted(fpq.E2M5) and not accepted(fpq.Format(5, 2, 16, fpq.SAT_PAPER))
     assert not accepted(fpq.Format(4, 3, 7, fpq.SAT_PAPER)) and not accepted(fpq.Format(4, 3, 8, fpq.SAT_NATIVE))
     # E3M4 / E2M5 weights are prepared as two E4M3 terms: twice the bytes, twice the activation codes
     d = fpq._CLayerDesc(fpq.LINEAR, 8, 200, 1, 1)
     assert L.fpq_prepared_size(fpq.E3M4.c(), ctypes.byref(d)) == 2 * 8 * 256
-    assert L.fpq_prepared_size(fpq.E5M2.c(), ctypes.byref(d)) == 8 * 256       # CUDA-core route: codes as they are
+    assert L.fpq_prepared_size(fpq.E5M2.c(), ctypes.byref(d)) == 8 * 256       # read as it is
     # the paper's default E4M3 (bias 8): two terms after a factor of two that the dequantization scale takes back
     assert L.fpq_prepared_size(fpq.Format(4, 3, 8, fpq.SAT_PAPER).c(), ctypes.byref(d)) == 2 * 8 * 256
-    assert L.fpq_prepared_size(fpq.Format(5, 2, 16, fpq.SAT_PAPER).c(), ctypes.byref(d)) == 8 * 256
+    # the paper's E5M2 (bias 16, all exponent fields finite): two terms of the tensor cores' own E5M2
+    assert L.fpq_prepared_size(fpq.Format(5, 2, 16, fpq.SAT_PAPER).c(), ctypes.byref(d)) == 2 * 8 * 256
+    # 7 significant bits are 4 + 3: two terms again
+    assert L.fpq_prepared_size(fpq.Format(1, 6, 1, fpq.SAT_PAPER).c(), ctypes.byref(d)) == 2 * 8 * 256
+    # 64 binades fit no two terms of a tensor-core type: CUDA cores, codes as they are
+    assert L.fpq_prepared_size(fpq.Format(6, 1, 31, fpq.SAT_PAPER).c(), ctypes.byref(d)) == 8 * 256
     assert fpq.fpq_linear_workspace_size(100, 64, 200, fpq.E4M3, fpq.E2M5) == 100 * 512
     assert L.fpq_prepared_size(fpq.E2M1.c(), ctypes.byref(d)) == 8 * 256 // 2
     assert L.fpq_prepared_size(fpq.E1M2.c(), ctypes.byref(d)) == 8 * 256      # one E4M3 byte per weight

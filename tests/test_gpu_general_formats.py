@@ -16,10 +16,13 @@ pytestmark = pytest.mark.gpu
 E4M3_PAPER = fpq.Format(4, 3, 7, fpq.SAT_PAPER)
 E4M3_B8 = fpq.Format(4, 3, 8, fpq.SAT_PAPER)        # the paper's default bias 2^(e-1)
 E5M2_B16 = fpq.Format(5, 2, 16, fpq.SAT_PAPER)
-E2M1_TINY = fpq.Format(2, 1, 12, fpq.SAT_PAPER)      # a 4-bit format whose values E4M3 cannot hold
+E2M1_TINY = fpq.Format(2, 1, 12, fpq.SAT_PAPER)      # a 4-bit format whose values E4M3 cannot hold as they are
+E1M6 = fpq.Format(1, 6, 1, fpq.SAT_PAPER)            # 7 significant bits = 4 + 3: two E4M3 terms
+E6M1 = fpq.Format(6, 1, 31, fpq.SAT_PAPER)           # 64 binades: beyond any two tensor-core terms, CUDA cores
+E5M2_B40 = fpq.Format(5, 2, 40, fpq.SAT_PAPER)       # needs a factor beyond the 2^16 the split tries
 
 PAIRS = [(fpq.E4M3, fpq.E3M4), (fpq.E4M3, fpq.E2M5), (fpq.E4M3, fpq.E5M2), (fpq.E4M3, E5M2_B16), (fpq.E4M3, E4M3_PAPER),
-         (fpq.E4M3, E4M3_B8), (fpq.E4M3, E2M1_TINY),
+         (fpq.E4M3, E4M3_B8), (fpq.E4M3, E2M1_TINY), (fpq.E4M3, E1M6), (fpq.E4M3, E6M1), (fpq.E4M3, E5M2_B40), (fpq.E3M4, E5M2_B16),
          (fpq.E5M2, fpq.E4M3), (fpq.E3M4, fpq.E2M1), (E4M3_PAPER, fpq.E1M2), (fpq.E2M5, fpq.E3M4)]
 
 

@@ -68,3 +68,19 @@ def test_search_result_runs_as_a_layer():
         L.x, L.w, L.bias, L.bits = x, w, np.zeros(N, np.float32), None
         assert FMT[L.wfmt][0].c().exp_bits == g.c().exp_bits and FMT[L.wfmt][0].c().exp_bias == g.c().exp_bias
         _check_full(L, use_bias=False)
+
+
+# OCP E5M2 (bias 15, native saturation) is the tensor cores' second 8-bit operand type: read as it is
+@pytest.mark.parametrize("M,K,N", [(130, 200, 72), (300, 320, 960), (2, 1280, 320), (257, 1000, 4)])
+def test_linear_e5m2_native_weights(M, K, N):
+    L = I.linear_layer("t", M, K, N, "e5m2", rounding=True)
+    I.draw(L, 23, M + K + N, "normal", 0.02, True, 0.01, (0.001, 20.0))
+    _check_full(L)
+
+
+@pytest.mark.parametrize("shape", [(2, 40, 12, 12, 72, 3, 1), (1, 130, 9, 11, 33, 3, 2), (2, 256, 8, 8, 256, 3, 1)])
+def test_conv_e5m2_native_weights(shape):
+    B, C, H, W, Co, R, stride = shape
+    L = I.conv_layer("t", B, C, H, W, Co, R, stride=stride, wfmt="e5m2", rounding=True)
+    I.draw(L, 24, B + C + Co, "silu", 0.03, True, 0.01)
+    _check_full(L)
