@@ -102,3 +102,29 @@ def test_empty_and_nan_inputs(gfw):
     y2 = fpq.fpq_linear(x, prep, ws, 0.01, fpq.E4M3, gfw, None, N)
     assert fpq.fpq_read_status() == fpq.OK
     assert torch.equal(y, y2)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_search_choice_for_the_weights_runs_as_the_layer(bits):
+    # Sec. V-A end to end: Algorithm 1 picks an encoding and a clipping value for the weight tensor (per tensor, as
+    # in the paper), the clipping value becomes the scale, and the layer runs with exactly that format
+    L = I.linear_layer("t", 160, 384, 96)
+    I.draw(L, 34, bits, "normal", 0.02, False, 0.01)
+    encs_o = O.FP8_ENCODINGS if bits == 8 else O.FP4_ENCODINGS
+    encs_g = [fpq.Format(f.e, f.m, f.B, fpq.SAT_PAPER) for f in encs_o]
+    clips = fpq.fpq_search_clip_candidates(float(np.abs(L.w).max()), 111)
+    _, best = fpq.fpq_search_format(torch.from_numpy(L.w.reshape(-1)).cuda(), encs_g, clips.cuda())
+    i, j = (int(v) for v in best.cpu().numpy())
+    gfw, ofw = encs_g[i], encs_o[i]
+    scale = np.float32(clips.numpy()[j]) / np.float32(O.cmax(ofw))          # c = scale * c(F)
+    ws = np.full(L.N, scale, dtype=np.float32)
+    xs = fpq.fpq_scale_from_max(float(np.abs(L.x).max()), fpq.E4M3)
+    d = "cuda"
+    codes = fpq.fpq_quantize_weight(torch.from_numpy(L.w).to(d), torch.from_numpy(ws).to(d), gfw, None)
+    assert np.array_equal(codes.cpu().numpy(), O.quantize_weight(L.w, ws, ofw, None))
+    prep = fpq.fpq_prepare_weight(codes, gfw, fpq.LINEAR, L.N, L.K)
+    y = fpq.fpq_linear(torch.from_numpy(L.x).to(d), prep, torch.from_numpy(ws).to(d), xs, fpq.E4M3, gfw,
+                       torch.from_numpy(L.bias).to(d), L.N)
+    assert fpq.fpq_read_status() == fpq.OK
+    yr, ab = O.linear(L.x, L.w, ws, xs, O.E4M3, ofw, L.bias, None)
+    assert_close(y.cpu().numpy(), yr, ab)
