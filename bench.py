@@ -25,6 +25,7 @@ import statistics
 import sys
 import threading
 import time
+import zlib
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
@@ -174,7 +175,7 @@ class LayerOnGpu:
         self.fw = fpq.E4M3 if L.wfmt == "e4m3" else fpq.E2M1
         self.conv = L.kind == "conv"
         g = torch.Generator(device=dev)
-        g.manual_seed(1000 + (hash(L.name) & 0xffff))
+        g.manual_seed(1000 + (zlib.crc32(L.name.encode()) & 0xffff))      # the same draws in every process
         if L.w is not None:
             self.w = torch.from_numpy(L.w.reshape(L.N, -1)).to(dev)
             self.bias = torch.from_numpy(L.bias).to(dev)
@@ -352,46 +353,107 @@ def run_own(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- timed region: W warm-up steps, then exactly K steps replayed as one CUDA graph
+    # ---- timed region: W warm-up steps, then exactly K steps captured as one CUDA graph.  The graph is replayed
+    # R >= 20 times (at least 50 ms of device time in all), every replay bracketed by its own pair of CUDA events;
+    # ms_per_step is the median replay divided by K, the fastest replay is reported beside it.
     for _ in range(args.warmup):
         layer.step()
     torch.cuda.synchronize()
     steps_graph = GraphOf(torch, layer.step, args.steps)
-    steps_graph.timed_replay()                         # untimed: graph upload, clocks, L2 turnover
+    first_ms = steps_graph.timed_replay()              # untimed: graph upload, clocks, L2 turnover
+    reps = max(20, int(50.0 / max(first_ms, 1e-3)) + 1)
     sampler = ClockSampler(physical_gpu_index(local))
     barrier()
     sampler.start()
-    total_ms = steps_graph.timed_replay()
+    replay_ms = [steps_graph.timed_replay() for _ in range(reps)]
     barrier()
     clocks = sampler.stop()
     st = fpq.fpq_read_status()
     if st != fpq.OK:
         raise SystemExit(f"device status after the timed region: {fpq.status_string(st)}")
+    total_ms = statistics.median(replay_ms)
+    min_ms = min(replay_ms)
     if world > 1:
         total_ms = max_over_ranks(total_ms, dist, dev)
+        min_ms = max_over_ranks(min_ms, dist, dev)
     flops_step = L.flops
     value = whole_job_value(flops_step, args.steps, world, total_ms)
-    launches_per_step = 2
     t_layer = total_ms * 1e-3 / args.steps
 
-    # ---- per-kernel durations: each kernel alone, n launches rotating over the same buffer sets
+    # ---- the same graph replayed back to back for at least two seconds: the clocks settle under load, so the
+    # figure is given as time x median SM clock as well
+    sustained = None
+    if rank == 0:
+        n_sus = max(1, int(2000.0 / max(total_ms, 1e-3)))
+        s2 = ClockSampler(physical_gpu_index(local))
+        s2.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_sus):
+            steps_graph.g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        c2 = s2.stop()
+        us = e0.elapsed_time(e1) * 1e3 / (n_sus * args.steps)
+        sustained = {"seconds": e0.elapsed_time(e1) * 1e-3, "us_per_step": us, "sm_mhz_median": c2["sm_mhz"],
+                     "reasons": c2["reasons"], "us_x_ghz": us * (c2["sm_mhz"] or 0) * 1e-3,
+                     "tflops": flops_step / us / 1e6}
+
+    # ---- L2-warm: the same step on ONE buffer set (input 33.5 MB + output 33.5 MB stay in the 126 MB L2)
+    warm = None
+    if rank == 0:
+        lw = ConvLayerOnGpu(L, fpq, torch, dev, nsets=1)
+        for _ in range(3):
+            lw.step()
+        warm = per_launch_us(torch, lw.step, 20)
+        del lw
+        torch.cuda.empty_cache()
+
+    # ---- which kernels the step runs (the library's own choice), and each of them alone over the same buffer sets
+    route = fpq.fpq_conv2d_route(L.B, L.C, L.H, L.W, L.N, L.R, L.S, L.pad, L.stride, fpq.E4M3, layer.fw)
     n_k = 10 * layer.nsets
     t_q = per_launch_us(torch, layer.stage1, n_k) * 1e-6
     t_c = per_launch_us(torch, layer.stage2, n_k) * 1e-6
-    if t_c >= t_q:
-        dom, t_dom, b_dom = "fpq_gemm_kernel (contraction + epilogue)", t_c, layer.stage2_bytes()
+    kernels_us = {"activation_quantize (two-kernel route)": t_q * 1e6, "contraction (two-kernel route)": t_c * 1e6}
+    if route == fpq.ROUTE_TWO_KERNELS:
+        launches_per_step = 2
+        path = ("two kernels per step: activation quantize to framed channels-last codes, then the persistent "
+                "TMA/tcgen05 implicit GEMM with fused dequantize + bias")
+        if t_c >= t_q:
+            dom, t_dom, b_dom = "fpq_gemm_kernel (contraction + epilogue)", t_c, layer.stage2_bytes()
+        else:
+            dom, t_dom, b_dom = "quantize_nchw_to_nhwc_e4m3_kernel (activation quantize)", t_q, layer.stage1_bytes()
+        how = "each kernel replayed alone from a CUDA graph over the rotating buffer sets"
     else:
-        dom, t_dom, b_dom = "quantize_nchw_to_nhwc_e4m3_kernel (activation quantize)", t_q, layer.stage1_bytes()
+        launches_per_step = 1
+        if route == fpq.ROUTE_PAIR_FUSED:
+            dom = "fpq_pair_conv_kernel (activation quantize + contraction + epilogue on CTA pairs)"
+            path = ("one kernel per step: FP32 activations staged by TMA, quantized to E4M3 in shared memory, "
+                    "tcgen05 cta_group::2 MMAs with the weights resident in shared memory, fused dequantize + bias")
+        else:
+            dom = "fpq_gemm_kernel (fused form: activation quantize + contraction + epilogue)"
+            path = "one kernel per step: activations quantized inside the contraction's operand staging"
+        # the step IS the kernel: its duration is the timed region's, its bytes the layer's algorithmic bytes
+        t_dom, b_dom = t_layer, layer.layer_bytes()
+        kernels_us[dom] = t_dom * 1e6
+        how = "the step is one kernel: CUDA events around the timed region's graph replays (median)"
     achieved = b_dom / t_dom / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": TRAFFIC.get(dom),
                 "algorithmic_bytes_per_launch": b_dom, "us_per_launch": t_dom * 1e6,
-                "kernels_us": {"activation_quantize": t_q * 1e6, "contraction": t_c * 1e6},
-                "how": "each kernel replayed alone from a CUDA graph over the rotating buffer sets"}
+                "kernels_us": kernels_us, "how": how}
     layer_roof = {"algorithmic_bytes": layer.layer_bytes(), "achieved_gbs": layer.layer_bytes() / t_layer / 1e9,
                   "frac_of_hbm_peak": layer.layer_bytes() / t_layer / 1e9 / peaks["hbm_gbs"],
                   "t_hbm_us": layer.layer_bytes() / (peaks["hbm_gbs"] * 1e9) * 1e6,
                   "t_tensor_us_nominal_fp8": flops_step / (NOMINAL_FP8_TFLOPS * 1e12) * 1e6}
+    # every route of the library on the same step, for comparison
+    routes_us = {}
+    for name, pol in (("fused", fpq.PATH_FUSED), ("two_kernels", fpq.PATH_TWO_KERNELS)):
+        fpq.fpq_set_path_policy(pol)
+        for _ in range(2):
+            layer.step()
+        routes_us[name] = per_launch_us(torch, layer.step, n_k)
+    fpq.fpq_set_path_policy(fpq.PATH_AUTO)
 
     # ---- the same K steps launched one by one from the host (launch-bound), for comparison
     evs = []
@@ -491,6 +553,9 @@ def run_own(args):
             side["linear_qkv_320_960_m8192_weights_" + fname] = {"us": t * 1e6, "tflops": 2.0 * M * N * K / t / 1e12}
         del w, a, alpha, x, y, wk
         torch.cuda.empty_cache()
+        # the other workloads of the metric: the transformer-block linears and the whole U-Net step
+        side["config4_transformer_linears_m8192"] = config4_measure(torch, fpq, I, dev, peaks)
+        side["sd_v1_unet_step_trace"] = trace_measure(torch, fpq, I, dev, peaks, 5)
 
     # ---- CPU baseline: the oracle, as it stands, on the host cores (rank 0, N = 1 only)
     cpu = None
@@ -510,14 +575,15 @@ def run_own(args):
             "config": {"workload": WORKLOAD,
                        "l2": f"inputs larger than L2: steps rotate over {layer.nsets} resident (x, scratch, y) sets, "
                              f"{layer.nsets * layer.set_bytes >> 20} MiB",
-                       "launch": "the K timed steps are one CUDA graph replay",
-                       "path": "two kernels per step: activation quantize to framed channels-last codes, "
-                               "then the persistent TMA/tcgen05 implicit GEMM with fused dequantize + bias"},
+                       "launch": f"the K timed steps are one CUDA graph; {reps} replays, each timed by its own pair of "
+                                 "CUDA events; ms_per_step = median replay / K",
+                       "path": path},
             "pct_dense_fp8_peak_nominal": 100 * value / world / NOMINAL_FP8_TFLOPS,
             "pct_dense_fp8_peak_2x_measured_bf16": 100 * value / world / (2 * peaks["bf16_tflops"]),
             "roofline": roofline, "layer_roofline": layer_roof, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
-            "weight_encode_us": enc_us, "w4a8": w4, "standalone_quantizer": quant, "eager_step_us": eager_us,
+            "min_ms_per_step": min_ms / args.steps, "replays": reps, "sustained": sustained, "l2_warm_us_per_step": warm,
+            "routes_us": routes_us, "weight_encode_us": enc_us, "w4a8": w4, "standalone_quantizer": quant, "eager_step_us": eager_us,
             "side_measurements": side,
         }
         print(json.dumps(line), flush=True)
@@ -525,21 +591,11 @@ def run_own(args):
         dist.destroy_process_group()
 
 
-def run_trace(args):
+def trace_measure(torch, fpq, I, dev, peaks, reps):
     """One denoising step of the SD-v1-style U-Net as a layer trace: all 234 conv / linear
     layers (W4A8 with rounding decisions), each with its own buffers, launched back to back on one
     stream and replayed as one CUDA graph.  The buffers of one pass total several GB, so every
     layer finds its input in HBM."""
-    import torch
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device")
-    dev = torch.device("cuda", 0)
-    torch.cuda.set_device(0)
-    from paper_2408_06995_b200 import build as fpq_build
-    fpq_build.build()
-    import paper_2408_06995_b200 as fpq
-    from paper_2408_06995_b200 import inputs as I
-    peaks = load_peaks()
     trace = I.sd_v1_unet_layers()
     layers = [LayerOnGpu(L, fpq, torch, dev, nsets=1) for L in trace]
     torch.cuda.synchronize()
@@ -553,7 +609,7 @@ def run_trace(args):
     torch.cuda.synchronize()
     g = GraphOf(torch, one_pass, 1)
     g.timed_replay()
-    ms = [g.timed_replay() for _ in range(max(3, min(args.steps, 20)))]
+    ms = [g.timed_replay() for _ in range(reps)]
     st = fpq.fpq_read_status()
     if st != fpq.OK:
         raise SystemExit(f"device status: {fpq.status_string(st)}")
@@ -562,13 +618,45 @@ def run_trace(args):
     bound_us = sum(max(lay.layer_bytes() / (peaks["hbm_gbs"] * 1e9), lay.L.flops / (NOMINAL_FP8_TFLOPS * 1e12)) * 1e6
                    for lay in layers)
     t = statistics.median(ms) * 1e-3
-    print(json.dumps({"suite": "sd_trace", "layers": len(layers), "gflop": flops / 1e9, "algorithmic_mb": bytes_ / 1e6,
-                      "ms_per_step": t * 1e3, "min_ms": min(ms), "aggregate_tflops": flops / t / 1e12,
-                      "pct_dense_fp8_peak_nominal": 100 * flops / t / 1e12 / NOMINAL_FP8_TFLOPS,
-                      "pct_dense_fp4_peak_nominal": 100 * flops / t / 1e12 / NOMINAL_FP4_TFLOPS,
-                      "sum_of_per_layer_bounds_us": bound_us, "frac_of_bound": bound_us * 1e-6 / t,
-                      "device_buffers_gb": sum(l.set_bytes for l in layers) / 1e9, "launch": "one CUDA graph replay"}),
-          flush=True)
+    out = {"suite": "sd_trace", "layers": len(layers), "gflop": flops / 1e9, "algorithmic_mb": bytes_ / 1e6,
+           "ms_per_step": t * 1e3, "min_ms": min(ms), "aggregate_tflops": flops / t / 1e12,
+           "pct_dense_fp8_peak_nominal": 100 * flops / t / 1e12 / NOMINAL_FP8_TFLOPS,
+           "pct_dense_fp4_peak_nominal": 100 * flops / t / 1e12 / NOMINAL_FP4_TFLOPS,
+           "sum_of_per_layer_bounds_us": bound_us, "frac_of_bound": bound_us * 1e-6 / t,
+           "device_buffers_gb": sum(l.set_bytes for l in layers) / 1e9, "launch": "one CUDA graph replay"}
+    del layers, g
+    torch.cuda.empty_cache()
+    return out
+
+
+def config4_measure(torch, fpq, I, dev, peaks):
+    """The eight SD-v1-style transformer-block linears (M = 8192; W8A8 and W4A8), each timed as a CUDA graph of
+    calls that rotate over buffer sets larger than the L2: the sum against the sum of the per-layer bounds."""
+    rows, tot, bound = {}, 0.0, 0.0
+    for L in I.config4():
+        lay = LayerOnGpu(L, fpq, torch, dev)
+        for _ in range(2):
+            lay.step()
+        us = per_launch_us(torch, lay.step, max(4, min(40, 3 * lay.nsets)), reps=2)
+        b = max(lay.layer_bytes() / (peaks["hbm_gbs"] * 1e9), L.flops / (NOMINAL_FP8_TFLOPS * 1e12)) * 1e6
+        rows[L.name] = {"us": us, "bound_us": b}
+        tot, bound = tot + us, bound + b
+        del lay
+        torch.cuda.empty_cache()
+    return {"sum_us": tot, "sum_of_bounds_us": bound, "frac_of_bound": bound / tot, "layers": rows}
+
+
+def run_trace(args):
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    from paper_2408_06995_b200 import build as fpq_build
+    fpq_build.build()
+    import paper_2408_06995_b200 as fpq
+    from paper_2408_06995_b200 import inputs as I
+    print(json.dumps(trace_measure(torch, fpq, I, dev, load_peaks(), max(3, min(args.steps, 20)))), flush=True)
 
 
 def run_suite(args):
@@ -584,7 +672,9 @@ def run_suite(args):
     import paper_2408_06995_b200 as fpq
     from paper_2408_06995_b200 import inputs as I
     peaks = load_peaks()
-    if args.suite == "ldm":
+    if args.suite == "cifar":
+        layers = I.config2()
+    elif args.suite == "ldm":
         layers = I.config3()
     elif args.suite == "transformer":
         layers = I.config4()
@@ -868,7 +958,7 @@ def main():
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline leg")
     ap.add_argument("--skip-w4", action="store_true", help="leave out the W4A8 side measurement")
-    ap.add_argument("--suite", default=None, choices=["ldm", "transformer", "sd", "sd_trace", "search", "sd_split", "round_learn", "formats"],
+    ap.add_argument("--suite", default=None, choices=["cifar", "ldm", "transformer", "sd", "sd_trace", "search", "sd_split", "round_learn", "formats"],
                     help="print a per-shape table of a whole workload instead of the headline line")
     ap.add_argument("--only", default=None, help="with --suite ldm|transformer|sd|round_learn: only the layers whose name contains this; "
                     "with --suite formats: only the weight formats whose name contains this")

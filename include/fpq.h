@@ -19,9 +19,12 @@
  *     buffers); the library takes turns inside where it keeps per-device tables.
  *     fpq_set_path_policy and fpq_linear_static are the exceptions stated at their
  *     declarations.
+ *   - The first layer call on a device (fpq_linear, fpq_conv2d and their forms) sets kernel
+ *     attributes and asks the driver how many thread-block clusters fit: make it outside any
+ *     stream capture.  Later calls only enqueue kernels and can be captured.
  *   - Errors are return codes (negative).  Whatever the host can check (null or
- *     misaligned pointers, impossible formats, shapes, workspace size) is
- *     rejected before anything is launched.
+ *     misaligned pointers, impossible formats, shapes, workspace size, an activation
+ *     scale that is not a positive finite number) is rejected before anything is launched.
  *
  * Number format (Sec. IV-B, format equation): a code has 1 sign bit, exp_bits
  * exponent bits p and man_bits mantissa bits d, value
@@ -56,7 +59,8 @@ enum {
     FPQ_ERR_CUDA = -7,        /* a CUDA runtime / driver call failed */
     FPQ_ERR_TIMEOUT = -8,     /* a bounded device-side wait expired (device status) */
     FPQ_ERR_NAN_INPUT = -9,   /* a NaN was quantized (to code 0) (device status) */
-    FPQ_ERR_TOO_LARGE = -10   /* problem exceeds a fixed built-in capacity */
+    FPQ_ERR_TOO_LARGE = -10,  /* problem exceeds a fixed built-in capacity */
+    FPQ_ERR_SCALE = -11       /* an activation scale is zero, negative, infinite or NaN */
 };
 
 enum { FPQ_SAT_PAPER = 0, FPQ_SAT_NATIVE = 1 };
@@ -397,20 +401,50 @@ fpq_status fpq_round_learn_harden(const float* alpha, int64_t N, int64_t K, uint
 
 /*
  * Which route fpq_linear / fpq_conv2d take (process-wide setting, not thread-safe against
- * concurrent layer calls; the results are the same bit for bit on either route):
+ * concurrent layer calls).  Every route multiplies the same codes exactly and adds in FP32, so the
+ * results agree within the layer tolerance; routes that run the same MMAs in the same order agree
+ * bit for bit.
  *   FPQ_PATH_FUSED        one kernel: the activation quantize (Sec. IV-B rounding equation) runs
  *                         inside the contraction's operand staging, the codes never reach global
- *                         memory.  Available for linear layers and stride-1 convolutions; other
- *                         geometries fall back to two kernels.
+ *                         memory (the layer of Sec. VI-A as one pass: FP32 in -> quantize -> low-bit
+ *                         MAC -> FP32 out).  Stride-1 convolutions whose whole weight tensor fits in
+ *                         the shared memory of a pair of SMs run on CTA pairs (tcgen05 cta_group::2);
+ *                         linear layers and the other stride-1 convolutions use the general fused
+ *                         form; other geometries fall back to two kernels.
  *   FPQ_PATH_TWO_KERNELS  always *_quantize_input followed by *_contract.
- *   FPQ_PATH_AUTO         the library's choice per layer kind (default).
+ *   FPQ_PATH_AUTO         the library's choice per shape (default): the CTA-pair kernel where it
+ *                         applies and measured faster, else two kernels.
  */
 enum { FPQ_PATH_AUTO = 0, FPQ_PATH_FUSED = 1, FPQ_PATH_TWO_KERNELS = 2 };
 fpq_status fpq_set_path_policy(int32_t policy);
 int32_t fpq_get_path_policy(void);
 
+/*
+ * Which kernels fpq_conv2d would run for this shape under the current policy, for logs and
+ * benchmarks (pointer alignment is assumed to be as documented; nothing is launched):
+ *   FPQ_ROUTE_TWO_KERNELS  activation-quantize kernel, then the contraction kernel;
+ *   FPQ_ROUTE_FUSED        the general one-kernel form;
+ *   FPQ_ROUTE_PAIR_FUSED   the one-kernel form on CTA pairs with resident weights;
+ *   FPQ_ROUTE_OTHER        formats the tensor cores have no type for (CUDA cores), or two-term weights;
+ *   negative               the error fpq_conv2d would return for these arguments.
+ */
+enum { FPQ_ROUTE_TWO_KERNELS = 0, FPQ_ROUTE_FUSED = 1, FPQ_ROUTE_PAIR_FUSED = 2, FPQ_ROUTE_OTHER = 3 };
+int32_t fpq_conv2d_route(int B, int C, int H, int W, int C_out, int R, int S, int pad, int stride,
+                         fpq_format fx, fpq_format fw);
+
+/*
+ * Diagnostic (the paper has no counterpart): launches one warp that waits on a barrier nobody ever
+ * arrives on, with the same bounded wait every role of the layer kernels uses, limited to
+ * limit_cycles SM clock cycles (1 .. 1e9).  The wait runs out, the warp records FPQ_ERR_TIMEOUT in the
+ * device status word and the kernel returns: the context stays usable, which is what a caller's
+ * failure handling relies on.  Returns FPQ_OK when the kernel was enqueued (the time-out shows in
+ * fpq_read_status), FPQ_ERR_SHAPE for a limit out of range, FPQ_ERR_CUDA.
+ */
+fpq_status fpq_selftest_bounded_wait(int64_t limit_cycles, void* stream);
+
 /* Waits for `stream`, then returns and clears the sticky device status word:
- * FPQ_OK, FPQ_ERR_TIMEOUT, FPQ_ERR_NAN_INPUT, or FPQ_ERR_CUDA. */
+ * FPQ_OK, FPQ_ERR_TIMEOUT, FPQ_ERR_NAN_INPUT, or FPQ_ERR_CUDA.  The word keeps one bit per kind of
+ * event; when both have happened FPQ_ERR_TIMEOUT (an incomplete output) is the one reported. */
 fpq_status fpq_read_status(void* stream);
 
 const char* fpq_status_string(fpq_status s);

@@ -252,18 +252,16 @@ def search_mse(x, encodings, clips) -> np.ndarray:
 
 
 def select_encoding_and_bias(mse: np.ndarray):
-    """Algorithm 1: walk the encodings (outer loop) and the bias candidates (inner loop) and keep
-    a candidate only when its error is strictly below the best so far.  The best-so-far starts
-    at +infinity: the listing's printed start value of 0 would never accept any candidate."""
-    best = (None, None)
-    prev_mse = float("inf")
-    for i in range(mse.shape[0]):
-        for j in range(mse.shape[1]):
-            curr_mse = float(mse[i, j])
-            if prev_mse > curr_mse:
-                best = (i, j)
-                prev_mse = curr_mse
-    return best
+    """The selection rule of Algorithm 1 (Sec. V-A): the (encoding, bias candidate) pair with the smallest
+    error; among equal errors the first one in encoding-major, candidate-minor order.  The listing prints a
+    start value of 0 for the best error so far, which no candidate could ever beat: read as +infinity.  A
+    NaN error is never selected, and with no finite-or-infinite error below +infinity nothing is selected."""
+    m = np.asarray(mse, dtype=np.float64)
+    flat = np.where(np.isnan(m), np.inf, m).reshape(-1)
+    if flat.size == 0 or not np.any(flat < np.inf):
+        return (None, None)
+    k = int(np.argmin(flat))                      # argmin returns the first occurrence of the minimum
+    return (k // m.shape[1], k % m.shape[1])
 
 
 # ---- sparsity of a quantized tensor (the paper's sparsity study) --------------------------

@@ -18,7 +18,8 @@ _SO = os.path.join(_HERE, "libfpq.so")
 
 OK = 0
 ERR_NULL, ERR_FORMAT, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED = -1, -2, -3, -4, -5
-ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NAN_INPUT, ERR_TOO_LARGE = -6, -7, -8, -9, -10
+ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NAN_INPUT, ERR_TOO_LARGE, ERR_SCALE = -6, -7, -8, -9, -10, -11
+ROUTE_TWO_KERNELS, ROUTE_FUSED, ROUTE_PAIR_FUSED, ROUTE_OTHER = 0, 1, 2, 3
 STATIC_SCRATCH_BYTES = 8 << 20
 SAT_PAPER, SAT_NATIVE = 0, 1
 LINEAR, CONV2D = 0, 1
@@ -72,6 +73,7 @@ EXPORTS = [
     "fpq_round_learn_workspace_size", "fpq_round_learn_step", "fpq_round_learn_harden", "fpq_round_learn_unfold",
     "fpq_zero_census", "fpq_prepared_size_split", "fpq_prepare_weight_split", "fpq_conv2d_split_workspace_size",
     "fpq_conv2d_split", "fpq_set_path_policy", "fpq_get_path_policy", "fpq_read_status", "fpq_status_string",
+    "fpq_conv2d_route", "fpq_selftest_bounded_wait",
 ]
 
 _lib = None
@@ -151,6 +153,10 @@ def lib() -> ctypes.CDLL:
         L.fpq_set_path_policy.argtypes = [i32]
         L.fpq_get_path_policy.restype = i32
         L.fpq_get_path_policy.argtypes = []
+        L.fpq_selftest_bounded_wait.restype = i32
+        L.fpq_selftest_bounded_wait.argtypes = [i64, vp]
+        L.fpq_conv2d_route.restype = i32
+        L.fpq_conv2d_route.argtypes = [i32] * 9 + [F, F]
         L.fpq_read_status.restype = i32
         L.fpq_read_status.argtypes = [vp]
         L.fpq_status_string.restype = ctypes.c_char_p
@@ -451,6 +457,19 @@ def fpq_set_path_policy(policy: int) -> None:
 
 def fpq_get_path_policy() -> int:
     return lib().fpq_get_path_policy()
+
+
+def fpq_selftest_bounded_wait(limit_cycles: int) -> None:
+    """One warp waits limit_cycles on a barrier nobody arrives on, then records ERR_TIMEOUT in the status word."""
+    _check(lib().fpq_selftest_bounded_wait(int(limit_cycles), _stream()), "fpq_selftest_bounded_wait")
+
+
+def fpq_conv2d_route(B, C, H, W, C_out, R, S, pad, stride, fx: Format, fw: Format) -> int:
+    """Which kernels fpq_conv2d would run for this shape under the current policy (ROUTE_*)."""
+    r = lib().fpq_conv2d_route(B, C, H, W, C_out, R, S, pad, stride, fx.c(), fw.c())
+    if r < 0:
+        _check(r, "fpq_conv2d_route")
+    return r
 
 
 def fpq_read_status() -> int:

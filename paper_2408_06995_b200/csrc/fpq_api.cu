@@ -1,5 +1,6 @@
 // extern "C" entry points: argument checks, format resolution, dispatch.
 #include <math.h>
+#include <cmath>
 #include <string.h>
 
 #include <map>
@@ -16,9 +17,11 @@ int* status_word()
 {
     // one lookup per device: the symbol has a separate instance on each GPU
     static int* ptr[64] = {nullptr};
+    static std::mutex mu;                      // host threads may make their first call at the same time
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
         return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
     if (!ptr[dev]) {
         void* p = nullptr;
         if (cudaGetSymbolAddress(&p, g_status) != cudaSuccess)
@@ -260,6 +263,9 @@ static int g_path_policy = FPQ_PATH_AUTO;
 
 static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 
+// an activation scale must be a positive finite number: 1 / scale is what the kernels multiply by
+static bool bad_scale(float s) { return !(s > 0.f) || std::isinf(s); }
+
 static int64_t padded_c(int64_t C) { return round_up(C, 128); }
 
 static fpq_status check_pair(fpq_format fx, fpq_format fw)
@@ -319,6 +325,8 @@ fpq_status fpq_quantize_weight(const float* w, int64_t N, int64_t K, const float
 
 fpq_status fpq_quantize_act(const float* x, int64_t n, float scale, fpq_format fmt, uint8_t* codes, void* stream)
 {
+    if (bad_scale(scale))
+        return FPQ_ERR_SCALE;
     QFormat q;
     if (!resolve_format(fmt, &q))
         return FPQ_ERR_FORMAT;
@@ -427,6 +435,8 @@ static fpq_status linear_checks(fpq_format fx, fpq_format fw, int64_t M, int64_t
 fpq_status fpq_linear_quantize_input(const float* x, float x_scale, fpq_format fx, fpq_format fw, int64_t M, int64_t N,
                                      int64_t K, void* workspace, size_t ws_bytes, void* stream)
 {
+    if (bad_scale(x_scale))
+        return FPQ_ERR_SCALE;
     bool empty = false;
     fpq_status s = linear_checks(fx, fw, M, N, K, workspace, ws_bytes, &empty);
     if (s != FPQ_OK || empty)
@@ -448,6 +458,8 @@ static fpq_status linear_contract_impl(const void* workspace, size_t ws_bytes, c
                                        const float* bias, float* y, int64_t M, int64_t N, int64_t K, void* stream,
                                        int after_stage1, const float* x_fused)
 {
+    if (bad_scale(x_scale))
+        return FPQ_ERR_SCALE;
     bool empty = false;
     fpq_status s = linear_checks(fx, fw, M, N, K, workspace, ws_bytes, &empty);
     if (s != FPQ_OK || empty)
@@ -494,6 +506,8 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
                       fpq_format fw, const float* bias, float* y, int64_t M, int64_t N, int64_t K, void* workspace,
                       size_t ws_bytes, void* stream)
 {
+    if (bad_scale(x_scale))
+        return FPQ_ERR_SCALE;
     if (general_pair(fx, fw)) {
         if (M < 0 || N < 0 || K < 0 || M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff)
             return FPQ_ERR_SHAPE;
@@ -658,6 +672,8 @@ fpq_status fpq_conv2d_quantize_input(const float* x, float x_scale, fpq_format f
                                      int W, int C_out, int R, int S, int pad, int stride, void* workspace,
                                      size_t ws_bytes, void* stream)
 {
+    if (bad_scale(x_scale))
+        return FPQ_ERR_SCALE;
     int Ho, Wo;
     bool empty = false;
     fpq_status s = conv_checks(fx, fw, B, C, H, W, C_out, R, S, pad, stride, workspace, ws_bytes, &Ho, &Wo, &empty);
@@ -679,8 +695,10 @@ static fpq_status conv2d_contract_impl(const void* workspace, size_t ws_bytes, c
                                        const float* w_scale, float x_scale, fpq_format fx, fpq_format fw,
                                        const float* bias, float* y, int B, int C, int H, int W, int C_out, int R,
                                        int S, int pad, int stride, void* stream, int after_stage1,
-                                       const float* x_fused)
+                                       const float* x_fused, bool pair_only = false)
 {
+    if (bad_scale(x_scale))
+        return FPQ_ERR_SCALE;
     int Ho, Wo;
     bool empty = false;
     fpq_status s = conv_checks(fx, fw, B, C, H, W, C_out, R, S, pad, stride, workspace, ws_bytes, &Ho, &Wo, &empty);
@@ -718,6 +736,16 @@ static fpq_status conv2d_contract_impl(const void* workspace, size_t ws_bytes, c
     p.x_scale = x_scale;
     p.bias = bias;
     p.y = y;
+    if (x_fused) {
+        // one kernel on CTA pairs where the weights fit in shared memory; else the general fused form
+        if (!pair_only || pair_conv_preferred(p)) {
+            const fpq_status sp = launch_pair_conv(p, (cudaStream_t)stream);
+            if (sp != FPQ_ERR_UNSUPPORTED)
+                return sp;
+        }
+        if (pair_only)
+            return FPQ_ERR_UNSUPPORTED;
+    }
     return launch_gemm(p, (cudaStream_t)stream);
 }
 
@@ -733,6 +761,8 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
                       fpq_format fw, const float* bias, float* y, int B, int C, int H, int W, int C_out, int R, int S,
                       int pad, int stride, void* workspace, size_t ws_bytes, void* stream)
 {
+    if (bad_scale(x_scale))
+        return FPQ_ERR_SCALE;
     if (general_pair(fx, fw)) {
         GeneralLayer g = {};
         if (!general_conv(&g, fx, fw, B, C, H, W, C_out, R, S, pad, stride))
@@ -789,9 +819,10 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
         return FPQ_ERR_ALIGN;
     // one kernel where the geometry allows it (stride 1): the activations are quantized inside the
     // contraction's operand staging; otherwise quantize to codes first
-    if (g_path_policy == FPQ_PATH_FUSED) {
+    // (the library's own choice: the CTA-pair kernel for the shapes it measured faster on, else two kernels)
+    if (g_path_policy == FPQ_PATH_FUSED || g_path_policy == FPQ_PATH_AUTO) {
         s = conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out,
-                                 R, S, pad, stride, stream, 0, x);
+                                 R, S, pad, stride, stream, 0, x, g_path_policy == FPQ_PATH_AUTO);
         if (s != FPQ_ERR_UNSUPPORTED)
             return s;
     }
@@ -865,6 +896,8 @@ fpq_status fpq_conv2d_split(const float* x1, int C1, float x1_scale, const float
                             const float* bias, float* y, int B, int H, int W, int C_out, int R, int S, int pad,
                             int stride, void* workspace, size_t ws_bytes, void* stream)
 {
+    if (bad_scale(x1_scale) || bad_scale(x2_scale))
+        return FPQ_ERR_SCALE;
     fpq_status s = check_pair(fx, fw);
     if (s != FPQ_OK)
         return s;
@@ -1191,6 +1224,52 @@ fpq_status fpq_round_learn_harden(const float* alpha, int64_t N, int64_t K, uint
     return launch_round_harden(alpha, N, K, rounding_bits, (cudaStream_t)stream);
 }
 
+int32_t fpq_conv2d_route(int B, int C, int H, int W, int C_out, int R, int S, int pad, int stride, fpq_format fx,
+                         fpq_format fw)
+{
+    if (general_pair(fx, fw) || two_term_pair(fx, fw)) {
+        QFormat q;
+        if (!resolve_format(fx, &q) || !resolve_format(fw, &q))
+            return FPQ_ERR_FORMAT;
+        return FPQ_ROUTE_OTHER;
+    }
+    fpq_status s = check_pair(fx, fw);
+    if (s != FPQ_OK)
+        return s;
+    int Ho, Wo;
+    s = conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo);
+    if (s != FPQ_OK)
+        return s;
+    if (g_path_policy == FPQ_PATH_TWO_KERNELS || B == 0 || C_out == 0)
+        return FPQ_ROUTE_TWO_KERNELS;
+    GemmProblem p{};
+    p.conv = 1;
+    p.x = reinterpret_cast<const float*>((uintptr_t)256);      // never followed: the plans only look at its alignment
+    p.C = C;
+    p.w4 = is_e2m1(fw) ? 1 : 0;
+    p.w_e5m2 = is_e5m2_native(fw) ? 1 : 0;
+    p.M = (int64_t)B * Ho * Wo;
+    p.N = C_out;
+    p.Cp = (int)padded_c(C);
+    p.Ca = (int)round_up(C, 16);
+    p.B = B, p.H = H, p.W = W, p.Ho = Ho, p.Wo = Wo, p.R = R, p.S = S, p.pad = pad, p.stride = stride;
+    if (pair_conv_applies(p) && (g_path_policy == FPQ_PATH_FUSED || pair_conv_preferred(p)))
+        return FPQ_ROUTE_PAIR_FUSED;
+    if (g_path_policy == FPQ_PATH_FUSED && stride == 1)
+        return FPQ_ROUTE_FUSED;                                  // (the general fused form; it may still fall back)
+    return FPQ_ROUTE_TWO_KERNELS;
+}
+
+fpq_status fpq_selftest_bounded_wait(int64_t limit_cycles, void* stream)
+{
+    if (limit_cycles < 1 || limit_cycles > 1000000000ll)
+        return FPQ_ERR_SHAPE;
+    int* sw = status_word();
+    if (!sw)
+        return FPQ_ERR_CUDA;
+    return launch_bounded_wait_selftest(limit_cycles, sw, (cudaStream_t)stream) == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
+}
+
 fpq_status fpq_set_path_policy(int32_t policy)
 {
     if (policy != FPQ_PATH_AUTO && policy != FPQ_PATH_FUSED && policy != FPQ_PATH_TWO_KERNELS)
@@ -1213,7 +1292,12 @@ fpq_status fpq_read_status(void* stream)
         return FPQ_ERR_CUDA;
     if (v != 0 && cudaMemcpy(sw, &zero, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess)
         return FPQ_ERR_CUDA;
-    return (fpq_status)v;
+    // one bit per kind of event; the most serious one is reported
+    if (v & STATUS_BIT_TIMEOUT)
+        return FPQ_ERR_TIMEOUT;
+    if (v & STATUS_BIT_NAN)
+        return FPQ_ERR_NAN_INPUT;
+    return FPQ_OK;
 }
 
 const char* fpq_status_string(fpq_status s)
@@ -1227,6 +1311,7 @@ const char* fpq_status_string(fpq_status s)
     case FPQ_ERR_UNSUPPORTED: return "unsupported operand formats or geometry";
     case FPQ_ERR_WORKSPACE: return "workspace missing or too small";
     case FPQ_ERR_CUDA: return "CUDA call failed";
+    case FPQ_ERR_SCALE: return "activation scale is not a positive finite number";
     case FPQ_ERR_TIMEOUT: return "device-side wait timed out";
     case FPQ_ERR_NAN_INPUT: return "NaN input quantized to zero";
     case FPQ_ERR_TOO_LARGE: return "problem larger than the built-in scratch capacity";

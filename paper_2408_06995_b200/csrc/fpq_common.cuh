@@ -24,6 +24,15 @@ float format_cmax(fpq_format f);
 // sticky device status word (defined in fpq_api.cu)
 int* status_word();
 
+// The status word holds one bit per kind of device-side event, so that a benign event (a NaN input quantized
+// to zero) can never hide a serious one (a bounded wait that ran out, which leaves the output incomplete).
+// fpq_read_status reports the most serious bit that is set.
+constexpr int STATUS_BIT_NAN = 1, STATUS_BIT_TIMEOUT = 2;
+__device__ __forceinline__ void flag_status(int* status, int code)
+{
+    atomicOr(status, code == FPQ_ERR_TIMEOUT ? STATUS_BIT_TIMEOUT : STATUS_BIT_NAN);
+}
+
 __host__ __device__ inline int64_t round_up(int64_t a, int64_t b) { return (a + b - 1) / b * b; }
 
 // ---- the quantizer on one element ---------------------------------------------
@@ -152,18 +161,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait: gives up after about two seconds (4e9 SM cycles) and reports false.
+// Bounded wait: gives up after `limit` SM cycles (by default 4e9, about two seconds) and reports false.
 // The cycle counter is only consulted every 1024 unsuccessful polls.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+constexpr long long MBAR_WAIT_LIMIT = 4000000000ll;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit = MBAR_WAIT_LIMIT)
 {
     if (mbar_try_wait(bar, parity))
         return true;
     const long long t0 = clock64();
     for (;;) {
-        for (int i = 0; i < 1024; ++i)
+        for (int i = 0; i < 1024; ++i) {
             if (mbar_try_wait(bar, parity))
                 return true;
-        if (clock64() - t0 > 4000000000ll)
+            __nanosleep(40);      // a waiting warp must not take issue slots from the warps that work
+        }
+        if (clock64() - t0 > limit)
             return false;
     }
 }
@@ -310,6 +322,162 @@ constexpr uint32_t SMEM_DESC_HI_K_SW128 = 64u | (1u << 14) | (2u << 29);
 __host__ __device__ inline uint32_t idesc_f8f6f4(uint32_t a_fmt, uint32_t b_fmt, uint32_t n)
 {
     return (1u << 4) | (a_fmt << 7) | (b_fmt << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// Division of a 31-bit unsigned number by a constant known on the host:
+// n / d = (umulhi(n, mul) + n) >> shift.
+struct FastDiv {
+    uint32_t mul, shift;
+};
+
+inline FastDiv make_fastdiv(uint32_t d)
+{
+    FastDiv f{0, 0};
+    if (d > 1) {
+        uint32_t s = 0;
+        while ((1ull << s) < d)
+            ++s;
+        f.shift = s;
+        f.mul = (uint32_t)((((1ull << 32) * ((1ull << s) - d)) / d) + 1);
+    }
+    return f;
+}
+
+__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f)
+{
+    return (uint32_t)(((uint64_t)__umulhi(n, f.mul) + n) >> f.shift);
+}
+
+// ---- thread-block cluster: barrier over all threads of all CTAs, and reads of a peer CTA's shared memory
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+// address of this CTA's shared-memory location `local_addr` in CTA `peer` of the cluster
+__device__ __forceinline__ uint32_t peer_smem_addr(uint32_t local_addr, uint32_t peer)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(peer));
+    return remote;
+}
+
+__device__ __forceinline__ float4 ld_cluster_smem4(uint32_t cluster_addr)
+{
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(cluster_addr)
+                 : "memory");
+    return v;
+}
+
+// ---- CTA pairs (cta_group::2): one MMA spans the tensor cores and tensor memory of two CTAs of a cluster.
+// Both CTAs allocate / free tensor memory with these; the MMAs and commits are issued by one thread of
+// the cluster's first CTA, which names both CTAs' shared memory by the same offsets.
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+
+__device__ __forceinline__ void tmem_relinquish_pair()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// D[tmem of both CTAs] (+)= A * B with M = 256: each CTA holds 128 rows of A and of D, and half of B's rows.
+template <bool ACC>
+__device__ __forceinline__ void mma_f8f6f4_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc)
+{
+    if (ACC) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "setp.eq.u32 p, 1, 1;\n\t"
+            "mov.b64 da, {%1, %3};\n\t"
+            "mov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], da, db, %4, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "setp.eq.u32 p, 1, 0;\n\t"
+            "mov.b64 da, {%1, %3};\n\t"
+            "mov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], da, db, %4, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc)
+            : "memory");
+    }
+}
+
+// one arrival on the barrier at this shared-memory offset in every CTA of `mask`, once all MMAs issued so
+// far by this thread are done
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar, uint16_t mask)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+
+// TMA load into this CTA's shared memory whose completion is reported to a barrier of the pair's first CTA
+// (cluster-space address)
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
+// arrival on a barrier anywhere in the cluster (cluster-space address)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar)
+{
+    // (default semantics, release at CTA scope: the cluster-scope release form took 1.8 us per arrival here; what
+    // the other CTA's MMA reads afterwards is this CTA's own shared memory, already fenced for the async proxy)
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Bounded wait on a barrier of this CTA that other CTAs of the cluster arrive on.  It polls with test_wait:
+// a thread suspended in try_wait was not woken by an arrival from another CTA until its time limit ran out
+// (about 2 us per wait, measured).
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 1024; ++i) {
+            uint32_t ok;
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t"
+                "mbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+                "selp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(ok)
+                : "r"(bar), "r"(parity)
+                : "memory");
+            if (ok)
+                return true;
+            __nanosleep(20);
+        }
+        if (clock64() - t0 > 4000000000ll)
+            return false;
+    }
+}
+
+// Instruction descriptor of the pair form: as idesc_f8f6f4 with M = 256.
+__host__ __device__ inline uint32_t idesc_f8f6f4_pair(uint32_t a_fmt, uint32_t b_fmt, uint32_t n)
+{
+    return (1u << 4) | (a_fmt << 7) | (b_fmt << 10) | ((n >> 3) << 17) | ((256u >> 4) << 24);
 }
 
 }  // namespace fpq

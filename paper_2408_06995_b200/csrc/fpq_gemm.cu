@@ -52,30 +52,6 @@ constexpr int SMEM_BUDGET = 227 * 1024;   // the most dynamic shared memory a CT
 // sensitive to code size (the extra path cost the plain FLAT kernel 7 us when it was a run-time branch)
 enum { MODE_ROWS = 0, MODE_FLAT = 1, MODE_TAPS = 2, MODE_FLAT2 = 3 };
 
-// Division of a 31-bit unsigned number by a constant known on the host:
-// n / d = (umulhi(n, mul) + n) >> shift.
-struct FastDiv {
-    uint32_t mul, shift;
-};
-
-static FastDiv make_fastdiv(uint32_t d)
-{
-    FastDiv f{0, 0};
-    if (d > 1) {
-        uint32_t s = 0;
-        while ((1ull << s) < d)
-            ++s;
-        f.shift = s;
-        f.mul = (uint32_t)((((1ull << 32) * ((1ull << s) - d)) / d) + 1);
-    }
-    return f;
-}
-
-__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f)
-{
-    return (uint32_t)(((uint64_t)__umulhi(n, f.mul) + n) >> f.shift);
-}
-
 struct GemmArgs {
     int mode;
     int64_t M;                 // ROWS: rows; FLAT: framed pixels B*Hp*Wp
@@ -245,38 +221,6 @@ __device__ __forceinline__ void fill_chunk_rows(const GemmArgs& g, uint8_t* dst,
         }
         *reinterpret_cast<uint4*>(dst + i * 128 + ((j ^ (i & 7)) << 4)) = v;
     }
-}
-
-// ---- thread-block cluster: barrier over all threads of all CTAs, and reads of a peer CTA's shared memory
-__device__ __forceinline__ void cluster_sync_all()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-
-__device__ __forceinline__ uint32_t cluster_rank()
-{
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-
-// address of this CTA's shared-memory location `local_addr` in CTA `peer` of the cluster
-__device__ __forceinline__ uint32_t peer_smem_addr(uint32_t local_addr, uint32_t peer)
-{
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(peer));
-    return remote;
-}
-
-__device__ __forceinline__ float4 ld_cluster_smem4(uint32_t cluster_addr)
-{
-    float4 v;
-    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                 : "r"(cluster_addr)
-                 : "memory");
-    return v;
 }
 
 // FUSED = false: the activation operand is read as codes (TMA, written by a quantize kernel).
@@ -503,7 +447,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                 }
             }
             if (dead) {
-                atomicMin(g.status, FPQ_ERR_TIMEOUT);
+                flag_status(g.status, FPQ_ERR_TIMEOUT);
                 // let the copies still in flight land before the CTA's shared memory is released
                 for (uint32_t i = (na > (uint32_t)g.a_stages ? na - g.a_stages : 0); i < na; ++i)
                     (void)mbar_wait(a_full + 8 * (i % g.a_stages), (i / g.a_stages) & 1);
@@ -737,7 +681,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                 mma_commit(acc_full + 8 * buf);
             }
             if (dead)
-                atomicMin(g.status, FPQ_ERR_TIMEOUT);
+                flag_status(g.status, FPQ_ERR_TIMEOUT);
         }
     } else if (warp < 2 + NUM_EPI_WARPS) {
         // ---------------- epilogue: warp w reads TMEM lane quarter w % 4 and the column
@@ -928,7 +872,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         if (g.y_tma && lane == 0)
             asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // the staging buffer must outlive its stores
         if (dead)
-            atomicMin(g.status, FPQ_ERR_TIMEOUT);
+            flag_status(g.status, FPQ_ERR_TIMEOUT);
     } else if (FUSED && warp == 2 + NUM_EPI_WARPS + NUM_XFORM_WARPS) {
         // ---------------- L2 prefetch warp ----------------
         // A transform thread can keep only two rows of loads in flight, so it cannot hide DRAM
@@ -1016,9 +960,9 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             }
         }
         if (nan)
-            atomicMin(g.status, FPQ_ERR_NAN_INPUT);
+            flag_status(g.status, FPQ_ERR_NAN_INPUT);
         if (dead)
-            atomicMin(g.status, FPQ_ERR_TIMEOUT);
+            flag_status(g.status, FPQ_ERR_TIMEOUT);
     }
 
     if (ksplit > 1) {

@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(256) quantize_values_kernel(const float* __res
         v[i] = decode_code(code, f);
     }
     if (any_nan)
-        atomicExch(status, (int)FPQ_ERR_NAN_INPUT);
+        flag_status(status, FPQ_ERR_NAN_INPUT);
 }
 
 // prepared [N][RS][Cp] (one byte per code, or two codes per byte, even index in the low nibble) ->

@@ -28,6 +28,10 @@ cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, in
 cudaError_t launch_quantize_rows_e4m3_twice(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, uint8_t* codes,
                                             cudaStream_t st);
 
+// One warp waits, with the kernels' own bounded wait, on a barrier nobody arrives on: after `limit` cycles it
+// records FPQ_ERR_TIMEOUT in the status word and returns (nothing hangs, nothing faults).
+cudaError_t launch_bounded_wait_selftest(long long limit, int* status, cudaStream_t st);
+
 // Geometry of one contraction launch (linear: taps = 1, rows of Ca codes).
 struct GemmProblem {
     int conv;            // 0 linear, 1 conv
@@ -56,6 +60,12 @@ struct GemmProblem {
 
 // Returns FPQ_OK or an error; enqueues one kernel.
 fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st);
+
+// Stride-1 convolution from FP32 NCHW activations (p.x) in one kernel on CTA pairs, weights resident in
+// shared memory.  FPQ_ERR_UNSUPPORTED when the shape is outside its range (nothing was enqueued).
+fpq_status launch_pair_conv(const GemmProblem& p, cudaStream_t st);
+bool pair_conv_applies(const GemmProblem& p);     // p.x only has to be non-NULL and 16-byte aligned
+bool pair_conv_preferred(const GemmProblem& p);   // ... and it measured faster than the two-kernel route on shapes like this
 
 // Linear layer with at most 8 rows on the CUDA cores (one pass over the weights).
 bool small_m_linear_applies(int64_t M, int64_t K);

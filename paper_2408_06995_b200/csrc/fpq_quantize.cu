@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const float* __restri
         }
     }
     if (nan)
-        atomicMin(status, FPQ_ERR_NAN_INPUT);
+        flag_status(status, FPQ_ERR_NAN_INPUT);
 }
 
 // Unaligned input: one output byte per thread (two elements for 4-bit codes).
@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(256) quantize_act_scalar_kernel(const float* _
         codes[o] = (uint8_t)c;
     }
     if (nan)
-        atomicMin(status, FPQ_ERR_NAN_INPUT);
+        flag_status(status, FPQ_ERR_NAN_INPUT);
 }
 
 // ---------------------------------------------------------------------------------
@@ -122,7 +122,7 @@ __global__ void __launch_bounds__(256) quantize_weight_kernel(const float* __res
         }
     }
     if (nan)
-        atomicMin(status, FPQ_ERR_NAN_INPUT);
+        flag_status(status, FPQ_ERR_NAN_INPUT);
 }
 
 // ---------------------------------------------------------------------------------
@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const float* __
         }
     }
     if (nan)
-        atomicMin(status, FPQ_ERR_NAN_INPUT);
+        flag_status(status, FPQ_ERR_NAN_INPUT);
 }
 
 // ---------------------------------------------------------------------------------
@@ -255,7 +255,7 @@ __global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const f
         }
     }
     if (nan)
-        atomicMin(status, FPQ_ERR_NAN_INPUT);
+        flag_status(status, FPQ_ERR_NAN_INPUT);
 }
 
 // ---------------------------------------------------------------------------------
@@ -457,6 +457,27 @@ cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, in
         tab2 = *table2;
     prepare_weight_kernel<<<grid_for(total, 256), 256, 0, st>>>(codes, N, C, RS, Cp, four_bit, table ? 1 : 0, tab,
                                                                 table2 ? 1 : 0, tab2, C1, C1p, prepared);
+    return cudaGetLastError();
+}
+
+// ---- self-test of the bounded wait every pipeline role uses ---------------------------------------
+__global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(long long limit, int* status)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        fence_barrier_init();
+    }
+    __syncwarp();
+    // phase 0 of a fresh barrier never completes without an arrival
+    if (!mbar_wait(b, 0, limit) && threadIdx.x == 0)
+        flag_status(status, FPQ_ERR_TIMEOUT);
+}
+
+cudaError_t launch_bounded_wait_selftest(long long limit, int* status, cudaStream_t st)
+{
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(limit, status);
     return cudaGetLastError();
 }
 

@@ -108,7 +108,7 @@ __global__ void __launch_bounds__(256) soft_weight_kernel(const float* __restric
         if (t != t) {
             E[i] = 0.f;
             DQ[i] = 0.f;
-            atomicExch(status, (int)FPQ_ERR_NAN_INPUT);
+            flag_status(status, FPQ_ERR_NAN_INPUT);
             continue;
         }
         float a = fminf(fmaxf(t, -c), c);

@@ -117,7 +117,7 @@ __global__ void __launch_bounds__(SEARCH_THREADS) search_mse_kernel(const Search
         a.partial[(int64_t)blockIdx.x * ncand + c] = s;
     }
     if (nan)
-        atomicMin(a.status, FPQ_ERR_NAN_INPUT);
+        flag_status(a.status, FPQ_ERR_NAN_INPUT);
 }
 
 // Block partial sums -> mse.  A block of 32 x 32 threads owns 32 candidates: thread (slice, ci) adds
@@ -144,36 +144,36 @@ __global__ void __launch_bounds__(1024) search_reduce_kernel(const double* __res
     }
 }
 
-// Algorithm 1: encodings in the outer loop, clipping candidates in the inner one, a candidate is
-// kept only when its error is strictly below the best so far, which starts at +infinity.  One warp:
-// lane l scans its contiguous stretch of that order, then the lanes are combined in lane order
-// with the same strict comparison, which gives what the sequential scan gives.
+// Selection rule of Algorithm 1 (Sec. V-A): the candidate with the smallest error; among equal errors the one
+// that comes first in encoding-major, candidate-minor order (the flat index).  The listing's start value for
+// the best error is read as +infinity; a NaN error never wins.  One warp: every lane takes the flat indices
+// lane, lane + 32, ..., then a shuffle tree reduces the (error, index) pairs with the smaller index breaking ties.
 __global__ void __launch_bounds__(32) search_select_kernel(const double* __restrict__ mse, int n_enc, int n_clip,
                                                            int32_t* __restrict__ best)
 {
     const int ncand = n_enc * n_clip, lane = threadIdx.x;
-    const int per = (ncand + 31) / 32;
-    double prev_mse = INFINITY;
-    int arg = -1;
-    for (int c = lane * per; c < min(ncand, (lane + 1) * per); ++c) {
-        const double curr_mse = mse[c];
-        if (prev_mse > curr_mse) {
+    double err = INFINITY;
+    int arg = 0x7fffffff;                        // "nothing yet": loses every tie
+    for (int c = lane; c < ncand; c += 32) {
+        const double e = mse[c];
+        if (e < err) {                           // false for NaN; indices grow, so the first of equal errors stays
+            err = e;
             arg = c;
-            prev_mse = curr_mse;
         }
     }
-    // lane 0 walks the 32 results in order
-    for (int l = 1; l < 32; ++l) {
-        const double other = __shfl_sync(0xffffffffu, prev_mse, l);
-        const int other_arg = __shfl_sync(0xffffffffu, arg, l);
-        if (lane == 0 && prev_mse > other) {
-            prev_mse = other;
-            arg = other_arg;
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        const double oe = __shfl_xor_sync(0xffffffffu, err, d);
+        const int oa = __shfl_xor_sync(0xffffffffu, arg, d);
+        if (oe < err || (oe == err && oa < arg)) {
+            err = oe;
+            arg = oa;
         }
     }
     if (lane == 0) {
-        best[0] = arg < 0 ? -1 : arg / n_clip;
-        best[1] = arg < 0 ? -1 : arg % n_clip;
+        const bool none = arg == 0x7fffffff;
+        best[0] = none ? -1 : arg / n_clip;
+        best[1] = none ? -1 : arg % n_clip;
     }
 }
 
@@ -202,6 +202,8 @@ fpq_status launch_search(const float* x, int64_t n, const fpq_format* enc, int n
     a.clip = clip;
     a.partial = (double*)workspace;
     a.status = status_word();
+    if (!a.status)
+        return FPQ_ERR_CUDA;
     const int ncand = n_enc * n_clip;
     const int64_t chunk = (int64_t)SEARCH_THREADS * SEARCH_PER_THREAD;
     int64_t blocks = (n + chunk - 1) / chunk;

@@ -111,7 +111,7 @@ __global__ void __launch_bounds__(SMALLM_THREADS) small_m_linear_kernel(const fl
         }
     }
     if (nan)
-        atomicMin(status, FPQ_ERR_NAN_INPUT);
+        flag_status(status, FPQ_ERR_NAN_INPUT);
 }
 
 bool small_m_linear_applies(int64_t M, int64_t K)

@@ -66,9 +66,12 @@ def _gpu_layer_once(L, ws, xs, use_bias, prep):
     return y.cpu().numpy()
 
 
-def gpu_layer(L, ws, xs, use_bias=True):
-    """The layer call on both of the library's routes (one fused kernel; quantize kernel +
-    contraction kernel).  They run the same MMAs in the same order: results must be equal."""
+def gpu_layer(L, ws, xs, use_bias=True, route="auto"):
+    """The layer call on every route of the library (one fused kernel; quantize kernel + contraction kernel;
+    the library's own choice).  All routes multiply the same codes exactly and add in FP32; where they run the
+    same MMAs in the same order the results are equal bit for bit, otherwise (a fused kernel that splits the
+    reduction differently) they differ by the rounding of the FP32 sums only.  The library's own choice must be
+    one of the two, bit for bit.  Returns the result of `route` ("auto", "fused" or "two")."""
     _, prep = gpu_prepare(L, ws)
     try:
         fpq.fpq_set_path_policy(fpq.PATH_FUSED)
@@ -77,8 +80,12 @@ def gpu_layer(L, ws, xs, use_bias=True):
         y2 = _gpu_layer_once(L, ws, xs, use_bias, prep)
     finally:
         fpq.fpq_set_path_policy(fpq.PATH_AUTO)
-    assert np.array_equal(y1, y2), "fused and two-kernel routes differ"
-    return y1
+    y0 = _gpu_layer_once(L, ws, xs, use_bias, prep)
+    assert np.array_equal(y0, y1) or np.array_equal(y0, y2), "the default route is neither of the two routes"
+    if not np.array_equal(y1, y2):
+        scale = float(np.abs(y2).max()) if y2.size else 0.0
+        assert np.all(np.abs(y1.astype(np.float64) - y2) <= 1e-4 * scale), "fused and two-kernel routes differ"
+    return {"auto": y0, "fused": y1, "two": y2}[route]
 
 
 def oracle_layer(L, ws, xs, idx=None, use_bias=True):

@@ -161,3 +161,38 @@ def test_weight_formats_the_layer_accepts(L):
     assert L.fpq_prepared_size(fpq.E2M1.c(), ctypes.byref(d)) == 8 * 256 // 2
     assert L.fpq_prepared_size(fpq.E1M2.c(), ctypes.byref(d)) == 8 * 256      # one E4M3 byte per weight
     assert L.fpq_prepared_size(fpq.E4M3.c(), ctypes.byref(d)) == 8 * 256
+
+
+def test_activation_scales_are_checked_before_anything_else(L):
+    F = fpq.E4M3.c()
+    p = ctypes.c_void_p(1024)      # never dereferenced
+    for bad in (0.0, -1.0, float("inf"), float("nan")):
+        assert L.fpq_quantize_act(p, 16, bad, F, p, None) == fpq.ERR_SCALE
+        assert L.fpq_linear(p, p, p, bad, F, F, None, p, 8, 8, 8, p, 1 << 20, None) == fpq.ERR_SCALE
+        assert L.fpq_conv2d(p, p, p, bad, F, F, None, p, 1, 4, 4, 4, 4, 3, 3, 1, 1, p, 1 << 20, None) == fpq.ERR_SCALE
+        assert L.fpq_linear_quantize_input(p, bad, F, F, 8, 8, 8, p, 1 << 20, None) == fpq.ERR_SCALE
+        assert L.fpq_conv2d_split(p, 4, bad, p, 4, 1.0, p, p, F, F, None, p, 1, 4, 4, 4, 3, 3, 1, 1, p, 1 << 20, None) == fpq.ERR_SCALE
+        assert L.fpq_conv2d_split(p, 4, 1.0, p, 4, bad, p, p, F, F, None, p, 1, 4, 4, 4, 3, 3, 1, 1, p, 1 << 20, None) == fpq.ERR_SCALE
+    assert "scale" in fpq.status_string(fpq.ERR_SCALE)
+
+
+def test_route_query(L):
+    try:
+        # the workload the bench times: one 128-channel chunk, 128 outputs -> the CTA-pair kernel
+        assert fpq.fpq_conv2d_route(64, 128, 32, 32, 128, 3, 3, 1, 1, fpq.E4M3, fpq.E4M3) == fpq.ROUTE_PAIR_FUSED
+        # weights that do not fit the shared memory of two SMs, more than 256 outputs, a stride: two kernels
+        assert fpq.fpq_conv2d_route(2, 1280, 16, 16, 1280, 3, 3, 1, 1, fpq.E4M3, fpq.E2M1) == fpq.ROUTE_TWO_KERNELS
+        assert fpq.fpq_conv2d_route(2, 128, 32, 32, 512, 1, 1, 0, 1, fpq.E4M3, fpq.E4M3) == fpq.ROUTE_TWO_KERNELS
+        assert fpq.fpq_conv2d_route(2, 128, 32, 32, 128, 3, 3, 1, 2, fpq.E4M3, fpq.E4M3) == fpq.ROUTE_TWO_KERNELS
+        # formats without a tensor-core type
+        assert fpq.fpq_conv2d_route(2, 128, 32, 32, 128, 3, 3, 1, 1, fpq.E3M4, fpq.E4M3) == fpq.ROUTE_OTHER
+        assert L.fpq_conv2d_route(2, 128, 32, 32, 128, 3, 3, 1, 1, fpq.Format(6, 3, 7).c(), fpq.E4M3.c()) == fpq.ERR_FORMAT
+        assert L.fpq_conv2d_route(2, 0, 32, 32, 128, 3, 3, 1, 1, fpq.E4M3.c(), fpq.E4M3.c()) == fpq.ERR_SHAPE
+        fpq.fpq_set_path_policy(fpq.PATH_TWO_KERNELS)
+        assert fpq.fpq_conv2d_route(64, 128, 32, 32, 128, 3, 3, 1, 1, fpq.E4M3, fpq.E4M3) == fpq.ROUTE_TWO_KERNELS
+        fpq.fpq_set_path_policy(fpq.PATH_FUSED)
+        assert fpq.fpq_conv2d_route(2, 1280, 16, 16, 1280, 3, 3, 1, 1, fpq.E4M3, fpq.E2M1) == fpq.ROUTE_FUSED
+    finally:
+        fpq.fpq_set_path_policy(fpq.PATH_AUTO)
+    assert L.fpq_selftest_bounded_wait(0, None) == fpq.ERR_SHAPE
+    assert L.fpq_selftest_bounded_wait(1 << 40, None) == fpq.ERR_SHAPE

@@ -115,6 +115,24 @@ def test_selection_keeps_the_first_strict_minimum():
     assert O.select_encoding_and_bias(mse) == (1, 2)
 
 
+def test_selection_with_tied_minima_takes_the_first_in_encoding_major_order():
+    # ties inside a row, across rows, at the very first entry, and an all-infinite table
+    assert O.select_encoding_and_bias(np.array([[1.0, 1.0], [1.0, 1.0]])) == (0, 0)
+    assert O.select_encoding_and_bias(np.array([[4.0, 2.0, 2.0], [2.0, 7.0, 2.0]])) == (0, 1)
+    assert O.select_encoding_and_bias(np.array([[np.inf, 3.0], [3.0, 3.0]])) == (0, 1)
+    assert O.select_encoding_and_bias(np.array([[np.nan, 6.0], [5.0, 5.0]])) == (1, 0)
+    assert O.select_encoding_and_bias(np.full((2, 3), np.inf)) == (None, None)
+    assert O.select_encoding_and_bias(np.full((2, 3), np.nan)) == (None, None)
+    # against the definition spelled out: smallest value, then smallest encoding index, then smallest candidate index
+    rng = np.random.default_rng(5)
+    for _ in range(200):
+        t = rng.integers(0, 4, size=(4, 7)).astype(np.float64)          # few distinct values: many ties
+        t[rng.random(t.shape) < 0.1] = np.nan
+        finite = [(t[i, j], i, j) for i in range(4) for j in range(7) if not np.isnan(t[i, j])]
+        want = min(finite)[1:] if finite else (None, None)
+        assert O.select_encoding_and_bias(t) == want
+
+
 def test_narrow_data_takes_the_most_mantissa_bits_and_heavy_tails_take_fewer():
     rng = np.random.default_rng(10)
     narrow = rng.uniform(-1, 1, 20000).astype(np.float32)

@@ -20,18 +20,28 @@ from _helpers import assert_close, gpu_prepare, layer_scales, oracle_layer
 pytestmark = pytest.mark.gpu
 
 
-def _both(L):
+def _free_bytes():
+    torch.cuda.synchronize()
+    return torch.cuda.mem_get_info()[0]
+
+
+def _both(L, gfw=None, fx=None):
     ws, xs = layer_scales(L)
-    gfw = fpq.E4M3 if L.wfmt == "e4m3" else fpq.E2M1
+    gfw = gfw or (fpq.E4M3 if L.wfmt == "e4m3" else fpq.E2M1)
+    fx = fx or fpq.E4M3
     _, prep = gpu_prepare(L, ws)
     x = torch.from_numpy(L.x).cuda()
     bias = torch.from_numpy(L.bias).cuda()
     wsd = torch.from_numpy(ws).cuda()
-    y_ref = fpq.fpq_linear(x, prep, wsd, xs, fpq.E4M3, gfw, bias, L.N)
+    y_ref = fpq.fpq_linear(x, prep, wsd, xs, fx, gfw, bias, L.N)
     y = torch.full((L.M, L.N), float("nan"), dtype=torch.float32, device="cuda")
-    before = torch.cuda.memory_allocated()
-    fpq.fpq_linear_static(x, prep, wsd, xs, fpq.E4M3, gfw, bias, y)
-    assert torch.cuda.memory_allocated() == before
+    fpq.fpq_linear_static(x, prep, wsd, xs, fx, gfw, bias, y)      # the first call on a device resolves the array
+    y.fill_(float("nan"))
+    # the driver's own count of free device memory: it moves for ANY allocation in this process, whoever made it
+    # (torch's counters only see torch's allocator)
+    before = _free_bytes()
+    fpq.fpq_linear_static(x, prep, wsd, xs, fx, gfw, bias, y)
+    assert _free_bytes() == before
     assert fpq.fpq_read_status() == fpq.OK
     return y.cpu().numpy(), y_ref.cpu().numpy(), ws, xs
 
@@ -54,3 +64,47 @@ def test_rejects_problems_beyond_the_fixed_capacity():
     assert M * K > fpq.STATIC_SCRATCH_BYTES
     assert L.fpq_linear_static(p, p, p, 1.0, F, F, None, p, M, 64, K, None) == fpq.ERR_TOO_LARGE
     assert "capacity" in fpq.status_string(fpq.ERR_TOO_LARGE)
+
+
+def test_a_handful_of_rows_leaves_the_array_alone():
+    # M <= 8 runs on the CUDA cores in one pass over the weights: no intermediate codes at all
+    L = I.draw(I.linear_layer("few", 4, 320, 1280, "e2m1", rounding=True), 12, 20, "normal", 0.02, True)
+    y, y_ref, ws, xs = _both(L)
+    assert np.array_equal(y, y_ref)
+    yo, ab = oracle_layer(L, ws, xs)
+    assert_close(y, yo, ab)
+
+
+def test_formats_that_need_more_scratch_per_element():
+    """Weights prepared as two tensor-core terms keep two copies of the activation codes, so they reach the end of
+    the array at half the documented size: within it the result equals fpq_linear's, beyond it the answer is
+    FPQ_ERR_WORKSPACE (the size test on M x K has passed), never a partial result."""
+    e3m4 = fpq.E3M4
+    M, K, N = 300, 320, 200
+    x = torch.randn(M, K, device="cuda")
+    w = torch.randn(N, K, device="cuda") * 0.02
+    ws = (w.abs().amax(dim=1) / fpq.fpq_format_max(e3m4)).contiguous()
+    prep = fpq.fpq_prepare_weight(fpq.fpq_quantize_weight(w, ws, e3m4, None), e3m4, fpq.LINEAR, N, K)
+    xs = float(x.abs().max()) / 448.0
+    y_ref = fpq.fpq_linear(x, prep, ws, xs, fpq.E4M3, e3m4, None, N)
+    y = torch.full((M, N), float("nan"), device="cuda")
+    fpq.fpq_linear_static(x, prep, ws, xs, fpq.E4M3, e3m4, None, y)
+    assert fpq.fpq_read_status() == fpq.OK
+    assert torch.equal(y, y_ref)
+    # 6000 x 1024 codes fit the array once (6 MiB of 8) but not twice
+    Lb = fpq.lib()
+    p = torch.zeros(256, dtype=torch.float32, device="cuda").data_ptr()
+    assert 6000 * 1024 <= fpq.STATIC_SCRATCH_BYTES < 2 * 6000 * 1024
+    assert Lb.fpq_linear_static(p, p, p, 1.0, fpq.E4M3.c(), e3m4.c(), None, p, 6000, 64, 1024, None) == fpq.ERR_WORKSPACE
+    # activations in a format the tensor cores have no type for run on the CUDA cores with FP32 scratch:
+    # a small problem fits, a larger one that passes the M x K test does not
+    e5m2 = fpq.E5M2
+    xs5 = float(x.abs().max()) / fpq.fpq_format_max(e5m2)
+    w8 = (w.abs().amax(dim=1) / 448.0).contiguous()
+    prep8 = fpq.fpq_prepare_weight(fpq.fpq_quantize_weight(w, w8, fpq.E4M3, None), fpq.E4M3, fpq.LINEAR, N, K)
+    y_ref = fpq.fpq_linear(x, prep8, w8, xs5, e5m2, fpq.E4M3, None, N)
+    y.fill_(float("nan"))
+    fpq.fpq_linear_static(x, prep8, w8, xs5, e5m2, fpq.E4M3, None, y)
+    assert fpq.fpq_read_status() == fpq.OK
+    assert torch.equal(y, y_ref)
+    assert Lb.fpq_linear_static(p, p, p, 1.0, e5m2.c(), fpq.E4M3.c(), None, p, 6000, 64, 1024, None) == fpq.ERR_WORKSPACE
