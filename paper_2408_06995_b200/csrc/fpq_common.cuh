@@ -170,11 +170,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long lo
         return true;
     const long long t0 = clock64();
     for (;;) {
-        for (int i = 0; i < 1024; ++i) {
+        for (int i = 0; i < 1024; ++i)
             if (mbar_try_wait(bar, parity))
                 return true;
-            __nanosleep(40);      // a waiting warp must not take issue slots from the warps that work
-        }
         if (clock64() - t0 > limit)
             return false;
     }
