@@ -412,10 +412,12 @@ fpq_status fpq_round_learn_harden(const float* alpha, int64_t N, int64_t K, uint
  *                         linear layers and the other stride-1 convolutions use the general fused
  *                         form; other geometries fall back to two kernels.
  *   FPQ_PATH_TWO_KERNELS  always *_quantize_input followed by *_contract.
+ *   FPQ_PATH_TWO_KERNELS_NARROW  the same, and the contraction never takes its CTA-pair form (M = 256
+ *                         MMAs for long reductions with many tiles): for measurements and tests.
  *   FPQ_PATH_AUTO         the library's choice per shape (default): the CTA-pair kernel where it
  *                         applies and measured faster, else two kernels.
  */
-enum { FPQ_PATH_AUTO = 0, FPQ_PATH_FUSED = 1, FPQ_PATH_TWO_KERNELS = 2 };
+enum { FPQ_PATH_AUTO = 0, FPQ_PATH_FUSED = 1, FPQ_PATH_TWO_KERNELS = 2, FPQ_PATH_TWO_KERNELS_NARROW = 3 };
 fpq_status fpq_set_path_policy(int32_t policy);
 int32_t fpq_get_path_policy(void);
 

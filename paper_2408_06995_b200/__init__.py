@@ -23,7 +23,7 @@ ROUTE_TWO_KERNELS, ROUTE_FUSED, ROUTE_PAIR_FUSED, ROUTE_OTHER = 0, 1, 2, 3
 STATIC_SCRATCH_BYTES = 8 << 20
 SAT_PAPER, SAT_NATIVE = 0, 1
 LINEAR, CONV2D = 0, 1
-PATH_AUTO, PATH_FUSED, PATH_TWO_KERNELS = 0, 1, 2
+PATH_AUTO, PATH_FUSED, PATH_TWO_KERNELS, PATH_TWO_KERNELS_NARROW = 0, 1, 2, 3
 
 
 class FpqError(RuntimeError):

@@ -745,6 +745,11 @@ static fpq_status conv2d_contract_impl(const void* workspace, size_t ws_bytes, c
         }
         if (pair_only)
             return FPQ_ERR_UNSUPPORTED;
+    } else if (g_path_policy != FPQ_PATH_TWO_KERNELS_NARROW && pair_gemm_preferred(p)) {
+        // long reductions with enough tiles: the wide MMAs of a CTA pair
+        const fpq_status sp = launch_pair_gemm(p, (cudaStream_t)stream);
+        if (sp != FPQ_ERR_UNSUPPORTED)
+            return sp;
     }
     return launch_gemm(p, (cudaStream_t)stream);
 }
@@ -1240,7 +1245,7 @@ int32_t fpq_conv2d_route(int B, int C, int H, int W, int C_out, int R, int S, in
     s = conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo);
     if (s != FPQ_OK)
         return s;
-    if (g_path_policy == FPQ_PATH_TWO_KERNELS || B == 0 || C_out == 0)
+    if (g_path_policy == FPQ_PATH_TWO_KERNELS || g_path_policy == FPQ_PATH_TWO_KERNELS_NARROW || B == 0 || C_out == 0)
         return FPQ_ROUTE_TWO_KERNELS;
     GemmProblem p{};
     p.conv = 1;
@@ -1272,7 +1277,8 @@ fpq_status fpq_selftest_bounded_wait(int64_t limit_cycles, void* stream)
 
 fpq_status fpq_set_path_policy(int32_t policy)
 {
-    if (policy != FPQ_PATH_AUTO && policy != FPQ_PATH_FUSED && policy != FPQ_PATH_TWO_KERNELS)
+    if (policy != FPQ_PATH_AUTO && policy != FPQ_PATH_FUSED && policy != FPQ_PATH_TWO_KERNELS &&
+        policy != FPQ_PATH_TWO_KERNELS_NARROW)
         return FPQ_ERR_UNSUPPORTED;
     g_path_policy = policy;
     return FPQ_OK;

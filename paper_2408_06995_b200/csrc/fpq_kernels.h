@@ -67,6 +67,11 @@ fpq_status launch_pair_conv(const GemmProblem& p, cudaStream_t st);
 bool pair_conv_applies(const GemmProblem& p);     // p.x only has to be non-NULL and 16-byte aligned
 bool pair_conv_preferred(const GemmProblem& p);   // ... and it measured faster than the two-kernel route on shapes like this
 
+// The contraction of a stride-1 convolution (activation codes already in the workspace) on CTA pairs with
+// M = 256 MMAs.  FPQ_ERR_UNSUPPORTED when the shape is outside its range (nothing was enqueued).
+fpq_status launch_pair_gemm(const GemmProblem& p, cudaStream_t st);
+bool pair_gemm_preferred(const GemmProblem& p);   // in range, and faster than the general contraction on shapes like this
+
 // Linear layer with at most 8 rows on the CUDA cores (one pass over the weights).
 bool small_m_linear_applies(int64_t M, int64_t K);
 fpq_status launch_small_m_linear(const float* x, int M, int K, const void* w_prepared, int w4, int N, const float* w_scale,
