@@ -683,7 +683,7 @@ def run_suite(args):
     else:
         raise SystemExit("unknown suite")
     rows = []
-    tot = {"auto": 0.0, "fused": 0.0, "two_kernels": 0.0, "best": 0.0, "flops": 0.0, "bytes": 0.0, "bound": 0.0}
+    tot = {"auto": 0.0, "fused": 0.0, "two_kernels": 0.0, "two_kernels_narrow": 0.0, "best": 0.0, "flops": 0.0, "bytes": 0.0, "bound": 0.0}
     if args.only:
         layers = [L for L in layers if args.only in L.name]
         if not layers:
@@ -692,7 +692,8 @@ def run_suite(args):
         lay = LayerOnGpu(L, fpq, torch, dev, l2_bytes=(128 << 20) if args.suite != "sd" else (48 << 20))
         n = max(4, min(40, 3 * lay.nsets))
         res = {}
-        for name, pol in (("fused", fpq.PATH_FUSED), ("two_kernels", fpq.PATH_TWO_KERNELS), ("auto", fpq.PATH_AUTO)):
+        for name, pol in (("fused", fpq.PATH_FUSED), ("two_kernels", fpq.PATH_TWO_KERNELS),
+                          ("two_kernels_narrow", fpq.PATH_TWO_KERNELS_NARROW), ("auto", fpq.PATH_AUTO)):
             fpq.fpq_set_path_policy(pol)
             for _ in range(2):
                 lay.step()
@@ -703,11 +704,11 @@ def run_suite(args):
             raise SystemExit(f"{L.name}: device status {fpq.status_string(st)}")
         t_hbm = lay.layer_bytes() / (peaks["hbm_gbs"] * 1e9) * 1e6
         t_tc = L.flops / (NOMINAL_FP8_TFLOPS * 1e12) * 1e6
-        best = min(res["fused"], res["two_kernels"])
+        best = min(res["fused"], res["two_kernels"], res["two_kernels_narrow"])
         rows.append({"name": L.name, "kind": L.kind, "M": L.M, "N": L.N, "K": L.K, "count": L.count, "wfmt": L.wfmt,
                      "us": res, "tflops_auto": L.flops / res["auto"] / 1e6, "t_hbm_us": t_hbm, "t_tensor_us": t_tc,
                      "frac_of_bound_auto": max(t_hbm, t_tc) / res["auto"]})
-        for k in ("auto", "fused", "two_kernels"):
+        for k in ("auto", "fused", "two_kernels", "two_kernels_narrow"):
             tot[k] += res[k] * L.count
         tot["best"] += best * L.count
         tot["flops"] += L.flops * L.count
@@ -716,7 +717,7 @@ def run_suite(args):
         del lay
         torch.cuda.empty_cache()
     summary = {"suite": args.suite, "layers": sum(r["count"] for r in rows), "distinct_shapes": len(rows),
-               "sum_us": {k: tot[k] for k in ("auto", "fused", "two_kernels", "best")},
+               "sum_us": {k: tot[k] for k in ("auto", "fused", "two_kernels", "two_kernels_narrow", "best")},
                "aggregate_tflops_auto": tot["flops"] / tot["auto"] / 1e6, "sum_bound_us": tot["bound"],
                "frac_of_bound_auto": tot["bound"] / tot["auto"], "gflop": tot["flops"] / 1e9, "rows": rows}
     print(json.dumps(summary), flush=True)
