@@ -35,12 +35,10 @@ WORKLOAD = "ddim_cifar_conv3x3_w8a8: x fp32 NCHW [64,128,32,32] SiLU(N(0,1)), w 
 NOMINAL_FP8_TFLOPS = 4500.0
 NOMINAL_FP4_TFLOPS = 9000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
-# profiles/ (a kernel is absent here until a capture of its current form exists).  ncu starts each
-# launch with flushed caches and stops counting when the kernel ends, so output that is still in L2
-# at that point (all of it, for these sizes) is missing from the write side.
+# profiles/ (a kernel is absent here until a capture of its current form exists).
 TRAFFIC = {
-    "fpq_gemm_kernel (contraction + epilogue)": 9712640 + 12800,
-    "quantize_nchw_to_nhwc_e4m3_kernel (activation quantize)": 33567232 + 0,
+    # --cache-control none capture, second of three launches taken mid-rotation (write-backs included)
+    "fpq_pair_conv_kernel (activation quantize + contraction + epilogue on CTA pairs)": 33718784 + 32794880,
 }
 
 
