@@ -151,8 +151,10 @@ fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_la
  * fpq_quantize_act does; products are exact and accumulated in FP32 on the
  * tensor cores (layers of at most 8 rows with K a multiple of 4 run on the CUDA
  * cores instead: the same exact products, another order of the FP32 additions;
- * the workspace is then left untouched).  Supported operand pairs: fx = E4M3 bias 7 FPQ_SAT_NATIVE with
- * fw = the same, fw = E5M2 bias 15 FPQ_SAT_NATIVE, fw = E2M1 bias 1, or any fw that fpq_prepare_weight
+ * the workspace is then left untouched).  Supported operand pairs: fx = E4M3 bias 7 FPQ_SAT_NATIVE or
+ * fx = E5M2 bias 15 FPQ_SAT_NATIVE (the two 8-bit types the tensor cores read; Sec. V-A searches the
+ * activation encodings too) with
+ * fw = E4M3 bias 7 FPQ_SAT_NATIVE, fw = E5M2 bias 15 FPQ_SAT_NATIVE, fw = E2M1 bias 1, or any fw that fpq_prepare_weight
  * re-encodes exactly into one or two terms of those types (see there) run on the tensor cores.  Every other valid pair (any fx, any fw) runs on the CUDA
  * cores: activations quantized to their grid values in FP32, weights decoded to FP32, an FP32 multiply-add
  * contraction - the same arithmetic model (exact products, FP32 sums) at roughly a tenth of the speed; the

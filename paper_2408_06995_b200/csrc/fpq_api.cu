@@ -77,6 +77,10 @@ static bool is_e5m2_native(fpq_format f)
     return f.exp_bits == 5 && f.man_bits == 2 && f.exp_bias == 15 && f.sat_mode == FPQ_SAT_NATIVE;
 }
 
+// activation formats the tensor cores read as they are: E4M3 (bias 7) and the OCP E5M2 (bias 15), both saturating
+// at the type's largest finite value
+static bool act_native(fpq_format f) { return is_e4m3_native(f) || is_e5m2_native(f); }
+
 static bool is_e2m1(fpq_format f)
 {
     return f.exp_bits == 2 && f.man_bits == 1 && f.exp_bias == 1;
@@ -237,13 +241,13 @@ static bool general_pair(fpq_format fx, fpq_format fw)
     QFormat q;
     if (!resolve_format(fx, &q) || !resolve_format(fw, &q))
         return false;
-    return !(is_e4m3_native(fx) && (weight_native(fw) || weight_reencoded(fw) || weight_two_term(fw)));
+    return !(act_native(fx) && (weight_native(fw) || weight_reencoded(fw) || weight_two_term(fw)));
 }
 
 static bool two_term_pair(fpq_format fx, fpq_format fw)
 {
     QFormat q;
-    return resolve_format(fx, &q) && resolve_format(fw, &q) && is_e4m3_native(fx) && weight_two_term(fw);
+    return resolve_format(fx, &q) && resolve_format(fw, &q) && act_native(fx) && weight_two_term(fw);
 }
 
 // Format of the codes in the prepared copy: re-encoded weights are E4M3 there.
@@ -273,7 +277,7 @@ static fpq_status check_pair(fpq_format fx, fpq_format fw)
     QFormat q;
     if (!resolve_format(fx, &q) || !resolve_format(fw, &q))
         return FPQ_ERR_FORMAT;
-    if (!is_e4m3_native(fx))
+    if (!act_native(fx))
         return FPQ_ERR_UNSUPPORTED;
     if (!weight_native(fw) && !weight_reencoded(fw))
         return FPQ_ERR_UNSUPPORTED;
@@ -447,8 +451,8 @@ fpq_status fpq_linear_quantize_input(const float* x, float x_scale, fpq_format f
         return FPQ_ERR_ALIGN;
     if (!status_word())
         return FPQ_ERR_CUDA;
-    return launch_quantize_rows_e4m3(x, M, K, round_up(K, 16), x_scale, (uint8_t*)workspace, (cudaStream_t)stream) ==
-                   cudaSuccess
+    return launch_quantize_rows_e4m3(x, M, K, round_up(K, 16), x_scale, (uint8_t*)workspace, (cudaStream_t)stream,
+                                     is_e5m2_native(fx) ? 1 : 0) == cudaSuccess
                ? FPQ_OK
                : FPQ_ERR_CUDA;
 }
@@ -477,6 +481,7 @@ static fpq_status linear_contract_impl(const void* workspace, size_t ws_bytes, c
     p.after_stage1 = after_stage1;
     p.w4 = is_e2m1(fw) ? 1 : 0;
     p.w_e5m2 = is_e5m2_native(fw) ? 1 : 0;
+    p.a_e5m2 = is_e5m2_native(fx) ? 1 : 0;
     p.M = M;
     p.N = (int)N;
     p.Cp = (int)padded_c(K);
@@ -551,8 +556,8 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
             return FPQ_ERR_ALIGN;
         if (!status_word())
             return FPQ_ERR_CUDA;
-        if (launch_quantize_rows_e4m3_twice(x, M, K, K2 / 2, x_scale, (uint8_t*)workspace, (cudaStream_t)stream) !=
-            cudaSuccess)
+        if (launch_quantize_rows_e4m3_twice(x, M, K, K2 / 2, x_scale, (uint8_t*)workspace, (cudaStream_t)stream,
+                                            is_e5m2_native(fx) ? 1 : 0) != cudaSuccess)
             return FPQ_ERR_CUDA;
         // (the contraction uses the activation scale only to dequantize: the weights' power of two goes there)
         return linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale * two_term_unshift(fw), fx, term, bias,
@@ -570,7 +575,7 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
         return FPQ_ERR_ALIGN;
     // a handful of rows (time-embedding projections): one pass over the weights on the CUDA cores,
     // whatever the route policy says; the workspace is not touched
-    if (small_m_linear_applies(M, K) && N <= 0x7fffffff && !is_e5m2_native(fw)) {
+    if (small_m_linear_applies(M, K) && N <= 0x7fffffff && !is_e5m2_native(fw) && is_e4m3_native(fx)) {
         if (!status_word())
             return FPQ_ERR_CUDA;
         return launch_small_m_linear(x, (int)M, (int)K, w_prepared, is_e2m1(fw) ? 1 : 0, (int)N, w_scale, x_scale, bias, y,
@@ -578,7 +583,7 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
     }
     // one kernel: the activations are quantized inside the contraction's operand staging
     // (AUTO takes the two-kernel route: measured faster on B200 so far)
-    if (g_path_policy == FPQ_PATH_FUSED) {
+    if (g_path_policy == FPQ_PATH_FUSED && is_e4m3_native(fx)) {
         s = linear_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, M, N, K, stream, 0,
                                  x);
         if (s != FPQ_ERR_UNSUPPORTED)
@@ -686,7 +691,7 @@ fpq_status fpq_conv2d_quantize_input(const float* x, float x_scale, fpq_format f
     if (!status_word())
         return FPQ_ERR_CUDA;
     return launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H, W, pad, (int)round_up(C, 16), (int)round_up(C, 16), 0, x_scale,
-                                             (uint8_t*)workspace, (cudaStream_t)stream) == cudaSuccess
+                                             (uint8_t*)workspace, (cudaStream_t)stream, is_e5m2_native(fx) ? 1 : 0) == cudaSuccess
                ? FPQ_OK
                : FPQ_ERR_CUDA;
 }
@@ -717,6 +722,7 @@ static fpq_status conv2d_contract_impl(const void* workspace, size_t ws_bytes, c
     p.after_stage1 = after_stage1;
     p.w4 = is_e2m1(fw) ? 1 : 0;
     p.w_e5m2 = is_e5m2_native(fw) ? 1 : 0;
+    p.a_e5m2 = is_e5m2_native(fx) ? 1 : 0;
     p.M = (int64_t)B * Ho * Wo;
     p.N = C_out;
     p.Cp = (int)padded_c(C);
@@ -804,9 +810,10 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
         if (!status_word())
             return FPQ_ERR_CUDA;
         cudaStream_t st = (cudaStream_t)stream;
-        if (launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H, W, pad, Cp, C2, 0, x_scale, (uint8_t*)workspace, st) !=
+        const int e5 = is_e5m2_native(fx) ? 1 : 0;
+        if (launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H, W, pad, Cp, C2, 0, x_scale, (uint8_t*)workspace, st, e5) !=
                 cudaSuccess ||
-            launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H, W, pad, Cp, C2, Cp, x_scale, (uint8_t*)workspace, st) !=
+            launch_quantize_nchw_to_nhwc_e4m3(x, B, C, H, W, pad, Cp, C2, Cp, x_scale, (uint8_t*)workspace, st, e5) !=
                 cudaSuccess)
             return FPQ_ERR_CUDA;
         return conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale * two_term_unshift(fw), fx, term, bias,
@@ -825,7 +832,7 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
     // one kernel where the geometry allows it (stride 1): the activations are quantized inside the
     // contraction's operand staging; otherwise quantize to codes first
     // (the library's own choice: the CTA-pair kernel for the shapes it measured faster on, else two kernels)
-    if (g_path_policy == FPQ_PATH_FUSED || g_path_policy == FPQ_PATH_AUTO) {
+    if ((g_path_policy == FPQ_PATH_FUSED || g_path_policy == FPQ_PATH_AUTO) && is_e4m3_native(fx)) {
         s = conv2d_contract_impl(workspace, ws_bytes, w_prepared, w_scale, x_scale, fx, fw, bias, y, B, C, H, W, C_out,
                                  R, S, pad, stride, stream, 0, x, g_path_policy == FPQ_PATH_AUTO);
         if (s != FPQ_ERR_UNSUPPORTED)
@@ -931,16 +938,18 @@ fpq_status fpq_conv2d_split(const float* x1, int C1, float x1_scale, const float
     const int C1p = (int)padded_c(C1);
     // each tensor is quantized with its own scale into its own channel range of the framed
     // channels-last codes; the concatenated FP32 tensor is never formed
-    if (launch_quantize_nchw_to_nhwc_e4m3(x1, B, C1, H, W, pad, C1p, (int)row, 0, x1_scale, (uint8_t*)workspace, st) !=
+    const int e5 = is_e5m2_native(fx) ? 1 : 0;
+    if (launch_quantize_nchw_to_nhwc_e4m3(x1, B, C1, H, W, pad, C1p, (int)row, 0, x1_scale, (uint8_t*)workspace, st, e5) !=
             cudaSuccess ||
         launch_quantize_nchw_to_nhwc_e4m3(x2, B, C2, H, W, pad, (int)round_up(C2, 16), (int)row, C1p, x2_scale,
-                                          (uint8_t*)workspace, st) != cudaSuccess)
+                                          (uint8_t*)workspace, st, e5) != cudaSuccess)
         return FPQ_ERR_CUDA;
     GemmProblem p{};
     p.conv = 1;
     p.after_stage1 = 1;
     p.w4 = is_e2m1(fw) ? 1 : 0;
     p.w_e5m2 = is_e5m2_native(fw) ? 1 : 0;
+    p.a_e5m2 = is_e5m2_native(fx) ? 1 : 0;
     p.M = (int64_t)B * Ho * Wo;
     p.N = C_out;
     p.Cp = C1p + (int)padded_c(C2);
@@ -1245,7 +1254,8 @@ int32_t fpq_conv2d_route(int B, int C, int H, int W, int C_out, int R, int S, in
     s = conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo);
     if (s != FPQ_OK)
         return s;
-    if (g_path_policy == FPQ_PATH_TWO_KERNELS || g_path_policy == FPQ_PATH_TWO_KERNELS_NARROW || B == 0 || C_out == 0)
+    if (g_path_policy == FPQ_PATH_TWO_KERNELS || g_path_policy == FPQ_PATH_TWO_KERNELS_NARROW || B == 0 || C_out == 0 ||
+        !is_e4m3_native(fx))
         return FPQ_ROUTE_TWO_KERNELS;
     GemmProblem p{};
     p.conv = 1;

@@ -127,6 +127,31 @@ __device__ __forceinline__ uint32_t e4m3x4_from_scaled(float t0, float t1, float
     return mag | (v & nonzero);
 }
 
+// The same for the OCP E5M2 type (bias 15, saturating at 57344): a magnitude above 0x7b can only come from a NaN.
+__device__ __forceinline__ uint32_t e5m2x4_from_scaled(float t0, float t1, float t2, float t3, bool& nan)
+{
+    uint16_t lo, hi;
+    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(t1), "f"(t0));
+    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(t3), "f"(t2));
+    const uint32_t v = (uint32_t)lo | ((uint32_t)hi << 16);
+    const uint32_t mag = v & 0x7f7f7f7fu;
+    const uint32_t nonzero = (mag + 0x7f7f7f7fu) & 0x80808080u;
+    const uint32_t nan_bytes = (mag + 0x04040404u) & 0x80808080u;
+    if (nan_bytes) {
+        nan = true;
+        const uint32_t full = (nan_bytes >> 7) * 0xffu;
+        return (mag | (v & nonzero)) & ~full;
+    }
+    return mag | (v & nonzero);
+}
+
+// E5 = false: E4M3 codes; E5 = true: E5M2 codes (the tensor cores' two 8-bit activation types)
+template <bool E5>
+__device__ __forceinline__ uint32_t fp8x4_from_scaled(float t0, float t1, float t2, float t3, bool& nan)
+{
+    return E5 ? e5m2x4_from_scaled(t0, t1, t2, t3, nan) : e4m3x4_from_scaled(t0, t1, t2, t3, nan);
+}
+
 // ---- PTX wrappers ----------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p)
 {

@@ -1376,7 +1376,7 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
 
     const int BN = (p.N <= 64) ? 64 : 128;
     g.n_tiles = (p.N + BN - 1) / BN;
-    g.idesc = idesc_f8f6f4(0u, p.w4 ? 5u : (p.w_e5m2 ? 1u : 0u), (uint32_t)BN);
+    g.idesc = idesc_f8f6f4(p.a_e5m2 ? 1u : 0u, p.w4 ? 5u : (p.w_e5m2 ? 1u : 0u), (uint32_t)BN);
     g.b_block_tx = (uint32_t)(BN * BK) / (p.w4 ? 2 : 1);
 
     CUtensorMap tmA, tmB;
@@ -1510,6 +1510,8 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
         g.y_tma = 1;
     }
 
+    if (p.x != nullptr && p.a_e5m2)
+        return FPQ_ERR_UNSUPPORTED;     // the fused forms convert to E4M3
     const bool fused = p.x != nullptr && g.mode != MODE_TAPS;
     if (fused) {
         g.x = p.x;

@@ -12,10 +12,11 @@ cudaError_t launch_quantize_act(const float* x, int64_t n, float scale, const QF
                                 cudaStream_t st);
 cudaError_t launch_quantize_weight(const float* w, int64_t N, int64_t K, const float* scale, const QFormat& f,
                                    const uint8_t* rbits, uint8_t* codes, cudaStream_t st);
+// (e5m2 != 0: the codes are OCP E5M2 instead of E4M3, the tensor cores' other 8-bit activation type)
 cudaError_t launch_quantize_rows_e4m3(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, uint8_t* codes,
-                                      cudaStream_t st);
+                                      cudaStream_t st, int e5m2 = 0);
 cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int H, int W, int pad, int Cp, int row,
-                                              int c_off, float scale, uint8_t* codes, cudaStream_t st);
+                                              int c_off, float scale, uint8_t* codes, cudaStream_t st, int e5m2 = 0);
 cudaError_t launch_zero_census(const uint8_t* codes, int64_t n, int four_bit, unsigned long long* count, cudaStream_t st);
 // Code-to-code table of an exact re-encode (weight format -> E4M3), passed to the kernel by value.
 struct CodeTable {
@@ -26,7 +27,7 @@ struct CodeTable {
 cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, int C1, int C1p,
                                   const CodeTable* table, const CodeTable* table2, uint8_t* prepared, cudaStream_t st);
 cudaError_t launch_quantize_rows_e4m3_twice(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, uint8_t* codes,
-                                            cudaStream_t st);
+                                            cudaStream_t st, int e5m2 = 0);
 
 // One warp waits, with the kernels' own bounded wait, on a barrier nobody arrives on: after `limit` cycles it
 // records FPQ_ERR_TIMEOUT in the status word and returns (nothing hangs, nothing faults).
@@ -38,6 +39,7 @@ struct GemmProblem {
     int after_stage1;    // launched right behind this library's own activation-quantize kernel
     int w4;              // weights are E2M1
     int w_e5m2;          // weights are E5M2 (bias 15, native saturation): the tensor cores' second 8-bit type
+    int a_e5m2;          // activation codes are E5M2 (bias 15, native saturation) instead of E4M3
     int64_t M;           // linear rows
     int N;               // outputs / out channels
     int Cp;              // padded reduction length per tap in the weight copy (multiple of 128)

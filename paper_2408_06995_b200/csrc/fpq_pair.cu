@@ -506,7 +506,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 // Geometry and shared-memory plan (no CUDA calls, no pointer is followed); FPQ_ERR_UNSUPPORTED outside the kernel's range.
 static fpq_status plan_pair(const GemmProblem& p, PairArgs& g, int* dyn_bytes)
 {
-    if (!p.conv || p.x == nullptr || p.stride != 1 || p.c_seg != 0 || p.Cp / BK > MAX_CHUNKS || p.R * p.S > 256)
+    if (!p.conv || p.x == nullptr || p.a_e5m2 || p.stride != 1 || p.c_seg != 0 || p.Cp / BK > MAX_CHUNKS || p.R * p.S > 256)
         return FPQ_ERR_UNSUPPORTED;
     if (p.W % 4 != 0 || p.W > 256 || (uintptr_t)p.x % 16 != 0 || p.N > 256 || p.N < 1)
         return FPQ_ERR_UNSUPPORTED;

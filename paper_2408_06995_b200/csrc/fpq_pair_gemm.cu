@@ -333,7 +333,7 @@ fpq_status plan_pg(const GemmProblem& p, int nsm, PGArgs& g, int* dyn_bytes)
         if (g.b_stages > 8)
             g.b_stages = 8;
     }
-    g.idesc = idesc_f8f6f4_pair(0u, p.w4 ? 5u : (p.w_e5m2 ? 1u : 0u), (uint32_t)g.BN);
+    g.idesc = idesc_f8f6f4_pair(p.a_e5m2 ? 1u : 0u, p.w4 ? 5u : (p.w_e5m2 ? 1u : 0u), (uint32_t)g.BN);
     g.tmem_cols = 2u * (uint32_t)g.BN;
     g.wait_prior_grid = p.after_stage1;
     *dyn_bytes = ctl + g.a_stages * g.a_stage_bytes + g.b_stages * g.b_stage_bytes;

@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(256) quantize_weight_kernel(const float* __res
 // ---------------------------------------------------------------------------------
 // TWICE: every row is written two times side by side, [M][2 Kp] (Kp a multiple of 128), for weights that
 // are the sum of two E4M3 terms: the reduction then runs over (x | x) against (first terms | second terms).
-template <bool TWICE>
+template <bool TWICE, bool E5>
 __global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const float* __restrict__ x, int64_t M, int64_t K,
                                                                  int64_t Kp, float rinv, uint8_t* __restrict__ codes,
                                                                  int* status)
@@ -159,8 +159,8 @@ __global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const float* __
                 if (k + 2 < K) a2 = __ldg(px + 4 * j + 2);
                 if (k + 3 < K) a3 = __ldg(px + 4 * j + 3);
             }
-            out[j] = e4m3x4_from_scaled(__fmul_rn(a0, rinv), __fmul_rn(a1, rinv), __fmul_rn(a2, rinv),
-                                        __fmul_rn(a3, rinv), nan);
+            out[j] = fp8x4_from_scaled<E5>(__fmul_rn(a0, rinv), __fmul_rn(a1, rinv), __fmul_rn(a2, rinv),
+                                           __fmul_rn(a3, rinv), nan);
         }
         if (TWICE) {
             int64_t o = row * 2 * vec_per_row + v % vec_per_row;
@@ -182,6 +182,7 @@ __global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const float* __
 // shared memory: loads are coalesced along pixels (16 in flight per thread), stores
 // are whole 128-byte channel rows.  The blocks also share out the frame pixels.
 // ---------------------------------------------------------------------------------
+template <bool E5>
 __global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const float* __restrict__ x, int C, int H,
                                                                          int W, int pad, int Cp, int row, int c_off,
                                                                          float rinv, uint8_t* __restrict__ codes,
@@ -214,10 +215,10 @@ __global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_e4m3_kernel(const f
                 a[q] = (c0 + cl + q < C && p < HW) ? __ldg(px + (int64_t)q * HW) : 0.f;
         }
         uint4 v;
-        v.x = e4m3x4_from_scaled(__fmul_rn(a[0], rinv), __fmul_rn(a[1], rinv), __fmul_rn(a[2], rinv), __fmul_rn(a[3], rinv), nan);
-        v.y = e4m3x4_from_scaled(__fmul_rn(a[4], rinv), __fmul_rn(a[5], rinv), __fmul_rn(a[6], rinv), __fmul_rn(a[7], rinv), nan);
-        v.z = e4m3x4_from_scaled(__fmul_rn(a[8], rinv), __fmul_rn(a[9], rinv), __fmul_rn(a[10], rinv), __fmul_rn(a[11], rinv), nan);
-        v.w = e4m3x4_from_scaled(__fmul_rn(a[12], rinv), __fmul_rn(a[13], rinv), __fmul_rn(a[14], rinv), __fmul_rn(a[15], rinv), nan);
+        v.x = fp8x4_from_scaled<E5>(__fmul_rn(a[0], rinv), __fmul_rn(a[1], rinv), __fmul_rn(a[2], rinv), __fmul_rn(a[3], rinv), nan);
+        v.y = fp8x4_from_scaled<E5>(__fmul_rn(a[4], rinv), __fmul_rn(a[5], rinv), __fmul_rn(a[6], rinv), __fmul_rn(a[7], rinv), nan);
+        v.z = fp8x4_from_scaled<E5>(__fmul_rn(a[8], rinv), __fmul_rn(a[9], rinv), __fmul_rn(a[10], rinv), __fmul_rn(a[11], rinv), nan);
+        v.w = fp8x4_from_scaled<E5>(__fmul_rn(a[12], rinv), __fmul_rn(a[13], rinv), __fmul_rn(a[14], rinv), __fmul_rn(a[15], rinv), nan);
         *reinterpret_cast<uint4*>(&tile[tx][cl]) = v;
     }
     __syncthreads();
@@ -356,29 +357,41 @@ cudaError_t launch_quantize_weight(const float* w, int64_t N, int64_t K, const f
 }
 
 cudaError_t launch_quantize_rows_e4m3(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, uint8_t* codes,
-                                      cudaStream_t st)
+                                      cudaStream_t st, int e5m2)
 {
     int64_t total = M * (Kp / 16);
-    quantize_rows_e4m3_kernel<false><<<grid_for(total, 256), 256, 0, st>>>(x, M, K, Kp, 1.0f / scale, codes,
-                                                                          status_word());
+    if (e5m2)
+        quantize_rows_e4m3_kernel<false, true><<<grid_for(total, 256), 256, 0, st>>>(x, M, K, Kp, 1.0f / scale, codes,
+                                                                                    status_word());
+    else
+        quantize_rows_e4m3_kernel<false, false><<<grid_for(total, 256), 256, 0, st>>>(x, M, K, Kp, 1.0f / scale, codes,
+                                                                                     status_word());
     return cudaGetLastError();
 }
 
 cudaError_t launch_quantize_rows_e4m3_twice(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, uint8_t* codes,
-                                            cudaStream_t st)
+                                            cudaStream_t st, int e5m2)
 {
     int64_t total = M * (Kp / 16);
-    quantize_rows_e4m3_kernel<true><<<grid_for(total, 256), 256, 0, st>>>(x, M, K, Kp, 1.0f / scale, codes,
-                                                                         status_word());
+    if (e5m2)
+        quantize_rows_e4m3_kernel<true, true><<<grid_for(total, 256), 256, 0, st>>>(x, M, K, Kp, 1.0f / scale, codes,
+                                                                                   status_word());
+    else
+        quantize_rows_e4m3_kernel<true, false><<<grid_for(total, 256), 256, 0, st>>>(x, M, K, Kp, 1.0f / scale, codes,
+                                                                                    status_word());
     return cudaGetLastError();
 }
 
 cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int H, int W, int pad, int Cp, int row,
-                                              int c_off, float scale, uint8_t* codes, cudaStream_t st)
+                                              int c_off, float scale, uint8_t* codes, cudaStream_t st, int e5m2)
 {
     dim3 grid((H * W + 31) / 32, (Cp + 127) / 128, B);
-    quantize_nchw_to_nhwc_e4m3_kernel<<<grid, 256, 0, st>>>(x, C, H, W, pad, Cp, row, c_off, 1.0f / scale, codes,
-                                                            status_word());
+    if (e5m2)
+        quantize_nchw_to_nhwc_e4m3_kernel<true><<<grid, 256, 0, st>>>(x, C, H, W, pad, Cp, row, c_off, 1.0f / scale, codes,
+                                                                      status_word());
+    else
+        quantize_nchw_to_nhwc_e4m3_kernel<false><<<grid, 256, 0, st>>>(x, C, H, W, pad, Cp, row, c_off, 1.0f / scale, codes,
+                                                                       status_word());
     return cudaGetLastError();
 }
 

@@ -110,6 +110,7 @@ def test_sizes(L):
     assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E4M3, fpq.E4M3) == 100 * 320
     assert fpq.fpq_linear_workspace_size(100, 64, 321, fpq.E4M3, fpq.E2M1) == 100 * 336
     assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E3M4, fpq.E4M3) > 100 * 320     # CUDA-core route: FP32 scratch
+    assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E5M2, fpq.E2M1) == 100 * 320    # OCP E5M2 activations: tensor cores
     assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.Format(6, 3, 7), fpq.E4M3) == 0
     assert fpq.fpq_conv2d_workspace_size(2, 4, 8, 8, 16, 3, 3, 1, 1, fpq.E4M3, fpq.E2M1) == 2 * 100 * 16
     assert fpq.fpq_prepared_size(fpq.E4M3, fpq.LINEAR, 10, 320) == 10 * 384

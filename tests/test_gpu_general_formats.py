@@ -23,7 +23,9 @@ E5M2_B40 = fpq.Format(5, 2, 40, fpq.SAT_PAPER)       # needs a factor beyond the
 
 PAIRS = [(fpq.E4M3, fpq.E3M4), (fpq.E4M3, fpq.E2M5), (fpq.E4M3, fpq.E5M2), (fpq.E4M3, E5M2_B16), (fpq.E4M3, E4M3_PAPER),
          (fpq.E4M3, E4M3_B8), (fpq.E4M3, E2M1_TINY), (fpq.E4M3, E1M6), (fpq.E4M3, E6M1), (fpq.E4M3, E5M2_B40), (fpq.E3M4, E5M2_B16),
-         (fpq.E5M2, fpq.E4M3), (fpq.E3M4, fpq.E2M1), (E4M3_PAPER, fpq.E1M2), (fpq.E2M5, fpq.E3M4)]
+         (fpq.E5M2, fpq.E4M3), (fpq.E3M4, fpq.E2M1), (E4M3_PAPER, fpq.E1M2), (fpq.E2M5, fpq.E3M4),
+         # OCP E5M2 activations are read by the tensor cores as they are, with every kind of weight preparation
+         (fpq.E5M2, fpq.E5M2), (fpq.E5M2, fpq.E2M1), (fpq.E5M2, fpq.E1M2), (fpq.E5M2, fpq.E3M4), (fpq.E5M2, E5M2_B16)]
 
 
 def _run(L, gfx, gfw, use_bias=True):
@@ -65,13 +67,26 @@ def test_linear(gfx, gfw, M, K, N):
 
 
 @pytest.mark.parametrize("gfx,gfw", [(fpq.E4M3, fpq.E3M4), (fpq.E4M3, E5M2_B16), (fpq.E4M3, E4M3_B8), (fpq.E5M2, fpq.E2M1),
-                                     (fpq.E3M4, fpq.E1M2)])
+                                     (fpq.E3M4, fpq.E1M2), (fpq.E5M2, fpq.E4M3), (fpq.E5M2, fpq.E3M4)])
 @pytest.mark.parametrize("shape", [(2, 40, 12, 12, 72, 3, 1), (1, 130, 9, 11, 33, 3, 2), (3, 64, 8, 8, 130, 1, 1)])
 def test_conv(gfx, gfw, shape):
     B, C, H, W, Co, R, stride = shape
     L = I.conv_layer("t", B, C, H, W, Co, R, stride=stride, rounding=(stride == 2))
     I.draw(L, 32, B + C + Co, "silu", 0.03, True, 0.01)
     _run(L, gfx, gfw)
+
+
+def test_e5m2_activations_at_a_size_that_spans_many_tiles():
+    # the tensor-core route for OCP E5M2 activations on shapes with several tiles per CTA and a ragged tail
+    L = I.linear_layer("t", 1000, 320, 960, "e4m3")
+    I.draw(L, 35, 1, "normal", 0.02, True, 0.01, (0.001, 20.0))
+    _run(L, fpq.E5M2, fpq.E4M3)
+    L = I.conv_layer("t", 9, 256, 32, 32, 256, 3, wfmt="e2m1", rounding=True)      # wide-MMA contraction (CTA pairs)
+    I.draw(L, 35, 2, "silu", 0.03, True, 0.01)
+    _run(L, fpq.E5M2, fpq.E2M1)
+    # the scratch is one byte per activation: the tensor-core route, not the FP32 scratch of the CUDA-core route
+    assert fpq.fpq_linear_workspace_size(1000, 960, 320, fpq.E5M2, fpq.E4M3) == 1000 * 320
+    assert fpq.fpq_linear_workspace_size(1000, 960, 320, fpq.E3M4, fpq.E4M3) > 4 * 1000 * 320
 
 
 def test_every_fp8_search_candidate_runs_as_a_layer():

@@ -98,13 +98,14 @@ def test_formats_that_need_more_scratch_per_element():
     assert Lb.fpq_linear_static(p, p, p, 1.0, fpq.E4M3.c(), e3m4.c(), None, p, 6000, 64, 1024, None) == fpq.ERR_WORKSPACE
     # activations in a format the tensor cores have no type for run on the CUDA cores with FP32 scratch:
     # a small problem fits, a larger one that passes the M x K test does not
-    e5m2 = fpq.E5M2
-    xs5 = float(x.abs().max()) / fpq.fpq_format_max(e5m2)
+    e2m5 = fpq.E2M5
+    xs5 = float(x.abs().max()) / fpq.fpq_format_max(e2m5)
     w8 = (w.abs().amax(dim=1) / 448.0).contiguous()
     prep8 = fpq.fpq_prepare_weight(fpq.fpq_quantize_weight(w, w8, fpq.E4M3, None), fpq.E4M3, fpq.LINEAR, N, K)
-    y_ref = fpq.fpq_linear(x, prep8, w8, xs5, e5m2, fpq.E4M3, None, N)
+    y_ref = fpq.fpq_linear(x, prep8, w8, xs5, e2m5, fpq.E4M3, None, N)
     y.fill_(float("nan"))
-    fpq.fpq_linear_static(x, prep8, w8, xs5, e5m2, fpq.E4M3, None, y)
+    fpq.fpq_linear_static(x, prep8, w8, xs5, e2m5, fpq.E4M3, None, y)
     assert fpq.fpq_read_status() == fpq.OK
     assert torch.equal(y, y_ref)
-    assert Lb.fpq_linear_static(p, p, p, 1.0, e5m2.c(), fpq.E4M3.c(), None, p, 6000, 64, 1024, None) == fpq.ERR_WORKSPACE
+    assert fpq.fpq_linear_workspace_size(6000, 64, 1024, e2m5, fpq.E4M3) > fpq.STATIC_SCRATCH_BYTES
+    assert Lb.fpq_linear_static(p, p, p, 1.0, e2m5.c(), fpq.E4M3.c(), None, p, 6000, 64, 1024, None) == fpq.ERR_WORKSPACE
