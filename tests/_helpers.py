@@ -51,6 +51,31 @@ def gpu_prepare(L, ws):
     return codes, prep
 
 
+GUARD = 256          # bytes of guard band on each side of an output or workspace buffer
+CANARY = 0xA5        # every guard byte (as FP32 words: 0xA5A5A5A5, a pattern no result produces)
+
+
+class Guarded:
+    """A device buffer with a guard band in front of it and behind it.  The library gets the inner view; after
+    the call the bands must still hold the canary bytes: a store one element before or past a ragged output,
+    or past the workspace size the library itself asked for, is caught on the host."""
+
+    def __init__(self, nbytes, dev="cuda"):
+        self.n = int(nbytes)
+        pad = (-self.n) % 256                          # the band behind starts on a 256-byte boundary
+        self.raw = torch.full((GUARD + self.n + pad + GUARD,), CANARY, dtype=torch.uint8, device=dev)
+        self.inner = self.raw[GUARD:GUARD + self.n]
+
+    def f32(self, shape):
+        return self.inner.view(torch.float32).view(shape)
+
+    def check(self, what):
+        front = self.raw[:GUARD]
+        back = self.raw[GUARD + self.n:]
+        assert bool((front == CANARY).all()), f"{what}: bytes in front of the buffer were overwritten"
+        assert bool((back == CANARY).all()), f"{what}: bytes behind the buffer were overwritten"
+
+
 def _gpu_layer_once(L, ws, xs, use_bias, prep):
     gfw, _ = FMT[L.wfmt]
     dev = "cuda"
@@ -58,11 +83,19 @@ def _gpu_layer_once(L, ws, xs, use_bias, prep):
     bias = torch.from_numpy(L.bias).to(dev) if use_bias else None
     wsd = torch.from_numpy(ws).to(dev)
     if L.kind == "linear":
-        y = fpq.fpq_linear(x, prep, wsd, xs, fpq.E4M3, gfw, bias, L.N)
+        yg = Guarded(4 * L.M * L.N)
+        wg = Guarded(max(1, fpq.fpq_linear_workspace_size(L.M, L.N, L.K, fpq.E4M3, gfw)))
+        y = fpq.fpq_linear(x, prep, wsd, xs, fpq.E4M3, gfw, bias, L.N, y=yg.f32((L.M, L.N)), workspace=wg.inner)
     else:
-        y = fpq.fpq_conv2d(x, prep, wsd, xs, fpq.E4M3, gfw, bias, L.N, L.R, L.S, L.pad, L.stride)
+        yg = Guarded(4 * L.B * L.N * L.Ho * L.Wo)
+        wg = Guarded(max(1, fpq.fpq_conv2d_workspace_size(L.B, L.C, L.H, L.W, L.N, L.R, L.S, L.pad, L.stride,
+                                                           fpq.E4M3, gfw)))
+        y = fpq.fpq_conv2d(x, prep, wsd, xs, fpq.E4M3, gfw, bias, L.N, L.R, L.S, L.pad, L.stride,
+                           y=yg.f32((L.B, L.N, L.Ho, L.Wo)), workspace=wg.inner)
     st = fpq.fpq_read_status()
     assert st == fpq.OK, fpq.status_string(st)
+    yg.check(f"{L.name} output")
+    wg.check(f"{L.name} workspace")
     return y.cpu().numpy()
 
 

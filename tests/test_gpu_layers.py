@@ -10,7 +10,7 @@ import torch
 import oracle as O
 import paper_2408_06995_b200 as fpq
 from paper_2408_06995_b200 import inputs as I
-from _helpers import FMT, assert_close, gpu_layer, gpu_prepare, layer_scales, oracle_layer, sample_indices
+from _helpers import FMT, Guarded, assert_close, gpu_layer, gpu_prepare, layer_scales, oracle_layer, sample_indices
 
 pytestmark = pytest.mark.gpu
 
@@ -325,12 +325,14 @@ def test_host_forms_equal_the_device_forms(kind, shape):
     wsd = torch.from_numpy(ws).cuda()
     bias = torch.from_numpy(L.bias).cuda()
     if kind == "conv":
-        yd = torch.empty((L.B, L.N, L.Ho, L.Wo), dtype=torch.float32, device="cuda")
-        wk = torch.empty(fpq.fpq_conv2d_workspace_size(L.B, L.C, L.H, L.W, L.N, L.R, L.S, L.pad, L.stride, fpq.E4M3, gfw),
-                         dtype=torch.uint8, device="cuda")
+        yg = Guarded(4 * L.B * L.N * L.Ho * L.Wo)
+        yd = yg.f32((L.B, L.N, L.Ho, L.Wo))
+        wg = Guarded(fpq.fpq_conv2d_workspace_size(L.B, L.C, L.H, L.W, L.N, L.R, L.S, L.pad, L.stride, fpq.E4M3, gfw))
     else:
-        yd = torch.empty((L.M, L.N), dtype=torch.float32, device="cuda")
-        wk = torch.empty(max(1, fpq.fpq_linear_workspace_size(L.M, L.N, L.K, fpq.E4M3, gfw)), dtype=torch.uint8, device="cuda")
+        yg = Guarded(4 * L.M * L.N)
+        yd = yg.f32((L.M, L.N))
+        wg = Guarded(max(1, fpq.fpq_linear_workspace_size(L.M, L.N, L.K, fpq.E4M3, gfw)))
+    wk = wg.inner
     yh = torch.empty(yd.shape, dtype=torch.float32).pin_memory()
     for _ in range(2):                                    # twice: the pipeline's streams and events are reused
         yh.fill_(float("nan"))
@@ -340,3 +342,5 @@ def test_host_forms_equal_the_device_forms(kind, shape):
             fpq.fpq_linear_host(xh, xd, prep, wsd, xs, fpq.E4M3, gfw, bias, yd, yh, wk)
         assert fpq.fpq_read_status() == fpq.OK
         assert np.array_equal(yh.numpy(), want)
+        yg.check("host form: device output")
+        wg.check("host form: workspace")

@@ -7,7 +7,7 @@ import torch
 
 import oracle as O
 import paper_2408_06995_b200 as fpq
-from _helpers import FMT, assert_close
+from _helpers import FMT, assert_close, Guarded
 
 pytestmark = pytest.mark.gpu
 
@@ -41,14 +41,16 @@ def _gpu(x1, x2, w, bias, bits, ws, s1, s2, gfw, pad, stride):
                                     torch.from_numpy(O.pack_bits(bits)).to(dev))
     prep = fpq.fpq_prepare_weight_split(codes, gfw, Co, C1, C2, R, S)
     Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
-    y = torch.empty((B, Co, Ho, Wo), dtype=torch.float32, device=dev)
-    wk = torch.empty(fpq.fpq_conv2d_split_workspace_size(B, C1, C2, H, W, Co, R, S, pad, stride, fpq.E4M3, gfw),
-                     dtype=torch.uint8, device=dev)
+    yg = Guarded(4 * B * Co * Ho * Wo)                                   # guard bands around output and scratch
+    wg = Guarded(fpq.fpq_conv2d_split_workspace_size(B, C1, C2, H, W, Co, R, S, pad, stride, fpq.E4M3, gfw))
+    y, wk = yg.f32((B, Co, Ho, Wo)), wg.inner
     wk.fill_(0xAB)                                                       # the call must not rely on a clean scratch
     fpq.fpq_conv2d_split(torch.from_numpy(x1).to(dev), s1, torch.from_numpy(x2).to(dev), s2, prep,
                          torch.from_numpy(ws).to(dev), fpq.E4M3, gfw, torch.from_numpy(bias).to(dev), y, R, S, pad,
                          stride, wk)
     assert fpq.fpq_read_status() == fpq.OK
+    yg.check("two-tensor convolution output")
+    wg.check("two-tensor convolution workspace")
     return y.cpu().numpy()
 
 
