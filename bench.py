@@ -513,11 +513,23 @@ def run_own(args):
         xq = torch.randn(nq, device=dev, dtype=torch.float32)
         cq = torch.empty(nq, device=dev, dtype=torch.uint8)
         quant = {}
-        for name, fmt, by in (("act_e4m3_native", fpq.E4M3, 5.0), ("act_e5m2_general", fpq.E5M2, 5.0),
-                              ("act_e2m1_general", fpq.E2M1, 4.5)):
+        for name, fmt, by in (("act_e4m3_hw_convert", fpq.E4M3, 5.0), ("act_e5m2_hw_convert", fpq.E5M2, 5.0),
+                              ("act_e2m1_hw_convert", fpq.E2M1, 4.5), ("act_e3m4_general", fpq.E3M4, 5.0),
+                              ("act_e1m2_general", fpq.E1M2, 4.5)):
             tq = per_launch_us(torch, lambda: fpq.fpq_quantize_act(xq, 0.01, fmt, cq), 10) * 1e-6
             quant[name] = {"elements": nq, "us": tq * 1e6, "gbs": by * nq / tq / 1e9,
                            "frac_of_hbm_peak": by * nq / tq / 1e9 / peaks["hbm_gbs"], "bytes_per_element": by}
+        # the weight encoder (Sec. V-B: nearest, or signed floor + learned decision) on an 8192 x 8192 matrix
+        wq = xq.view(8192, 8192)
+        wsq = torch.full((8192,), 0.01, device=dev)
+        rbq = torch.randint(0, 256, (8192, 1024), device=dev, dtype=torch.uint8)
+        for name, fmt, rb, by in (("weight_e4m3_nearest", fpq.E4M3, None, 5.0), ("weight_e2m1_nearest", fpq.E2M1, None, 4.5),
+                                  ("weight_e2m1_learned", fpq.E2M1, rbq, 4.625), ("weight_e3m4_learned", fpq.E3M4, rbq, 5.125)):
+            out = fpq.fpq_quantize_weight(wq, wsq, fmt, rb)
+            tq = per_launch_us(torch, lambda: fpq.fpq_quantize_weight(wq, wsq, fmt, rb, out), 10) * 1e-6
+            quant[name] = {"elements": nq, "us": tq * 1e6, "gbs": by * nq / tq / 1e9,
+                           "frac_of_hbm_peak": by * nq / tq / 1e9 / peaks["hbm_gbs"], "bytes_per_element": by}
+        del wq, wsq, rbq, out
         del xq, cq
         torch.cuda.empty_cache()
 

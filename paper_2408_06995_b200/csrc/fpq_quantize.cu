@@ -9,7 +9,69 @@ namespace fpq {
 // Activation quantize, flat: 16 elements per thread, 4 x 128-bit loads, one
 // 128-bit store.  HBM-bound: 5 bytes per element.
 // ---------------------------------------------------------------------------------
-template <bool FAST_E4M3>
+// MODE selects the conversion: 0 the general rounding arithmetic (any format), 1 E4M3, 2 OCP E5M2 and
+// 3 E2M1 with the hardware converts (round to nearest even, saturating at the type's largest finite value:
+// the same function of t, -0 and NaN mapped to code 0 afterwards).
+constexpr int Q_GENERAL = 0, Q_E4M3 = 1, Q_E5M2 = 2, Q_E2M1 = 3;
+
+// Eight E2M1 codes (bias 1, grid 0 .. 6) from eight scaled floats, element j in nibble j.
+__device__ __forceinline__ uint32_t e2m1x8_from_scaled(const float (&t)[8], bool& nan)
+{
+    uint32_t v = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        uint32_t b;
+        asm("{\n\t.reg .b8 q;\n\t"
+            "cvt.rn.satfinite.e2m1x2.f32 q, %1, %2;\n\t"
+            "cvt.u32.u8 %0, q;\n\t}"
+            : "=r"(b)
+            : "f"(t[2 * j + 1]), "f"(t[2 * j]));
+        v |= b << (8 * j);
+        nan |= (t[2 * j] != t[2 * j]) | (t[2 * j + 1] != t[2 * j + 1]);
+    }
+    // a NaN converts to the largest magnitude: those nibbles are cleared; -0 becomes +0
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        if (t[j] != t[j])
+            v &= ~(0xfu << (4 * j));
+    const uint32_t mag = v & 0x77777777u;
+    const uint32_t nonzero = (mag + 0x77777777u) & 0x88888888u;
+    return mag | (v & nonzero);
+}
+
+// 16 scaled values -> their codes: four words of bytes, or two words of nibbles for 4-bit formats
+template <int MODE>
+__device__ __forceinline__ void encode16_rne(const float (&t)[16], const QFormat& f, uint32_t (&out)[4], bool& nan)
+{
+    if constexpr (MODE == Q_E2M1) {
+        const float lo[8] = {t[0], t[1], t[2], t[3], t[4], t[5], t[6], t[7]};
+        const float hi[8] = {t[8], t[9], t[10], t[11], t[12], t[13], t[14], t[15]};
+        out[0] = e2m1x8_from_scaled(lo, nan);
+        out[1] = e2m1x8_from_scaled(hi, nan);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (MODE == Q_E4M3)
+                out[j] = e4m3x4_from_scaled(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3], nan);
+            else if (MODE == Q_E5M2)
+                out[j] = e5m2x4_from_scaled(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3], nan);
+            else
+                out[j] = quantize_rne_bits(t[4 * j], f, nan) | (quantize_rne_bits(t[4 * j + 1], f, nan) << 8) |
+                         (quantize_rne_bits(t[4 * j + 2], f, nan) << 16) | (quantize_rne_bits(t[4 * j + 3], f, nan) << 24);
+        }
+        if (f.four_bit) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const uint32_t a0 = out[2 * j], a1 = out[2 * j + 1];
+                out[j] = (a0 & 0xf) | ((a0 >> 4) & 0xf0) | ((a0 >> 8) & 0xf00) | ((a0 >> 12) & 0xf000) |
+                         ((a1 & 0xf) << 16) | (((a1 >> 4) & 0xf0) << 16) | (((a1 >> 8) & 0xf00) << 16) |
+                         (((a1 >> 12) & 0xf000) << 16);
+            }
+        }
+    }
+}
+
+template <int MODE>
 __global__ void __launch_bounds__(256) quantize_act_kernel(const float* __restrict__ x, int64_t n, float rinv,
                                                            QFormat f, uint8_t* __restrict__ codes, int* status)
 {
@@ -22,31 +84,20 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const float* __restri
 #pragma unroll
         for (int j = 0; j < 4; ++j)
             a[j] = __ldg(px + j);
-        uint32_t out[4];
+        float t[16];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            float t0 = __fmul_rn(a[j].x, rinv), t1 = __fmul_rn(a[j].y, rinv);
-            float t2 = __fmul_rn(a[j].z, rinv), t3 = __fmul_rn(a[j].w, rinv);
-            if (FAST_E4M3) {
-                out[j] = e4m3x4_from_scaled(t0, t1, t2, t3, nan);
-            } else {
-                out[j] = quantize_rne_bits(t0, f, nan) | (quantize_rne_bits(t1, f, nan) << 8) |
-                         (quantize_rne_bits(t2, f, nan) << 16) | (quantize_rne_bits(t3, f, nan) << 24);
-            }
+            t[4 * j] = __fmul_rn(a[j].x, rinv);
+            t[4 * j + 1] = __fmul_rn(a[j].y, rinv);
+            t[4 * j + 2] = __fmul_rn(a[j].z, rinv);
+            t[4 * j + 3] = __fmul_rn(a[j].w, rinv);
         }
-        if (!f.four_bit) {
+        uint32_t out[4];
+        encode16_rne<MODE>(t, f, out, nan);
+        if (!f.four_bit)
             reinterpret_cast<uint4*>(codes)[v] = make_uint4(out[0], out[1], out[2], out[3]);
-        } else {
-            uint32_t p[2];
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                uint32_t a0 = out[2 * j], a1 = out[2 * j + 1];
-                p[j] = (a0 & 0xf) | ((a0 >> 4) & 0xf0) | ((a0 >> 8) & 0xf00) | ((a0 >> 12) & 0xf000) |
-                       ((a1 & 0xf) << 16) | (((a1 >> 4) & 0xf0) << 16) | (((a1 >> 8) & 0xf00) << 16) |
-                       (((a1 >> 12) & 0xf000) << 16);
-            }
-            reinterpret_cast<uint2*>(codes)[v] = make_uint2(p[0], p[1]);
-        }
+        else
+            reinterpret_cast<uint2*>(codes)[v] = make_uint2(out[0], out[1]);
     }
     // tail (fewer than 16 elements): one thread, in order, so nibbles never race
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -120,6 +171,69 @@ __global__ void __launch_bounds__(256) quantize_weight_kernel(const float* __res
             for (int j = 0; j < (cnt + 1) / 2; ++j)
                 po[j] = (uint8_t)(c[2 * j] | (c[2 * j + 1] << 4));
         }
+    }
+    if (nan)
+        flag_status(status, FPQ_ERR_NAN_INPUT);
+}
+
+// The same for rows whose length is a multiple of 16 (aligned buffers): one thread per 16 weights of a row (two
+// rounding bytes), 4 x 128-bit loads, one 128-bit (64-bit for 4-bit codes) store.  HBM-bound: 4 bytes in,
+// 1 or 0.5 out, 1/8 of rounding decisions per weight.  LEARNED: the rounding decisions are given.
+template <int MODE, bool LEARNED>
+__global__ void __launch_bounds__(256) quantize_weight_vec_kernel(const float* __restrict__ w, int64_t N, int64_t K,
+                                                                  const float* __restrict__ scale, QFormat f,
+                                                                  const uint8_t* __restrict__ rbits,
+                                                                  uint8_t* __restrict__ codes, int* status)
+{
+    bool nan = false;
+    const int64_t per_row = K / 16;
+    const int64_t total = N * per_row;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < total; v += stride) {
+        const int64_t n = v / per_row;
+        const float rinv = __fdiv_rn(1.0f, __ldg(scale + n));
+        const float4* pw = reinterpret_cast<const float4*>(w) + v * 4;
+        float4 a[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            a[j] = __ldg(pw + j);
+        float t[16];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            t[4 * j] = __fmul_rn(a[j].x, rinv);
+            t[4 * j + 1] = __fmul_rn(a[j].y, rinv);
+            t[4 * j + 2] = __fmul_rn(a[j].z, rinv);
+            t[4 * j + 3] = __fmul_rn(a[j].w, rinv);
+        }
+        uint32_t out[4];
+        if (!LEARNED) {
+            encode16_rne<MODE>(t, f, out, nan);
+        } else {
+            // 16 decisions: the row's bytes 2 g and 2 g + 1 (K / 8 is even, so the pair is 2-byte aligned)
+            const uint32_t hb = __ldg(reinterpret_cast<const uint16_t*>(rbits) + v);
+            uint32_t c[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                c[j] = quantize_bits(t[j], f, (int)((hb >> j) & 1u), nan);
+            if (!f.four_bit) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    out[j] = c[4 * j] | (c[4 * j + 1] << 8) | (c[4 * j + 2] << 16) | (c[4 * j + 3] << 24);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    uint32_t o = 0;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        o |= c[8 * j + q] << (4 * q);
+                    out[j] = o;
+                }
+            }
+        }
+        if (!f.four_bit)
+            reinterpret_cast<uint4*>(codes)[v] = make_uint4(out[0], out[1], out[2], out[3]);
+        else
+            reinterpret_cast<uint2*>(codes)[v] = make_uint2(out[0], out[1]);
     }
     if (nan)
         flag_status(status, FPQ_ERR_NAN_INPUT);
@@ -329,6 +443,18 @@ static int grid_for(int64_t work_items, int threads)
     return (int)blocks;
 }
 
+// which conversion a format's round-to-nearest encode may use
+static int rne_mode(const QFormat& f)
+{
+    if (f.native_e4m3)
+        return Q_E4M3;
+    if (f.e == 5 && f.m == 2 && f.B == 15 && f.code_max == 0x7B)
+        return Q_E5M2;
+    if (f.e == 2 && f.m == 1 && f.B == 1)
+        return Q_E2M1;
+    return Q_GENERAL;
+}
+
 cudaError_t launch_quantize_act(const float* x, int64_t n, float scale, const QFormat& f, uint8_t* codes,
                                 cudaStream_t st)
 {
@@ -336,12 +462,16 @@ cudaError_t launch_quantize_act(const float* x, int64_t n, float scale, const QF
         return cudaSuccess;
     float rinv = 1.0f / scale;
     bool aligned = ((uintptr_t)x % 16 == 0) && ((uintptr_t)codes % 16 == 0);
+    const int grid = grid_for(n / 16 + 1, 256);
     if (!aligned) {
         quantize_act_scalar_kernel<<<grid_for(n, 256), 256, 0, st>>>(x, n, rinv, f, codes, status_word());
-    } else if (f.native_e4m3) {
-        quantize_act_kernel<true><<<grid_for(n / 16 + 1, 256), 256, 0, st>>>(x, n, rinv, f, codes, status_word());
     } else {
-        quantize_act_kernel<false><<<grid_for(n / 16 + 1, 256), 256, 0, st>>>(x, n, rinv, f, codes, status_word());
+        switch (rne_mode(f)) {
+        case Q_E4M3: quantize_act_kernel<Q_E4M3><<<grid, 256, 0, st>>>(x, n, rinv, f, codes, status_word()); break;
+        case Q_E5M2: quantize_act_kernel<Q_E5M2><<<grid, 256, 0, st>>>(x, n, rinv, f, codes, status_word()); break;
+        case Q_E2M1: quantize_act_kernel<Q_E2M1><<<grid, 256, 0, st>>>(x, n, rinv, f, codes, status_word()); break;
+        default: quantize_act_kernel<Q_GENERAL><<<grid, 256, 0, st>>>(x, n, rinv, f, codes, status_word()); break;
+        }
     }
     return cudaGetLastError();
 }
@@ -351,6 +481,21 @@ cudaError_t launch_quantize_weight(const float* w, int64_t N, int64_t K, const f
 {
     if (N == 0 || K == 0)
         return cudaSuccess;
+    const bool vec = K % 16 == 0 && (uintptr_t)w % 16 == 0 && (uintptr_t)codes % 16 == 0 && (uintptr_t)rbits % 2 == 0;
+    if (vec) {
+        const int grid = grid_for(N * (K / 16), 256);
+        if (rbits) {
+            quantize_weight_vec_kernel<Q_GENERAL, true><<<grid, 256, 0, st>>>(w, N, K, scale, f, rbits, codes, status_word());
+        } else {
+            switch (rne_mode(f)) {
+            case Q_E4M3: quantize_weight_vec_kernel<Q_E4M3, false><<<grid, 256, 0, st>>>(w, N, K, scale, f, rbits, codes, status_word()); break;
+            case Q_E5M2: quantize_weight_vec_kernel<Q_E5M2, false><<<grid, 256, 0, st>>>(w, N, K, scale, f, rbits, codes, status_word()); break;
+            case Q_E2M1: quantize_weight_vec_kernel<Q_E2M1, false><<<grid, 256, 0, st>>>(w, N, K, scale, f, rbits, codes, status_word()); break;
+            default: quantize_weight_vec_kernel<Q_GENERAL, false><<<grid, 256, 0, st>>>(w, N, K, scale, f, rbits, codes, status_word()); break;
+            }
+        }
+        return cudaGetLastError();
+    }
     int64_t total = N * ((K + 7) / 8);
     quantize_weight_kernel<<<grid_for(total, 256), 256, 0, st>>>(w, N, K, scale, f, rbits, codes, status_word());
     return cudaGetLastError();

@@ -33,8 +33,10 @@ def _sweep(f):
 def test_weight_encode_sweep_all_modes(f):
     of = to_oracle(f)
     pts = _sweep(f)
-    for scale in (1.0, 0.25, 0.0371, 3.3):
+    for scale, pad16 in ((1.0, False), (0.25, True), (0.0371, True), (3.3, False)):
         x = (pts * np.float32(scale)).astype(np.float32)
+        if pad16:       # rows of a multiple of 16 weights take the 16-per-thread kernels
+            x = np.concatenate([x, np.zeros(-x.size % 16, np.float32)])
         N = 3
         K = x.size
         w = np.stack([x, x[::-1], np.roll(x, 5)]).astype(np.float32)
@@ -85,34 +87,46 @@ def test_act_quantize_random(f, n):
     assert np.array_equal(got2.reshape(-1), want.reshape(-1))
 
 
-def test_act_quantize_sweep_e4m3_fast_path():
-    pts = _sweep(fpq.E4M3)
+@pytest.mark.parametrize("f", FORMATS)
+def test_act_quantize_sweep(f):
+    """Every grid value, every tie and their FP32 neighbours, both signs (the hardware-convert kernels of E4M3, the
+    OCP E5M2 and E2M1 and the general arithmetic alike)."""
+    pts = _sweep(f)
     for scale in (1.0, 0.5, 0.0371, 11.0):
         x = np.tile((pts * np.float32(scale)).astype(np.float32), 3)
-        want = O.quantize_act(x, scale, O.E4M3)
-        got = fpq.fpq_quantize_act(torch.from_numpy(x).cuda(), scale, fpq.E4M3).cpu().numpy()
-        assert np.array_equal(got, want)
+        want = O.quantize_act(x, scale, to_oracle(f))
+        got = fpq.fpq_quantize_act(torch.from_numpy(x).cuda(), scale, f).cpu().numpy()
+        assert np.array_equal(got.reshape(-1), want.reshape(-1))
 
 
 def test_special_values_and_status_flag():
     assert fpq.fpq_read_status() == fpq.OK
     x = np.zeros(64, dtype=np.float32)
     x[3], x[4], x[5], x[6], x[20] = np.inf, -np.inf, -0.0, -1e-30, 1.0
-    for f in (fpq.E4M3, fpq.E2M1, fpq.E3M4):
+    for f in (fpq.E4M3, fpq.E5M2, fpq.E2M1, fpq.E3M4):
         got = fpq.fpq_quantize_act(torch.from_numpy(x).cuda(), 1.0, f).cpu().numpy()
         want = O.quantize_act(x, 1.0, to_oracle(f))
         assert np.array_equal(got.reshape(-1), want.reshape(-1))
         assert fpq.fpq_read_status() == fpq.OK
-    x[7] = np.nan
-    for f in (fpq.E4M3, fpq.E3M4):
+    x[7] = x[40] = x[41] = np.nan
+    for f in (fpq.E4M3, fpq.E5M2, fpq.E2M1, fpq.E3M4):
         got = fpq.fpq_quantize_act(torch.from_numpy(x).cuda(), 1.0, f).cpu().numpy()
         want = O.quantize_act(x, 1.0, to_oracle(f))
-        assert got[7] == 0 and np.array_equal(got, want)
+        assert np.array_equal(got.reshape(-1), want.reshape(-1))
+        if f is not fpq.E2M1:
+            assert got[7] == 0
         assert fpq.fpq_read_status() == fpq.ERR_NAN_INPUT
         assert fpq.fpq_read_status() == fpq.OK          # reading clears it
-    w = torch.from_numpy(x.reshape(1, -1)).cuda()
-    fpq.fpq_quantize_weight(w, torch.ones(1, device="cuda"), fpq.E2M1)
-    assert fpq.fpq_read_status() == fpq.ERR_NAN_INPUT
+    # the weight encoders: rows of 64 (16 per thread) and of 63 (8 per thread), with and without rounding decisions
+    for f in (fpq.E4M3, fpq.E5M2, fpq.E2M1, fpq.E3M4):
+        for K in (64, 63):
+            w = np.stack([x[:K], x[:K][::-1]]).astype(np.float32)
+            sc = np.ones(2, np.float32)
+            for rb in (None, O.pack_bits(np.ones((2, K), np.uint8))):
+                got = fpq.fpq_quantize_weight(torch.from_numpy(w).cuda(), torch.from_numpy(sc).cuda(), f,
+                                              None if rb is None else torch.from_numpy(rb).cuda()).cpu().numpy()
+                assert np.array_equal(got, O.quantize_weight(w, sc, to_oracle(f), rb))
+                assert fpq.fpq_read_status() == fpq.ERR_NAN_INPUT
 
 
 def test_empty_inputs():
