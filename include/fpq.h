@@ -32,6 +32,9 @@
  *     (-1)^s d 2^(1 - exp_bias - man_bits)                    for p = 0
  * bit (e+m) = sign, bits [m, e+m) = p, bits [0, m) = d.  1 + e + m <= 8; formats
  * of up to 4 bits are stored two per byte (even index in the low nibble).
+ * exp_bias is limited to 2^exp_bits - man_bits - 104 <= exp_bias <= 126 - man_bits
+ * (every grid value and the rounding constants of its binades are normal FP32
+ * numbers); anything else is FPQ_ERR_FORMAT.
  * `scale` is the real value of one unit of the code domain: real = scale *
  * value(code).  It plays the role of the paper's real-valued exponent bias:
  * b_paper = exp_bias - log2(scale).

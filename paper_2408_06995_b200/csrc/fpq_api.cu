@@ -48,8 +48,9 @@ bool resolve_format(fpq_format f, QFormat* q)
     if (f.sat_mode != FPQ_SAT_PAPER && f.sat_mode != FPQ_SAT_NATIVE)
         return false;
     int top = (1 << f.exp_bits) - 1;
-    // every grid value must be a normal FP32 number
-    if (top - f.exp_bias > 126 || 1 - f.exp_bias - f.man_bits < -125)
+    // every grid value must be a normal FP32 number, and so must 1.5 * 2^23 steps of the top binade (the
+    // rounding constant of the quantizer kernels)
+    if (top - f.exp_bias + 23 - f.man_bits > 126 || 1 - f.exp_bias - f.man_bits < -125)
         return false;
     q->e = f.exp_bits;
     q->m = f.man_bits;

@@ -39,6 +39,101 @@ __device__ __forceinline__ uint32_t e2m1x8_from_scaled(const float (&t)[8], bool
     return mag | (v & nonzero);
 }
 
+// ---- the general rounding arithmetic, four elements at a time ---------------------------------------
+// The magic-number addition of quantize_rne_bits with everything that depends on the format alone taken
+// out of the loop and as much as possible on the floating-point pipe.  With E the power of two at or below
+// max(|a|, smallest normal of the format), C = E * 1.5 * 2^(23-m) is 1.5 * 2^23 steps of the element's
+// binade, the FP32 sum |a| + C is a whole number of steps (rounded as the add's rounding mode says) and
+// (bits(E) >> sh) + (bits(sum) - bits(C)) - c2 is the code.  These forms assume finite inputs: the caller
+// looks for NaN and infinity once per thread item and falls back on the element-wise functions.
+struct WordConsts {
+    float cmax, lo, kmul;
+    uint32_t c2, code_max, mag4, sign4, pow_m;
+    int sh, sign_down, sign_shift;
+};
+__device__ __forceinline__ WordConsts word_consts(const QFormat& f)
+{
+    WordConsts c;
+    c.cmax = __uint_as_float(f.cmax_bits);
+    c.lo = __uint_as_float((uint32_t)(128 - f.B) << 23);
+    c.kmul = __uint_as_float(((uint32_t)(127 + 23 - f.m) << 23) | 0x400000u);
+    c.c2 = (uint32_t)(128 - f.B) << f.m;
+    c.code_max = (uint32_t)f.code_max;
+    c.sign4 = 0x01010101u << f.sign_shift;
+    c.mag4 = c.sign4 - 0x01010101u;
+    c.pow_m = 1u << f.m;
+    c.sh = 23 - f.m;
+    c.sign_down = 7 - f.sign_shift;
+    c.sign_shift = f.sign_shift;
+    return c;
+}
+
+// the sign bits of four floats at bit `sign_shift` of the four bytes of a word
+__device__ __forceinline__ uint32_t signs4(uint32_t u0, uint32_t u1, uint32_t u2, uint32_t u3, const WordConsts& c)
+{
+    const uint32_t t01 = __byte_perm(u0, u1, 0x0073), t23 = __byte_perm(u2, u3, 0x0073);
+    return (__byte_perm(t01, t23, 0x5410) & 0x80808080u) >> c.sign_down;
+}
+
+// Round to nearest even: four byte codes in one word (sign included; a zero magnitude has no sign).  The clipping
+// value is the largest code's value, so no code can come out above it.
+__device__ __forceinline__ uint32_t rne_word(float t0, float t1, float t2, float t3, const WordConsts& c)
+{
+    const float t[4] = {t0, t1, t2, t3};
+    uint32_t w = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float a = fminf(fabsf(t[j]), c.cmax);
+        const uint32_t ebits = __float_as_uint(fmaxf(a, c.lo)) & 0x7f800000u;
+        const float C = __fmul_rn(__uint_as_float(ebits), c.kmul);
+        const uint32_t k = __float_as_uint(__fadd_rn(a, C)) - __float_as_uint(C);
+        w |= ((ebits >> c.sh) + k - c.c2) << (8 * j);
+    }
+    const uint32_t nonzero = ((w & c.mag4) + c.mag4) & c.sign4;
+    return w | (signs4(__float_as_uint(t0), __float_as_uint(t1), __float_as_uint(t2), __float_as_uint(t3), c) & nonzero);
+}
+
+// Signed floor plus the learned decision h (Sec. V-B): the sum a + C rounded toward minus infinity is
+// floor(a / step) steps above C for either sign of a (a minus zero counts as zero), h is added to that whole
+// number and the magnitude is encoded.  One step above a binade's lower edge toward zero lies in the finer
+// binade below (k < 2^m in a normal binade): there the code is one less than the plain sum.
+__device__ __forceinline__ uint32_t floor_word(float t0, float t1, float t2, float t3, uint32_t h4, const WordConsts& c)
+{
+    const float t[4] = {t0, t1, t2, t3};
+    uint32_t w = 0, sg = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float a = fminf(fabsf(t[j]), c.cmax);
+        const uint32_t ebits = __float_as_uint(fmaxf(a, c.lo)) & 0x7f800000u;
+        const float C = __fmul_rn(__uint_as_float(ebits), c.kmul);
+        const int k = (int)(__float_as_uint(__fadd_rd(copysignf(a, t[j]), C)) - __float_as_uint(C)) + (int)((h4 >> j) & 1u);
+        const uint32_t kmag = (uint32_t)abs(k);
+        const uint32_t base = (ebits >> c.sh) - c.c2;          // (exponent field - 1 of the binade) << m
+        const uint32_t code = min(base + kmag - ((kmag < c.pow_m && base >= c.pow_m) ? 1u : 0u), c.code_max);
+        w |= code << (8 * j);
+        sg |= (k < 0 ? 1u : 0u) << (8 * j);
+    }
+    const uint32_t nonzero = ((w & c.mag4) + c.mag4) & c.sign4;
+    return w | ((sg << c.sign_shift) & nonzero);
+}
+
+// 0 if all sixteen values are finite (anything else otherwise): x * 0 is 0 for a finite x and NaN for the rest
+__device__ __forceinline__ float nonfinite_probe(const float (&t)[16])
+{
+    float acc = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+        acc = fmaf(t[j], 0.0f, acc);
+    return acc;
+}
+
+// four byte codes of a 4-bit format -> 16 bits of nibbles
+__device__ __forceinline__ uint32_t nibbles_of(uint32_t w)
+{
+    const uint32_t x = (w | (w >> 4)) & 0x00ff00ffu;
+    return (x | (x >> 8)) & 0xffffu;
+}
+
 // 16 scaled values -> their codes: four words of bytes, or two words of nibbles for 4-bit formats
 template <int MODE>
 __device__ __forceinline__ void encode16_rne(const float (&t)[16], const QFormat& f, uint32_t (&out)[4], bool& nan)
@@ -49,24 +144,23 @@ __device__ __forceinline__ void encode16_rne(const float (&t)[16], const QFormat
         out[0] = e2m1x8_from_scaled(lo, nan);
         out[1] = e2m1x8_from_scaled(hi, nan);
     } else {
+        const WordConsts c = word_consts(f);
+        const bool slow = MODE == Q_GENERAL && nonfinite_probe(t) != 0.0f;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             if (MODE == Q_E4M3)
                 out[j] = e4m3x4_from_scaled(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3], nan);
             else if (MODE == Q_E5M2)
                 out[j] = e5m2x4_from_scaled(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3], nan);
+            else if (!slow)
+                out[j] = rne_word(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3], c);
             else
                 out[j] = quantize_rne_bits(t[4 * j], f, nan) | (quantize_rne_bits(t[4 * j + 1], f, nan) << 8) |
                          (quantize_rne_bits(t[4 * j + 2], f, nan) << 16) | (quantize_rne_bits(t[4 * j + 3], f, nan) << 24);
         }
         if (f.four_bit) {
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const uint32_t a0 = out[2 * j], a1 = out[2 * j + 1];
-                out[j] = (a0 & 0xf) | ((a0 >> 4) & 0xf0) | ((a0 >> 8) & 0xf00) | ((a0 >> 12) & 0xf000) |
-                         ((a1 & 0xf) << 16) | (((a1 >> 4) & 0xf0) << 16) | (((a1 >> 8) & 0xf00) << 16) |
-                         (((a1 >> 12) & 0xf000) << 16);
-            }
+            out[0] = nibbles_of(out[0]) | (nibbles_of(out[1]) << 16);
+            out[1] = nibbles_of(out[2]) | (nibbles_of(out[3]) << 16);
         }
     }
 }
@@ -211,23 +305,23 @@ __global__ void __launch_bounds__(256) quantize_weight_vec_kernel(const float* _
         } else {
             // 16 decisions: the row's bytes 2 g and 2 g + 1 (K / 8 is even, so the pair is 2-byte aligned)
             const uint32_t hb = __ldg(reinterpret_cast<const uint16_t*>(rbits) + v);
-            uint32_t c[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-                c[j] = quantize_bits(t[j], f, (int)((hb >> j) & 1u), nan);
-            if (!f.four_bit) {
+            const WordConsts c = word_consts(f);
+            if (nonfinite_probe(t) == 0.0f) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
-                    out[j] = c[4 * j] | (c[4 * j + 1] << 8) | (c[4 * j + 2] << 16) | (c[4 * j + 3] << 24);
+                    out[j] = floor_word(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3], hb >> (4 * j), c);
             } else {
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    uint32_t o = 0;
+                for (int j = 0; j < 4; ++j) {
+                    out[j] = 0;
 #pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        o |= c[8 * j + q] << (4 * q);
-                    out[j] = o;
+                    for (int q = 0; q < 4; ++q)
+                        out[j] |= quantize_bits(t[4 * j + q], f, (int)((hb >> (4 * j + q)) & 1u), nan) << (8 * q);
                 }
+            }
+            if (f.four_bit) {
+                out[0] = nibbles_of(out[0]) | (nibbles_of(out[1]) << 16);
+                out[1] = nibbles_of(out[2]) | (nibbles_of(out[3]) << 16);
             }
         }
         if (!f.four_bit)

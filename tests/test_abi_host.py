@@ -39,6 +39,11 @@ def test_format_max_and_scale(L):
     assert fpq.fpq_format_max(fpq.E2M5) == 3.9375
     assert fpq.fpq_format_max(fpq.Format(5, 3, 7)) == 0.0          # 9 bits
     assert fpq.fpq_format_max(fpq.Format(4, 3, 7, 5)) == 0.0        # unknown saturation mode
+    # the documented range of exp_bias: 2^e - m - 104 <= exp_bias <= 126 - m
+    assert fpq.fpq_format_max(fpq.Format(4, 3, 16 - 3 - 104)) == 1.875 * 2.0 ** (15 + 91)
+    assert fpq.fpq_format_max(fpq.Format(4, 3, 16 - 3 - 105)) == 0.0
+    assert fpq.fpq_format_max(fpq.Format(4, 3, 123)) == 1.875 * 2.0 ** (15 - 123)
+    assert fpq.fpq_format_max(fpq.Format(4, 3, 124)) == 0.0
     import numpy as np
     assert fpq.fpq_scale_from_max(3.0, fpq.E4M3) == float(np.float32(3.0) / np.float32(448.0))
 

@@ -99,6 +99,28 @@ def test_act_quantize_sweep(f):
         assert np.array_equal(got.reshape(-1), want.reshape(-1))
 
 
+@pytest.mark.parametrize("f", [fpq.Format(4, 3, -91), fpq.Format(4, 3, 123), fpq.Format(2, 1, -101), fpq.Format(2, 1, 125),
+                               fpq.Format(1, 6, -108), fpq.Format(1, 6, 120)])
+def test_exponent_bias_at_the_ends_of_its_range(f):
+    """The smallest and largest exponent bias the library accepts: grid values next to the ends of FP32's normal
+    range, flat quantizer and weight encoder (nearest and learned), 16-per-thread kernels."""
+    of = to_oracle(f)
+    pts = _sweep(f)
+    pts = pts[np.isfinite(pts)]
+    x = np.concatenate([pts, np.zeros(-pts.size % 16, np.float32)])
+    want = O.quantize_act(x, 1.0, of)
+    got = fpq.fpq_quantize_act(torch.from_numpy(x).cuda(), 1.0, f).cpu().numpy()
+    assert np.array_equal(got.reshape(-1), want.reshape(-1))
+    w = np.stack([x, x[::-1]]).astype(np.float32)
+    sc = np.ones(2, np.float32)
+    rng = np.random.default_rng(11)
+    for rb in (None, O.pack_bits(rng.integers(0, 2, w.shape, dtype=np.uint8))):
+        got = fpq.fpq_quantize_weight(torch.from_numpy(w).cuda(), torch.from_numpy(sc).cuda(), f,
+                                      None if rb is None else torch.from_numpy(rb).cuda()).cpu().numpy()
+        assert np.array_equal(got, O.quantize_weight(w, sc, of, rb))
+    assert fpq.fpq_read_status() == fpq.OK
+
+
 def test_special_values_and_status_flag():
     assert fpq.fpq_read_status() == fpq.OK
     x = np.zeros(64, dtype=np.float32)
