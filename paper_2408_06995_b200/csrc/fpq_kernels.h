@@ -99,6 +99,17 @@ fpq_status launch_sgemm_nt(const float* P, int64_t ldp, const float* Q, int64_t 
                            int64_t J, int64_t R, cudaStream_t st);
 fpq_status launch_round_harden(const float* alpha, int64_t N, int64_t K, uint8_t* bits, cudaStream_t st);
 
+// C = P Q^T in FP32 on the tensor cores (three TF32 products per term): P [I][ldp], Q [J][ldq], reduction of
+// length R contiguous in both, cut into slices of kb_per_split 32-wide blocks.  epi 0: slice z is written to
+// C + z * split_stride, row-major [I][ldc]; epi 1 (one slice): C[j][i] (leading dimension ldc) and *sq_sum +=
+// the sum of the squared outputs.  FPQ_ERR_UNSUPPORTED (nothing enqueued) unless tf32x3_applies.
+bool tf32x3_applies(const float* P, int64_t ldp, const float* Q, int64_t ldq, int64_t I, int64_t J, int64_t R);
+fpq_status launch_tf32x3(const float* P, int64_t ldp, const float* Q, int64_t ldq, int64_t I, int64_t J, int64_t R,
+                         int kb_per_split, int epi, float* C, int64_t ldc, int64_t split_stride, double* sq_sum,
+                         cudaStream_t st);
+// XT[k][m] = X[m][k] for X [M][K] with leading dimension ldx, XT with leading dimension ldt
+cudaError_t launch_transpose(const float* X, int64_t ldx, int64_t M, int64_t K, float* XT, int64_t ldt, cudaStream_t st);
+
 // Layer on the CUDA cores for operand formats the tensor-core contraction has no type for (any valid pair):
 // activations quantized to their grid values in FP32, weight codes decoded to FP32, FP32 multiply-add
 // contraction (exact products, FP32 sums, as on the tensor cores), dequantize + bias.

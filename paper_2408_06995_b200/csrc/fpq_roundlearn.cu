@@ -381,6 +381,11 @@ struct Plan {
     int splits;             // slices of M in the second contraction
     int64_t r_per_split;
     size_t off_E, off_DQ, off_D, off_DP, off_GP, bytes;
+    // tensor-core route (K a multiple of 4): A^T and D^T with rows of Mp floats, slices of 32-wide blocks of M
+    int64_t Mp;
+    int kb_per_split_tc, splits_tc;
+    int kb_per_split1_tc, splits1_tc;       // first contraction: sliced too when it has few output tiles
+    size_t off_AT, off_DT;
 };
 
 // As many slices of a reduction of length R as still fit into one wave of two resident blocks per SM (one more
@@ -412,11 +417,42 @@ Plan make_plan(int64_t M, int64_t N, int64_t K)
     o += (size_t)round_up(N * K * 4, 256);
     p.off_D = o;
     o += (size_t)round_up(M * p.N4 * 4, 256);
+    {
+        const int64_t tiles1 = ((M + 127) / 128) * ((N + 255) / 256);       // 128 x 256 output tiles
+        const int64_t kblocks = (K + 31) / 32;
+        p.kb_per_split1_tc = (int)kblocks;
+        p.splits1_tc = 1;
+        if (tiles1 * 2 <= 148 && kblocks >= 16) {
+            int64_t per = (kblocks + 148 / tiles1 - 1) / (148 / tiles1);
+            per = per < 8 ? 8 : per;
+            p.kb_per_split1_tc = (int)per;
+            p.splits1_tc = (int)((kblocks + per - 1) / per);
+        }
+    }
     p.off_DP = o;
-    if (p.splits1 > 1)
-        o += (size_t)round_up((int64_t)p.splits1 * M * p.N4 * 4, 256);
+    {
+        const int slices = p.splits1 > p.splits1_tc ? p.splits1 : p.splits1_tc;
+        if (slices > 1)
+            o += (size_t)round_up((int64_t)slices * M * p.N4 * 4, 256);
+    }
+    // second contraction on the tensor cores: one CTA per SM, so about 148 / tiles slices of at least 4 blocks
+    p.Mp = round_up(M, 4);
+    {
+        const int64_t tiles2 = ((N + 127) / 128) * ((K + 255) / 256);       // 128 x 256 output tiles
+        const int64_t kblocks = (M + 31) / 32;
+        int64_t want = 148 / tiles2;
+        want = want < 1 ? 1 : (want > 64 ? 64 : want);
+        int64_t per = (kblocks + want - 1) / want;
+        per = per < 4 ? 4 : per;
+        p.kb_per_split_tc = (int)per;
+        p.splits_tc = (int)((kblocks + per - 1) / per);
+    }
     p.off_GP = o;
-    o += (size_t)round_up((int64_t)p.splits * N * K * 4, 256);
+    o += (size_t)round_up((int64_t)(p.splits > p.splits_tc ? p.splits : p.splits_tc) * N * K * 4, 256);
+    p.off_AT = o;
+    o += (size_t)round_up(K * p.Mp * 4, 256);
+    p.off_DT = o;
+    o += (size_t)round_up(N * p.Mp * 4, 256);
     p.bytes = o;
     return p;
 }
@@ -442,6 +478,36 @@ fpq_status launch_round_learn(const float* w, const float* scale, const QFormat&
     if (cudaMemsetAsync(loss, 0, 2 * sizeof(double), st) != cudaSuccess)
         return FPQ_ERR_CUDA;
     soft_weight_kernel<<<grid_for(N * K), 256, 0, st>>>(w, scale, f, alpha, E, DQ, loss + 1, N, K, status);
+    double inv_mn = 1.0 / ((double)M * (double)N);
+    if (tf32x3_applies(a, K, E, K, M, N, K) && M <= (1 << 21) && N <= (1 << 21) && K <= (1 << 21)) {
+        // Both contractions on the tensor cores (three TF32 products per FP32 product): D^T = (A E^T)^T is written
+        // transposed by the first one's epilogue and A^T by a transpose kernel, so that the second one, D^T A,
+        // again reduces over the contiguous index of both operands.
+        float* AT = (float*)(ws + p.off_AT);
+        float* DT = (float*)(ws + p.off_DT);
+        if (launch_transpose(a, K, M, K, AT, p.Mp, st) != cudaSuccess)
+            return FPQ_ERR_CUDA;
+        fpq_status s1;
+        if (p.splits1_tc == 1) {
+            s1 = launch_tf32x3(a, K, E, K, M, N, K, p.kb_per_split1_tc, 1, DT, p.Mp, 0, loss, st);
+        } else {
+            // few output tiles and a long reduction: slices of it, added up in a fixed order, then transposed
+            s1 = launch_tf32x3(a, K, E, K, M, N, K, p.kb_per_split1_tc, 0, DP, p.N4, M * p.N4, nullptr, st);
+            if (s1 == FPQ_OK) {
+                reduce_d_kernel<<<grid_for(M * p.N4), 256, 0, st>>>(DP, p.splits1_tc, D, M * p.N4, N, p.N4, loss);
+                if (launch_transpose(D, p.N4, M, N, DT, p.Mp, st) != cudaSuccess)
+                    return FPQ_ERR_CUDA;
+            }
+        }
+        if (s1 != FPQ_OK)
+            return s1;
+        s1 = launch_tf32x3(DT, p.Mp, AT, p.Mp, N, K, M, p.kb_per_split_tc, 0, GP, K, N * K, nullptr, st);
+        if (s1 != FPQ_OK)
+            return s1;
+        grad_finalize_kernel<<<grid_for(N * K), 256, 0, st>>>(GP, p.splits_tc, DQ, alpha, grad, loss, N * K,
+                                                              (float)(2.0 * inv_mn), inv_mn, reg, lr);
+        return cudaGetLastError() == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;
+    }
     dim3 g1((unsigned)((M + TILE - 1) / TILE), (unsigned)((N + TILE - 1) / TILE), (unsigned)p.splits1);
     if (p.splits1 == 1) {
         sgemm128<true><<<g1, 256, 0, st>>>(a, K, E, K, D, p.N4, (int)M, (int)N, K, K, loss);
@@ -451,7 +517,6 @@ fpq_status launch_round_learn(const float* w, const float* scale, const QFormat&
     }
     dim3 g2((unsigned)((N + TILE - 1) / TILE), (unsigned)((K + TILE - 1) / TILE), (unsigned)p.splits);
     sgemm128<false><<<g2, 256, 0, st>>>(D, p.N4, a, K, GP, K, (int)N, (int)K, M, p.r_per_split, nullptr);
-    double inv_mn = 1.0 / ((double)M * (double)N);
     grad_finalize_kernel<<<grid_for(N * K), 256, 0, st>>>(GP, p.splits, DQ, alpha, grad, loss, N * K,
                                                           (float)(2.0 * inv_mn), inv_mn, reg, lr);
     return cudaGetLastError() == cudaSuccess ? FPQ_OK : FPQ_ERR_CUDA;

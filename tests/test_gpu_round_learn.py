@@ -84,6 +84,24 @@ def test_round_learn_step_at_transformer_block_sizes(shape):
     _check(M, N, K, fpq.E2M1, O.E2M1, seed=5)
 
 
+def test_tensor_core_contractions_keep_fp32_accuracy():
+    """Rows of a multiple of 4 floats take the tensor cores (three TF32 products per FP32 product, the reduction
+    accumulated in chunks): the result must stay at FP32 accuracy, far inside the bounds above.  A two-product
+    split, an operand read with other than its leading TF32 bits, or one long truncating accumulation would show
+    here as errors of 1e-4 and more."""
+    for (M, N, K) in [(512, 256, 1280), (1024, 320, 5120), (300, 130, 324)]:
+        w, scale, alpha, a = _case(M, N, K, O.E2M1, 7)
+        d = "cuda"
+        grad, loss = fpq.fpq_round_learn_step(torch.from_numpy(w).to(d), torch.from_numpy(scale).to(d), fpq.E2M1,
+                                              torch.from_numpy(alpha.copy()).to(d), torch.from_numpy(a).to(d), 0.0, 0.0)
+        assert fpq.fpq_read_status() == fpq.OK
+        r = O.round_learn_step(w, scale, O.E2M1, alpha, a, 0.0)
+        assert loss.cpu().numpy()[0] == pytest.approx(r["mse"], rel=1e-5)
+        err = np.abs(grad.cpu().numpy().astype(np.float64) - r["grad"])
+        assert np.all(err <= 2e-5 * r["absum"] + 4.0 * np.spacing(np.abs(r["grad"]).astype(np.float32)).astype(np.float64) + 1e-16)
+        assert np.median(err[r["absum"] > 0] / r["absum"][r["absum"] > 0]) < 2e-6
+
+
 def test_two_calls_on_one_workspace_agree():
     w, scale, alpha, a = _case(500, 130, 72, O.E2M1, 9)
     d = "cuda"
