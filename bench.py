@@ -34,6 +34,8 @@ METRIC = "W8A8 and W4A8 quantized-layer TFLOP/s on 1 B200 and % of dense FP8/FP4
 WORKLOAD = "ddim_cifar_conv3x3_w8a8: x fp32 NCHW [64,128,32,32] SiLU(N(0,1)), w [128,128,3,3] e4m3 + rounding bits, pad 1"
 NOMINAL_FP8_TFLOPS = 4500.0
 NOMINAL_FP4_TFLOPS = 9000.0
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_TF32_TFLOPS = 1100.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
 # profiles/ (a kernel is absent here until a capture of its current form exists).
 TRAFFIC = {
@@ -548,8 +550,12 @@ def run_own(args):
                           10) * 1e-6
         fp32_peak = torch.cuda.get_device_properties(dev).multi_processor_count * 128 * 2 * \
             (clocks.get("sm_mhz") or 1965.0) * 1e6
-        side["round_learn_step_qkv_320_960_m4096"] = {"us": t * 1e6, "tflops_fp32": 4.0 * M * N * K / t / 1e12,
-                                                      "frac_of_fp32_fma_peak": 4.0 * M * N * K / t / fp32_peak}
+        tf32_peak = peaks["bf16_tflops"] * (NOMINAL_TF32_TFLOPS / NOMINAL_BF16_TFLOPS)
+        side["round_learn_step_qkv_320_960_m4096"] = {
+            "us": t * 1e6, "tflops_fp32_equivalent": 4.0 * M * N * K / t / 1e12,
+            "x_fp32_fma_peak": 4.0 * M * N * K / t / fp32_peak,
+            "frac_of_tf32_peak_3_products": 3 * 4.0 * M * N * K / t / 1e12 / tf32_peak,
+            "how": "both contractions on the tensor cores, three TF32 products per FP32 product"}
         M = 8192
         x = torch.randn((M, K), device=dev)
         y = torch.empty((M, N), device=dev)
@@ -824,11 +830,23 @@ def run_round_learn(args):
         out["rows"].append({"name": name, "M": M, "N": N, "K": K, "us": t * 1e6, "tflops": flop / t / 1e12,
                             "steps_per_s": 1.0 / t})
     clocks = sampler.stop()
-    peak = props.multi_processor_count * 128 * 2 * (clocks["sm_mhz"] or 1965.0) * 1e6
+    # Rows of a multiple of 4 floats run on the tensor cores, every FP32 product as three TF32 products: the
+    # tensor work is 3 x 4 M N K flop against the TF32 peak (the measured bf16 peak x the nominal 1.1 / 2.25).
+    # `tflops` stays the FP32-equivalent figure; the CUDA cores' own FP32 multiply-add peak is given for scale.
+    peaks = load_peaks()
+    tf32_peak = peaks["bf16_tflops"] * (NOMINAL_TF32_TFLOPS / NOMINAL_BF16_TFLOPS)
+    fma_peak = props.multi_processor_count * 128 * 2 * (clocks["sm_mhz"] or 1965.0) * 1e6 / 1e12
     for row in out["rows"]:
-        row["roofline"] = {"bound": "alu", "achieved": row["tflops"], "peak": peak / 1e12, "unit": "TFLOP/s",
-                           "frac": row["tflops"] * 1e12 / peak,
-                           "peak_source": "SM count x 128 FP32 lanes x 2 flop x sampled SM clock"}
+        on_tensor = row["K"] % 4 == 0
+        if on_tensor:
+            row["roofline"] = {"bound": "tensor", "achieved": 3.0 * row["tflops"], "peak": tf32_peak, "unit": "TFLOP/s",
+                               "frac": 3.0 * row["tflops"] / tf32_peak,
+                               "peak_source": peaks["source"] + " bf16 x 1.1/2.25 (TF32)", "traffic": None,
+                               "fp32_fma_peak_tflops": fma_peak}
+        else:
+            row["roofline"] = {"bound": "alu", "achieved": row["tflops"], "peak": fma_peak, "unit": "TFLOP/s",
+                               "frac": row["tflops"] / fma_peak,
+                               "peak_source": "SM count x 128 FP32 lanes x 2 flop x sampled SM clock"}
     out["clocks"] = clocks
     if not args.skip_cpu:
         name, M, N, K = min(shapes, key=lambda sh: sh[1] * sh[2] * sh[3])
