@@ -360,9 +360,12 @@ fpq_status fpq_search_clip_candidates(float maxabs, int32_t count, float* clip_h
  * The paper prints "+ lambda(alpha)" without saying how the per-weight terms combine or how they
  * are weighted: they are summed and the caller gives the weight `reg`.  The activations are used as
  * given (FP32, the same on both sides of the difference, as in the paper's equations).
- * Everything is computed in FP32, the precision the method is stated in: the two contractions are
- * FP32 multiply-adds (A (Wq - W)^T, which is A Wq^T - A W^T by linearity, and its transpose product
- * with A), the sums of squares and of lambda are accumulated in double.
+ * Everything is computed at FP32 accuracy, the precision the method is stated in.  The two
+ * contractions (A (Wq - W)^T, which is A Wq^T - A W^T by linearity, and its transpose product with A)
+ * run on the tensor cores when K is a multiple of 4 and `a` is 16-byte aligned: every FP32 product as
+ * the sum of three TF32 products of exact operand splits, the reduction added up in FP32 (errors of a
+ * few 1e-6 of the sum of absolute terms); otherwise they are FP32 multiply-adds on the CUDA cores.
+ * The sums of squares and of lambda are accumulated in double.
  *   w       [N][K] FP32 weights, scale [N] (as fpq_quantize_weight)
  *   fmt     weight format (any valid format; the paper learns rounding for FP4 only)
  *   alpha   [N][K] FP32, read; overwritten by alpha - lr * grad when lr != 0 (plain gradient descent)
@@ -371,7 +374,7 @@ fpq_status fpq_search_clip_candidates(float maxabs, int32_t count, float* clip_h
  *   grad    out, [N][K] FP32
  *   loss    out, 2 doubles (8-byte aligned): {mse, sum of lambda}
  *   workspace  fpq_round_learn_workspace_size(M, N, K) bytes, 256-byte aligned, contents not kept
- * One memset and four kernels on `stream`; no allocation, no host synchronisation.  A NaN weight
+ * One memset and four to seven kernels on `stream`; no allocation, no host synchronisation.  A NaN weight
  * contributes nothing and sets FPQ_ERR_NAN_INPUT in the device status.  Limits: 1 <= M < 2^31 - 128,
  * 1 <= N, K <= 65535 * 128, N * K < 2^40.  Errors: FPQ_ERR_FORMAT, FPQ_ERR_SHAPE, FPQ_ERR_NULL,
  * FPQ_ERR_ALIGN, FPQ_ERR_WORKSPACE, FPQ_ERR_CUDA.  The workspace size is 0 for shapes out of range.
