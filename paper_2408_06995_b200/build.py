@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 SO = os.path.join(HERE, "libfpq.so")
 SOURCES = ["fpq_api.cu", "fpq_quantize.cu", "fpq_gemm.cu", "fpq_pair.cu", "fpq_pair_gemm.cu", "fpq_noalloc.cu", "fpq_search.cu", "fpq_smallm.cu",
-           "fpq_roundlearn.cu", "fpq_general.cu", "fpq_tf32.cu"]
+           "fpq_roundlearn.cu", "fpq_general.cu", "fpq_tf32.cu", "fpq_tensormap.cu"]
 
 
 def _newest_source_mtime() -> float:

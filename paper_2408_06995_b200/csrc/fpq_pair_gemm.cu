@@ -17,6 +17,7 @@
 
 #include "fpq_common.cuh"
 #include "fpq_kernels.h"
+#include "fpq_tensormap.h"
 
 namespace fpq {
 
@@ -271,10 +272,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) fpq_pair_gemm_kernel(const __grid
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 // geometry and shared-memory plan; FPQ_ERR_UNSUPPORTED outside the kernel's range
 fpq_status plan_pg(const GemmProblem& p, int nsm, PGArgs& g, int* dyn_bytes)
 {
@@ -363,12 +360,9 @@ fpq_status launch_pair_gemm(const GemmProblem& p, cudaStream_t st)
     {
         std::lock_guard<std::mutex> lock(mu);
         if (!enc) {
-            void* fn = nullptr;
-            cudaDriverEntryPointQueryResult q;
-            if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
-                q != cudaDriverEntryPointSuccess)
+            enc = tensor_map_encoder();
+            if (!enc)
                 return FPQ_ERR_CUDA;
-            enc = (EncodeTiledFn)fn;
         }
         if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
             return FPQ_ERR_CUDA;

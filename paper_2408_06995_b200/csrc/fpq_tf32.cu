@@ -23,6 +23,7 @@
 
 #include "fpq_common.cuh"
 #include "fpq_kernels.h"
+#include "fpq_tensormap.h"
 
 namespace fpq {
 
@@ -304,10 +305,6 @@ __global__ void __launch_bounds__(256) transpose_kernel(const float* __restrict_
             XT[(k0 + r) * ldt + m0 + tx] = tile[tx][r];
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 // rows x R floats, row-major with leading dimension ld: boxes of box_rows rows x 32 floats, zeros outside
 bool encode_rows(EncodeTiledFn enc, CUtensorMap* tm, const float* base, int64_t rows, int64_t R, int64_t ld, int box_rows)
 {
@@ -342,12 +339,9 @@ fpq_status launch_tf32x3(const float* P, int64_t ldp, const float* Q, int64_t ld
     {
         std::lock_guard<std::mutex> lock(mu);
         if (!enc) {
-            void* fn = nullptr;
-            cudaDriverEntryPointQueryResult q;
-            if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
-                q != cudaDriverEntryPointSuccess)
+            enc = tensor_map_encoder();
+            if (!enc)
                 return FPQ_ERR_CUDA;
-            enc = (EncodeTiledFn)fn;
         }
         int dev = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
