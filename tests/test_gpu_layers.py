@@ -73,6 +73,36 @@ def test_linear_ragged_shapes(wfmt, M, K, N):
     _check_full(L, use_bias=False)
 
 
+def test_same_addresses_other_shapes():
+    """Layers of different shapes called one after the other on the same device addresses (one arena for inputs,
+    scratch and outputs, as a network's allocator would hand out): the library remembers the TMA descriptors it
+    has made per (address, shape), so a descriptor of an earlier shape at the same address must never be taken.
+    Every result must equal, bit for bit, the one computed in buffers of its own."""
+    shapes = [(300, 320, 960), (300, 960, 320), (150, 640, 960), (300, 320, 960), (256, 128, 128), (128, 128, 256)]
+    arena_x = torch.empty(1 << 20, dtype=torch.float32, device="cuda")
+    arena_y = torch.empty(1 << 20, dtype=torch.float32, device="cuda")
+    arena_w = torch.empty(4 << 20, dtype=torch.uint8, device="cuda")
+    arena_p = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    for wfmt in ("e4m3", "e2m1"):
+        gfw, _ = FMT[wfmt]
+        for j, (M, K, N) in enumerate(shapes):
+            L = I.linear_layer("t", M, K, N, wfmt, rounding=False)
+            I.draw(L, 9, 10 * j, "normal", 0.02, True, 0.01)
+            ws, xs = layer_scales(L)
+            want = gpu_layer(L, ws, xs)
+            codes = fpq.fpq_quantize_weight(torch.from_numpy(L.w.reshape(N, K)).cuda(), torch.from_numpy(ws).cuda(), gfw, None)
+            nprep = fpq.fpq_prepared_size(gfw, fpq.LINEAR, N, K)
+            prep = fpq.fpq_prepare_weight(codes, gfw, fpq.LINEAR, N, K, prepared=arena_p[:nprep])
+            x = arena_x[:M * K].view(M, K)
+            x.copy_(torch.from_numpy(L.x))
+            y = arena_y[:M * N].view(M, N)
+            nws = max(256, fpq.fpq_linear_workspace_size(M, N, K, fpq.E4M3, gfw))
+            fpq.fpq_linear(x, prep, torch.from_numpy(ws).cuda(), xs, fpq.E4M3, gfw, torch.from_numpy(L.bias).cuda(), N, y=y,
+                           workspace=arena_w[:nws])
+            assert fpq.fpq_read_status() == fpq.OK
+            assert np.array_equal(y.cpu().numpy(), want), (wfmt, M, K, N)
+
+
 # at most 8 rows: one pass over the weights on the CUDA cores instead of the tensor-core kernel
 @pytest.mark.parametrize("wfmt", ["e4m3", "e2m1"])
 @pytest.mark.parametrize("M,K,N", [(1, 128, 8), (2, 320, 1280), (3, 1000, 77), (8, 1280, 320), (8, 3072, 40), (5, 130, 1),
