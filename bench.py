@@ -561,7 +561,7 @@ def run_own(args):
         y = torch.empty((M, N), device=dev)
         for fname, f in (("e4m3", fpq.E4M3), ("e1m2_reencoded", fpq.E1M2), ("e3m4_two_terms", fpq.E3M4),
                          ("e5m2_bias16_two_terms", fpq.Format(5, 2, 16, fpq.SAT_PAPER)),
-                         ("e6m1_cuda_cores", fpq.Format(6, 1, 31, fpq.SAT_PAPER))):
+                         ("e6m1_fp32_grid_values_tf32", fpq.Format(6, 1, 31, fpq.SAT_PAPER))):
             ws = (w.abs().amax(dim=1) / fpq.fpq_format_max(f)).contiguous()
             prep = fpq.fpq_prepare_weight(fpq.fpq_quantize_weight(w, ws, f, None), f, fpq.LINEAR, N, K)
             wk = torch.empty(max(256, fpq.fpq_linear_workspace_size(M, N, K, fpq.E4M3, f)), dtype=torch.uint8, device=dev)
@@ -885,7 +885,7 @@ def run_formats(args):
                ("e2m5", fpq.E2M5, "tensor cores, weights prepared as two E4M3 terms"),
                ("e4m3_bias8", fpq.Format(4, 3, 8, fpq.SAT_PAPER), "tensor cores, weights prepared as two E4M3 terms"),
                ("e5m2_bias16", fpq.Format(5, 2, 16, fpq.SAT_PAPER), "tensor cores, weights prepared as two E5M2 terms"),
-               ("e6m1", fpq.Format(6, 1, 31, fpq.SAT_PAPER), "CUDA cores (FP32 multiply-adds)")]
+               ("e6m1", fpq.Format(6, 1, 31, fpq.SAT_PAPER), "FP32 grid values, one TF32 tensor-core product per term")]
     if args.only:
         formats = [f for f in formats if args.only in f[0]]
         if not formats:

@@ -1,12 +1,13 @@
 // Quantized layer for operand formats the tensor cores have no type for (E3M4, E2M5, E5M2, the paper's
 // E4M3 with its code for 480, or any activation format other than native E4M3).  Same arithmetic model
 // as the tensor-core path - operands are exact grid values, every product is exact in FP32 (at most
-// 7 + 7 significant bits), sums are FP32 - carried out on the CUDA cores:
+// 7 + 8 significant bits), sums are FP32 - carried out on FP32 values:
 //   quantize_values_kernel   x -> value of q(x / scale) in code units, FP32 (Sec. IV-B rounding equation)
 //   decode_prepared_kernel   prepared weight codes -> FP32 values, [N][C*R*S] in the boundary's order
 //   unfold (convolutions)    input rows written out
-//   FP32 contraction         rows x weights^T
-//   dequant_store_kernel     y = acc * (scale_x * scale_w[n]) + bias[n], row-major or NCHW
+//   contraction              rows x weights^T with y = acc * (scale_x * scale_w[n]) + bias[n] in its epilogue, on the
+//                            tensor cores (grid values are TF32 numbers: one exact product per term); rows that are
+//                            not a multiple of 4 floats: FP32 multiply-adds on the CUDA cores, then dequant_store_kernel
 #include "fpq_kernels.h"
 
 namespace fpq {
@@ -142,6 +143,17 @@ fpq_status launch_general_layer(const GeneralLayer& g, void* workspace, cudaStre
         if (s != FPQ_OK)
             return s;
         a = rows;
+    }
+    // Grid values of formats of up to 8 bits have at most 8 significant bits: they are TF32 numbers, their products
+    // are exact in FP32, and one tensor-core product per term computes what the FP32 multiply-add computes (the sums
+    // differ in the order and rounding of the FP32 additions only).  Rows that are not a multiple of 4 floats stay
+    // on the CUDA cores.  The tensor-core kernel's epilogue dequantizes and adds the bias itself.
+    if (tf32x3_applies(a, g.K, wv, g.K, g.M, g.N, g.K) && g.M <= (1 << 21) && g.N <= (1 << 21) &&
+        (int64_t)g.Ho * g.Wo < (1 << 30)) {
+        const fpq_status s = launch_tf32x3(a, g.K, wv, g.K, g.M, g.N, g.K, (int)((g.K + 31) / 32), 2, g.y, g.N, 0, nullptr, st,
+                                           1, g.w_scale, g.x_scale, g.bias, g.conv ? g.Ho * g.Wo : 0);
+        if (s != FPQ_ERR_UNSUPPORTED)
+            return s;
     }
     fpq_status s = launch_sgemm_nt(a, g.K, wv, g.K, acc, p.N4, g.M, g.N, g.K, st);
     if (s != FPQ_OK)

@@ -102,11 +102,14 @@ fpq_status launch_round_harden(const float* alpha, int64_t N, int64_t K, uint8_t
 // C = P Q^T in FP32 on the tensor cores (three TF32 products per term): P [I][ldp], Q [J][ldq], reduction of
 // length R contiguous in both, cut into slices of kb_per_split 32-wide blocks.  epi 0: slice z is written to
 // C + z * split_stride, row-major [I][ldc]; epi 1 (one slice): C[j][i] (leading dimension ldc) and *sq_sum +=
-// the sum of the squared outputs.  FPQ_ERR_UNSUPPORTED (nothing enqueued) unless tf32x3_applies.
+// the sum of the squared outputs.  passes = 1: the operands hold TF32 numbers (at most 11 significant bits) and one
+// product per term is exact.  epi 2 (one slice): C is the layer's output, sum * (x_scale * w_scale[j]) + bias[j], row-major
+// [I][ldc] (howo = 0) or NCHW with i = image * howo + pixel.  FPQ_ERR_UNSUPPORTED (nothing enqueued) unless tf32x3_applies.
 bool tf32x3_applies(const float* P, int64_t ldp, const float* Q, int64_t ldq, int64_t I, int64_t J, int64_t R);
 fpq_status launch_tf32x3(const float* P, int64_t ldp, const float* Q, int64_t ldq, int64_t I, int64_t J, int64_t R,
                          int kb_per_split, int epi, float* C, int64_t ldc, int64_t split_stride, double* sq_sum,
-                         cudaStream_t st);
+                         cudaStream_t st, int passes = 3, const float* w_scale = nullptr, float x_scale = 1.0f,
+                         const float* bias = nullptr, int howo = 0);
 // XT[k][m] = X[m][k] for X [M][K] with leading dimension ldx, XT with leading dimension ldt
 cudaError_t launch_transpose(const float* X, int64_t ldx, int64_t M, int64_t K, float* XT, int64_t ldt, cudaStream_t st);
 

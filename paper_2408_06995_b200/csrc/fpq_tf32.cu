@@ -45,6 +45,13 @@ struct Tf32Args {
     int kb_per_split;          // blocks per slice (blockIdx.y)
     int tiles_j;
     int epi;                   // 0: C[z][i][j] = the slice's sum, row-major;  1: C[j][i] (transposed) and the sum of squares
+    int passes;                // 3: full FP32 products;  1: the operands are TF32 numbers already (hi * hi is all there is)
+    // epi 2: the layer's output y = sum * (x_scale * w_scale[j]) + bias[j], row-major [I][J] (howo = 0) or NCHW with
+    // i = image * howo + pixel
+    const float* w_scale;
+    const float* bias;
+    float x_scale;
+    int howo;
     float* C;
     int64_t ldc, split_stride;
     double* sq_sum;
@@ -163,9 +170,12 @@ __global__ void __launch_bounds__(T_THREADS, 1) tf32x3_gemm_kernel(const __grid_
 #pragma unroll
                 for (uint32_t kk = 0; kk < 4; ++kk) {
                     // 8 floats = 32 bytes per MMA: two 16-byte units further along the row
-                    mma_tf32(d, p_lo + 2 * kk, q_hi + 2 * kk, SMEM_DESC_HI_K_SW128, g.idesc, acc);
-                    mma_tf32(d, p_hi + 2 * kk, q_lo + 2 * kk, SMEM_DESC_HI_K_SW128, g.idesc, 1u);
-                    mma_tf32(d, p_hi + 2 * kk, q_hi + 2 * kk, SMEM_DESC_HI_K_SW128, g.idesc, 1u);
+                    if (g.passes == 3) {
+                        mma_tf32(d, p_lo + 2 * kk, q_hi + 2 * kk, SMEM_DESC_HI_K_SW128, g.idesc, acc);
+                        mma_tf32(d, p_hi + 2 * kk, q_lo + 2 * kk, SMEM_DESC_HI_K_SW128, g.idesc, 1u);
+                        acc = 1u;
+                    }
+                    mma_tf32(d, p_hi + 2 * kk, q_hi + 2 * kk, SMEM_DESC_HI_K_SW128, g.idesc, acc);
                     acc = 1u;
                 }
                 mma_commit(empty + 8 * s);          // the stage is free once these MMAs have read it
@@ -217,10 +227,12 @@ __global__ void __launch_bounds__(T_THREADS, 1) tf32x3_gemm_kernel(const __grid_
             if (!mbar_wait(full + 8 * s, ph)) { dead = true; break; }
             float4* raw = reinterpret_cast<float4*>(smem + s * T_STAGE_BYTES);
             float4* low = raw + T_RAW_BYTES / 16;
+            if (g.passes == 3) {
 #pragma unroll
-            for (int q = 0; q < T_RAW_BYTES / 16 / (32 * T_NUM_XF); ++q) {
-                const int e = q * (32 * T_NUM_XF) + tid;
-                low[e] = tail4(raw[e]);
+                for (int q = 0; q < T_RAW_BYTES / 16 / (32 * T_NUM_XF); ++q) {
+                    const int e = q * (32 * T_NUM_XF) + tid;
+                    low[e] = tail4(raw[e]);
+                }
             }
             fence_proxy_async();
             __syncwarp();
@@ -254,6 +266,35 @@ __global__ void __launch_bounds__(T_THREADS, 1) tf32x3_gemm_kernel(const __grid_
                             for (int v = 0; v < 32; ++v)
                                 if (j0 + v < g.J)
                                     dst[v] = r[v];
+                        }
+                    }
+                } else if (g.epi == 2) {
+                    if (i < g.I) {
+                        float o[32];
+#pragma unroll
+                        for (int v = 0; v < 32; ++v) {
+                            const int j = min(j0 + v, g.J - 1);
+                            o[v] = fmaf(r[v], g.x_scale * __ldg(g.w_scale + j), g.bias ? __ldg(g.bias + j) : 0.f);
+                        }
+                        if (g.howo == 0) {
+                            float* dst = g.C + (int64_t)i * g.ldc + j0;
+                            if ((g.ldc & 3) == 0 && j0 + 32 <= g.J) {
+#pragma unroll
+                                for (int v = 0; v < 8; ++v)
+                                    reinterpret_cast<float4*>(dst)[v] = make_float4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+                            } else {
+#pragma unroll
+                                for (int v = 0; v < 32; ++v)
+                                    if (j0 + v < g.J)
+                                        dst[v] = o[v];
+                            }
+                        } else {
+                            // NCHW: for one channel the 32 lanes write 32 consecutive pixels (of one image, mostly)
+                            const int b = i / g.howo, pix = i - b * g.howo;
+#pragma unroll
+                            for (int v = 0; v < 32; ++v)
+                                if (j0 + v < g.J)
+                                    g.C[((int64_t)b * g.J + j0 + v) * g.howo + pix] = o[v];
                         }
                     }
                 } else {
@@ -329,12 +370,12 @@ bool tf32x3_applies(const float* P, int64_t ldp, const float* Q, int64_t ldq, in
 // dimension ldc; epi 1 (splits must be 1): C[j][i] with leading dimension ldc, and *sq_sum += sum of squares.
 fpq_status launch_tf32x3(const float* P, int64_t ldp, const float* Q, int64_t ldq, int64_t I, int64_t J, int64_t R,
                          int kb_per_split, int epi, float* C, int64_t ldc, int64_t split_stride, double* sq_sum,
-                         cudaStream_t st)
+                         cudaStream_t st, int passes, const float* w_scale, float x_scale, const float* bias, int howo)
 {
     static std::mutex mu;
     static EncodeTiledFn enc = nullptr;
     static bool attr_set[64] = {};
-    if (!tf32x3_applies(P, ldp, Q, ldq, I, J, R) || kb_per_split < 1)
+    if (!tf32x3_applies(P, ldp, Q, ldq, I, J, R) || kb_per_split < 1 || (passes != 1 && passes != 3))
         return FPQ_ERR_UNSUPPORTED;
     {
         std::lock_guard<std::mutex> lock(mu);
@@ -362,6 +403,11 @@ fpq_status launch_tf32x3(const float* P, int64_t ldp, const float* Q, int64_t ld
     g.kb_per_split = kb_per_split;
     g.tiles_j = (int)((J + TN - 1) / TN);
     g.epi = epi;
+    g.passes = passes;
+    g.w_scale = w_scale;
+    g.x_scale = x_scale;
+    g.bias = bias;
+    g.howo = howo;
     g.C = C;
     g.ldc = ldc;
     g.split_stride = split_stride;
@@ -372,7 +418,7 @@ fpq_status launch_tf32x3(const float* P, int64_t ldp, const float* Q, int64_t ld
     // kind::tf32: FP32 accumulator, TF32 (format 2) on both sides, K-major, N = 256, M = 128
     g.idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
     const int splits = (g.kblocks + kb_per_split - 1) / kb_per_split;
-    if (epi == 1 && splits != 1)
+    if ((epi == 1 || epi == 2) && splits != 1)
         return FPQ_ERR_UNSUPPORTED;
     const int64_t tiles = ((I + TM - 1) / TM) * (int64_t)g.tiles_j;
     if (tiles > 0x7fffffff || splits > 65535)
