@@ -908,6 +908,22 @@ def run_formats(args):
             t = per_launch_us(torch, lambda: fpq.fpq_linear(x, prep, ws, xs, fpq.E4M3, f, bias, N, y, wk), 10) * 1e-6
             rows.append({"name": name, "weights": fname, "route": route, "M": M, "N": N, "K": K, "us": t * 1e6,
                          "tflops": 2.0 * M * N * K / t / 1e12, "weight_bytes": prep.numel()})
+        if args.only:
+            continue
+        # the activation encodings of the search (Sec. V-A) against E4M3 / E2M1 weights
+        for aname, fa, fwt, route in (("e4m3", fpq.E4M3, fpq.E2M1, "tensor cores"), ("e5m2_ocp", fpq.E5M2, fpq.E2M1, "tensor cores"),
+                                      ("e3m4", fpq.E3M4, fpq.E4M3, "tensor cores, activations as two E4M3 terms"),
+                                      ("e2m5", fpq.E2M5, fpq.E2M1, "tensor cores, activations as two E4M3 terms"),
+                                      ("e4m3_all_finite", fpq.Format(4, 3, 7, fpq.SAT_PAPER), fpq.E2M1,
+                                       "tensor cores, activations as two E4M3 terms"),
+                                      ("e3m4", fpq.E3M4, fpq.E3M4, "FP32 grid values, one TF32 tensor-core product per term")):
+            ws = (w.abs().amax(dim=1) / fpq.fpq_format_max(fwt)).contiguous()
+            prep = fpq.fpq_prepare_weight(fpq.fpq_quantize_weight(w, ws, fwt, None), fwt, fpq.LINEAR, N, K)
+            xsa = float(x.abs().max()) / fpq.fpq_format_max(fa)
+            wk = torch.empty(max(256, fpq.fpq_linear_workspace_size(M, N, K, fa, fwt)), dtype=torch.uint8, device=dev)
+            t = per_launch_us(torch, lambda: fpq.fpq_linear(x, prep, ws, xsa, fa, fwt, bias, N, y, wk), 10) * 1e-6
+            rows.append({"name": name, "activations": aname, "weights": "e4m3" if fwt is fpq.E4M3 else ("e2m1" if fwt is fpq.E2M1 else "e3m4"),
+                         "route": route, "M": M, "N": N, "K": K, "us": t * 1e6, "tflops": 2.0 * M * N * K / t / 1e12})
     clocks = sampler.stop()
     fp32_peak = props.multi_processor_count * 128 * 2 * (clocks["sm_mhz"] or 1965.0) * 1e6
     for r in rows:

@@ -140,7 +140,7 @@ fpq_status fpq_quantize_act(const float* x, int64_t n, float scale, fpq_format f
  * fpq_conv2d then contract over twice the reduction length on the tensor cores - exact products,
  * FP32 sums, as for one term.  The paper's E5M2 (bias 16, all exponent fields finite) is prepared
  * the same way as two terms of the tensor cores' own E5M2.  Every other format (beyond two such
- * terms, e.g. 6 exponent bits) is copied unchanged and runs on the CUDA cores.
+ * terms, e.g. 6 exponent bits) is copied unchanged and takes the FP32 grid-value route of the layer calls.
  */
 size_t fpq_prepared_size(fpq_format fmt, const fpq_layer_desc* d);
 fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_layer_desc* d,
@@ -158,10 +158,17 @@ fpq_status fpq_prepare_weight(const uint8_t* codes, fpq_format fmt, const fpq_la
  * fx = E5M2 bias 15 FPQ_SAT_NATIVE (the two 8-bit types the tensor cores read; Sec. V-A searches the
  * activation encodings too) with
  * fw = E4M3 bias 7 FPQ_SAT_NATIVE, fw = E5M2 bias 15 FPQ_SAT_NATIVE, fw = E2M1 bias 1, or any fw that fpq_prepare_weight
- * re-encodes exactly into one or two terms of those types (see there) run on the tensor cores.  Every other valid pair (any fx, any fw) runs on the CUDA
- * cores: activations quantized to their grid values in FP32, weights decoded to FP32, an FP32 multiply-add
- * contraction - the same arithmetic model (exact products, FP32 sums) at roughly a tenth of the speed; the
- * workspace is then FP32 scratch (fpq_linear_workspace_size says how much) and must be 256-byte aligned.
+ * re-encodes exactly into one or two terms of those types (see there) run on the tensor cores.  An activation
+ * format fx whose every value is one value or the sum of two values of such a type (the same classification:
+ * E3M4 bias 4, E2M5 bias 2, E4M3 with all exponent fields finite, the small formats inside E4M3) with a weight
+ * format that is read directly or re-encoded into one term runs there too: the activations are quantized with the
+ * general arithmetic, written as [first terms | second terms], and contracted over twice the reduction length
+ * against the weights repeated (a copy in the workspace, which must then be 256-byte aligned).  Every other valid
+ * pair (any fx, any fw) works on FP32 grid values: activations quantized to their grid values in FP32, weights
+ * decoded to FP32, one FP32 contraction (on the tensor cores as exact TF32 products when K is a multiple of 4,
+ * else FP32 multiply-adds on the CUDA cores) - the same arithmetic model (exact products, FP32 sums) at roughly a
+ * third of the speed; the workspace is then FP32 scratch (fpq_linear_workspace_size says how much) and must be
+ * 256-byte aligned.
  * This holds for fpq_linear and fpq_conv2d and their host-buffer forms (and for fpq_linear_static as far as
  * its fixed scratch reaches: FPQ_ERR_WORKSPACE beyond); the staged (quantize_input / contract) and two-tensor
  * forms take only the pairs the tensor cores read directly or after the one-term re-encode, and return
@@ -435,7 +442,8 @@ int32_t fpq_get_path_policy(void);
  *   FPQ_ROUTE_TWO_KERNELS  activation-quantize kernel, then the contraction kernel;
  *   FPQ_ROUTE_FUSED        the general one-kernel form;
  *   FPQ_ROUTE_PAIR_FUSED   the one-kernel form on CTA pairs with resident weights;
- *   FPQ_ROUTE_OTHER        formats the tensor cores have no type for (CUDA cores), or two-term weights;
+ *   FPQ_ROUTE_OTHER        operand formats that are not read as they are: weights or activations as one or two
+ *                          terms of a tensor-core type, or the FP32 grid-value route;
  *   negative               the error fpq_conv2d would return for these arguments.
  */
 enum { FPQ_ROUTE_TWO_KERNELS = 0, FPQ_ROUTE_FUSED = 1, FPQ_ROUTE_PAIR_FUSED = 2, FPQ_ROUTE_OTHER = 3 };

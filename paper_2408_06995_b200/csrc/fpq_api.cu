@@ -237,10 +237,30 @@ static bool weight_two_term(fpq_format f) { return classify_weight(f).kind == W_
 
 // Operand pairs the tensor-core contraction has no type for run on the CUDA cores (fpq_linear and fpq_conv2d
 // only; the staged, host-buffer, two-tensor and built-in-scratch forms keep to the tensor-core pairs).
+// Activations of a format whose every value is one value (terms = 1) or the sum of two values (terms = 2) of a
+// tensor-core type - the classification the weights use: E3M4, E2M5, the paper's all-finite E4M3 as two E4M3
+// terms, the small formats inside E4M3 as one - against weights the tensor cores read as they are (or re-encoded):
+// fpq_linear and fpq_conv2d quantize with the general arithmetic, write the terms as operand codes
+// [first terms | second terms] and run the ordinary contraction over that against the weights repeated.
+static bool act_terms_pair(fpq_format fx, fpq_format fw, int* terms)
+{
+    QFormat q;
+    if (!resolve_format(fx, &q) || !resolve_format(fw, &q) || act_native(fx))
+        return false;
+    const WeightClass& c = classify_weight(fx);
+    if (c.kind != W_ONE_TERM && c.kind != W_TWO_TERM)
+        return false;
+    if (terms)
+        *terms = c.kind == W_TWO_TERM ? 2 : 1;
+    return weight_native(fw) || weight_reencoded(fw);
+}
+
 static bool general_pair(fpq_format fx, fpq_format fw)
 {
     QFormat q;
     if (!resolve_format(fx, &q) || !resolve_format(fw, &q))
+        return false;
+    if (act_terms_pair(fx, fw, nullptr))
         return false;
     return !(act_native(fx) && (weight_native(fw) || weight_reencoded(fw) || weight_two_term(fw)));
 }
@@ -272,6 +292,27 @@ static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 static bool bad_scale(float s) { return !(s > 0.f) || std::isinf(s); }
 
 static int64_t padded_c(int64_t C) { return round_up(C, 128); }
+
+// Scratch of the term-activation route: the operand codes [units][terms * Cp] (units = rows or framed pixels), then,
+// with two terms, the prepared weights with every (output, tap) row written twice side by side.
+struct TermsPlan {
+    int terms;
+    int64_t Cp;
+    size_t codes_bytes, w_off, w_row_bytes, bytes;
+};
+static TermsPlan terms_plan(fpq_format fx, fpq_format fw, int64_t units, int64_t C, int64_t w_rows)
+{
+    TermsPlan t = {};
+    act_terms_pair(fx, fw, &t.terms);
+    QFormat q;
+    resolve_format(fw, &q);
+    t.Cp = padded_c(C);
+    t.codes_bytes = (size_t)units * t.terms * t.Cp;
+    t.w_row_bytes = (size_t)((q.four_bit && !weight_reencoded(fw)) ? t.Cp / 2 : t.Cp);
+    t.w_off = (size_t)round_up((int64_t)t.codes_bytes, 256);
+    t.bytes = t.terms == 2 ? t.w_off + (size_t)w_rows * 2 * t.w_row_bytes : t.codes_bytes;
+    return t;
+}
 
 static fpq_status check_pair(fpq_format fx, fpq_format fw)
 {
@@ -411,6 +452,9 @@ size_t fpq_linear_workspace_size(int64_t M, int64_t N, int64_t K, fpq_format fx,
     }
     if (two_term_pair(fx, fw))
         return (M < 0 || K < 0 || K > 0x3fffffff) ? 0 : (size_t)(M * 2 * padded_c(K));
+    if (act_terms_pair(fx, fw, nullptr))
+        return (M < 0 || N < 0 || K < 1 || M > 0x7fffffff || N > 0x7fffffff || K > 0x3fffffff) ? 0
+                                                                                              : terms_plan(fx, fw, M, K, N).bytes;
     (void)N;
     if (check_pair(fx, fw) != FPQ_OK || M < 0 || K < 0)
         return 0;
@@ -537,6 +581,40 @@ fpq_status fpq_linear(const float* x, const void* w_prepared, const float* w_sca
             return FPQ_ERR_WORKSPACE;
         return launch_general_layer(g, workspace, (cudaStream_t)stream);
     }
+    if (act_terms_pair(fx, fw, nullptr)) {
+        if (M < 0 || N < 0 || K < 0 || M > 0x7fffffff || N > 0x7fffffff || K > 0x3fffffff)
+            return FPQ_ERR_SHAPE;
+        if (M == 0 || N == 0)
+            return FPQ_OK;
+        if (K == 0)
+            return FPQ_ERR_SHAPE;
+        if (!x || !w_prepared || !w_scale || !y)
+            return FPQ_ERR_NULL;
+        if (!aligned(x, 16) || !aligned(y, 16) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
+            (bias && !aligned(bias, 4)) || !aligned(workspace, 256))
+            return FPQ_ERR_ALIGN;
+        const TermsPlan t = terms_plan(fx, fw, M, K, N);
+        if (!workspace || ws_bytes < t.bytes)
+            return FPQ_ERR_WORKSPACE;
+        if (!status_word())
+            return FPQ_ERR_CUDA;
+        const WeightClass& cx = classify_weight(fx);
+        const fpq_format term = cx.e5m2 ? kE5M2Native : kE4M3Native;
+        QFormat qx;
+        resolve_format(fx, &qx);
+        cudaStream_t st = (cudaStream_t)stream;
+        const void* wp = w_prepared;
+        if (t.terms == 2) {
+            if (launch_repeat_rows(w_prepared, N, (int64_t)t.w_row_bytes, (uint8_t*)workspace + t.w_off, st) != cudaSuccess)
+                return FPQ_ERR_CUDA;
+            wp = (const uint8_t*)workspace + t.w_off;
+        }
+        if (launch_quantize_rows_terms(x, M, K, t.Cp, x_scale, qx, cx.t1, t.terms == 2 ? &cx.t2 : nullptr,
+                                       (uint8_t*)workspace, st) != cudaSuccess)
+            return FPQ_ERR_CUDA;
+        return linear_contract_impl(workspace, ws_bytes, wp, w_scale, x_scale * ldexpf(1.0f, -cx.shift), term, fw, bias, y, M,
+                                    N, t.terms * t.Cp, stream, 1, nullptr);
+    }
     if (two_term_pair(fx, fw)) {
         // weights prepared as two E4M3 terms: activation codes written twice per row, then the ordinary
         // contraction over twice the (padded) reduction length
@@ -646,6 +724,11 @@ size_t fpq_conv2d_workspace_size(int B, int C, int H, int W, int C_out, int R, i
         if (conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo) != FPQ_OK)
             return 0;
         return (size_t)B * (H + 2 * pad) * (W + 2 * pad) * (size_t)(2 * padded_c(C));
+    }
+    if (act_terms_pair(fx, fw, nullptr)) {
+        if (conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo) != FPQ_OK || C > 0x3fffffff / 2)
+            return 0;
+        return terms_plan(fx, fw, (int64_t)B * (H + 2 * pad) * (W + 2 * pad), C, (int64_t)C_out * R * S).bytes;
     }
     if (check_pair(fx, fw) != FPQ_OK || conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho, &Wo) != FPQ_OK)
         return 0;
@@ -790,6 +873,48 @@ fpq_status fpq_conv2d(const float* x, const void* w_prepared, const float* w_sca
         if (!workspace || ws_bytes < general_layer_workspace_bytes(g))
             return FPQ_ERR_WORKSPACE;
         return launch_general_layer(g, workspace, (cudaStream_t)stream);
+    }
+    if (act_terms_pair(fx, fw, nullptr)) {
+        // activations as one or two terms of a tensor-core type: term codes in the framed channels-last scratch
+        // ([first terms | second terms] per pixel), the weights' rows repeated behind it, then the ordinary
+        // convolution over terms * (padded C) channels
+        if (C < 1 || C > 0x3fffffff / 2)
+            return FPQ_ERR_SHAPE;
+        int Ho3, Wo3;
+        fpq_status s3 = conv_shape(B, C, H, W, C_out, R, S, pad, stride, &Ho3, &Wo3);
+        if (s3 != FPQ_OK)
+            return s3;
+        if (B == 0 || C_out == 0)
+            return FPQ_OK;
+        if (B > 65535)
+            return FPQ_ERR_SHAPE;
+        if (!x || !w_prepared || !w_scale || !y)
+            return FPQ_ERR_NULL;
+        if (!aligned(x, 4) || !aligned(y, 4) || !aligned(w_prepared, 128) || !aligned(w_scale, 4) ||
+            (bias && !aligned(bias, 4)) || !aligned(workspace, 256))
+            return FPQ_ERR_ALIGN;
+        const TermsPlan t = terms_plan(fx, fw, (int64_t)B * (H + 2 * pad) * (W + 2 * pad), C, (int64_t)C_out * R * S);
+        if (!workspace || ws_bytes < t.bytes)
+            return FPQ_ERR_WORKSPACE;
+        if (!status_word())
+            return FPQ_ERR_CUDA;
+        const WeightClass& cx = classify_weight(fx);
+        const fpq_format term = cx.e5m2 ? kE5M2Native : kE4M3Native;
+        QFormat qx;
+        resolve_format(fx, &qx);
+        cudaStream_t st = (cudaStream_t)stream;
+        const void* wp = w_prepared;
+        if (t.terms == 2) {
+            if (launch_repeat_rows(w_prepared, (int64_t)C_out * R * S, (int64_t)t.w_row_bytes, (uint8_t*)workspace + t.w_off,
+                                   st) != cudaSuccess)
+                return FPQ_ERR_CUDA;
+            wp = (const uint8_t*)workspace + t.w_off;
+        }
+        if (launch_quantize_nchw_to_nhwc_terms(x, B, C, H, W, pad, (int)t.Cp, x_scale, qx, cx.t1,
+                                               t.terms == 2 ? &cx.t2 : nullptr, (uint8_t*)workspace, st) != cudaSuccess)
+            return FPQ_ERR_CUDA;
+        return conv2d_contract_impl(workspace, ws_bytes, wp, w_scale, x_scale * ldexpf(1.0f, -cx.shift), term, fw, bias, y, B,
+                                    (int)(t.terms * t.Cp), H, W, C_out, R, S, pad, stride, stream, 1, nullptr);
     }
     if (two_term_pair(fx, fw)) {
         // weights prepared as two E4M3 terms per tap: the activation codes fill two channel ranges of the
@@ -1242,7 +1367,7 @@ fpq_status fpq_round_learn_harden(const float* alpha, int64_t N, int64_t K, uint
 int32_t fpq_conv2d_route(int B, int C, int H, int W, int C_out, int R, int S, int pad, int stride, fpq_format fx,
                          fpq_format fw)
 {
-    if (general_pair(fx, fw) || two_term_pair(fx, fw)) {
+    if (general_pair(fx, fw) || two_term_pair(fx, fw) || act_terms_pair(fx, fw, nullptr)) {
         QFormat q;
         if (!resolve_format(fx, &q) || !resolve_format(fw, &q))
             return FPQ_ERR_FORMAT;

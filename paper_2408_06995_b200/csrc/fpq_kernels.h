@@ -26,6 +26,15 @@ struct CodeTable {
 // well: Cp counts two halves per row, the first filled through table, the second through table2.
 cudaError_t launch_prepare_weight(const uint8_t* codes, int N, int C, int RS, int Cp, int four_bit, int C1, int C1p,
                                   const CodeTable* table, const CodeTable* table2, uint8_t* prepared, cudaStream_t st);
+// Activations of a format that is one term or the sum of two terms of a tensor-core type: general quantizer, then
+// the tables (t2 == NULL: one term).  Rows / pixels hold [first terms | second terms], Kp (Cp) positions each.
+cudaError_t launch_quantize_rows_terms(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, const QFormat& f,
+                                       const CodeTable& t1, const CodeTable* t2, uint8_t* codes, cudaStream_t st);
+cudaError_t launch_quantize_nchw_to_nhwc_terms(const float* x, int B, int C, int H, int W, int pad, int Cp, float scale,
+                                               const QFormat& f, const CodeTable& t1, const CodeTable* t2, uint8_t* codes,
+                                               cudaStream_t st);
+// every row of src [rows][row_bytes] (row_bytes a multiple of 16) twice side by side in dst [rows][2 * row_bytes]
+cudaError_t launch_repeat_rows(const void* src, int64_t rows, int64_t row_bytes, void* dst, cudaStream_t st);
 cudaError_t launch_quantize_rows_e4m3_twice(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, uint8_t* codes,
                                             cudaStream_t st, int e5m2 = 0);
 

@@ -635,6 +635,219 @@ cudaError_t launch_quantize_nchw_to_nhwc_e4m3(const float* x, int B, int C, int 
 }
 
 // ---------------------------------------------------------------------------------
+// Activations in a format the tensor cores have no type for, whose every value is one value or the sum of two
+// values of a tensor-core type (tables: code of the format -> code of each term; the same classification as for
+// weights): quantize with the general arithmetic, look the terms up, and write them as operand codes.  TERMS = 2:
+// every row (pixel) holds [first terms | second terms], Kp (Cp) positions each, and the contraction runs over
+// twice the padded reduction length against the weights repeated.
+// ---------------------------------------------------------------------------------
+// 16 scaled values -> 16 codes of any format, one per byte (4-bit formats too), four per word
+__device__ __forceinline__ void codes16_bytes(const float (&t)[16], const QFormat& f, uint32_t (&w)[4], bool& nan)
+{
+    if (nonfinite_probe(t) == 0.0f) {
+        const WordConsts c = word_consts(f);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            w[j] = rne_word(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3], c);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            w[j] = quantize_rne_bits(t[4 * j], f, nan) | (quantize_rne_bits(t[4 * j + 1], f, nan) << 8) |
+                   (quantize_rne_bits(t[4 * j + 2], f, nan) << 16) | (quantize_rne_bits(t[4 * j + 3], f, nan) << 24);
+    }
+}
+
+// the same four positions of a table-mapped word
+__device__ __forceinline__ uint32_t map4(uint32_t w, const uint8_t* tab)
+{
+    return (uint32_t)tab[w & 0xffu] | ((uint32_t)tab[(w >> 8) & 0xffu] << 8) | ((uint32_t)tab[(w >> 16) & 0xffu] << 16) |
+           ((uint32_t)tab[w >> 24] << 24);
+}
+
+template <int TERMS>
+__global__ void __launch_bounds__(256) quantize_rows_terms_kernel(const float* __restrict__ x, int64_t M, int64_t K,
+                                                                  int64_t Kp, float rinv, QFormat f, CodeTable tab1,
+                                                                  CodeTable tab2, uint8_t* __restrict__ codes, int* status)
+{
+    __shared__ uint8_t s1[256], s2[256];
+    s1[threadIdx.x] = tab1.t[threadIdx.x];
+    s2[threadIdx.x] = tab2.t[threadIdx.x];
+    __syncthreads();
+    asm volatile("griddepcontrol.launch_dependents;");
+    bool nan = false;
+    const int64_t vec_per_row = Kp / 16;
+    const int64_t total = M * vec_per_row;
+    const bool aligned = (K % 4) == 0;
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < total; v += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = v / vec_per_row, k0 = (v - row * vec_per_row) * 16;
+        const float* px = x + row * K + k0;
+        float t[16];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+            const int64_t k = k0 + 4 * j;
+            if (aligned && k + 4 <= K) {
+                const float4 q = __ldg(reinterpret_cast<const float4*>(px + 4 * j));
+                a0 = q.x; a1 = q.y; a2 = q.z; a3 = q.w;
+            } else {
+                if (k + 0 < K) a0 = __ldg(px + 4 * j + 0);
+                if (k + 1 < K) a1 = __ldg(px + 4 * j + 1);
+                if (k + 2 < K) a2 = __ldg(px + 4 * j + 2);
+                if (k + 3 < K) a3 = __ldg(px + 4 * j + 3);
+            }
+            t[4 * j] = __fmul_rn(a0, rinv);
+            t[4 * j + 1] = __fmul_rn(a1, rinv);
+            t[4 * j + 2] = __fmul_rn(a2, rinv);
+            t[4 * j + 3] = __fmul_rn(a3, rinv);
+        }
+        // (positions past K hold 0.0: code 0, and every table maps code 0 to 0)
+        uint32_t w[4], o1[4], o2[4];
+        codes16_bytes(t, f, w, nan);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            o1[j] = map4(w[j], s1);
+            o2[j] = TERMS == 2 ? map4(w[j], s2) : 0u;
+        }
+        uint4* dst = reinterpret_cast<uint4*>(codes + row * (TERMS * Kp) + k0);
+        dst[0] = make_uint4(o1[0], o1[1], o1[2], o1[3]);
+        if (TERMS == 2)
+            dst[Kp / 16] = make_uint4(o2[0], o2[1], o2[2], o2[3]);
+    }
+    if (nan)
+        flag_status(status, FPQ_ERR_NAN_INPUT);
+}
+
+// NCHW FP32 -> zero-framed channels-last term codes [B][Hp][Wp][TERMS * Cp] (as quantize_nchw_to_nhwc_e4m3_kernel,
+// with the conversion above)
+template <int TERMS>
+__global__ void __launch_bounds__(256) quantize_nchw_to_nhwc_terms_kernel(const float* __restrict__ x, int C, int H, int W,
+                                                                          int pad, int Cp, float rinv, QFormat f,
+                                                                          CodeTable tab1, CodeTable tab2,
+                                                                          uint8_t* __restrict__ codes, int* status)
+{
+    __shared__ __align__(16) uint8_t tile[2][32][128 + 16];
+    __shared__ uint8_t s1[256], s2[256];
+    s1[threadIdx.x] = tab1.t[threadIdx.x];
+    s2[threadIdx.x] = tab2.t[threadIdx.x];
+    __syncthreads();
+    asm volatile("griddepcontrol.launch_dependents;");
+    bool nan = false;
+    const int HW = H * W, Wp = W + 2 * pad, Hp = H + 2 * pad;
+    const int row = TERMS * Cp;
+    const int b = blockIdx.z;
+    const int c0 = blockIdx.y * 128;
+    const int p0 = blockIdx.x * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 pixels x 8 channel groups of 16
+    const float* xb = x + (int64_t)b * C * HW;
+    uint8_t* ob = codes + (int64_t)b * Hp * Wp * row;
+    const int p = p0 + tx;
+    {
+        const int cl = ty * 16;
+        float t[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q)
+            t[q] = (c0 + cl + q < C && p < HW) ? __fmul_rn(__ldg(xb + (int64_t)(c0 + cl + q) * HW + p), rinv) : 0.f;
+        uint32_t w[4], o1[4], o2[4];
+        codes16_bytes(t, f, w, nan);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            o1[j] = map4(w[j], s1);
+            o2[j] = TERMS == 2 ? map4(w[j], s2) : 0u;
+        }
+        *reinterpret_cast<uint4*>(&tile[0][tx][cl]) = make_uint4(o1[0], o1[1], o1[2], o1[3]);
+        if (TERMS == 2)
+            *reinterpret_cast<uint4*>(&tile[1][tx][cl]) = make_uint4(o2[0], o2[1], o2[2], o2[3]);
+    }
+    __syncthreads();
+    {
+        // 32 pixels x 8 chunks of 16 channels: 8 consecutive threads write one pixel's row
+        const int pl = threadIdx.x >> 3, ch = (threadIdx.x & 7) * 16;
+        const int pp = p0 + pl, c = c0 + ch;
+        if (pp < HW && c < Cp) {
+            const int yy = pp / W, xx = pp - yy * W;
+            uint8_t* dst = ob + ((int64_t)(yy + pad) * Wp + (xx + pad)) * row + c;
+            *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(&tile[0][pl][ch]);
+            if (TERMS == 2)
+                *reinterpret_cast<uint4*>(dst + Cp) = *reinterpret_cast<const uint4*>(&tile[1][pl][ch]);
+        }
+    }
+    // frame pixels of this image, shared out over the blocks of the image's pixel axis
+    if (pad > 0) {
+        const int nframe = Hp * Wp - HW;
+        const int chunks = (min(Cp - c0, 128)) / 16;
+        const int total = nframe * chunks;
+        for (int t = blockIdx.x * 256 + threadIdx.x; t < total; t += gridDim.x * 256) {
+            const int j = t / chunks, ch = (t - j * chunks) * 16;
+            int yp, xp;
+            const int top = pad * Wp;
+            if (j < top) {
+                yp = j / Wp; xp = j - yp * Wp;
+            } else if (j < 2 * top) {
+                const int k = j - top;
+                yp = H + pad + k / Wp; xp = k % Wp;
+            } else {
+                const int k = j - 2 * top;             // 2*pad frame pixels per interior row
+                yp = pad + k / (2 * pad);
+                const int e = k % (2 * pad);
+                xp = (e < pad) ? e : W + e;
+            }
+            uint8_t* dst = ob + ((int64_t)yp * Wp + xp) * row + c0 + ch;
+            *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+            if (TERMS == 2)
+                *reinterpret_cast<uint4*>(dst + Cp) = make_uint4(0, 0, 0, 0);
+        }
+    }
+    if (nan)
+        flag_status(status, FPQ_ERR_NAN_INPUT);
+}
+
+// Prepared weights [rows][row_bytes] -> [rows][2 * row_bytes] with every row written twice side by side (the
+// weights' side of a contraction over [first terms | second terms] of the activations).  16 bytes per thread.
+__global__ void __launch_bounds__(256) repeat_rows_kernel(const uint4* __restrict__ src, int64_t rows, int64_t vec_per_row,
+                                                          uint4* __restrict__ dst)
+{
+    const int64_t total = rows * vec_per_row;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / vec_per_row, c = i - r * vec_per_row;
+        const uint4 v = __ldg(src + i);
+        dst[r * 2 * vec_per_row + c] = v;
+        dst[r * 2 * vec_per_row + vec_per_row + c] = v;
+    }
+}
+
+cudaError_t launch_quantize_rows_terms(const float* x, int64_t M, int64_t K, int64_t Kp, float scale, const QFormat& f,
+                                       const CodeTable& t1, const CodeTable* t2, uint8_t* codes, cudaStream_t st)
+{
+    const int grid = grid_for(M * (Kp / 16), 256);
+    if (t2)
+        quantize_rows_terms_kernel<2><<<grid, 256, 0, st>>>(x, M, K, Kp, 1.0f / scale, f, t1, *t2, codes, status_word());
+    else
+        quantize_rows_terms_kernel<1><<<grid, 256, 0, st>>>(x, M, K, Kp, 1.0f / scale, f, t1, t1, codes, status_word());
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_nchw_to_nhwc_terms(const float* x, int B, int C, int H, int W, int pad, int Cp, float scale,
+                                               const QFormat& f, const CodeTable& t1, const CodeTable* t2, uint8_t* codes,
+                                               cudaStream_t st)
+{
+    dim3 grid((H * W + 31) / 32, (Cp + 127) / 128, B);
+    if (t2)
+        quantize_nchw_to_nhwc_terms_kernel<2><<<grid, 256, 0, st>>>(x, C, H, W, pad, Cp, 1.0f / scale, f, t1, *t2, codes,
+                                                                     status_word());
+    else
+        quantize_nchw_to_nhwc_terms_kernel<1><<<grid, 256, 0, st>>>(x, C, H, W, pad, Cp, 1.0f / scale, f, t1, t1, codes,
+                                                                     status_word());
+    return cudaGetLastError();
+}
+
+cudaError_t launch_repeat_rows(const void* src, int64_t rows, int64_t row_bytes, void* dst, cudaStream_t st)
+{
+    const int64_t vec = row_bytes / 16;
+    repeat_rows_kernel<<<grid_for(rows * vec, 256), 256, 0, st>>>((const uint4*)src, rows, vec, (uint4*)dst);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------
 // Zero census of a code tensor (the sparsity measurement): how many of the n values are the
 // code 0.  16 bytes per thread and step, one atomic per block.  *count must be 0 at the start.
 // ---------------------------------------------------------------------------------

@@ -1,7 +1,8 @@
 """Layers whose operand formats the tensor cores have no type for (E3M4, E2M5, E5M2, the paper's E4M3 with
 all exponent fields finite - what the FP8 encoding search of Sec. V-A may select - or activations in a format
-other than native E4M3): fpq_linear / fpq_conv2d run them on the CUDA cores with the same arithmetic model
-(exact products of grid values, FP32 sums), so the bar is the one of the tensor-core path."""
+other than native E4M3): fpq_linear / fpq_conv2d run them as terms of a tensor-core type where the format splits
+into one or two, else on FP32 grid values, always with the same arithmetic model (exact products of grid values, FP32
+sums), so the bar is the one of the native path."""
 import numpy as np
 import pytest
 import torch
@@ -20,12 +21,18 @@ E2M1_TINY = fpq.Format(2, 1, 12, fpq.SAT_PAPER)      # a 4-bit format whose valu
 E1M6 = fpq.Format(1, 6, 1, fpq.SAT_PAPER)            # 7 significant bits = 4 + 3: two E4M3 terms
 E6M1 = fpq.Format(6, 1, 31, fpq.SAT_PAPER)           # 64 binades: beyond any two tensor-core terms, CUDA cores
 E5M2_B40 = fpq.Format(5, 2, 40, fpq.SAT_PAPER)       # needs a factor beyond the 2^16 the split tries
+E3M2_B3 = fpq.Format(3, 2, 3, fpq.SAT_PAPER)         # 6-bit formats whose every value is an E4M3 value: one term
+E2M3_B1 = fpq.Format(2, 3, 1, fpq.SAT_PAPER)
 
 PAIRS = [(fpq.E4M3, fpq.E3M4), (fpq.E4M3, fpq.E2M5), (fpq.E4M3, fpq.E5M2), (fpq.E4M3, E5M2_B16), (fpq.E4M3, E4M3_PAPER),
          (fpq.E4M3, E4M3_B8), (fpq.E4M3, E2M1_TINY), (fpq.E4M3, E1M6), (fpq.E4M3, E6M1), (fpq.E4M3, E5M2_B40), (fpq.E3M4, E5M2_B16),
          (fpq.E5M2, fpq.E4M3), (fpq.E3M4, fpq.E2M1), (E4M3_PAPER, fpq.E1M2), (fpq.E2M5, fpq.E3M4),
          # OCP E5M2 activations are read by the tensor cores as they are, with every kind of weight preparation
-         (fpq.E5M2, fpq.E5M2), (fpq.E5M2, fpq.E2M1), (fpq.E5M2, fpq.E1M2), (fpq.E5M2, fpq.E3M4), (fpq.E5M2, E5M2_B16)]
+         (fpq.E5M2, fpq.E5M2), (fpq.E5M2, fpq.E2M1), (fpq.E5M2, fpq.E1M2), (fpq.E5M2, fpq.E3M4), (fpq.E5M2, E5M2_B16),
+         # activations that are one or two terms of a tensor-core type, against weights read as they are or re-encoded:
+         # the terms are written as operand codes and the ordinary contraction runs over them
+         (fpq.E3M4, fpq.E4M3), (fpq.E2M5, fpq.E4M3), (fpq.E2M5, fpq.E2M1), (fpq.E2M5, fpq.E5M2), (E4M3_PAPER, fpq.E4M3),
+         (E4M3_B8, fpq.E4M3), (E5M2_B16, fpq.E2M1), (E3M2_B3, fpq.E4M3), (E2M3_B1, fpq.E2M1), (E1M6, fpq.E1M2)]
 
 
 def _run(L, gfx, gfw, use_bias=True):
@@ -67,7 +74,8 @@ def test_linear(gfx, gfw, M, K, N):
 
 
 @pytest.mark.parametrize("gfx,gfw", [(fpq.E4M3, fpq.E3M4), (fpq.E4M3, E5M2_B16), (fpq.E4M3, E4M3_B8), (fpq.E5M2, fpq.E2M1),
-                                     (fpq.E3M4, fpq.E1M2), (fpq.E5M2, fpq.E4M3), (fpq.E5M2, fpq.E3M4)])
+                                     (fpq.E3M4, fpq.E1M2), (fpq.E5M2, fpq.E4M3), (fpq.E5M2, fpq.E3M4),
+                                     (fpq.E2M5, fpq.E4M3), (fpq.E3M4, fpq.E2M1), (E3M2_B3, fpq.E4M3), (E5M2_B16, fpq.E4M3)])
 @pytest.mark.parametrize("shape", [(2, 40, 12, 12, 72, 3, 1), (1, 130, 9, 11, 33, 3, 2), (3, 64, 8, 8, 130, 1, 1)])
 def test_conv(gfx, gfw, shape):
     B, C, H, W, Co, R, stride = shape
@@ -87,6 +95,28 @@ def test_e5m2_activations_at_a_size_that_spans_many_tiles():
     # the scratch is one byte per activation: the tensor-core route, not the FP32 scratch of the CUDA-core route
     assert fpq.fpq_linear_workspace_size(1000, 960, 320, fpq.E5M2, fpq.E4M3) == 1000 * 320
     assert fpq.fpq_linear_workspace_size(1000, 960, 320, fpq.E3M4, fpq.E4M3) > 4 * 1000 * 320
+
+
+@pytest.mark.parametrize("gfx", [fpq.E3M4, fpq.E2M5])
+def test_two_term_activations_at_a_size_that_spans_many_tiles(gfx):
+    # the FP8 activation encodings of the search that the tensor cores have no type for, as two E4M3 terms:
+    # several tiles per CTA, a ragged tail, both weight widths; and a convolution with a split reduction
+    L = I.linear_layer("t", 1000, 320, 960, "e4m3")
+    I.draw(L, 36, 1, "normal", 0.02, True, 0.01, (0.001, 20.0))
+    _run(L, gfx, fpq.E4M3)
+    _run(L, gfx, fpq.E2M1)
+    L = I.conv_layer("t", 2, 320, 16, 16, 320, 3)
+    I.draw(L, 36, 2, "silu", 0.03, True, 0.01)
+    _run(L, gfx, fpq.E2M1)
+
+
+def test_four_bit_activation_format_as_one_term():
+    # E1M2 activations (every value an E4M3 value): the oracle's layer reads 4-bit activation codes packed per row,
+    # which equals the flat packing of its quantizer for even row lengths only
+    L = I.linear_layer("t", 130, 200, 72)
+    I.draw(L, 37, 1, "normal", 0.02, True, 0.01, (0.001, 20.0))
+    _run(L, fpq.E1M2, fpq.E4M3)
+    _run(L, fpq.E1M2, fpq.E2M1)
 
 
 def test_every_fp8_search_candidate_runs_as_a_layer():
