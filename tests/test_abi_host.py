@@ -114,7 +114,15 @@ def test_search_host_side(L):
 def test_sizes(L):
     assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E4M3, fpq.E4M3) == 100 * 320
     assert fpq.fpq_linear_workspace_size(100, 64, 321, fpq.E4M3, fpq.E2M1) == 100 * 336
-    assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E3M4, fpq.E4M3) > 100 * 320     # CUDA-core route: FP32 scratch
+    # E3M4 activations as two E4M3 terms: codes [100][2 * 384], then the weights' rows repeated [64][2 * 384]
+    assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E3M4, fpq.E4M3) == 100 * 768 + 64 * 768
+    assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E3M4, fpq.E2M1) == 100 * 768 + 64 * 384      # packed FP4 weights
+    # a 6-bit format inside E4M3: one term, no copy of the weights
+    assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.Format(3, 2, 3), fpq.E4M3) == 100 * 384
+    # term activations against two-term weights, or activations beyond two terms: FP32 scratch of the grid-value route
+    assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E3M4, fpq.E3M4) > 4 * 100 * 320
+    assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.Format(6, 1, 31), fpq.E4M3) > 4 * 100 * 320
+    assert fpq.fpq_conv2d_workspace_size(2, 4, 8, 8, 16, 3, 3, 1, 1, fpq.E2M5, fpq.E4M3) == 2 * 100 * 256 + 16 * 9 * 256
     assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.E5M2, fpq.E2M1) == 100 * 320    # OCP E5M2 activations: tensor cores
     assert fpq.fpq_linear_workspace_size(100, 64, 320, fpq.Format(6, 3, 7), fpq.E4M3) == 0
     assert fpq.fpq_conv2d_workspace_size(2, 4, 8, 8, 16, 3, 3, 1, 1, fpq.E4M3, fpq.E2M1) == 2 * 100 * 16
