@@ -719,10 +719,29 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             float* yrow;
             int64_t nstride;
             row_target(pair ? 2 * mt : mt, row, row_valid, yrow, nstride);
+            const int ncol0 = n0 + half * HALF;    // first output column of this warp
+
+            // With more output columns than the shared-memory table holds, the warp fetches the scales and biases
+            // of its own columns of this tile now, while the tile's MMAs still run (fetched after the accumulator was
+            // complete they cost 0.7 us per 32 columns): [HALF] x_scale * w_scale, then [HALF] bias, in the warp's
+            // own slice of shared memory (nobody else reads it: no barrier).
+            float* w_sc = s_scale + (warp - 2) * 2 * HALF;
+            if (!g.stage_scales && ksplit == 1) {
+                __syncwarp();
+#pragma unroll
+                for (int q = 0; q < 2 * HALF / 32; ++q) {
+                    const int i = q * 32 + lane;                   // [0, HALF): scale, [HALF, 2 HALF): bias
+                    const int col = ncol0 + (i < HALF ? i : i - HALF);
+                    float v = 0.f;
+                    if (col < g.N)
+                        v = i < HALF ? g.x_scale * __ldg(g.w_scale + col) : (g.bias ? __ldg(g.bias + col) : 0.f);
+                    w_sc[i] = v;
+                }
+                __syncwarp();
+            }
 
             if (!mbar_wait(acc_full + 8 * buf, aph)) { dead = true; }
             tc_fence_after();
-            const int ncol0 = n0 + half * HALF;    // first output column of this warp
             if (ksplit > 1) {
                 // partial sums of this CTA's chunk range: column-major [BN][128] at the start of the
                 // rings, which are idle once the accumulator is complete; the cluster adds them up below
@@ -765,9 +784,10 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                                 break;
                             const bool full = nb + 32 <= g.N;
                             // dequantize + bias in place
-                            if (g.stage_scales) {
-                                const float4* s4 = reinterpret_cast<const float4*>(s_scale + nb);
-                                const float4* b4 = reinterpret_cast<const float4*>(s_bias + nb);
+                            {
+                                // (from the table of all columns, or from the warp's copy for this tile)
+                                const float4* s4 = reinterpret_cast<const float4*>(g.stage_scales ? s_scale + nb : w_sc + (nb - ncol0));
+                                const float4* b4 = reinterpret_cast<const float4*>(g.stage_scales ? s_bias + nb : w_sc + HALF + (nb - ncol0));
 #pragma unroll
                                 for (int j = 0; j < 8; ++j) {
                                     const float4 sv = s4[j], bv = b4[j];
@@ -775,26 +795,6 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                                     r[cl][4 * j + 1] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 1]), sv.y, bv.y));
                                     r[cl][4 * j + 2] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 2]), sv.z, bv.z));
                                     r[cl][4 * j + 3] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 3]), sv.w, bv.w));
-                                }
-                            } else if (full && g.vec_scale) {
-                                const float4* s4 = reinterpret_cast<const float4*>(g.w_scale + nb);
-                                const float4* b4 = reinterpret_cast<const float4*>(g.bias + nb);
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) {
-                                    const float4 sv = __ldg(s4 + j);
-                                    const float4 bv = g.bias ? __ldg(b4 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-                                    r[cl][4 * j + 0] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 0]), g.x_scale * sv.x, bv.x));
-                                    r[cl][4 * j + 1] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 1]), g.x_scale * sv.y, bv.y));
-                                    r[cl][4 * j + 2] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 2]), g.x_scale * sv.z, bv.z));
-                                    r[cl][4 * j + 3] = __float_as_uint(fmaf(__uint_as_float(r[cl][4 * j + 3]), g.x_scale * sv.w, bv.w));
-                                }
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) {
-                                    const bool in = nb + j < g.N;
-                                    const float sv = in ? __ldg(g.w_scale + nb + j) : 0.f;
-                                    const float bv = (in && g.bias) ? __ldg(g.bias + nb + j) : 0.f;
-                                    r[cl][j] = __float_as_uint(fmaf(__uint_as_float(r[cl][j]), g.x_scale * sv, bv));
                                 }
                             }
                             if (!FUSED && g.seg_acc) {
@@ -1145,7 +1145,9 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
         return FPQ_ERR_CUDA;
     const int n_pad = (g.N + 31) & ~31;
     g.stage_scales = (n_pad * 8 <= 16384) ? 1 : 0;
-    const int ctl = 512 + 1024 + (g.y_tma ? epi_warps(FUSED) * 8192 : 0) + (g.stage_scales ? n_pad * 8 : 0);
+    // (without the table of all columns: every epilogue warp's copy of its own columns' scales and biases, 2 * BN floats
+    // per group of four warps)
+    const int ctl = 512 + 1024 + (g.y_tma ? epi_warps(FUSED) * 8192 : 0) + (g.stage_scales ? n_pad * 8 : 4 * 2 * BN * 4);
     const int budget = SMEM_BUDGET - ctl;
     const int b_block = BN * BK;
     const int a_min_span = (g.mode == MODE_FLAT) ? g.taps : 1;
