@@ -36,7 +36,8 @@ constexpr int T_STAGE_BYTES = 2 * T_RAW_BYTES;       // P | Q as loaded (read by
 constexpr int T_STAGES = 2;
 constexpr int T_XF_W0 = 2, T_NUM_XF = 8;
 constexpr int T_THREADS = 32 * (T_XF_W0 + T_NUM_XF);
-constexpr int T_SMEM = T_STAGES * T_STAGE_BYTES + 1024 + 256;
+constexpr int T_SCALE_BYTES = T_NUM_XF * 2 * (TN / 2) * 4;      // per epilogue warp: scales and biases of its columns (epi 2)
+constexpr int T_SMEM = T_STAGES * T_STAGE_BYTES + 1024 + 256 + T_SCALE_BYTES;
 constexpr int T_CHUNK = 8;                           // 32-wide blocks accumulated in tensor memory before they are added up
 
 struct Tf32Args {
@@ -222,6 +223,20 @@ __global__ void __launch_bounds__(T_THREADS, 1) tf32x3_gemm_kernel(const __grid_
             if (lane == 0)
                 mbar_arrive(acc_empty + 8 * buf);
         };
+        // epi 2: the warp's own copy of x_scale * w_scale | bias of its columns, fetched before the main loop
+        float* w_sc = reinterpret_cast<float*>(smem + T_STAGES * T_STAGE_BYTES + 256) + (warp - T_XF_W0) * 2 * HALF;
+        if (g.epi == 2) {
+#pragma unroll
+            for (int q = 0; q < 2 * HALF / 32; ++q) {
+                const int e = q * 32 + lane;                       // [0, HALF): scale, [HALF, 2 HALF): bias
+                const int col = tj * TN + half * HALF + (e < HALF ? e : e - HALF);
+                float v = 0.f;
+                if (col < g.J)
+                    v = e < HALF ? g.x_scale * __ldg(g.w_scale + col) : (g.bias ? __ldg(g.bias + col) : 0.f);
+                w_sc[e] = v;
+            }
+            __syncwarp();
+        }
         uint32_t s = 0, ph = 0;
         for (int kb = kb_lo; kb < kb_hi && !dead; ++kb) {
             if (!mbar_wait(full + 8 * s, ph)) { dead = true; break; }
@@ -272,10 +287,8 @@ __global__ void __launch_bounds__(T_THREADS, 1) tf32x3_gemm_kernel(const __grid_
                     if (i < g.I) {
                         float o[32];
 #pragma unroll
-                        for (int v = 0; v < 32; ++v) {
-                            const int j = min(j0 + v, g.J - 1);
-                            o[v] = fmaf(r[v], g.x_scale * __ldg(g.w_scale + j), g.bias ? __ldg(g.bias + j) : 0.f);
-                        }
+                        for (int v = 0; v < 32; ++v)
+                            o[v] = fmaf(r[v], w_sc[c * 32 + v], w_sc[HALF + c * 32 + v]);
                         if (g.howo == 0) {
                             float* dst = g.C + (int64_t)i * g.ldc + j0;
                             if ((g.ldc & 3) == 0 && j0 + 32 <= g.J) {
