@@ -73,6 +73,9 @@ struct GemmArgs {
     // weight ring: a stage holds b_span consecutive blocks; resident = the whole reduction,
     // reloaded only when the column tile changes
     int b_span, b_stage_bytes, b_stages, b_resident;
+    // one weight load covers b_box_t taps x b_box_c chunks of the column tile (a TMA load costs its SM about 400
+    // cycles whatever its size): b_box_t > 1 inside a chunk's taps, b_box_c > 1 over chunks of a tap-less layer
+    int b_box_t, b_box_c;
     int y_tma;                 // row-major output leaves through TMA stores
     int vec_scale;             // w_scale / bias are 16-byte aligned
     int stage_scales;          // x_scale * w_scale[n] and bias[n] of all N columns sit in shared memory
@@ -366,6 +369,15 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
             int resident_nt = -1, resident_mt = -1;
             bool dead = false;
             bool prior_done = !g.wait_prior_grid;
+            // `count` consecutive weight blocks (chunk c2, tap t2 onward; taps fastest) of column tile n0, one load per box
+            const int b_box = g.b_box_t * g.b_box_c;
+            auto load_weights = [&](uint32_t dst, uint32_t bar, int n0, int c2, int t2, int count) {
+                for (int l = 0; l < count; l += b_box, dst += b_box * B_BLOCK_BYTES) {
+                    tma_load_4d(dst, &tmB, bar, 0, n0, t2, c2);
+                    t2 += g.b_box_t;
+                    if (t2 >= g.taps) { t2 = 0; c2 += g.b_box_c; }
+                }
+            };
             for (int t = t_lo; t < t_hi && !dead; t += t_step) {
                 int mt, nt;
                 decode_tile(t, mt, nt);
@@ -390,12 +402,7 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                         // the weights do not depend on the kernel in front: fetch them before waiting for it
                         if (!mbar_wait(b_empty + 8 * sb, pb ^ 1)) { dead = true; break; }
                         mbar_expect_tx(b_full + 8 * sb, (uint32_t)g.nblk * g.b_block_tx);
-                        uint32_t dst = b_ring + sb * g.b_stage_bytes;
-                        int c2 = 0, t2 = 0;
-                        for (int l = 0; l < g.nblk; ++l, dst += B_BLOCK_BYTES) {
-                            tma_load_3d(dst, &tmB, b_full + 8 * sb, c2 * BK, t2, n0);
-                            if (++t2 == g.taps) { t2 = 0; ++c2; }
-                        }
+                        load_weights(b_ring + sb * g.b_stage_bytes, b_full + 8 * sb, n0, 0, 0, g.nblk);
                         ++nb;
                         if (++sb == (uint32_t)g.b_stages) { sb = 0; pb ^= 1; }
                         early_b = true;
@@ -430,14 +437,10 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                     }
                     if (jb == 0 && load_b && !early_b) {
                         if (!mbar_wait(b_empty + 8 * sb, pb ^ 1)) { dead = true; break; }
-                        const int nblocks = min(g.b_span, nblk - j);
+                        // (a box that reaches past the last chunk is filled with zeros there and reports its full size)
+                        const int nblocks = (min(g.b_span, nblk - j) + b_box - 1) / b_box * b_box;
                         mbar_expect_tx(b_full + 8 * sb, (uint32_t)nblocks * g.b_block_tx);
-                        uint32_t dst = b_ring + sb * g.b_stage_bytes;
-                        int c2 = cc, t2 = tap;
-                        for (int l = 0; l < nblocks; ++l, dst += B_BLOCK_BYTES) {
-                            tma_load_3d(dst, &tmB, b_full + 8 * sb, c2 * BK, t2, n0);
-                            if (++t2 == g.taps) { t2 = 0; ++c2; }
-                        }
+                        load_weights(b_ring + sb * g.b_stage_bytes, b_full + 8 * sb, n0, cc, tap, nblocks);
                         ++nb;
                         if (++sb == (uint32_t)g.b_stages) { sb = 0; pb ^= 1; }
                     }
@@ -1133,8 +1136,14 @@ static int max_clusters(DeviceInfo* di, int size)
     return slot;
 }
 
+// what the weight tensor map is made from (its box depends on the plan, so it is encoded after planning)
+struct WeightSpec {
+    const void* w;      // prepared weights [N][taps][Cp]
+    int w4, Cp, N;
+};
+
 template <int BN, bool FUSED, int MODE>
-static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY, GemmArgs& g,
+static fpq_status launch_mode(const CUtensorMap& tmA, const WeightSpec& wspec, const CUtensorMap& tmY, GemmArgs& g,
                                  cudaStream_t st)
 {
     // Split the shared-memory budget between the two rings.  A barrier handshake costs the
@@ -1284,6 +1293,34 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
     const int dyn = g.a_stages * g.a_stage_bytes + g.b_stages * g.b_stage_bytes + ctl;
     if (!allow_max_smem<BN, FUSED, MODE>(di))
         return FPQ_ERR_CUDA;
+    // Blocks per weight load.  A stage of b_span blocks is a run of taps inside one chunk (3 x 3 layers: three taps) or
+    // a run of chunks of a tap-less layer; the resident form holds whole chunks, so one load takes all taps of a chunk.
+    g.b_box_t = g.b_box_c = 1;
+    if (g.b_resident) {
+        if (g.taps > 1 && g.taps <= 16)
+            g.b_box_t = g.taps;
+    } else if (g.taps > 1) {
+        if (g.b_span > 1 && g.taps % g.b_span == 0)
+            g.b_box_t = g.b_span;
+    } else if (g.b_span > 1) {
+        g.b_box_c = g.b_span;
+    }
+    // prepared weights [N][taps][Cp] as (position in chunk, output, tap, chunk): a box lands as [chunk][tap][output][128 B]
+    CUtensorMap tmB;
+    {
+        EncodeTiledFn enc = encode_fn();
+        if (!enc)
+            return FPQ_ERR_CUDA;
+        const cuuint64_t rowB = wspec.w4 ? (cuuint64_t)wspec.Cp / 2 : (cuuint64_t)wspec.Cp;
+        cuuint64_t dimsB[4] = {(cuuint64_t)BK, (cuuint64_t)wspec.N, (cuuint64_t)g.taps, (cuuint64_t)(wspec.Cp / BK)};
+        cuuint64_t stridesB[3] = {rowB * g.taps, rowB, wspec.w4 ? (cuuint64_t)BK / 2 : (cuuint64_t)BK};
+        cuuint32_t boxB[4] = {BK, (cuuint32_t)BN, (cuuint32_t)g.b_box_t, (cuuint32_t)g.b_box_c};
+        cuuint32_t estrB[4] = {1, 1, 1, 1};
+        if (enc(&tmB, wspec.w4 ? CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B : CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, (void*)wspec.w, dimsB,
+                stridesB, boxB, estrB, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return FPQ_ERR_CUDA;
+    }
     const int64_t tiles = (int64_t)g.m_tiles * g.n_tiles;
     if (g.ksplit > 1 && tiles * g.ksplit > 0x7fffff00ll)
         return FPQ_ERR_SHAPE;
@@ -1314,23 +1351,23 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, co
 }
 
 template <int BN, bool FUSED>
-static fpq_status launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY, GemmArgs& g,
+static fpq_status launch_variant(const CUtensorMap& tmA, const WeightSpec& wspec, const CUtensorMap& tmY, GemmArgs& g,
                                  cudaStream_t st)
 {
     // one instantiation per addressing mode keeps every kernel's code small: the single MMA-issuing
     // thread is sensitive to instruction fetch
     if (g.mode == MODE_ROWS)
-        return launch_mode<BN, FUSED, MODE_ROWS>(tmA, tmB, tmY, g, st);
+        return launch_mode<BN, FUSED, MODE_ROWS>(tmA, wspec, tmY, g, st);
     if (g.mode == MODE_FLAT && g.pair) {
         if (FUSED)
             return FPQ_ERR_UNSUPPORTED;
-        return launch_mode<BN, false, MODE_FLAT2>(tmA, tmB, tmY, g, st);
+        return launch_mode<BN, false, MODE_FLAT2>(tmA, wspec, tmY, g, st);
     }
     if (g.mode == MODE_FLAT)
-        return launch_mode<BN, FUSED, MODE_FLAT>(tmA, tmB, tmY, g, st);
+        return launch_mode<BN, FUSED, MODE_FLAT>(tmA, wspec, tmY, g, st);
     if (FUSED)
         return FPQ_ERR_UNSUPPORTED;
-    return launch_mode<BN, false, MODE_TAPS>(tmA, tmB, tmY, g, st);
+    return launch_mode<BN, false, MODE_TAPS>(tmA, wspec, tmY, g, st);
 }
 
 fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
@@ -1367,7 +1404,7 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
     g.idesc = idesc_f8f6f4(p.a_e5m2 ? 1u : 0u, p.w4 ? 5u : (p.w_e5m2 ? 1u : 0u), (uint32_t)BN);
     g.b_block_tx = (uint32_t)(BN * BK) / (p.w4 ? 2 : 1);
 
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA;
     cuuint64_t dimsA[4], stridesA[3];
     cuuint32_t boxA[4], estrA[4] = {1, 1, 1, 1};
     const int Hp = p.H + 2 * p.pad, Wp = p.W + 2 * p.pad;
@@ -1470,17 +1507,8 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return FPQ_ERR_CUDA;
 
-    // prepared weights [N][taps][Cp]
-    cuuint64_t dimsB[3] = {(cuuint64_t)p.Cp, (cuuint64_t)g.taps, (cuuint64_t)p.N};
-    cuuint64_t rowB = p.w4 ? (cuuint64_t)p.Cp / 2 : (cuuint64_t)p.Cp;
-    cuuint64_t stridesB[2] = {rowB, rowB * g.taps};
-    cuuint32_t boxB[3] = {BK, 1, (cuuint32_t)BN};
-    cuuint32_t estrB[3] = {1, 1, 1};
-    if (enc(&tmB, p.w4 ? CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B : CU_TENSOR_MAP_DATA_TYPE_UINT8, 3,
-            (void*)p.w_prepared, dimsB, stridesB, boxB, estrB, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return FPQ_ERR_CUDA;
+    // (the weight map is encoded once the plan has fixed how many blocks one load covers)
+    const WeightSpec wspec = {p.w_prepared, p.w4, p.Cp, p.N};
 
     // row-major output through TMA stores
     CUtensorMap tmY = tmA;
@@ -1509,11 +1537,11 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
         g.W = p.W;
         g.pad = p.pad;
         g.wait_prior_grid = 0;
-        return BN == 64 ? launch_variant<64, true>(tmA, tmB, tmY, g, st) : launch_variant<128, true>(tmA, tmB, tmY, g, st);
+        return BN == 64 ? launch_variant<64, true>(tmA, wspec, tmY, g, st) : launch_variant<128, true>(tmA, wspec, tmY, g, st);
     }
     if (p.x != nullptr)
         return FPQ_ERR_UNSUPPORTED;     // the caller falls back to the two-kernel route
-    return BN == 64 ? launch_variant<64, false>(tmA, tmB, tmY, g, st) : launch_variant<128, false>(tmA, tmB, tmY, g, st);
+    return BN == 64 ? launch_variant<64, false>(tmA, wspec, tmY, g, st) : launch_variant<128, false>(tmA, wspec, tmY, g, st);
 }
 
 }  // namespace fpq
