@@ -76,6 +76,7 @@ struct GemmArgs {
     // one weight load covers b_box_t taps x b_box_c chunks of the column tile (a TMA load costs its SM about 400
     // cycles whatever its size): b_box_t > 1 inside a chunk's taps, b_box_c > 1 over chunks of a tap-less layer
     int b_box_t, b_box_c;
+    int a_box_c;               // row-major activations: one load covers the a_box_c chunks of a stage (1 = one per chunk)
     int y_tma;                 // row-major output leaves through TMA stores
     int vec_scale;             // w_scale / bias are 16-byte aligned
     int stage_scales;          // x_scale * w_scale[n] and bias[n] of all N columns sit in shared memory
@@ -417,9 +418,13 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
                         if (!mbar_wait(a_empty + 8 * sa, pa ^ 1)) { dead = true; break; }
                         const int nblocks = min(g.a_span, nblk - j);
                         const int nloads = (MODE == MODE_TAPS) ? nblocks : nblocks / g.taps;
-                        mbar_expect_tx(a_full + 8 * sa, (uint32_t)nloads * g.a_chunk_tx);
+                        const bool a_wide = MODE == MODE_ROWS && g.a_box_c > 1;
+                        mbar_expect_tx(a_full + 8 * sa, (uint32_t)(a_wide ? g.a_box_c : nloads) * g.a_chunk_tx);
                         uint32_t dst = a_ring + sa * g.a_stage_bytes;
-                        if (MODE == MODE_TAPS) {
+                        if (a_wide) {
+                            // all chunks of the stage in one box (chunks past the last one read as zeros)
+                            tma_load_4d(dst, &tmA, a_full + 8 * sa, 0, mt * tile_rows, cc, 0);
+                        } else if (MODE == MODE_TAPS) {
                             int c2 = cc, t2 = tap, r2 = r, s2 = sx;
                             for (int l = 0; l < nloads; ++l, dst += g.a_chunk_bytes) {
                                 tma_load_4d(dst, &tmA, a_full + 8 * sa, c2 * BK, x0 + s2, y0 + r2, b0);
@@ -1140,6 +1145,9 @@ static int max_clusters(DeviceInfo* di, int size)
 struct WeightSpec {
     const void* w;      // prepared weights [N][taps][Cp]
     int w4, Cp, N;
+    const void* a;      // row-major activation codes [M][Ca] (linear layers), else NULL
+    int Ca;
+    int64_t M;
 };
 
 template <int BN, bool FUSED, int MODE>
@@ -1306,11 +1314,24 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const WeightSpec& wspec, c
         g.b_box_c = g.b_span;
     }
     // prepared weights [N][taps][Cp] as (position in chunk, output, tap, chunk): a box lands as [chunk][tap][output][128 B]
-    CUtensorMap tmB;
+    CUtensorMap tmB, tmA2 = tmA;
+    g.a_box_c = 1;
     {
         EncodeTiledFn enc = encode_fn();
         if (!enc)
             return FPQ_ERR_CUDA;
+        if (MODE == MODE_ROWS && !FUSED && wspec.a && wspec.Ca % BK == 0 && g.taps == 1 && g.a_span > 1 && g.a_span <= 8) {
+            // rows of whole chunks: the chunks of a stage as one box, (position in chunk, row, chunk)
+            cuuint64_t dimsA[4] = {(cuuint64_t)BK, (cuuint64_t)wspec.M, (cuuint64_t)(wspec.Ca / BK), 1};
+            cuuint64_t stridesA[3] = {(cuuint64_t)wspec.Ca, (cuuint64_t)BK, (cuuint64_t)wspec.Ca * (cuuint64_t)wspec.M};
+            cuuint32_t boxA[4] = {BK, BM, (cuuint32_t)g.a_span, 1};
+            cuuint32_t estrA[4] = {1, 1, 1, 1};
+            if (enc(&tmA2, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, (void*)wspec.a, dimsA, stridesA, boxA, estrA,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return FPQ_ERR_CUDA;
+            g.a_box_c = g.a_span;
+        }
         const cuuint64_t rowB = wspec.w4 ? (cuuint64_t)wspec.Cp / 2 : (cuuint64_t)wspec.Cp;
         cuuint64_t dimsB[4] = {(cuuint64_t)BK, (cuuint64_t)wspec.N, (cuuint64_t)g.taps, (cuuint64_t)(wspec.Cp / BK)};
         cuuint64_t stridesB[3] = {rowB * g.taps, rowB, wspec.w4 ? (cuuint64_t)BK / 2 : (cuuint64_t)BK};
@@ -1346,7 +1367,7 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const WeightSpec& wspec, c
     }
     cfg.attrs = attr;
     cfg.numAttrs = (unsigned)nattr;
-    return cudaLaunchKernelEx(&cfg, fpq_gemm_kernel<BN, FUSED, MODE>, tmA, tmB, tmY, (const GemmArgs)g) == cudaSuccess ? FPQ_OK
+    return cudaLaunchKernelEx(&cfg, fpq_gemm_kernel<BN, FUSED, MODE>, tmA2, tmB, tmY, (const GemmArgs)g) == cudaSuccess ? FPQ_OK
                                                                                                       : FPQ_ERR_CUDA;
 }
 
@@ -1508,7 +1529,7 @@ fpq_status launch_gemm(const GemmProblem& p, cudaStream_t st)
         return FPQ_ERR_CUDA;
 
     // (the weight map is encoded once the plan has fixed how many blocks one load covers)
-    const WeightSpec wspec = {p.w_prepared, p.w4, p.Cp, p.N};
+    const WeightSpec wspec = {p.w_prepared, p.w4, p.Cp, p.N, (!p.conv && p.x == nullptr) ? p.a_codes : nullptr, p.Ca, p.M};
 
     // row-major output through TMA stores
     CUtensorMap tmY = tmA;
