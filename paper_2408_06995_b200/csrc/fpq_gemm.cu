@@ -1307,6 +1307,8 @@ static fpq_status launch_mode(const CUtensorMap& tmA, const WeightSpec& wspec, c
     if (g.b_resident) {
         if (g.taps > 1 && g.taps <= 16)
             g.b_box_t = g.taps;
+        else if (g.taps == 1 && g.cchunks > 1 && g.cchunks <= 8)
+            g.b_box_c = g.cchunks;
     } else if (g.taps > 1) {
         if (g.b_span > 1 && g.taps % g.b_span == 0)
             g.b_box_t = g.b_span;
