@@ -472,6 +472,10 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         // loop shapes (3x3 taps over one loaded chunk; one block per chunk) are
         // straight-line code.
         if (elect_one()) {
+            // (the limits of this role's waits start counting once the kernel in front has finished: its run time
+            // is not this kernel's)
+            if (g.wait_prior_grid)
+                asm volatile("griddepcontrol.wait;" ::: "memory");
             uint32_t sa = 0, pa = 0, sb = 0, pb = 0, it = 0;
             uint32_t sa0 = 0, pa0 = 0;                 // ring position of the resident activation panel
             int resident_nt = -1, resident_mt = -1;
@@ -713,6 +717,9 @@ __global__ void __launch_bounds__(num_threads(FUSED), 1) fpq_gemm_kernel(const _
         // buffer and leaves as one TMA store (whole 128-byte lines; rows past M and columns
         // past N are clipped by the tensor map)
         uint8_t* stage0 = smem + ctl_off + (warp - 2) * 8192;     // two 4 KiB buffers, used in turn
+        // (as in the MMA role: bounded waits start counting after the kernel in front)
+        if (g.wait_prior_grid)
+            asm volatile("griddepcontrol.wait;" ::: "memory");
         uint32_t nstore = 0;
         uint32_t it = 0;
         bool dead = false;
